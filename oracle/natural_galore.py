@@ -1,0 +1,219 @@
+"""fp64 CPU oracle of the Natural GaLore per-matrix optimizer update.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+optimizer computes, written from the paper's equations; the tests, the smoke
+check and the benchmark's CPU-baseline leg are its only callers.  It shares no
+code with the CUDA path and must never be imported by the product package.
+
+Every quantity is float64.  One ``MatrixState`` holds the state of one weight
+matrix W (M x N); ``step`` advances it by one optimizer step in the order the
+paper gives:
+
+  O0  every T steps: P <- first r' left singular vectors of G        (Sec. 1 "GaLore" paragraph; Sec. 2.2)
+  O1  R = P^T G                                                        (Sec. 1, low-rank projection equation)
+  O2  push R into the history of the last s low-rank gradients         (Sec. 2.4, stacked matrix G)
+  O3  K_ij = <H_i, H_j> / c                                            (Sec. 2.2 empirical FIM, mean of outer products)
+  O4  S = I + K / lambda,  y = U^T vec(R),  solve S z = y (Cholesky)   (Sec. 2.4)
+  O5  N~ = R / lambda - (1 / lambda^2) U z                             (Sec. 2.4, last equation)
+  O6  m, v, u = m / sqrt(v + eps)                                      (Sec. 2.2, Adam equations as printed)
+  O7  W <- W - eta P u - eta wd W                                      (Sec. 2.2 update equation; decoupled decay as in AdamW)
+
+with U = [vec(H_1) ... vec(H_c)] / sqrt(c) and c the number of gradients held.
+
+Readings taken where the paper is silent or inconsistent (each is listed in the
+design notes): left projection only; r' = min(r, M, N); the empirical Fisher is
+the *mean* of outer products plus lambda I (the 1/h of the Sec. 2.2 definition
+carried into Sec. 2.4); exactly s columns, the current gradient among them;
+divide by the number of gradients actually held while the history fills; eps
+inside the square root and no bias correction, as printed; scale factor alpha = 1;
+decoupled weight decay on the pre-update W; refresh when k mod T == 0 from the
+current gradient; moments and history are kept across a refresh.
+
+Parity pins: every function below is pinned by tests/test_oracle_pins.py
+(Woodbury against a dense solve, Sherman-Morrison closed forms, Eckart-Young,
+the GaLore/Adam reductions, a hand-worked step).  The absolute values of the
+update on the benchmark workloads are "parity unpinned" by the paper itself: it
+prints no worked example of the optimizer step.
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import List, Optional
+
+import numpy as np
+
+
+# ----------------------------------------------------------------------------- small pieces
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Values of x rounded to the nearest bf16 (ties to even), returned as float64.
+
+    Used only to hold the projection matrix in the storage format the update is
+    defined on (P is kept as bf16 by contract; see the design notes)."""
+    f = np.ascontiguousarray(x, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
+def left_singular_basis(G: np.ndarray, r: int) -> np.ndarray:
+    """First r' = min(r, M, N) left singular vectors of G (compact SVD G = P Sigma Q^T, Sec. 1)."""
+    G = np.asarray(G, dtype=np.float64)
+    rp = min(r, G.shape[0], G.shape[1])
+    U, _, _ = np.linalg.svd(G, full_matrices=False)
+    return np.ascontiguousarray(U[:, :rp])
+
+
+def project(P: np.ndarray, G: np.ndarray) -> np.ndarray:
+    """Low-rank gradient R = P^T G (Sec. 1)."""
+    return P.T @ G
+
+
+def gram_matrix(history: List[np.ndarray]) -> np.ndarray:
+    """K = U^T U with U = [vec(H_1) ... vec(H_c)] / sqrt(c): K_ij = <H_i, H_j>_F / c."""
+    c = len(history)
+    K = np.empty((c, c), dtype=np.float64)
+    for i in range(c):
+        for j in range(c):
+            K[i, j] = float(np.sum(history[i] * history[j])) / c
+    return K
+
+
+def cholesky_lower(S: np.ndarray) -> np.ndarray:
+    """Lower Cholesky factor L of a symmetric positive definite S (S = L L^T), written out."""
+    n = S.shape[0]
+    L = np.zeros((n, n), dtype=np.float64)
+    for j in range(n):
+        d = S[j, j] - float(np.dot(L[j, :j], L[j, :j]))
+        if not (d > 0.0) or not math.isfinite(d):
+            raise np.linalg.LinAlgError("matrix is not positive definite")
+        L[j, j] = math.sqrt(d)
+        for i in range(j + 1, n):
+            L[i, j] = (S[i, j] - float(np.dot(L[i, :j], L[j, :j]))) / L[j, j]
+    return L
+
+
+def cholesky_solve(S: np.ndarray, y: np.ndarray) -> np.ndarray:
+    """Solve S z = y through S = L L^T: forward then backward substitution (Sec. 2.4)."""
+    L = cholesky_lower(S)
+    n = S.shape[0]
+    t = np.zeros(n, dtype=np.float64)
+    for i in range(n):
+        t[i] = (y[i] - float(np.dot(L[i, :i], t[:i]))) / L[i, i]
+    z = np.zeros(n, dtype=np.float64)
+    for i in range(n - 1, -1, -1):
+        z[i] = (t[i] - float(np.dot(L[i + 1:, i], z[i + 1:]))) / L[i, i]
+    return z
+
+
+def natural_gradient(R: np.ndarray, history: List[np.ndarray], lam: float) -> np.ndarray:
+    """N~ = F^-1 vec(R) with F = lambda I + U U^T, by the Woodbury route of Sec. 2.4.
+
+    S = I + (1/lambda) U^T U,  y = U^T vec(R),  S z = y,
+    N~ = (1/lambda) R - (1/lambda^2) U z.
+    """
+    c = len(history)
+    rc = math.sqrt(c)
+    K = gram_matrix(history)
+    S = np.eye(c) + K / lam
+    y = np.array([float(np.sum(H * R)) / rc for H in history], dtype=np.float64)
+    z = cholesky_solve(S, y)
+    Uz = np.zeros_like(R)
+    for i in range(c):
+        Uz += (z[i] / rc) * history[i]
+    return R / lam - Uz / (lam * lam)
+
+
+def adam_moments(m, v, g, beta1, beta2, eps, *, step_index=0, bias_correction=False, eps_outside=False):
+    """m, v and the direction u of the Adam equations in Sec. 2.2.
+
+    As printed: u = m / sqrt(v + eps), no bias correction.  The two switches give
+    the textbook form and exist for the reduction pin only."""
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    mh, vh = m, v
+    if bias_correction:
+        mh = m / (1.0 - beta1 ** (step_index + 1))
+        vh = v / (1.0 - beta2 ** (step_index + 1))
+    u = mh / (np.sqrt(vh) + eps) if eps_outside else mh / np.sqrt(vh + eps)
+    return m, v, u
+
+
+# ----------------------------------------------------------------------------- the optimizer state
+
+@dataclasses.dataclass
+class Hyper:
+    r: int
+    s: int
+    T: int
+    lam: float = 1e-3
+    lr: float = 1e-3
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    wd: float = 0.0
+    bias_correction: bool = False
+    eps_outside: bool = False
+    reset_history_on_refresh: bool = False
+    store_P_as_bf16: bool = True
+
+
+class MatrixState:
+    """Optimizer state of one M x N weight matrix."""
+
+    def __init__(self, M: int, N: int, hp: Hyper):
+        self.M, self.N, self.hp = M, N, hp
+        self.rp = min(hp.r, M, N)
+        self.P: Optional[np.ndarray] = None
+        self.m = np.zeros((self.rp, N), dtype=np.float64)
+        self.v = np.zeros((self.rp, N), dtype=np.float64)
+        self.slots: List[Optional[np.ndarray]] = [None] * max(hp.s, 0)
+        self.head = 0
+        self.count = 0
+        self.k = 0
+        self.last_natural_gradient: Optional[np.ndarray] = None
+        self.last_direction: Optional[np.ndarray] = None
+
+    # -- subspace -------------------------------------------------------------
+    def set_subspace(self, P: np.ndarray) -> None:
+        P = np.asarray(P, dtype=np.float64)
+        assert P.shape == (self.M, self.rp), (P.shape, (self.M, self.rp))
+        self.P = round_to_bf16(P) if self.hp.store_P_as_bf16 else P.copy()
+
+    def refresh(self, G: np.ndarray) -> None:
+        self.set_subspace(left_singular_basis(G, self.hp.r))
+        if self.hp.reset_history_on_refresh:
+            self.slots = [None] * max(self.hp.s, 0)
+            self.head = 0
+            self.count = 0
+
+    def history(self) -> List[np.ndarray]:
+        return [self.slots[i] for i in range(self.count)]
+
+    # -- one step ---------------------------------------------------------------
+    def step(self, W: np.ndarray, G: np.ndarray, *, auto_refresh: bool = True) -> np.ndarray:
+        """Advance by one step; W (float64, M x N) is updated in place; returns Delta W."""
+        hp = self.hp
+        G = np.asarray(G, dtype=np.float64)
+        if auto_refresh and hp.T > 0 and self.k % hp.T == 0:           # O0
+            self.refresh(G)
+        if self.P is None:
+            raise RuntimeError("no subspace: refresh first")
+        R = project(self.P, G)                                          # O1
+        if hp.s > 0:
+            self.slots[self.head] = R                                   # O2
+            self.head = (self.head + 1) % hp.s
+            self.count = min(self.count + 1, hp.s)
+            Nt = natural_gradient(R, self.history(), hp.lam)            # O3-O5
+        else:
+            Nt = R
+        self.m, self.v, u = adam_moments(self.m, self.v, Nt, hp.beta1, hp.beta2, hp.eps,
+                                         step_index=self.k, bias_correction=hp.bias_correction,
+                                         eps_outside=hp.eps_outside)    # O6
+        dW = -hp.lr * (self.P @ u) - hp.lr * hp.wd * W                  # O7
+        W += dW
+        self.k += 1
+        self.last_natural_gradient = Nt
+        self.last_direction = u
+        return dW
