@@ -1,0 +1,166 @@
+/*
+ * ngalore.h -- C ABI of the Natural GaLore optimizer step for NVIDIA B200 (sm_100a).
+ *
+ * One ngalore_state owns, on the current CUDA device, the optimizer state of a
+ * set of 2-D weight matrices.  For a matrix W (rows x cols = M x N, row-major,
+ * fp32) with gradient G (M x N, row-major, bf16) one step computes
+ *
+ *   R  = P^T G                                   low-rank projection        (Sec. 1, "GaLore" paragraph)
+ *   H[head] <- R, ring of the s latest R         stacked gradient matrix    (Sec. 2.4)
+ *   K_ij = <H_i, H_j> / c                        empirical Fisher, mean of outer products (Sec. 2.2)
+ *   (lambda I + K) w = e_cur, by Cholesky        the s x s system           (Sec. 2.4; equals S z = y after scaling)
+ *   N~ = sum_i w_i H_i                           natural gradient F^-1 R    (Sec. 2.4, Woodbury identity)
+ *   m, v, u = m / sqrt(v + eps)                  Adam moments as printed    (Sec. 2.2)
+ *   W <- (1 - lr wd) W - lr P u                  update with decoupled decay (Sec. 2.2 update equation; AdamW)
+ *
+ * and, every T steps, first refreshes P to an orthonormal basis of the
+ * dominant r'-dimensional left singular subspace of G, r' = min(r, M, N)
+ * (Sec. 1: P from the compact SVD of the gradient, "updated periodically").
+ *
+ * Conventions
+ *  - All matrix pointers are DEVICE pointers unless a parameter says "host".
+ *    Arrays of pointers (W, G below) are HOST arrays of device pointers.
+ *  - W and G are dense row-major with leading dimension cols; cols must be a
+ *    multiple of 8 and every pointer 16-byte aligned.  The caller owns W and G;
+ *    the library owns everything else and frees it in ngalore_destroy.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    ngalore_step and ngalore_refresh_subspace enqueue work and return; they do
+ *    not synchronise and do not allocate.
+ *  - Host-detectable errors are returned at once and leave the state untouched.
+ *    Errors found on the device (a non-finite gradient, a non-positive Cholesky
+ *    pivot, a wait that ran out) set a per-matrix status word; that matrix's W,
+ *    m and v are left unchanged for the step and ngalore_poll_status reports it.
+ *    No call traps or aborts.
+ *  - A state is bound to the device that was current in ngalore_create and is
+ *    not safe for concurrent calls from several threads.
+ */
+#ifndef NGALORE_H
+#define NGALORE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ngalore_state ngalore_state;
+
+typedef struct {
+  int64_t rows; /* M */
+  int64_t cols; /* N, multiple of 8 */
+} ngalore_shape;
+
+typedef enum {
+  NGALORE_OK = 0,
+  NGALORE_ERR_INVALID_ARG = 1,
+  NGALORE_ERR_ALLOC = 2,
+  NGALORE_ERR_CUDA = 3,
+  NGALORE_ERR_UNSUPPORTED_DEVICE = 4, /* the device is not compute capability 10.x */
+  NGALORE_ERR_NO_SUBSPACE = 5,        /* step before any refresh / set_subspace with T == 0 */
+  NGALORE_ERR_NOT_SPD = 6,            /* device: Cholesky pivot <= 0 */
+  NGALORE_ERR_NONFINITE = 7,          /* device: NaN or Inf reached the Gram matrix */
+  NGALORE_ERR_TIMEOUT = 8             /* device: a bounded wait inside a kernel ran out */
+} ngalore_status;
+
+/* Optional settings; pass NULL to ngalore_create for the defaults shown. */
+typedef struct {
+  int32_t struct_size;              /* = sizeof(ngalore_options) */
+  int32_t gemm_impl;                /* 0 (default): tensor-core (tcgen05) projection GEMMs; 1: plain SIMT GEMMs (debug) */
+  int32_t power_iterations;         /* subspace-iteration sweeps in the refresh; <= 0 selects the default 4 */
+  int32_t reset_history_on_refresh; /* default 0: history, m and v survive a refresh */
+  uint64_t seed;                    /* seed of the refresh's random test matrix; 0 selects a fixed default */
+  int32_t stream_impl;              /* 0 (default): fused Gram/solve/moment kernel; 1: separate plain kernels (debug) */
+  int32_t reserved;
+} ngalore_options;
+
+/*
+ * Create the state for n_matrices weight matrices (Sec. 2.2-2.4 name the
+ * hyper-parameters: rank r, history length s, refresh period T, Tikhonov
+ * lambda, learning rate, Adam betas and eps, weight decay).
+ *   shapes      host array of n_matrices shapes
+ *   r >= 1      target rank; per matrix r' = min(r, rows, cols)
+ *   s in [0,32] history length; 0 disables the Fisher term (plain GaLore)
+ *   T >= 0      refresh period in steps; 0 = never refresh automatically
+ *   lambda > 0 when s > 0
+ * Moments and history start at zero / empty; P is unset until the first
+ * refresh or ngalore_set_subspace.  Allocates all device memory the state will
+ * ever need (cudaMalloc) on the current device.
+ */
+ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r, int s, int T,
+                              double lambda, double lr, double beta1, double beta2, double eps,
+                              double wd, const ngalore_options* opt, ngalore_state** out);
+
+/* Free the state and all its device memory (synchronises the device). NULL is allowed. */
+void ngalore_destroy(ngalore_state* st);
+
+/*
+ * One optimizer step over every matrix (equations at the top of this file).
+ *   W  host array of n_matrices device pointers, fp32 M x N, updated in place
+ *   G  host array of n_matrices device pointers, bf16 bit patterns M x N, read only
+ * If T > 0 and the step index k satisfies k mod T == 0, the subspace of every
+ * matrix is refreshed from G first.  Increments k.
+ */
+ngalore_status ngalore_step(ngalore_state* st, float* const* W, const uint16_t* const* G, void* stream);
+
+/*
+ * Refresh P from G without stepping (Sec. 1: P spans the leading left singular
+ * vectors of the gradient).  matrix_index = -1 refreshes all matrices, else one
+ * (G is still the full array of n_matrices pointers; only entry matrix_index is read).
+ * Uses a randomized subspace iteration; P is orthonormal to fp32 accuracy and is
+ * stored both as an fp32 master and as the bf16 working copy the step reads.
+ */
+ngalore_status ngalore_refresh_subspace(ngalore_state* st, const uint16_t* const* G, int matrix_index,
+                                        void* stream);
+
+/*
+ * Same step with HOST buffers: copies W and G to internal device staging,
+ * steps, copies W back and waits.  W_host / G_host are host arrays of HOST
+ * pointers (pinned memory gives asynchronous copies).  Needs staging memory of
+ * the size of all W and G, allocated on first use.
+ */
+ngalore_status ngalore_step_host(ngalore_state* st, float* const* W_host, const uint16_t* const* G_host,
+                                 void* stream);
+
+/* Wait for the state's work and copy the per-matrix status words (ngalore_status values)
+ * to the host array `per_matrix` (n_matrices ints; may be NULL); clears them on the device.
+ * Returns NGALORE_OK when all are OK, else the first non-OK status. */
+ngalore_status ngalore_poll_status(ngalore_state* st, int* per_matrix);
+
+/* Copy the fp32 master of P (rows x r', row-major) of matrix i to / from the device buffer P.
+ * set also rebuilds the bf16 working copies; the step uses the bf16 values. */
+ngalore_status ngalore_get_subspace(ngalore_state* st, int i, float* P, void* stream);
+ngalore_status ngalore_set_subspace(ngalore_state* st, int i, const float* P, void* stream);
+/* Copy the bf16 working copy of P, widened to fp32 (rows x r'), to the device buffer P. */
+ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, void* stream);
+
+/* Checkpoint: with blob == NULL stores the needed size in *bytes; else copies the whole state
+ * (P, m, v, history, Gram matrices, counters) into the HOST buffer blob (synchronises).
+ * import restores it into a state created with identical shapes and r, s. */
+ngalore_status ngalore_state_export(ngalore_state* st, void* blob, size_t* bytes);
+ngalore_status ngalore_state_import(ngalore_state* st, const void* blob, size_t bytes);
+
+/* Change the learning rate used from the next step on. */
+ngalore_status ngalore_set_lr(ngalore_state* st, double lr);
+
+/* Introspection (host values, no device work). */
+int ngalore_num_matrices(const ngalore_state* st);
+int ngalore_rank(const ngalore_state* st, int i);          /* r' of matrix i, -1 if i is out of range */
+int64_t ngalore_step_count(const ngalore_state* st);        /* k */
+size_t ngalore_device_bytes(const ngalore_state* st);       /* device memory held by the state */
+/* Kernels launched by the library on behalf of this state since creation. */
+int64_t ngalore_launch_count(const ngalore_state* st);
+
+/* Per-phase timing of ngalore_step with CUDA events recorded on the launching stream.
+ * phase: 0 projection GEMM (R = P^T G), 1 Gram / solve / moment kernels, 2 back-projection + W update.
+ * ngalore_last_phase_ms waits for the step and returns milliseconds, or a negative value when
+ * profiling is off or no step has run. */
+ngalore_status ngalore_set_profiling(ngalore_state* st, int on);
+double ngalore_last_phase_ms(ngalore_state* st, int phase);
+
+const char* ngalore_status_string(ngalore_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NGALORE_H */

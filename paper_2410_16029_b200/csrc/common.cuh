@@ -1,0 +1,64 @@
+// Shared device-side structures of the Natural GaLore step library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ngalore {
+
+constexpr int kMaxHistory = 32;       // s <= 32: one warp lane per Gram row in the solve
+constexpr int kStreamThreads = 256;   // threads per CTA of the streaming kernels
+
+// Per-matrix device descriptor (array in device memory, one entry per weight matrix).
+struct MatDesc {
+  int M, N, rp, s;            // rows, cols, r' = min(r, M, N), history length
+  long long rn;               // rp * N, elements of one low-rank matrix
+  float* H;                   // history ring: s slots of rp x N fp32 (one slot when s == 0)
+  float* m;                   // first moment, rp x N
+  float* v;                   // second moment, rp x N
+  __nv_bfloat16* u_hi;        // direction u = m / sqrt(v + eps), high bf16 part, rp x N
+  __nv_bfloat16* u_lo;        // low part: bf16(u - hi)
+  __nv_bfloat16* P16;         // working copy of P, M x rp row-major
+  __nv_bfloat16* Pt16;        // working copy of P^T, rp x M row-major
+  float* P32;                 // fp32 master of P, M x rp row-major
+  double* Kraw;               // s x s raw inner products <H_i, H_j>
+  float* wsol;                // kMaxHistory solution weights of (lambda I + K) w = e_cur
+  double* gpart;              // per-tile partial Gram rows: ntiles x s
+  int* status;                // sticky ngalore_status word
+  int* step_bad;              // 1 when this step must leave W, m, v untouched
+  int* gram_done;             // fused kernel: count of finished Gram tiles of this step
+  int* w_ready;               // fused kernel: set to the step epoch once wsol is valid
+  int tile0, ntiles;          // range of streaming tiles owned by this matrix
+};
+
+struct Ctrl {
+  long long n_appended;       // low-rank gradients pushed into the ring so far
+  long long k;                // optimizer step index
+  int epoch;                  // increments every step; flags of the fused kernel compare against it
+  int timeout_flag;           // set when a bounded wait ran out
+  unsigned int work_counter;  // dynamic tile counter of the fused streaming kernel
+  unsigned int gemm_counter;  // dynamic tile counter of the tensor-core GEMMs
+};
+
+struct Hyper {
+  float lr, wd, beta1, beta2, eps;
+  float pad;
+  double lambda;
+};
+
+struct StreamTile {
+  int mat;    // matrix index
+  int local;  // tile index inside the matrix
+};
+
+__device__ __forceinline__ int ring_cur(const Ctrl* c, int s) {
+  return s > 0 ? static_cast<int>(c->n_appended % s) : 0;
+}
+__device__ __forceinline__ int ring_count(const Ctrl* c, int s) {
+  if (s <= 0) return 1;
+  long long n = c->n_appended + 1;
+  return n < s ? static_cast<int>(n) : s;
+}
+
+}  // namespace ngalore

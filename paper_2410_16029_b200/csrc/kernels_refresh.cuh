@@ -1,0 +1,247 @@
+// Pieces of the subspace refresh (Sec. 1: P spans the leading left singular vectors of G,
+// "updated periodically").  The refresh is a randomized subspace iteration; every application of
+// G or G^T is followed by an orthonormalisation Q = Y R^-1 with R^T R = Y^T Y (Cholesky QR with
+// the Gram matrix and the factorisation in fp64).
+#pragma once
+
+#include "common.cuh"
+
+namespace ngalore {
+
+// ---------------------------------------------------------------- random test matrix
+
+__device__ __forceinline__ unsigned long long splitmix64(unsigned long long x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+// Standard normal entries from a counter-based hash (Box-Muller on two hashed uniforms).
+__global__ void fill_normal_kernel(float* X, long long n, unsigned long long seed, unsigned long long stream_id) {
+  const long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (i >= n) return;
+  const unsigned long long h =
+      splitmix64(seed ^ splitmix64(stream_id * 0x100000001B3ull + static_cast<unsigned long long>(i)));
+  const float u1 = (static_cast<float>(h >> 40) + 1.0f) * (1.0f / 16777217.0f);
+  const float u2 = static_cast<float>((h >> 8) & 0xFFFFFFull) * (1.0f / 16777216.0f);
+  X[i] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+}
+
+// ---------------------------------------------------------------- batched Cholesky (fp64, one CTA per matrix)
+
+struct CholProblem {
+  double* C;  // L x L row-major; lower triangle in, lower Cholesky factor out (C = Lf Lf^T)
+  int L;
+};
+
+// Left-looking blocked Cholesky, block width 32, 512 threads.  A pivot that is not positive
+// (rank-deficient Y) is replaced by a tiny positive number so that the factor stays finite;
+// the caller runs a second orthonormalisation pass at the end of the refresh.
+__global__ void __launch_bounds__(512) chol_batched_kernel(const CholProblem* probs) {
+  constexpr int NB = 32;
+  __shared__ double D[NB][NB + 1];   // diagonal block, or rows j0..j0+31 of the factor for one k-chunk
+  __shared__ double Rs[64][NB + 1];  // 64 panel rows for one k-chunk
+  __shared__ double maxdiag_s;
+  const CholProblem p = probs[blockIdx.x];
+  double* C = p.C;
+  const int L = p.L;
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    double md = 0.0;
+    for (int i = 0; i < L; ++i) md = fmax(md, C[static_cast<long long>(i) * L + i]);
+    maxdiag_s = md;
+  }
+  __syncthreads();
+  const double tiny = fmax(maxdiag_s, 1e-300) * 1e-28;
+
+  for (int j0 = 0; j0 < L; j0 += NB) {
+    const int nbj = (L - j0 < NB) ? (L - j0) : NB;
+    // (a) panel update: C[i][j0+jj] -= sum_{k<j0} C[i][k] C[j0+jj][k], rows i >= j0.
+    for (int r0 = j0; r0 < L; r0 += 64) {
+      const int row = tid >> 3;      // 0..63
+      const int cg = (tid & 7) * 4;  // 4 consecutive panel columns
+      double acc[4] = {0.0, 0.0, 0.0, 0.0};
+      for (int k0 = 0; k0 < j0; k0 += NB) {
+        for (int x = tid; x < NB * NB; x += 512) {
+          const int a = x / NB, b = x % NB;
+          D[a][b] = (a < nbj) ? C[static_cast<long long>(j0 + a) * L + k0 + b] : 0.0;
+        }
+        for (int x = tid; x < 64 * NB; x += 512) {
+          const int a = x / NB, b = x % NB;
+          Rs[a][b] = (r0 + a < L) ? C[static_cast<long long>(r0 + a) * L + k0 + b] : 0.0;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int b = 0; b < NB; ++b) {
+          const double rv = Rs[row][b];
+          acc[0] += rv * D[cg + 0][b];
+          acc[1] += rv * D[cg + 1][b];
+          acc[2] += rv * D[cg + 2][b];
+          acc[3] += rv * D[cg + 3][b];
+        }
+        __syncthreads();
+      }
+      if (r0 + row < L) {
+#pragma unroll
+        for (int y = 0; y < 4; ++y)
+          if (cg + y < nbj) C[static_cast<long long>(r0 + row) * L + j0 + cg + y] -= acc[y];
+      }
+    }
+    __syncthreads();
+    // (b) factor the diagonal block in shared memory (warp 0, lane = row).
+    for (int x = tid; x < NB * NB; x += 512) {
+      const int a = x / NB, b = x % NB;
+      D[a][b] = (a < nbj && b < nbj) ? C[static_cast<long long>(j0 + a) * L + j0 + b] : 0.0;
+    }
+    __syncthreads();
+    if (tid < 32) {
+      const int lane = tid;
+      for (int k = 0; k < nbj; ++k) {
+        double dkk = D[k][k];
+        if (!(dkk > tiny)) dkk = tiny;
+        const double lkk = sqrt(dkk);
+        __syncwarp();
+        if (lane == k) D[k][k] = lkk;
+        if (lane > k && lane < nbj) D[lane][k] /= lkk;
+        __syncwarp();
+        if (lane > k && lane < nbj) {
+          const double lik = D[lane][k];
+          for (int j = k + 1; j <= lane; ++j) D[lane][j] -= lik * D[j][k];
+        }
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+    for (int x = tid; x < NB * NB; x += 512) {
+      const int a = x / NB, b = x % NB;
+      if (a < nbj && b <= a) C[static_cast<long long>(j0 + a) * L + j0 + b] = D[a][b];
+    }
+    // (c) rows below the block: x D^T = c, forward substitution, one thread per row.
+    for (int i = j0 + nbj + tid; i < L; i += 512) {
+      double xr[NB];
+      double* crow = C + static_cast<long long>(i) * L + j0;
+#pragma unroll
+      for (int jj = 0; jj < NB; ++jj) {
+        if (jj < nbj) {
+          double a = crow[jj];
+#pragma unroll
+          for (int t = 0; t < NB; ++t)
+            if (t < jj) a -= xr[t] * D[jj][t];
+          xr[jj] = a / D[jj][jj];
+        }
+      }
+#pragma unroll
+      for (int jj = 0; jj < NB; ++jj)
+        if (jj < nbj) crow[jj] = xr[jj];
+    }
+    __syncthreads();
+  }
+}
+
+// ---------------------------------------------------------------- Q = Y Lf^-T (rows are independent)
+
+// One CTA owns 32 rows of Y (rows x L, fp32) and produces the same rows of Q (fp32) with
+// Q Lf^T = Y, Lf the lower Cholesky factor of Y^T Y (fp64).  Column blocks of 32 are solved in
+// order; finished columns of Q stay in shared memory (fp64).
+struct OrthApply {
+  const float* Y;
+  float* Q;
+  const double* Lf;
+  int rows, L;
+};
+
+inline size_t orth_apply_smem_bytes(int L) {
+  return (static_cast<size_t>(32) * L + 32 * 33) * sizeof(double);
+}
+
+__global__ void __launch_bounds__(256) orth_apply_kernel(OrthApply p) {
+  constexpr int NB = 32, RB = 32;
+  extern __shared__ __align__(16) unsigned char orth_smem_raw[];
+  double* Qs = reinterpret_cast<double*>(orth_smem_raw);  // RB x L (finished columns)
+  double* Ls = Qs + static_cast<size_t>(RB) * p.L;        // NB x (NB + 1) chunk of Lf
+  const int tid = threadIdx.x;
+  const int r0 = blockIdx.x * RB;
+  const int L = p.L;
+  const int row = tid >> 3;      // 0..31
+  const int cg = (tid & 7) * 4;  // 4 columns of the current block
+  for (int j0 = 0; j0 < L; j0 += NB) {
+    const int nbj = (L - j0 < NB) ? (L - j0) : NB;
+    double acc[4];
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const int col = j0 + cg + y;
+      acc[y] = (r0 + row < p.rows && col < L)
+                   ? static_cast<double>(p.Y[static_cast<long long>(r0 + row) * L + col])
+                   : 0.0;
+    }
+    for (int k0 = 0; k0 < j0; k0 += NB) {
+      __syncthreads();
+      for (int x = tid; x < NB * NB; x += 256) {
+        const int a = x / NB, b = x % NB;
+        Ls[a * (NB + 1) + b] = (a < nbj) ? p.Lf[static_cast<long long>(j0 + a) * L + k0 + b] : 0.0;
+      }
+      __syncthreads();
+#pragma unroll 8
+      for (int b = 0; b < NB; ++b) {
+        const double qv = Qs[static_cast<size_t>(row) * L + k0 + b];
+        acc[0] -= qv * Ls[(cg + 0) * (NB + 1) + b];
+        acc[1] -= qv * Ls[(cg + 1) * (NB + 1) + b];
+        acc[2] -= qv * Ls[(cg + 2) * (NB + 1) + b];
+        acc[3] -= qv * Ls[(cg + 3) * (NB + 1) + b];
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int y = 0; y < 4; ++y)
+      if (cg + y < nbj) Qs[static_cast<size_t>(row) * L + j0 + cg + y] = acc[y];
+    for (int x = tid; x < NB * NB; x += 256) {
+      const int a = x / NB, b = x % NB;
+      Ls[a * (NB + 1) + b] = (a < nbj && b < nbj) ? p.Lf[static_cast<long long>(j0 + a) * L + j0 + b] : 0.0;
+    }
+    __syncthreads();
+    if (tid < RB) {
+      double* q = Qs + static_cast<size_t>(tid) * L + j0;
+      for (int jj = 0; jj < nbj; ++jj) {
+        double a = q[jj];
+        for (int t = 0; t < jj; ++t) a -= q[t] * Ls[jj * (NB + 1) + t];
+        q[jj] = a / Ls[jj * (NB + 1) + jj];
+      }
+    }
+    __syncthreads();
+  }
+  for (int x = tid; x < RB * L; x += 256) {
+    const int a = x / L, b = x % L;
+    if (r0 + a < p.rows)
+      p.Q[static_cast<long long>(r0 + a) * L + b] = static_cast<float>(Qs[static_cast<size_t>(a) * L + b]);
+  }
+}
+
+// ---------------------------------------------------------------- working copies of P
+
+// P16 = bf16(P32) (M x rp) and Pt16 = its transpose (rp x M).  Block (32, 8).
+__global__ void working_copies_kernel(const float* P32, __nv_bfloat16* P16, __nv_bfloat16* Pt16, int M, int rp) {
+  __shared__ float tile[32][33];
+  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
+  for (int a = threadIdx.y; a < 32; a += blockDim.y) {
+    const int i = i0 + a, j = j0 + threadIdx.x;
+    float val = 0.f;
+    if (i < M && j < rp) {
+      val = P32[static_cast<long long>(i) * rp + j];
+      P16[static_cast<long long>(i) * rp + j] = __float2bfloat16_rn(val);
+    }
+    tile[a][threadIdx.x] = val;
+  }
+  __syncthreads();
+  for (int a = threadIdx.y; a < 32; a += blockDim.y) {
+    const int j = j0 + a, i = i0 + threadIdx.x;
+    if (i < M && j < rp) Pt16[static_cast<long long>(j) * M + i] = __float2bfloat16_rn(tile[threadIdx.x][a]);
+  }
+}
+
+__global__ void widen_bf16_kernel(const __nv_bfloat16* src, float* dst, long long n) {
+  const long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (i < n) dst[i] = __bfloat162float(src[i]);
+}
+
+}  // namespace ngalore
