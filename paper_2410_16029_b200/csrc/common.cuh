@@ -38,7 +38,8 @@ struct Ctrl {
   int epoch;                  // increments every step; flags of the fused kernel compare against it
   int timeout_flag;           // set when a bounded wait ran out
   unsigned int work_counter;  // dynamic tile counter of the fused streaming kernel
-  unsigned int gemm_counter;  // dynamic tile counter of the tensor-core GEMMs
+  unsigned int gemm_counter0; // dynamic tile counter of the projection GEMM
+  unsigned int gemm_counter1; // dynamic tile counter of the back-projection GEMM
 };
 
 struct Hyper {

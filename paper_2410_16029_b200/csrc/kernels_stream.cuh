@@ -48,7 +48,10 @@ __device__ __forceinline__ void gram_tile(const MatDesc& d, int local, int cur, 
     double t = 0.0;
 #pragma unroll
     for (int w = 0; w < kStreamThreads / 32; ++w) t += red[w * SMAX + threadIdx.x];
-    if (static_cast<int>(threadIdx.x) < d.s) d.gpart[static_cast<long long>(local) * d.s + threadIdx.x] = t;
+    if (static_cast<int>(threadIdx.x) < d.s) {
+      d.gpart[static_cast<long long>(local) * d.s + threadIdx.x] = t;
+      __threadfence();  // a later reader may run in another CTA of the same launch
+    }
   }
   __syncthreads();
 }
@@ -67,7 +70,7 @@ __device__ __forceinline__ void solve_matrix(const MatDesc& d, int cur, int c, d
   if (d.s > 0) {
     double row = 0.0;
     if (lane < c) {
-      for (int t = 0; t < d.ntiles; ++t) row += d.gpart[static_cast<long long>(t) * d.s + lane];
+      for (int t = 0; t < d.ntiles; ++t) row += __ldcg(d.gpart + static_cast<long long>(t) * d.s + lane);
       if (!isfinite(row)) finite = false;
     }
     finite = __all_sync(0xffffffffu, finite);
@@ -152,7 +155,7 @@ __device__ __forceinline__ void combine_tile(const MatDesc& d, int local, int cu
                                              const Hyper& hp, const float* wsm /* smem weights */) {
   const long long e0 = static_cast<long long>(local) * tile_elems;
   const long long e1 = (e0 + tile_elems < d.rn) ? e0 + tile_elems : d.rn;
-  if (*d.step_bad) {
+  if (__ldcg(d.step_bad)) {
     float* Hc = d.H + static_cast<long long>(cur) * d.rn;
     for (long long e = e0 + threadIdx.x * 4; e < e1; e += kStreamThreads * 4) {
       *reinterpret_cast<float4*>(Hc + e) = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -240,7 +243,8 @@ __global__ void advance_kernel(Ctrl* ctrl) {
   ctrl->k += 1;
   ctrl->epoch += 1;
   ctrl->work_counter = 0u;
-  ctrl->gemm_counter = 0u;
+  ctrl->gemm_counter0 = 0u;
+  ctrl->gemm_counter1 = 0u;
 }
 
 }  // namespace ngalore

@@ -1,0 +1,738 @@
+// C-ABI entry points of the Natural GaLore step library: state layout, orchestration of one
+// optimizer step and of the subspace refresh.  See include/ngalore.h for the contract.
+#include "../../include/ngalore.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "kernels_refresh.cuh"
+#include "kernels_simt_gemm.cuh"
+#include "kernels_stream.cuh"
+#include "gemm_tcgen05.cuh"
+#include "kernels_fused_stream.cuh"
+
+using namespace ngalore;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct HostMat {
+  int M, N, rp;
+  long long rn;
+  // refresh scratch (device)
+  float *Ya, *Yb, *Xa, *Xb;
+  double* C;
+};
+
+struct BlobHeader {
+  uint64_t magic;
+  uint64_t arena_bytes;
+  int64_t k;
+  int64_t n_appended;
+  int32_t n, r, s, has_subspace;
+  uint64_t shape_hash;
+};
+constexpr uint64_t kBlobMagic = 0x4E47414C4F524531ull;  // "NGALORE1"
+
+}  // namespace
+
+struct ngalore_state {
+  int device = 0;
+  int n = 0, r = 0, s = 0, T = 0;
+  Hyper hyper{};
+  bool hyper_dirty = true;
+  ngalore_options opt{};
+  std::vector<HostMat> mats;
+  std::vector<MatDesc> h_desc;
+  MatDesc* d_desc = nullptr;
+  char* arena = nullptr;  // persistent optimizer state (exported by checkpoints)
+  size_t arena_bytes = 0;
+  char* work = nullptr;   // scratch, tables, per-step buffers
+  size_t work_bytes = 0;
+  Ctrl* d_ctrl = nullptr;
+  Hyper* d_hyper = nullptr;
+  int* d_status = nullptr;
+  int* d_step_bad = nullptr;
+  StreamTile* d_tiles = nullptr;
+  int n_tiles = 0, tile_elems = 0;
+  float** d_W = nullptr;
+  const __nv_bfloat16** d_G = nullptr;
+  std::vector<const void*> last_W, last_G;
+  CholProblem* d_chol = nullptr;
+  int64_t k = 0;
+  int64_t n_appended = 0;
+  bool has_subspace = false;
+  int64_t launches = 0;
+  uint64_t shape_hash = 0;
+  // tensor-core GEMM plan (tile tables, tensor maps)
+  TcPlan tc;
+  // fused streaming kernel plan
+  FusedPlan fused;
+  // host-buffer staging
+  char* stage = nullptr;
+  size_t stage_bytes = 0;
+  std::vector<float*> stage_W;
+  std::vector<uint16_t*> stage_G;
+  // profiling
+  bool profiling = false;
+  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  bool ev_valid = false;
+};
+
+namespace {
+
+#define NG_CUDA(expr)                                   \
+  do {                                                  \
+    cudaError_t e__ = (expr);                           \
+    if (e__ != cudaSuccess) return NGALORE_ERR_CUDA;    \
+  } while (0)
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+template <int SMAX>
+void launch_plain_stream(ngalore_state* st, cudaStream_t stream) {
+  if (st->s > 0) {
+    gram_kernel<SMAX><<<st->n_tiles, kStreamThreads, 0, stream>>>(st->d_desc, st->d_tiles, st->d_ctrl, st->tile_elems);
+    solve_kernel<<<(st->n + 3) / 4, 128, 0, stream>>>(st->d_desc, st->n, st->d_ctrl, st->d_hyper);
+    st->launches += 2;
+  }
+  combine_kernel<SMAX><<<st->n_tiles, kStreamThreads, 0, stream>>>(st->d_desc, st->d_tiles, st->d_ctrl, st->d_hyper,
+                                                                   st->tile_elems);
+  st->launches += 1;
+}
+
+ngalore_status upload_pointers(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream,
+                               bool* changed_out) {
+  bool changed = false;
+  for (int i = 0; i < st->n; ++i) {
+    if (W != nullptr && st->last_W[i] != W[i]) { st->last_W[i] = W[i]; changed = true; }
+    if (G != nullptr && st->last_G[i] != G[i]) { st->last_G[i] = G[i]; changed = true; }
+  }
+  if (changed) {
+    // Pageable source: the runtime stages the bytes before returning, so the vectors may change later.
+    NG_CUDA(cudaMemcpyAsync(st->d_W, st->last_W.data(), sizeof(void*) * st->n, cudaMemcpyHostToDevice, stream));
+    NG_CUDA(cudaMemcpyAsync(st->d_G, st->last_G.data(), sizeof(void*) * st->n, cudaMemcpyHostToDevice, stream));
+  }
+  if (changed_out) *changed_out = changed;
+  return NGALORE_OK;
+}
+
+ngalore_status upload_hyper(ngalore_state* st, cudaStream_t stream) {
+  if (!st->hyper_dirty) return NGALORE_OK;
+  NG_CUDA(cudaMemcpyAsync(st->d_hyper, &st->hyper, sizeof(Hyper), cudaMemcpyHostToDevice, stream));
+  st->hyper_dirty = false;
+  return NGALORE_OK;
+}
+
+ngalore_status make_working_copies(ngalore_state* st, int i, cudaStream_t stream) {
+  const HostMat& hm = st->mats[i];
+  const MatDesc& d = st->h_desc[i];
+  dim3 grid((hm.rp + 31) / 32, (hm.M + 31) / 32), block(32, 8);
+  working_copies_kernel<<<grid, block, 0, stream>>>(d.P32, d.P16, d.Pt16, hm.M, hm.rp);
+  st->launches += 1;
+  NG_CUDA(cudaGetLastError());
+  return NGALORE_OK;
+}
+
+// Q = orth(Y) for a list of matrices: Gram (fp64) -> batched Cholesky -> Q = Y Lf^-T.
+// side 0: Y is M x rp (Ya -> Yb or Yb -> Ya); side 1: Y is N x rp (Xa -> Xb).
+ngalore_status orthonormalise(ngalore_state* st, const std::vector<int>& idx, int side, bool from_a,
+                              cudaStream_t stream) {
+  for (int i : idx) {
+    const HostMat& hm = st->mats[i];
+    const float* Y = side == 0 ? (from_a ? hm.Ya : hm.Yb) : (from_a ? hm.Xa : hm.Xb);
+    const int rows = side == 0 ? hm.M : hm.N;
+    SimtGemm g{};
+    g.m = hm.rp; g.n = hm.rp; g.k = rows;
+    g.A = Y; g.a_rs = 1; g.a_cs = hm.rp; g.a_dt = DT_F32;
+    g.B = Y; g.b_rs = hm.rp; g.b_cs = 1; g.b_dt = DT_F32;
+    g.C = hm.C; g.c_rs = hm.rp; g.c_cs = 1; g.c_dt = DT_F64;
+    g.epilogue = EPI_STORE;
+    NG_CUDA(launch_simt_gemm<double>(g, stream));
+    st->launches += 1;
+  }
+  // The problem table holds every matrix; launch over the selected ones.
+  if (idx.size() == static_cast<size_t>(st->n)) {
+    chol_batched_kernel<<<st->n, 512, 0, stream>>>(st->d_chol);
+    st->launches += 1;
+  } else {
+    for (int i : idx) {
+      chol_batched_kernel<<<1, 512, 0, stream>>>(st->d_chol + i);
+      st->launches += 1;
+    }
+  }
+  NG_CUDA(cudaGetLastError());
+  for (int i : idx) {
+    const HostMat& hm = st->mats[i];
+    OrthApply p{};
+    p.Y = side == 0 ? (from_a ? hm.Ya : hm.Yb) : (from_a ? hm.Xa : hm.Xb);
+    p.Q = side == 0 ? (from_a ? hm.Yb : hm.Ya) : (from_a ? hm.Xb : hm.Xa);
+    p.Lf = hm.C;
+    p.rows = side == 0 ? hm.M : hm.N;
+    p.L = hm.rp;
+    orth_apply_kernel<<<(p.rows + 31) / 32, 256, orth_apply_smem_bytes(p.L), stream>>>(p);
+    st->launches += 1;
+  }
+  NG_CUDA(cudaGetLastError());
+  return NGALORE_OK;
+}
+
+enum RefreshBuf { BUF_YA, BUF_YB, BUF_XA, BUF_XB };
+inline float* refresh_buf(const HostMat& hm, RefreshBuf b) {
+  switch (b) {
+    case BUF_YA: return hm.Ya;
+    case BUF_YB: return hm.Yb;
+    case BUF_XA: return hm.Xa;
+    default: return hm.Xb;
+  }
+}
+
+// Y = G X (side 0: out M x rp from X N x rp) or X = G^T Y (side 1: out N x rp from Y M x rp).
+ngalore_status apply_gradient(ngalore_state* st, const std::vector<int>& idx, const uint16_t* const* G, int side,
+                              RefreshBuf src, RefreshBuf dst, cudaStream_t stream) {
+  for (int i : idx) {
+    const HostMat& hm = st->mats[i];
+    SimtGemm g{};
+    if (side == 0) {
+      g.m = hm.M; g.n = hm.rp; g.k = hm.N;
+      g.A = G[i]; g.a_rs = hm.N; g.a_cs = 1;
+    } else {
+      g.m = hm.N; g.n = hm.rp; g.k = hm.M;
+      g.A = G[i]; g.a_rs = 1; g.a_cs = hm.N;
+    }
+    g.a_dt = DT_BF16;
+    g.B = refresh_buf(hm, src); g.b_rs = hm.rp; g.b_cs = 1; g.b_dt = DT_F32;
+    g.C = refresh_buf(hm, dst); g.c_rs = hm.rp; g.c_cs = 1; g.c_dt = DT_F32;
+    g.epilogue = EPI_STORE;
+    NG_CUDA(launch_simt_gemm<float>(g, stream));
+    st->launches += 1;
+  }
+  return NGALORE_OK;
+}
+
+ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G, const std::vector<int>& idx,
+                            cudaStream_t stream) {
+  const int q = st->opt.power_iterations > 0 ? st->opt.power_iterations : 4;
+  // Random test matrix Omega (N x rp), one hashed stream per matrix and refresh.
+  for (int i : idx) {
+    const HostMat& hm = st->mats[i];
+    const long long cnt = static_cast<long long>(hm.N) * hm.rp;
+    fill_normal_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, stream>>>(
+        hm.Xa, cnt, st->opt.seed, static_cast<unsigned long long>(st->k) * 65536ull + static_cast<unsigned>(i));
+    st->launches += 1;
+  }
+  NG_CUDA(cudaGetLastError());
+  ngalore_status rc;
+  // Ya = G Omega; Yb = orth(Ya)
+  if ((rc = apply_gradient(st, idx, G, 0, BUF_XA, BUF_YA, stream))) return rc;
+  if ((rc = orthonormalise(st, idx, 0, true, stream))) return rc;
+  for (int it = 0; it < q; ++it) {
+    // Xa = G^T Yb; Xb = orth(Xa); Ya = G Xb; Yb = orth(Ya)
+    if ((rc = apply_gradient(st, idx, G, 1, BUF_YB, BUF_XA, stream))) return rc;
+    if ((rc = orthonormalise(st, idx, 1, true, stream))) return rc;
+    if ((rc = apply_gradient(st, idx, G, 0, BUF_XB, BUF_YA, stream))) return rc;
+    if ((rc = orthonormalise(st, idx, 0, true, stream))) return rc;
+  }
+  // Second pass Yb -> Ya so that a clamped pivot of the first pass cannot leave P non-orthonormal.
+  if ((rc = orthonormalise(st, idx, 0, false, stream))) return rc;
+  for (int i : idx) {
+    const HostMat& hm = st->mats[i];
+    NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, hm.Ya, sizeof(float) * hm.M * hm.rp, cudaMemcpyDeviceToDevice, stream));
+    if ((rc = make_working_copies(st, i, stream))) return rc;
+  }
+  if (st->opt.reset_history_on_refresh && idx.size() == static_cast<size_t>(st->n)) {
+    st->n_appended = 0;
+    NG_CUDA(cudaMemsetAsync(&st->d_ctrl->n_appended, 0, sizeof(long long), stream));
+  }
+  if (idx.size() == static_cast<size_t>(st->n)) st->has_subspace = true;
+  return NGALORE_OK;
+}
+
+ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream) {
+  ngalore_status rc;
+  if (st->T > 0 && st->k % st->T == 0) {
+    std::vector<int> all(st->n);
+    for (int i = 0; i < st->n; ++i) all[i] = i;
+    if ((rc = refresh_impl(st, G, all, stream))) return rc;
+  }
+  if (!st->has_subspace) return NGALORE_ERR_NO_SUBSPACE;
+  bool ptr_changed = false;
+  if ((rc = upload_pointers(st, W, G, stream, &ptr_changed))) return rc;
+  if ((rc = upload_hyper(st, stream))) return rc;
+  const int cur = st->s > 0 ? static_cast<int>(st->n_appended % st->s) : 0;
+
+  if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[0], stream));
+  // ---- phase 0: R = P^T G into ring slot `cur`
+  if (st->opt.gemm_impl == 1) {
+    for (int i = 0; i < st->n; ++i) {
+      const HostMat& hm = st->mats[i];
+      const MatDesc& d = st->h_desc[i];
+      SimtGemm g{};
+      g.m = hm.rp; g.n = hm.N; g.k = hm.M;
+      g.A = d.Pt16; g.a_rs = hm.M; g.a_cs = 1; g.a_dt = DT_BF16;
+      g.B = G[i]; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_BF16;
+      g.C = d.H + static_cast<long long>(cur) * hm.rn; g.c_rs = hm.N; g.c_cs = 1; g.c_dt = DT_F32;
+      g.epilogue = EPI_STORE;
+      NG_CUDA(launch_simt_gemm<float>(g, stream));
+      st->launches += 1;
+    }
+  } else {
+    if ((rc = tc_project(st->tc, st->d_desc, st->d_ctrl, G, ptr_changed, stream, &st->launches))) return rc;
+  }
+  if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[1], stream));
+  // ---- phase 1: Gram row, solve, natural gradient + moments
+  if (st->opt.stream_impl == 1) {
+    if (st->s <= 8) launch_plain_stream<8>(st, stream);
+    else if (st->s <= 16) launch_plain_stream<16>(st, stream);
+    else launch_plain_stream<32>(st, stream);
+  } else {
+    if ((rc = fused_stream_launch(st->fused, st->d_desc, st->n, st->d_ctrl, st->d_hyper, st->s, stream, &st->launches))) return rc;
+  }
+  NG_CUDA(cudaGetLastError());
+  if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[2], stream));
+  // ---- phase 2: W <- (1 - lr wd) W - lr P u
+  if (st->opt.gemm_impl == 1) {
+    for (int i = 0; i < st->n; ++i) {
+      const HostMat& hm = st->mats[i];
+      const MatDesc& d = st->h_desc[i];
+      SimtGemm g{};
+      g.m = hm.M; g.n = hm.N; g.k = hm.rp;
+      g.A = d.P16; g.a_rs = hm.rp; g.a_cs = 1; g.a_dt = DT_BF16;
+      g.B = d.u_hi; g.B2 = d.u_lo; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_BF16;
+      g.C = W[i]; g.c_rs = hm.N; g.c_cs = 1; g.c_dt = DT_F32;
+      g.epilogue = EPI_W_UPDATE;
+      g.hyper = st->d_hyper;
+      g.skip_flag = d.step_bad;
+      NG_CUDA(launch_simt_gemm<float>(g, stream));
+      st->launches += 1;
+    }
+  } else {
+    if ((rc = tc_backproject(st->tc, st->d_desc, st->d_ctrl, st->d_hyper, W, ptr_changed, stream, &st->launches))) return rc;
+  }
+  advance_kernel<<<1, 1, 0, stream>>>(st->d_ctrl);
+  st->launches += 1;
+  NG_CUDA(cudaGetLastError());
+  if (st->profiling) {
+    NG_CUDA(cudaEventRecord(st->ev[3], stream));
+    st->ev_valid = true;
+  }
+  st->k += 1;
+  st->n_appended += 1;
+  return NGALORE_OK;
+}
+
+}  // namespace
+
+// ======================================================================================= C ABI
+
+extern "C" {
+
+const char* ngalore_status_string(ngalore_status s) {
+  switch (s) {
+    case NGALORE_OK: return "ok";
+    case NGALORE_ERR_INVALID_ARG: return "invalid argument";
+    case NGALORE_ERR_ALLOC: return "device allocation failed";
+    case NGALORE_ERR_CUDA: return "CUDA runtime error";
+    case NGALORE_ERR_UNSUPPORTED_DEVICE: return "unsupported device (compute capability 10.x required)";
+    case NGALORE_ERR_NO_SUBSPACE: return "no subspace: refresh or set one first";
+    case NGALORE_ERR_NOT_SPD: return "Cholesky pivot not positive";
+    case NGALORE_ERR_NONFINITE: return "non-finite value in the Gram matrix";
+    case NGALORE_ERR_TIMEOUT: return "a bounded device wait ran out";
+  }
+  return "unknown status";
+}
+
+ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r, int s, int T, double lambda,
+                              double lr, double beta1, double beta2, double eps, double wd,
+                              const ngalore_options* opt, ngalore_state** out) {
+  if (out == nullptr) return NGALORE_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (shapes == nullptr || n_matrices <= 0 || r < 1 || s < 0 || s > kMaxHistory || T < 0) return NGALORE_ERR_INVALID_ARG;
+  if (s > 0 && !(lambda > 0.0)) return NGALORE_ERR_INVALID_ARG;
+  if (!(beta1 >= 0.0 && beta1 < 1.0 && beta2 >= 0.0 && beta2 < 1.0) || eps < 0.0) return NGALORE_ERR_INVALID_ARG;
+  for (int i = 0; i < n_matrices; ++i) {
+    if (shapes[i].rows < 1 || shapes[i].cols < 8 || shapes[i].cols % 8 != 0) return NGALORE_ERR_INVALID_ARG;
+    if (shapes[i].rows > (1 << 24) || shapes[i].cols > (1 << 24)) return NGALORE_ERR_INVALID_ARG;
+  }
+  if (opt != nullptr && opt->struct_size != static_cast<int32_t>(sizeof(ngalore_options))) return NGALORE_ERR_INVALID_ARG;
+
+  int dev = 0;
+  NG_CUDA(cudaGetDevice(&dev));
+  cudaDeviceProp prop{};
+  NG_CUDA(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return NGALORE_ERR_UNSUPPORTED_DEVICE;
+
+  ngalore_state* st = new (std::nothrow) ngalore_state();
+  if (st == nullptr) return NGALORE_ERR_ALLOC;
+  st->device = dev;
+  st->n = n_matrices; st->r = r; st->s = s; st->T = T;
+  st->hyper.lr = static_cast<float>(lr); st->hyper.wd = static_cast<float>(wd);
+  st->hyper.beta1 = static_cast<float>(beta1); st->hyper.beta2 = static_cast<float>(beta2);
+  st->hyper.eps = static_cast<float>(eps); st->hyper.lambda = lambda;
+  if (opt != nullptr) st->opt = *opt;
+  st->opt.struct_size = sizeof(ngalore_options);
+  if (st->opt.seed == 0) st->opt.seed = 0x9E3779B97F4A7C15ull;
+
+  // ---- streaming tile size: aim for at least ~8 tiles per SM overall, tiles of 2048..8192 elements
+  long long total_rn = 0;
+  st->mats.resize(n_matrices);
+  uint64_t hash = 1469598103934665603ull;
+  for (int i = 0; i < n_matrices; ++i) {
+    HostMat& hm = st->mats[i];
+    hm.M = static_cast<int>(shapes[i].rows); hm.N = static_cast<int>(shapes[i].cols);
+    hm.rp = r < hm.M ? r : hm.M;
+    if (hm.N < hm.rp) hm.rp = hm.N;
+    hm.rn = static_cast<long long>(hm.rp) * hm.N;
+    total_rn += hm.rn;
+    hash = (hash ^ static_cast<uint64_t>(hm.M)) * 1099511628211ull;
+    hash = (hash ^ static_cast<uint64_t>(hm.N)) * 1099511628211ull;
+  }
+  st->shape_hash = hash;
+  int te = 8192;
+  while (te > 2048 && total_rn / te < static_cast<long long>(prop.multiProcessorCount) * 8) te >>= 1;
+  st->tile_elems = te;
+
+  // ---- arena layout
+  const int slots = s > 0 ? s : 1;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  struct Offs { size_t H, m, v, P32, P16, Pt16, Kraw, wsol; };
+  std::vector<Offs> offs(n_matrices);
+  const size_t o_ctrl = take(sizeof(Ctrl));
+  const size_t o_status = take(sizeof(int) * n_matrices);
+  const size_t o_bad = take(sizeof(int) * n_matrices);
+  for (int i = 0; i < n_matrices; ++i) {
+    const HostMat& hm = st->mats[i];
+    offs[i].H = take(sizeof(float) * hm.rn * slots);
+    offs[i].m = take(sizeof(float) * hm.rn);
+    offs[i].v = take(sizeof(float) * hm.rn);
+    offs[i].P32 = take(sizeof(float) * hm.M * hm.rp);
+    offs[i].P16 = take(sizeof(__nv_bfloat16) * hm.M * hm.rp);
+    offs[i].Pt16 = take(sizeof(__nv_bfloat16) * hm.M * hm.rp);
+    offs[i].Kraw = take(sizeof(double) * slots * slots);
+    offs[i].wsol = take(sizeof(float) * kMaxHistory);
+  }
+  st->arena_bytes = off;
+
+  // ---- work layout
+  off = 0;
+  struct WOffs { size_t uhi, ulo, gpart, Ya, Yb, Xa, Xb, C; };
+  std::vector<WOffs> woffs(n_matrices);
+  const size_t o_hyper = take(sizeof(Hyper));
+  const size_t o_desc = take(sizeof(MatDesc) * n_matrices);
+  const size_t o_dW = take(sizeof(void*) * n_matrices);
+  const size_t o_dG = take(sizeof(void*) * n_matrices);
+  const size_t o_chol = take(sizeof(CholProblem) * n_matrices);
+  const size_t o_flags = take(sizeof(int) * 2 * n_matrices);
+  int n_tiles = 0;
+  std::vector<StreamTile> tiles;
+  std::vector<int> tile0(n_matrices), ntl(n_matrices);
+  for (int i = 0; i < n_matrices; ++i) {
+    const HostMat& hm = st->mats[i];
+    ntl[i] = static_cast<int>((hm.rn + te - 1) / te);
+    tile0[i] = n_tiles;
+    for (int t = 0; t < ntl[i]; ++t) tiles.push_back(StreamTile{i, t});
+    n_tiles += ntl[i];
+    woffs[i].uhi = take(sizeof(__nv_bfloat16) * hm.rn);
+    woffs[i].ulo = take(sizeof(__nv_bfloat16) * hm.rn);
+    woffs[i].gpart = take(sizeof(double) * ntl[i] * slots);
+    woffs[i].Ya = take(sizeof(float) * hm.M * hm.rp);
+    woffs[i].Yb = take(sizeof(float) * hm.M * hm.rp);
+    woffs[i].Xa = take(sizeof(float) * hm.N * hm.rp);
+    woffs[i].Xb = take(sizeof(float) * hm.N * hm.rp);
+    woffs[i].C = take(sizeof(double) * hm.rp * hm.rp);
+  }
+  st->n_tiles = n_tiles;
+  const size_t o_tiles = take(sizeof(StreamTile) * n_tiles);
+  st->work_bytes = off;
+
+  auto fail = [&](ngalore_status code) {
+    ngalore_destroy(st);
+    return code;
+  };
+  if (cudaMalloc(&st->arena, st->arena_bytes) != cudaSuccess) { st->arena = nullptr; return fail(NGALORE_ERR_ALLOC); }
+  if (cudaMalloc(&st->work, st->work_bytes) != cudaSuccess) { st->work = nullptr; return fail(NGALORE_ERR_ALLOC); }
+  if (cudaMemset(st->arena, 0, st->arena_bytes) != cudaSuccess) return fail(NGALORE_ERR_CUDA);
+  if (cudaMemset(st->work, 0, st->work_bytes) != cudaSuccess) return fail(NGALORE_ERR_CUDA);
+
+  st->d_ctrl = reinterpret_cast<Ctrl*>(st->arena + o_ctrl);
+  st->d_status = reinterpret_cast<int*>(st->arena + o_status);
+  st->d_step_bad = reinterpret_cast<int*>(st->arena + o_bad);
+  st->d_hyper = reinterpret_cast<Hyper*>(st->work + o_hyper);
+  st->d_desc = reinterpret_cast<MatDesc*>(st->work + o_desc);
+  st->d_W = reinterpret_cast<float**>(st->work + o_dW);
+  st->d_G = reinterpret_cast<const __nv_bfloat16**>(st->work + o_dG);
+  st->d_chol = reinterpret_cast<CholProblem*>(st->work + o_chol);
+  st->d_tiles = reinterpret_cast<StreamTile*>(st->work + o_tiles);
+  int* flags = reinterpret_cast<int*>(st->work + o_flags);
+
+  st->h_desc.resize(n_matrices);
+  std::vector<CholProblem> chol(n_matrices);
+  std::vector<float> w_init(kMaxHistory, 0.f);
+  w_init[0] = 1.f;
+  for (int i = 0; i < n_matrices; ++i) {
+    HostMat& hm = st->mats[i];
+    MatDesc& d = st->h_desc[i];
+    d.M = hm.M; d.N = hm.N; d.rp = hm.rp; d.s = s; d.rn = hm.rn;
+    d.H = reinterpret_cast<float*>(st->arena + offs[i].H);
+    d.m = reinterpret_cast<float*>(st->arena + offs[i].m);
+    d.v = reinterpret_cast<float*>(st->arena + offs[i].v);
+    d.P32 = reinterpret_cast<float*>(st->arena + offs[i].P32);
+    d.P16 = reinterpret_cast<__nv_bfloat16*>(st->arena + offs[i].P16);
+    d.Pt16 = reinterpret_cast<__nv_bfloat16*>(st->arena + offs[i].Pt16);
+    d.Kraw = reinterpret_cast<double*>(st->arena + offs[i].Kraw);
+    d.wsol = reinterpret_cast<float*>(st->arena + offs[i].wsol);
+    d.u_hi = reinterpret_cast<__nv_bfloat16*>(st->work + woffs[i].uhi);
+    d.u_lo = reinterpret_cast<__nv_bfloat16*>(st->work + woffs[i].ulo);
+    d.gpart = reinterpret_cast<double*>(st->work + woffs[i].gpart);
+    d.status = st->d_status + i;
+    d.step_bad = st->d_step_bad + i;
+    d.gram_done = flags + 2 * i;
+    d.w_ready = flags + 2 * i + 1;
+    d.tile0 = tile0[i]; d.ntiles = ntl[i];
+    hm.Ya = reinterpret_cast<float*>(st->work + woffs[i].Ya);
+    hm.Yb = reinterpret_cast<float*>(st->work + woffs[i].Yb);
+    hm.Xa = reinterpret_cast<float*>(st->work + woffs[i].Xa);
+    hm.Xb = reinterpret_cast<float*>(st->work + woffs[i].Xb);
+    hm.C = reinterpret_cast<double*>(st->work + woffs[i].C);
+    chol[i].C = hm.C; chol[i].L = hm.rp;
+    if (s == 0 && cudaMemcpy(d.wsol, w_init.data(), sizeof(float) * kMaxHistory, cudaMemcpyHostToDevice) != cudaSuccess)
+      return fail(NGALORE_ERR_CUDA);
+  }
+  if (cudaMemcpy(st->d_desc, st->h_desc.data(), sizeof(MatDesc) * n_matrices, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(st->d_chol, chol.data(), sizeof(CholProblem) * n_matrices, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(st->d_tiles, tiles.data(), sizeof(StreamTile) * n_tiles, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(st->d_hyper, &st->hyper, sizeof(Hyper), cudaMemcpyHostToDevice) != cudaSuccess)
+    return fail(NGALORE_ERR_CUDA);
+  st->hyper_dirty = false;
+  st->last_W.assign(n_matrices, nullptr);
+  st->last_G.assign(n_matrices, nullptr);
+
+  // kernels with large dynamic shared memory
+  int max_rp = 0;
+  for (const HostMat& hm : st->mats) max_rp = hm.rp > max_rp ? hm.rp : max_rp;
+  if (orth_apply_smem_bytes(max_rp) > static_cast<size_t>(prop.sharedMemPerBlockOptin)) return fail(NGALORE_ERR_INVALID_ARG);
+  if (cudaFuncSetAttribute(orth_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(orth_apply_smem_bytes(max_rp))) != cudaSuccess)
+    return fail(NGALORE_ERR_CUDA);
+
+  ngalore_status rc = tc_plan_create(st->tc, st->h_desc, st->d_desc, s, prop.multiProcessorCount);
+  if (rc != NGALORE_OK) return fail(rc);
+  rc = fused_plan_create(st->fused, st->h_desc, st->tile_elems, prop.multiProcessorCount);
+  if (rc != NGALORE_OK) return fail(rc);
+  for (int e = 0; e < 4; ++e)
+    if (cudaEventCreate(&st->ev[e]) != cudaSuccess) return fail(NGALORE_ERR_CUDA);
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(NGALORE_ERR_CUDA);
+  *out = st;
+  return NGALORE_OK;
+}
+
+void ngalore_destroy(ngalore_state* st) {
+  if (st == nullptr) return;
+  DeviceGuard guard(st->device);
+  cudaDeviceSynchronize();
+  tc_plan_destroy(st->tc);
+  fused_plan_destroy(st->fused);
+  for (int e = 0; e < 4; ++e)
+    if (st->ev[e]) cudaEventDestroy(st->ev[e]);
+  if (st->stage) cudaFree(st->stage);
+  if (st->work) cudaFree(st->work);
+  if (st->arena) cudaFree(st->arena);
+  delete st;
+}
+
+ngalore_status ngalore_step(ngalore_state* st, float* const* W, const uint16_t* const* G, void* stream) {
+  if (st == nullptr || W == nullptr || G == nullptr) return NGALORE_ERR_INVALID_ARG;
+  for (int i = 0; i < st->n; ++i) {
+    if (W[i] == nullptr || G[i] == nullptr) return NGALORE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(W[i]) | reinterpret_cast<uintptr_t>(G[i])) & 15u) return NGALORE_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
+  return step_impl(st, W, G, static_cast<cudaStream_t>(stream));
+}
+
+ngalore_status ngalore_refresh_subspace(ngalore_state* st, const uint16_t* const* G, int matrix_index, void* stream) {
+  if (st == nullptr || G == nullptr || matrix_index < -1 || matrix_index >= st->n) return NGALORE_ERR_INVALID_ARG;
+  std::vector<int> idx;
+  if (matrix_index < 0) {
+    for (int i = 0; i < st->n; ++i) idx.push_back(i);
+  } else {
+    idx.push_back(matrix_index);
+  }
+  for (int i : idx)
+    if (G[i] == nullptr || (reinterpret_cast<uintptr_t>(G[i]) & 15u)) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
+  return refresh_impl(st, G, idx, static_cast<cudaStream_t>(stream));
+}
+
+ngalore_status ngalore_step_host(ngalore_state* st, float* const* W_host, const uint16_t* const* G_host, void* stream) {
+  if (st == nullptr || W_host == nullptr || G_host == nullptr) return NGALORE_ERR_INVALID_ARG;
+  for (int i = 0; i < st->n; ++i)
+    if (W_host[i] == nullptr || G_host[i] == nullptr) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (st->stage == nullptr) {
+    size_t off = 0;
+    std::vector<size_t> ow(st->n), og(st->n);
+    for (int i = 0; i < st->n; ++i) {
+      const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+      ow[i] = off; off += align_up(mn * sizeof(float));
+      og[i] = off; off += align_up(mn * sizeof(uint16_t));
+    }
+    if (cudaMalloc(&st->stage, off) != cudaSuccess) { st->stage = nullptr; return NGALORE_ERR_ALLOC; }
+    st->stage_bytes = off;
+    st->stage_W.resize(st->n); st->stage_G.resize(st->n);
+    for (int i = 0; i < st->n; ++i) {
+      st->stage_W[i] = reinterpret_cast<float*>(st->stage + ow[i]);
+      st->stage_G[i] = reinterpret_cast<uint16_t*>(st->stage + og[i]);
+    }
+  }
+  for (int i = 0; i < st->n; ++i) {
+    const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+    NG_CUDA(cudaMemcpyAsync(st->stage_G[i], G_host[i], mn * sizeof(uint16_t), cudaMemcpyHostToDevice, s));
+    NG_CUDA(cudaMemcpyAsync(st->stage_W[i], W_host[i], mn * sizeof(float), cudaMemcpyHostToDevice, s));
+  }
+  ngalore_status rc = step_impl(st, st->stage_W.data(), st->stage_G.data(), s);
+  if (rc != NGALORE_OK) return rc;
+  for (int i = 0; i < st->n; ++i) {
+    const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+    NG_CUDA(cudaMemcpyAsync(W_host[i], st->stage_W[i], mn * sizeof(float), cudaMemcpyDeviceToHost, s));
+  }
+  NG_CUDA(cudaStreamSynchronize(s));
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_poll_status(ngalore_state* st, int* per_matrix) {
+  if (st == nullptr) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
+  NG_CUDA(cudaDeviceSynchronize());
+  std::vector<int> h(st->n);
+  NG_CUDA(cudaMemcpy(h.data(), st->d_status, sizeof(int) * st->n, cudaMemcpyDeviceToHost));
+  Ctrl c{};
+  NG_CUDA(cudaMemcpy(&c, st->d_ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost));
+  NG_CUDA(cudaMemset(st->d_status, 0, sizeof(int) * st->n));
+  if (c.timeout_flag != 0) NG_CUDA(cudaMemset(&st->d_ctrl->timeout_flag, 0, sizeof(int)));
+  ngalore_status first = NGALORE_OK;
+  for (int i = 0; i < st->n; ++i) {
+    if (per_matrix) per_matrix[i] = h[i];
+    if (first == NGALORE_OK && h[i] != 0) first = static_cast<ngalore_status>(h[i]);
+  }
+  if (first == NGALORE_OK && c.timeout_flag != 0) first = NGALORE_ERR_TIMEOUT;
+  return first;
+}
+
+ngalore_status ngalore_get_subspace(ngalore_state* st, int i, float* P, void* stream) {
+  if (st == nullptr || i < 0 || i >= st->n || P == nullptr) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  const HostMat& hm = st->mats[i];
+  NG_CUDA(cudaMemcpyAsync(P, st->h_desc[i].P32, sizeof(float) * hm.M * hm.rp, cudaMemcpyDeviceToDevice,
+                          static_cast<cudaStream_t>(stream)));
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, void* stream) {
+  if (st == nullptr || i < 0 || i >= st->n || P == nullptr) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  const HostMat& hm = st->mats[i];
+  const long long cnt = static_cast<long long>(hm.M) * hm.rp;
+  widen_bf16_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      st->h_desc[i].P16, P, cnt);
+  st->launches += 1;
+  NG_CUDA(cudaGetLastError());
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_set_subspace(ngalore_state* st, int i, const float* P, void* stream) {
+  if (st == nullptr || i < 0 || i >= st->n || P == nullptr) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  const HostMat& hm = st->mats[i];
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, P, sizeof(float) * hm.M * hm.rp, cudaMemcpyDeviceToDevice, s));
+  ngalore_status rc = make_working_copies(st, i, s);
+  if (rc != NGALORE_OK) return rc;
+  st->has_subspace = true;  // the caller is responsible for setting every matrix before stepping
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_state_export(ngalore_state* st, void* blob, size_t* bytes) {
+  if (st == nullptr || bytes == nullptr) return NGALORE_ERR_INVALID_ARG;
+  const size_t need = sizeof(BlobHeader) + st->arena_bytes;
+  if (blob == nullptr) { *bytes = need; return NGALORE_OK; }
+  if (*bytes < need) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  NG_CUDA(cudaDeviceSynchronize());
+  BlobHeader h{};
+  h.magic = kBlobMagic; h.arena_bytes = st->arena_bytes; h.k = st->k; h.n_appended = st->n_appended;
+  h.n = st->n; h.r = st->r; h.s = st->s; h.has_subspace = st->has_subspace ? 1 : 0; h.shape_hash = st->shape_hash;
+  std::memcpy(blob, &h, sizeof(h));
+  NG_CUDA(cudaMemcpy(static_cast<char*>(blob) + sizeof(h), st->arena, st->arena_bytes, cudaMemcpyDeviceToHost));
+  *bytes = need;
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_state_import(ngalore_state* st, const void* blob, size_t bytes) {
+  if (st == nullptr || blob == nullptr || bytes < sizeof(BlobHeader)) return NGALORE_ERR_INVALID_ARG;
+  BlobHeader h{};
+  std::memcpy(&h, blob, sizeof(h));
+  if (h.magic != kBlobMagic || h.arena_bytes != st->arena_bytes || h.n != st->n || h.r != st->r || h.s != st->s ||
+      h.shape_hash != st->shape_hash || bytes < sizeof(h) + h.arena_bytes)
+    return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  NG_CUDA(cudaDeviceSynchronize());
+  NG_CUDA(cudaMemcpy(st->arena, static_cast<const char*>(blob) + sizeof(h), st->arena_bytes, cudaMemcpyHostToDevice));
+  st->k = h.k; st->n_appended = h.n_appended; st->has_subspace = h.has_subspace != 0;
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_set_lr(ngalore_state* st, double lr) {
+  if (st == nullptr || !(lr == lr)) return NGALORE_ERR_INVALID_ARG;
+  st->hyper.lr = static_cast<float>(lr);
+  st->hyper_dirty = true;
+  return NGALORE_OK;
+}
+
+int ngalore_num_matrices(const ngalore_state* st) { return st ? st->n : 0; }
+int ngalore_rank(const ngalore_state* st, int i) { return (st && i >= 0 && i < st->n) ? st->mats[i].rp : -1; }
+int64_t ngalore_step_count(const ngalore_state* st) { return st ? st->k : -1; }
+size_t ngalore_device_bytes(const ngalore_state* st) { return st ? st->arena_bytes + st->work_bytes + st->stage_bytes + st->tc.device_bytes : 0; }
+int64_t ngalore_launch_count(const ngalore_state* st) { return st ? st->launches : 0; }
+
+ngalore_status ngalore_set_profiling(ngalore_state* st, int on) {
+  if (st == nullptr) return NGALORE_ERR_INVALID_ARG;
+  st->profiling = on != 0;
+  st->ev_valid = false;
+  return NGALORE_OK;
+}
+
+double ngalore_last_phase_ms(ngalore_state* st, int phase) {
+  if (st == nullptr || phase < 0 || phase > 2 || !st->profiling || !st->ev_valid) return -1.0;
+  DeviceGuard guard(st->device);
+  if (cudaEventSynchronize(st->ev[3]) != cudaSuccess) return -1.0;
+  float ms = 0.f;
+  if (cudaEventElapsedTime(&ms, st->ev[phase], st->ev[phase + 1]) != cudaSuccess) return -1.0;
+  return static_cast<double>(ms);
+}
+
+}  // extern "C"
