@@ -1,0 +1,217 @@
+"""Thin ctypes binding over the C-ABI library ``libngalore.so`` (see include/ngalore.h).
+
+Argument marshalling only: every step of the optimizer runs in the library's
+CUDA kernels.  torch is used for device memory and streams.  Importing this
+module fails loudly when the library has not been built; there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libngalore.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it first (python -c 'import __graft_entry__ as g; g.build()' "
+        "or python -m paper_2410_16029_b200.build). There is no CPU fallback.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK = 0
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "ALLOC", 3: "CUDA", 4: "UNSUPPORTED_DEVICE", 5: "NO_SUBSPACE",
+                6: "NOT_SPD", 7: "NONFINITE", 8: "TIMEOUT"}
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int64), ("cols", ctypes.c_int64)]
+
+
+class Options(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_int32), ("gemm_impl", ctypes.c_int32),
+                ("power_iterations", ctypes.c_int32), ("reset_history_on_refresh", ctypes.c_int32),
+                ("seed", ctypes.c_uint64), ("stream_impl", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+_vp = ctypes.c_void_p
+_lib.ngalore_create.restype = ctypes.c_int
+_lib.ngalore_create.argtypes = [ctypes.POINTER(Shape), ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                ctypes.c_double, ctypes.c_double, ctypes.POINTER(Options), ctypes.POINTER(_vp)]
+_lib.ngalore_destroy.restype = None
+_lib.ngalore_destroy.argtypes = [_vp]
+_lib.ngalore_step.restype = ctypes.c_int
+_lib.ngalore_step.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp]
+_lib.ngalore_refresh_subspace.restype = ctypes.c_int
+_lib.ngalore_refresh_subspace.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.c_int, _vp]
+_lib.ngalore_step_host.restype = ctypes.c_int
+_lib.ngalore_step_host.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp]
+_lib.ngalore_poll_status.restype = ctypes.c_int
+_lib.ngalore_poll_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_int)]
+for _name in ("ngalore_get_subspace", "ngalore_set_subspace", "ngalore_get_working_subspace"):
+    getattr(_lib, _name).restype = ctypes.c_int
+    getattr(_lib, _name).argtypes = [_vp, ctypes.c_int, _vp, _vp]
+_lib.ngalore_state_export.restype = ctypes.c_int
+_lib.ngalore_state_export.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_size_t)]
+_lib.ngalore_state_import.restype = ctypes.c_int
+_lib.ngalore_state_import.argtypes = [_vp, _vp, ctypes.c_size_t]
+_lib.ngalore_set_lr.restype = ctypes.c_int
+_lib.ngalore_set_lr.argtypes = [_vp, ctypes.c_double]
+_lib.ngalore_num_matrices.restype = ctypes.c_int
+_lib.ngalore_num_matrices.argtypes = [_vp]
+_lib.ngalore_rank.restype = ctypes.c_int
+_lib.ngalore_rank.argtypes = [_vp, ctypes.c_int]
+_lib.ngalore_step_count.restype = ctypes.c_int64
+_lib.ngalore_step_count.argtypes = [_vp]
+_lib.ngalore_device_bytes.restype = ctypes.c_size_t
+_lib.ngalore_device_bytes.argtypes = [_vp]
+_lib.ngalore_launch_count.restype = ctypes.c_int64
+_lib.ngalore_launch_count.argtypes = [_vp]
+_lib.ngalore_set_profiling.restype = ctypes.c_int
+_lib.ngalore_set_profiling.argtypes = [_vp, ctypes.c_int]
+_lib.ngalore_last_phase_ms.restype = ctypes.c_double
+_lib.ngalore_last_phase_ms.argtypes = [_vp, ctypes.c_int]
+_lib.ngalore_status_string.restype = ctypes.c_char_p
+_lib.ngalore_status_string.argtypes = [ctypes.c_int]
+
+
+class NGaLoreError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)} ({_lib.ngalore_status_string(code).decode()})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise NGaLoreError(code, where)
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _ptr_array(tensors: Sequence[torch.Tensor]):
+    arr = (_vp * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = t.data_ptr()
+    return arr
+
+
+class NGaLore:
+    """Optimizer state for a list of (rows, cols) weight matrices on the current CUDA device."""
+
+    def __init__(self, shapes, r, s, T, lam=1e-3, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, wd=0.0, *,
+                 gemm_impl=0, stream_impl=0, power_iterations=0, reset_history_on_refresh=False, seed=0):
+        self.shapes = [(int(M), int(N)) for M, N in shapes]
+        arr = (Shape * len(self.shapes))(*[Shape(M, N) for M, N in self.shapes])
+        opt = Options(ctypes.sizeof(Options), gemm_impl, power_iterations, int(reset_history_on_refresh), seed,
+                      stream_impl, 0)
+        handle = _vp()
+        _check(_lib.ngalore_create(arr, len(self.shapes), r, s, T, lam, lr, beta1, beta2, eps, wd,
+                                   ctypes.byref(opt), ctypes.byref(handle)), "ngalore_create")
+        self._h = handle
+        self.device = torch.device("cuda", torch.cuda.current_device())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            _lib.ngalore_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- checks ---------------------------------------------------------------
+    def _check_WG(self, W, G):
+        assert len(W) == len(self.shapes) and len(G) == len(self.shapes)
+        for (M, N), w, g in zip(self.shapes, W, G):
+            assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous() and tuple(w.shape) == (M, N)
+            assert g.is_cuda and g.dtype == torch.bfloat16 and g.is_contiguous() and tuple(g.shape) == (M, N)
+
+    # -- the three calls of the optimizer -------------------------------------------
+    def step(self, W: List[torch.Tensor], G: List[torch.Tensor], stream=None, check=True):
+        if check:
+            self._check_WG(W, G)
+        _check(_lib.ngalore_step(self._h, _ptr_array(W), _ptr_array(G), _stream_ptr(stream)), "ngalore_step")
+
+    def step_ptrs(self, W_ptrs, G_ptrs, stream=None):
+        """Step with pre-built pointer arrays (see ``pointer_array``): no per-call marshalling."""
+        _check(_lib.ngalore_step(self._h, W_ptrs, G_ptrs, _stream_ptr(stream)), "ngalore_step")
+
+    @staticmethod
+    def pointer_array(tensors):
+        return _ptr_array(tensors)
+
+    def refresh_subspace(self, G: List[torch.Tensor], matrix_index=-1, stream=None):
+        assert len(G) == len(self.shapes)
+        _check(_lib.ngalore_refresh_subspace(self._h, _ptr_array(G), matrix_index, _stream_ptr(stream)),
+               "ngalore_refresh_subspace")
+
+    def step_host(self, W_host: List[torch.Tensor], G_host: List[torch.Tensor], stream=None):
+        """Step with host tensors (fp32 W updated in place, bf16 G); copies run inside the call."""
+        for w, g in zip(W_host, G_host):
+            assert not w.is_cuda and not g.is_cuda and w.is_contiguous() and g.is_contiguous()
+        _check(_lib.ngalore_step_host(self._h, _ptr_array(W_host), _ptr_array(G_host), _stream_ptr(stream)),
+               "ngalore_step_host")
+
+    # -- state access -----------------------------------------------------------
+    def poll_status(self):
+        arr = (ctypes.c_int * len(self.shapes))()
+        code = _lib.ngalore_poll_status(self._h, arr)
+        return code, list(arr)
+
+    def rank(self, i):
+        return _lib.ngalore_rank(self._h, i)
+
+    def get_subspace(self, i, working=False) -> torch.Tensor:
+        M, _ = self.shapes[i]
+        out = torch.empty((M, self.rank(i)), dtype=torch.float32, device=self.device)
+        fn = _lib.ngalore_get_working_subspace if working else _lib.ngalore_get_subspace
+        _check(fn(self._h, i, out.data_ptr(), _stream_ptr(None)), "ngalore_get_subspace")
+        return out
+
+    def set_subspace(self, i, P: torch.Tensor):
+        M, _ = self.shapes[i]
+        P = P.to(device=self.device, dtype=torch.float32).contiguous()
+        assert tuple(P.shape) == (M, self.rank(i))
+        _check(_lib.ngalore_set_subspace(self._h, i, P.data_ptr(), _stream_ptr(None)), "ngalore_set_subspace")
+        torch.cuda.current_stream().synchronize()  # P may be freed by the caller
+
+    def export_state(self) -> bytes:
+        n = ctypes.c_size_t(0)
+        _check(_lib.ngalore_state_export(self._h, None, ctypes.byref(n)), "ngalore_state_export")
+        buf = ctypes.create_string_buffer(n.value)
+        _check(_lib.ngalore_state_export(self._h, buf, ctypes.byref(n)), "ngalore_state_export")
+        return buf.raw[: n.value]
+
+    def import_state(self, blob: bytes):
+        _check(_lib.ngalore_state_import(self._h, blob, len(blob)), "ngalore_state_import")
+
+    def set_lr(self, lr: float):
+        _check(_lib.ngalore_set_lr(self._h, lr), "ngalore_set_lr")
+
+    @property
+    def step_count(self) -> int:
+        return _lib.ngalore_step_count(self._h)
+
+    @property
+    def device_bytes(self) -> int:
+        return _lib.ngalore_device_bytes(self._h)
+
+    @property
+    def launch_count(self) -> int:
+        return _lib.ngalore_launch_count(self._h)
+
+    def set_profiling(self, on: bool):
+        _check(_lib.ngalore_set_profiling(self._h, int(on)), "ngalore_set_profiling")
+
+    def last_phase_ms(self, phase: int) -> float:
+        return _lib.ngalore_last_phase_ms(self._h, phase)
