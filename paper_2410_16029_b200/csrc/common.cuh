@@ -14,13 +14,14 @@ constexpr int kStreamThreads = 256;   // threads per CTA of the streaming kernel
 struct MatDesc {
   int M, N, rp, s;            // rows, cols, r' = min(r, M, N), history length
   long long rn;               // rp * N, elements of one low-rank matrix
+  int ldp, ldpt;              // leading dimensions of P16 (>= rp) and Pt16 (>= M), multiples of 8 for TMA
   float* H;                   // history ring: s slots of rp x N fp32 (one slot when s == 0)
   float* m;                   // first moment, rp x N
   float* v;                   // second moment, rp x N
   __nv_bfloat16* u_hi;        // direction u = m / sqrt(v + eps), high bf16 part, rp x N
   __nv_bfloat16* u_lo;        // low part: bf16(u - hi)
-  __nv_bfloat16* P16;         // working copy of P, M x rp row-major
-  __nv_bfloat16* Pt16;        // working copy of P^T, rp x M row-major
+  __nv_bfloat16* P16;         // working copy of P, M x ldp row-major (padding is zero)
+  __nv_bfloat16* Pt16;        // working copy of P^T, rp x ldpt row-major
   float* P32;                 // fp32 master of P, M x rp row-major
   double* Kraw;               // s x s raw inner products <H_i, H_j>
   float* wsol;                // kMaxHistory solution weights of (lambda I + K) w = e_cur

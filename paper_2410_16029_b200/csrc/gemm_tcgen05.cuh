@@ -1,12 +1,535 @@
-// Tensor-core (tcgen05 / TMEM / TMA) grouped GEMMs of the step -- placeholder plan while the SIMT path is brought up.
+// Grouped tensor-core GEMMs of the step for sm_100a: tcgen05.mma with the accumulator in TMEM,
+// operands staged in shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), one persistent
+// warp-specialised CTA per SM.
+//
+//   projection       R = P^T G          A = Pt16 (r' x M, K-major), B = G (M x N, N contiguous)
+//                    epilogue: store (or atomically add, when K is split) into ring slot `cur`   (Sec. 1)
+//   back-projection  W <- (1 - lr wd) W - lr P u     A = P16 (M x r'), B = u_hi and u_lo (r' x N)
+//                    epilogue: fused read-modify-write of W                                      (Sec. 2.2)
+//
+// Warp roles (192 threads): warp 0 issues TMA loads, warp 1 allocates TMEM and issues the MMAs,
+// warps 2..5 drain the accumulator (tcgen05.ld), transpose through shared memory and write
+// coalesced rows.  Two accumulator buffers let the epilogue of one tile overlap the MMAs of the next.
+// Every mbarrier wait is bounded: when it runs out the CTA raises Ctrl::timeout_flag, stops issuing
+// work, and still releases its TMEM.
 #pragma once
+
+#include <cuda.h>
+
+#include <algorithm>
 #include <vector>
+
 #include "../../include/ngalore.h"
 #include "common.cuh"
+
 namespace ngalore {
-struct TcPlan { size_t device_bytes = 0; };
-inline ngalore_status tc_plan_create(TcPlan&, const std::vector<MatDesc>&, const MatDesc*, int, int) { return NGALORE_OK; }
-inline void tc_plan_destroy(TcPlan&) {}
-inline ngalore_status tc_project(TcPlan&, const MatDesc*, Ctrl*, const uint16_t* const*, bool, cudaStream_t, int64_t*) { return NGALORE_ERR_INVALID_ARG; }
-inline ngalore_status tc_backproject(TcPlan&, const MatDesc*, Ctrl*, const Hyper*, float* const*, bool, cudaStream_t, int64_t*) { return NGALORE_ERR_INVALID_ARG; }
+
+constexpr int kTcBM = 128;        // rows of one accumulator tile (TMEM lanes)
+constexpr int kTcBK = 64;         // K elements per pipeline stage (one 128-byte swizzle row of bf16)
+constexpr int kTcThreads = 192;
+constexpr unsigned long long kTcWaitLimitNs = 2000000000ull;  // a wait on an mbarrier is abandoned after 2 s
+
+struct TcTile {
+  int mat;
+  int m0, n0;      // tile origin in the output
+  int k0;          // first K element
+  int kblocks;     // number of 64-wide K blocks
+  int atomic;      // 1: K is split, accumulate into the output with atomics
+};
+
+// ------------------------------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after kTcWaitLimitNs of wall time (or when another warp already gave up)
+// and returns false.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const uint32_t addr = smem_u32(bar);
+  unsigned long long t0 = 0;
+  for (unsigned it = 0;; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if ((it & 63u) == 63u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kTcWaitLimitNs) break;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (64-bit): start address, leading/stride byte offsets (>>4), descriptor
+// version 1 (bits 46-47), 128-byte swizzle (value 2 in bits 61-63).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  d |= 2ull << 61;
+  return d;
+}
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A (K-major) and B (MN-major), M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(kTcBM >> 4) << 24);
+}
+
+template <int BN, int NB, int STAGES>
+struct TcSmem {
+  static constexpr int kABytes = kTcBM * kTcBK * 2;           // 16 KB
+  static constexpr int kBChunkBytes = 64 * kTcBK * 2;         // one 64-column chunk: 64 K rows x 128 B
+  static constexpr int kBBytes = (BN / 64) * kBChunkBytes;    // per B operand
+  static constexpr int kStageBytes = kABytes + NB * kBBytes;
+  static constexpr int kEpiWarpBytes = 32 * 36 * 4;           // 32 rows x (32 + 4 pad) floats
+  static constexpr int kBarOffset = STAGES * kStageBytes + 4 * kEpiWarpBytes;
+  static constexpr int kTotal = kBarOffset + 256 + 1024;      // barriers + slack for 1024-byte alignment
+};
+
+enum { TC_EPI_PROJECT = 0, TC_EPI_WUPDATE = 1 };
+
+template <int BN, int NB, int STAGES, int EPI>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__ tiles, int n_tiles,
+               const MatDesc* __restrict__ mats, Ctrl* ctrl, const Hyper* __restrict__ hyper,
+               float* const* __restrict__ Wptrs) {
+  using L = TcSmem<BN, NB, STAGES>;
+  extern __shared__ unsigned char tc_smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
+  uint64_t* full_bar = bars;                   // [STAGES]
+  uint64_t* empty_bar = bars + STAGES;         // [STAGES]
+  uint64_t* tfull_bar = bars + 2 * STAGES;     // [2]
+  uint64_t* tempty_bar = bars + 2 * STAGES + 2;  // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+        const TcTile tile = tiles[t];
+        const MatDesc& d = mats[tile.mat];
+        const CUtensorMap* mapA = tmaps + tile.mat * 5 + (EPI == TC_EPI_PROJECT ? 0 : 2);
+        const CUtensorMap* mapB0 = tmaps + tile.mat * 5 + (EPI == TC_EPI_PROJECT ? 1 : 3);
+        const int n_rem = d.N - tile.n0;
+        const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
+        const int nchunks = (n_eff + 63) >> 6;
+        const uint32_t bytes = L::kABytes + NB * nchunks * L::kBChunkBytes;
+        for (int kb = 0; kb < tile.kblocks; ++kb) {
+          if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          unsigned char* sA = smem + stage * L::kStageBytes;
+          mbar_expect_tx(full_bar + stage, bytes);
+          const int k = tile.k0 + kb * kTcBK;
+          tma_load_2d(sA, mapA, k, tile.m0, full_bar + stage);
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb) {
+            unsigned char* sB = sA + L::kABytes + nb * L::kBBytes;
+            for (int c = 0; c < nchunks; ++c)
+              tma_load_2d(sB + c * L::kBChunkBytes, mapB0 + nb, tile.n0 + c * 64, k, full_bar + stage);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
+        const TcTile tile = tiles[t];
+        const MatDesc& d = mats[tile.mat];
+        const int n_rem = d.N - tile.n0;
+        const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
+        const uint32_t idesc = instr_desc(n_eff);
+        const int buf = local & 1;
+        const uint32_t tphase = (local >> 1) & 1u;
+        if (!mbar_wait(tempty_bar + buf, tphase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + buf * BN;
+        for (int kb = 0; kb < tile.kblocks; ++kb) {
+          if (!mbar_wait(full_bar + stage, phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t aaddr = smem_u32(smem + stage * L::kStageBytes);
+#pragma unroll
+          for (int nb = 0; nb < NB; ++nb) {
+            const uint32_t baddr = aaddr + L::kABytes + nb * L::kBBytes;
+#pragma unroll
+            for (int kk = 0; kk < kTcBK / 16; ++kk) {
+              const uint64_t adesc = smem_desc(aaddr + kk * 32, 16, 1024);
+              const uint64_t bdesc = smem_desc(baddr + kk * 2048, L::kBChunkBytes, 1024);
+              tc_mma_bf16(tmem_d, adesc, bdesc, idesc, (kb > 0 || nb > 0 || kk > 0) ? 1u : 0u);
+            }
+          }
+          tc_commit(empty_bar + stage);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit(tfull_bar + buf);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;  // TMEM lanes 32 * quarter .. + 31 belong to this warp
+    float* stg = reinterpret_cast<float*>(smem + STAGES * L::kStageBytes + (warp - 2) * L::kEpiWarpBytes);
+    float lr = 0.f, decay = 1.f;
+    if (EPI == TC_EPI_WUPDATE) { lr = hyper->lr; decay = 1.f - hyper->lr * hyper->wd; }
+    int local = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
+      const TcTile tile = tiles[t];
+      const MatDesc& d = mats[tile.mat];
+      const int n_rem = d.N - tile.n0;
+      const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
+      const int buf = local & 1;
+      const uint32_t tphase = (local >> 1) & 1u;
+      float* out;
+      int rows_total;
+      bool skip = false;
+      if (EPI == TC_EPI_PROJECT) {
+        out = d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn;
+        rows_total = d.rp;
+      } else {
+        out = Wptrs[tile.mat];
+        rows_total = d.M;
+        skip = __ldcg(d.step_bad) != 0;
+      }
+      if (!mbar_wait(tfull_bar + buf, tphase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row_base = tile.m0 + quarter * 32;
+      for (int c0 = 0; c0 < n_eff; c0 += 32) {
+        uint32_t r[32];
+        tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * BN + c0), r);
+        tc_wait_ld();
+        if (c0 + 32 >= n_eff) {
+          // all TMEM reads of this tile are done: hand the buffer back before the global traffic
+          tc_fence_before();
+          if (lane == 0) mbar_arrive(tempty_bar + buf);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          *reinterpret_cast<float4*>(stg + lane * 36 + j * 4) =
+              make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                          __uint_as_float(r[4 * j + 3]));
+        __syncwarp();
+        const int col = tile.n0 + c0 + (lane & 7) * 4;
+        if (!skip && col < d.N) {
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int rr = it * 4 + (lane >> 3);
+            const int row = row_base + rr;
+            if (row < rows_total) {
+              const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + (lane & 7) * 4);
+              float* p = out + static_cast<long long>(row) * d.N + col;
+              if (EPI == TC_EPI_PROJECT) {
+                if (tile.atomic) {
+                  atomicAdd(reinterpret_cast<float4*>(p), acc);
+                } else {
+                  *reinterpret_cast<float4*>(p) = acc;
+                }
+              } else {
+                float4 w = *reinterpret_cast<const float4*>(p);
+                w.x = decay * w.x - lr * acc.x;
+                w.y = decay * w.y - lr * acc.y;
+                w.z = decay * w.z - lr * acc.z;
+                w.w = decay * w.w - lr * acc.w;
+                *reinterpret_cast<float4*>(p) = w;
+              }
+            }
+          }
+        }
+        __syncwarp();
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // a wait ran out: give bulk copies that may still be in flight time to land before the CTA retires
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    if (threadIdx.x == 0) atomicExch(&ctrl->timeout_flag, 1);
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// Zero the ring slot the projection is about to accumulate into, for the matrices whose K is split.
+__global__ void zero_split_slots_kernel(const MatDesc* mats, const int* split_mats, const Ctrl* ctrl) {
+  const MatDesc& d = mats[split_mats[blockIdx.y]];
+  float4* p = reinterpret_cast<float4*>(d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn);
+  const long long n4 = d.rn / 4;
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n4;
+       i += static_cast<long long>(gridDim.x) * blockDim.x)
+    p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// ------------------------------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr int kProjBN = 256, kProjStages = 4;
+constexpr int kBackBN = 128, kBackStages = 4;
+
+struct TcPlan {
+  size_t device_bytes = 0;
+  EncodeTiledFn encode = nullptr;
+  int n_mats = 0;
+  std::vector<CUtensorMap> h_maps;  // 5 per matrix: A_proj, B_proj (G), A_back, B_hi, B_lo
+  std::vector<int> rowsN;           // per matrix: M, N for re-encoding G maps
+  std::vector<int> colsN;
+  std::vector<const void*> last_G;
+  CUtensorMap* d_maps = nullptr;
+  TcTile* d_tiles_proj = nullptr;
+  TcTile* d_tiles_back = nullptr;
+  int n_tiles_proj = 0, n_tiles_back = 0;
+  int grid_proj = 0, grid_back = 0;
+  int* d_split_mats = nullptr;
+  int n_split = 0;
+  bool maps_dirty = true;
+};
+
+inline bool tc_encode_2d(EncodeTiledFn fn, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer,
+                         uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {row_stride_bytes};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline void tc_plan_destroy(TcPlan& plan) {
+  if (plan.d_maps) cudaFree(plan.d_maps);
+  if (plan.d_tiles_proj) cudaFree(plan.d_tiles_proj);
+  if (plan.d_tiles_back) cudaFree(plan.d_tiles_back);
+  if (plan.d_split_mats) cudaFree(plan.d_split_mats);
+  plan.d_maps = nullptr; plan.d_tiles_proj = nullptr; plan.d_tiles_back = nullptr; plan.d_split_mats = nullptr;
+}
+
+inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& mats, const MatDesc* /*d_mats*/, int /*s*/,
+                                     int sm_count) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr)
+    return NGALORE_ERR_CUDA;
+  plan.encode = reinterpret_cast<EncodeTiledFn>(fn);
+  const int n = static_cast<int>(mats.size());
+  plan.n_mats = n;
+  plan.h_maps.resize(static_cast<size_t>(n) * 5);
+  plan.last_G.assign(n, nullptr);
+  std::memset(plan.h_maps.data(), 0, sizeof(CUtensorMap) * plan.h_maps.size());
+  for (int i = 0; i < n; ++i) {
+    const MatDesc& d = mats[i];
+    // A_proj: Pt16, r' rows x M (K) columns, row stride ldpt
+    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 0], d.Pt16, d.M, d.rp, static_cast<uint64_t>(d.ldpt) * 2, kTcBK, kTcBM))
+      return NGALORE_ERR_CUDA;
+    // A_back: P16, M rows x r' (K) columns, row stride ldp
+    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 2], d.P16, d.rp, d.M, static_cast<uint64_t>(d.ldp) * 2, kTcBK, kTcBM))
+      return NGALORE_ERR_CUDA;
+    // B_hi / B_lo: r' (K) rows x N columns
+    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 3], d.u_hi, d.N, d.rp, static_cast<uint64_t>(d.N) * 2, 64, kTcBK))
+      return NGALORE_ERR_CUDA;
+    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 4], d.u_lo, d.N, d.rp, static_cast<uint64_t>(d.N) * 2, 64, kTcBK))
+      return NGALORE_ERR_CUDA;
+  }
+
+  // ---- projection tiles: output r' x N, K = M; split K so that no tile dominates the schedule
+  std::vector<TcTile> proj, back;
+  long long total_kb = 0;
+  for (int i = 0; i < n; ++i) {
+    const MatDesc& d = mats[i];
+    const long long tiles_i = static_cast<long long>((d.rp + kTcBM - 1) / kTcBM) * ((d.N + kProjBN - 1) / kProjBN);
+    total_kb += tiles_i * ((d.M + kTcBK - 1) / kTcBK);
+  }
+  const long long per_cta = (total_kb + sm_count - 1) / sm_count;
+  long long target_kb = per_cta / 4;
+  if (target_kb < 16) target_kb = 16;
+  std::vector<int> split_mats;
+  for (int i = 0; i < n; ++i) {
+    const MatDesc& d = mats[i];
+    const int kb_total = (d.M + kTcBK - 1) / kTcBK;
+    int splits = static_cast<int>((kb_total + target_kb - 1) / target_kb);
+    if (splits < 1) splits = 1;
+    const int kb_per = (kb_total + splits - 1) / splits;
+    splits = (kb_total + kb_per - 1) / kb_per;
+    if (splits > 1) split_mats.push_back(i);
+    for (int n0 = 0; n0 < d.N; n0 += kProjBN)
+      for (int sp = 0; sp < splits; ++sp)
+        for (int m0 = 0; m0 < d.rp; m0 += kTcBM) {
+          const int kb0 = sp * kb_per;
+          const int kbn = std::min(kb_per, kb_total - kb0);
+          proj.push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0});
+        }
+  }
+  std::stable_sort(proj.begin(), proj.end(), [](const TcTile& a, const TcTile& b) { return a.kblocks > b.kblocks; });
+  for (int i = 0; i < n; ++i) {
+    const MatDesc& d = mats[i];
+    const int kbn = (d.rp + kTcBK - 1) / kTcBK;
+    for (int m0 = 0; m0 < d.M; m0 += kTcBM)
+      for (int n0 = 0; n0 < d.N; n0 += kBackBN) back.push_back(TcTile{i, m0, n0, 0, kbn, 0});
+  }
+  plan.n_tiles_proj = static_cast<int>(proj.size());
+  plan.n_tiles_back = static_cast<int>(back.size());
+  plan.grid_proj = std::min(plan.n_tiles_proj, sm_count);
+  plan.grid_back = std::min(plan.n_tiles_back, sm_count);
+  plan.n_split = static_cast<int>(split_mats.size());
+
+  const size_t maps_bytes = sizeof(CUtensorMap) * plan.h_maps.size();
+  if (cudaMalloc(&plan.d_maps, maps_bytes) != cudaSuccess) { plan.d_maps = nullptr; return NGALORE_ERR_ALLOC; }
+  if (cudaMalloc(&plan.d_tiles_proj, sizeof(TcTile) * proj.size()) != cudaSuccess) { plan.d_tiles_proj = nullptr; return NGALORE_ERR_ALLOC; }
+  if (cudaMalloc(&plan.d_tiles_back, sizeof(TcTile) * back.size()) != cudaSuccess) { plan.d_tiles_back = nullptr; return NGALORE_ERR_ALLOC; }
+  if (cudaMalloc(&plan.d_split_mats, sizeof(int) * (split_mats.size() + 1)) != cudaSuccess) { plan.d_split_mats = nullptr; return NGALORE_ERR_ALLOC; }
+  plan.device_bytes = maps_bytes + sizeof(TcTile) * (proj.size() + back.size()) + sizeof(int) * (split_mats.size() + 1);
+  if (cudaMemcpy(plan.d_tiles_proj, proj.data(), sizeof(TcTile) * proj.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_tiles_back, back.data(), sizeof(TcTile) * back.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  if (!split_mats.empty() &&
+      cudaMemcpy(plan.d_split_mats, split_mats.data(), sizeof(int) * split_mats.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  plan.rowsN.resize(n); plan.colsN.resize(n);
+  for (int i = 0; i < n; ++i) { plan.rowsN[i] = mats[i].M; plan.colsN[i] = mats[i].N; }
+
+  using LP = TcSmem<kProjBN, 1, kProjStages>;
+  using LB = TcSmem<kBackBN, 2, kBackStages>;
+  if (cudaFuncSetAttribute(tc_gemm_kernel<kProjBN, 1, kProjStages, TC_EPI_PROJECT>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_gemm_kernel<kBackBN, 2, kBackStages, TC_EPI_WUPDATE>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, LB::kTotal) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  plan.maps_dirty = true;
+  return NGALORE_OK;
+}
+
+// R = P^T G for every matrix, into ring slot `cur` (read on the device from Ctrl).
+inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const uint16_t* const* G,
+                                 cudaStream_t stream, int64_t* launches) {
+  bool changed = plan.maps_dirty;
+  for (int i = 0; i < plan.n_mats; ++i) {
+    if (plan.last_G[i] != G[i]) {
+      plan.last_G[i] = G[i];
+      if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 1], G[i], plan.colsN[i], plan.rowsN[i],
+                        static_cast<uint64_t>(plan.colsN[i]) * 2, 64, kTcBK))
+        return NGALORE_ERR_CUDA;
+      changed = true;
+    }
+  }
+  if (changed) {
+    if (cudaMemcpyAsync(plan.d_maps, plan.h_maps.data(), sizeof(CUtensorMap) * plan.h_maps.size(),
+                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return NGALORE_ERR_CUDA;
+    plan.maps_dirty = false;
+  }
+  if (plan.n_split > 0) {
+    zero_split_slots_kernel<<<dim3(64, plan.n_split), 256, 0, stream>>>(d_mats, plan.d_split_mats, d_ctrl);
+    *launches += 1;
+  }
+  using LP = TcSmem<kProjBN, 1, kProjStages>;
+  tc_gemm_kernel<kProjBN, 1, kProjStages, TC_EPI_PROJECT><<<plan.grid_proj, kTcThreads, LP::kTotal, stream>>>(
+      plan.d_maps, plan.d_tiles_proj, plan.n_tiles_proj, d_mats, d_ctrl, nullptr, nullptr);
+  *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
+}
+
+// W <- (1 - lr wd) W - lr P (u_hi + u_lo) for every matrix; d_W is the device array of W pointers.
+inline ngalore_status tc_backproject(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const Hyper* d_hyper,
+                                     float* const* d_W, cudaStream_t stream, int64_t* launches) {
+  if (plan.maps_dirty) {
+    if (cudaMemcpyAsync(plan.d_maps, plan.h_maps.data(), sizeof(CUtensorMap) * plan.h_maps.size(),
+                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return NGALORE_ERR_CUDA;
+    plan.maps_dirty = false;
+  }
+  using LB = TcSmem<kBackBN, 2, kBackStages>;
+  tc_gemm_kernel<kBackBN, 2, kBackStages, TC_EPI_WUPDATE><<<plan.grid_back, kTcThreads, LB::kTotal, stream>>>(
+      plan.d_maps, plan.d_tiles_back, plan.n_tiles_back, d_mats, d_ctrl, d_hyper, d_W);
+  *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
+}
+
 }  // namespace ngalore

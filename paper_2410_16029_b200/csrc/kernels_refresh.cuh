@@ -219,8 +219,10 @@ __global__ void __launch_bounds__(256) orth_apply_kernel(OrthApply p) {
 
 // ---------------------------------------------------------------- working copies of P
 
-// P16 = bf16(P32) (M x rp) and Pt16 = its transpose (rp x M).  Block (32, 8).
-__global__ void working_copies_kernel(const float* P32, __nv_bfloat16* P16, __nv_bfloat16* Pt16, int M, int rp) {
+// P16 = bf16(P32) (M x rp, leading dimension ldp) and Pt16 = its transpose (rp x M, leading dimension ldpt).
+// Block (32, 8).
+__global__ void working_copies_kernel(const float* P32, __nv_bfloat16* P16, __nv_bfloat16* Pt16, int M, int rp,
+                                      int ldp, int ldpt) {
   __shared__ float tile[32][33];
   const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
   for (int a = threadIdx.y; a < 32; a += blockDim.y) {
@@ -228,20 +230,21 @@ __global__ void working_copies_kernel(const float* P32, __nv_bfloat16* P16, __nv
     float val = 0.f;
     if (i < M && j < rp) {
       val = P32[static_cast<long long>(i) * rp + j];
-      P16[static_cast<long long>(i) * rp + j] = __float2bfloat16_rn(val);
+      P16[static_cast<long long>(i) * ldp + j] = __float2bfloat16_rn(val);
     }
     tile[a][threadIdx.x] = val;
   }
   __syncthreads();
   for (int a = threadIdx.y; a < 32; a += blockDim.y) {
     const int j = j0 + a, i = i0 + threadIdx.x;
-    if (i < M && j < rp) Pt16[static_cast<long long>(j) * M + i] = __float2bfloat16_rn(tile[threadIdx.x][a]);
+    if (i < M && j < rp) Pt16[static_cast<long long>(j) * ldpt + i] = __float2bfloat16_rn(tile[threadIdx.x][a]);
   }
 }
 
-__global__ void widen_bf16_kernel(const __nv_bfloat16* src, float* dst, long long n) {
+// dst (rows x cols, dense fp32) = src (rows x cols, leading dimension ld, bf16)
+__global__ void widen_bf16_kernel(const __nv_bfloat16* src, float* dst, long long n, int cols, int ld) {
   const long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  if (i < n) dst[i] = __bfloat162float(src[i]);
+  if (i < n) dst[i] = __bfloat162float(src[(i / cols) * ld + (i % cols)]);
 }
 
 }  // namespace ngalore

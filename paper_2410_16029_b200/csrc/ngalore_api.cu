@@ -146,7 +146,7 @@ ngalore_status make_working_copies(ngalore_state* st, int i, cudaStream_t stream
   const HostMat& hm = st->mats[i];
   const MatDesc& d = st->h_desc[i];
   dim3 grid((hm.rp + 31) / 32, (hm.M + 31) / 32), block(32, 8);
-  working_copies_kernel<<<grid, block, 0, stream>>>(d.P32, d.P16, d.Pt16, hm.M, hm.rp);
+  working_copies_kernel<<<grid, block, 0, stream>>>(d.P32, d.P16, d.Pt16, hm.M, hm.rp, d.ldp, d.ldpt);
   st->launches += 1;
   NG_CUDA(cudaGetLastError());
   return NGALORE_OK;
@@ -287,7 +287,7 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       const MatDesc& d = st->h_desc[i];
       SimtGemm g{};
       g.m = hm.rp; g.n = hm.N; g.k = hm.M;
-      g.A = d.Pt16; g.a_rs = hm.M; g.a_cs = 1; g.a_dt = DT_BF16;
+      g.A = d.Pt16; g.a_rs = d.ldpt; g.a_cs = 1; g.a_dt = DT_BF16;
       g.B = G[i]; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_BF16;
       g.C = d.H + static_cast<long long>(cur) * hm.rn; g.c_rs = hm.N; g.c_cs = 1; g.c_dt = DT_F32;
       g.epilogue = EPI_STORE;
@@ -295,7 +295,7 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       st->launches += 1;
     }
   } else {
-    if ((rc = tc_project(st->tc, st->d_desc, st->d_ctrl, G, ptr_changed, stream, &st->launches))) return rc;
+    if ((rc = tc_project(st->tc, st->d_desc, st->d_ctrl, G, stream, &st->launches))) return rc;
   }
   if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[1], stream));
   // ---- phase 1: Gram row, solve, natural gradient + moments
@@ -315,7 +315,7 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       const MatDesc& d = st->h_desc[i];
       SimtGemm g{};
       g.m = hm.M; g.n = hm.N; g.k = hm.rp;
-      g.A = d.P16; g.a_rs = hm.rp; g.a_cs = 1; g.a_dt = DT_BF16;
+      g.A = d.P16; g.a_rs = d.ldp; g.a_cs = 1; g.a_dt = DT_BF16;
       g.B = d.u_hi; g.B2 = d.u_lo; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_BF16;
       g.C = W[i]; g.c_rs = hm.N; g.c_cs = 1; g.c_dt = DT_F32;
       g.epilogue = EPI_W_UPDATE;
@@ -325,7 +325,7 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       st->launches += 1;
     }
   } else {
-    if ((rc = tc_backproject(st->tc, st->d_desc, st->d_ctrl, st->d_hyper, W, ptr_changed, stream, &st->launches))) return rc;
+    if ((rc = tc_backproject(st->tc, st->d_desc, st->d_ctrl, st->d_hyper, st->d_W, stream, &st->launches))) return rc;
   }
   advance_kernel<<<1, 1, 0, stream>>>(st->d_ctrl);
   st->launches += 1;
@@ -425,8 +425,8 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     offs[i].m = take(sizeof(float) * hm.rn);
     offs[i].v = take(sizeof(float) * hm.rn);
     offs[i].P32 = take(sizeof(float) * hm.M * hm.rp);
-    offs[i].P16 = take(sizeof(__nv_bfloat16) * hm.M * hm.rp);
-    offs[i].Pt16 = take(sizeof(__nv_bfloat16) * hm.M * hm.rp);
+    offs[i].P16 = take(sizeof(__nv_bfloat16) * hm.M * ((hm.rp + 7) / 8 * 8));
+    offs[i].Pt16 = take(sizeof(__nv_bfloat16) * hm.rp * ((hm.M + 7) / 8 * 8));
     offs[i].Kraw = take(sizeof(double) * slots * slots);
     offs[i].wsol = take(sizeof(float) * kMaxHistory);
   }
@@ -492,6 +492,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     HostMat& hm = st->mats[i];
     MatDesc& d = st->h_desc[i];
     d.M = hm.M; d.N = hm.N; d.rp = hm.rp; d.s = s; d.rn = hm.rn;
+    d.ldp = (hm.rp + 7) / 8 * 8; d.ldpt = (hm.M + 7) / 8 * 8;
     d.H = reinterpret_cast<float*>(st->arena + offs[i].H);
     d.m = reinterpret_cast<float*>(st->arena + offs[i].m);
     d.v = reinterpret_cast<float*>(st->arena + offs[i].v);
@@ -658,7 +659,7 @@ ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, 
   const HostMat& hm = st->mats[i];
   const long long cnt = static_cast<long long>(hm.M) * hm.rp;
   widen_bf16_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      st->h_desc[i].P16, P, cnt);
+      st->h_desc[i].P16, P, cnt, hm.rp, st->h_desc[i].ldp);
   st->launches += 1;
   NG_CUDA(cudaGetLastError());
   return NGALORE_OK;
