@@ -1,0 +1,353 @@
+#!/usr/bin/env python
+"""Throughput of the Natural GaLore optimizer step on synthetic Llama-shaped gradients.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 0..4] [--impl ours|reference]
+
+One "step" is one optimizer step over every weight matrix of the workload (projection, history
+Gram + solve, natural gradient + Adam moments, back-projection + W update).  Prints ONE JSON line.
+With --gpus N > 1 (launched under torchrun) every rank steps its own replica of the matrix set
+(weak scaling, no data-path collective); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "optimizer steps/sec over all matrices (device-timed)"
+UNIT = "steps/s"
+
+
+def measured_peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def byte_model(wl):
+    """Algorithmic bytes per step: every datum moved once (G bf16, W fp32, P bf16, history/m/v fp32)."""
+    tot = stream = 0
+    for i, (_, M, N) in enumerate(wl.shapes):
+        rp = wl.rank_of(i)
+        rn = rp * N
+        tot += 10 * M * N + 2 * M * rp + (4 * wl.s + 20) * rn
+        stream += (4 * wl.s + 16) * rn          # history read once + m, v read and written
+    return tot, stream
+
+
+def flop_model(wl):
+    f = 0
+    for i, (_, M, N) in enumerate(wl.shapes):
+        rp = wl.rank_of(i)
+        f += 4 * M * N * rp + 4 * wl.s * rp * N + 12 * rp * N
+    return f
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------- oracle arm
+
+def oracle_sample(wl, seed_shift=0, P_by_shape=None):
+    """Time the fp64 oracle on one matrix per distinct shape (history pre-filled to s slots) and scale by
+    the shape counts to one full step.  Returns (seconds per full step, description, threads)."""
+    from oracle import natural_galore as orc
+    from paper_2410_16029_b200 import workload as W
+
+    counts = {}
+    for _, M, N in wl.shapes:
+        counts[(M, N)] = counts.get((M, N), 0) + 1
+    total = 0.0
+    rng = np.random.default_rng(1234 + seed_shift)
+    for i, M, N in wl.distinct_shapes():
+        hp = orc.Hyper(r=wl.r, s=wl.s, T=0, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps)
+        st = orc.MatrixState(M, N, hp)
+        if P_by_shape is not None and (M, N) in P_by_shape:
+            P = P_by_shape[(M, N)]
+        else:
+            P, _ = np.linalg.qr(rng.standard_normal((M, st.rp)))
+        st.set_subspace(P)
+        for j in range(wl.s):                       # steady state: a full history
+            st.slots[j] = rng.standard_normal((st.rp, N))
+        st.count, st.head = wl.s, 0
+        G = W.bf16_bits_to_f64(W.gradient_bits(wl, i, 1))
+        Wm = np.zeros((M, N))
+        t0 = time.perf_counter()
+        st.step(Wm, G, auto_refresh=False)
+        total += (time.perf_counter() - t0) * counts[(M, N)]
+    try:
+        import threadpoolctl
+        threads = max(p["num_threads"] for p in threadpoolctl.threadpool_info())
+    except Exception:
+        threads = os.cpu_count()
+    desc = (f"one oracle step (full history of {wl.s}) on one matrix of each of the "
+            f"{len(counts)} distinct shapes, scaled by the shape counts to the {wl.n_matrices}-matrix step")
+    return total, desc, threads
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    desc, threads = "", 0
+    for k in range(args.warmup + args.steps):
+        t, desc, threads = oracle_sample(wl, seed_shift=k)
+        if k >= args.warmup:
+            times.append(t)
+    sec = float(np.mean(times))
+    val = 1.0 / sec
+    out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": wl.name, "matrices": wl.n_matrices, "r": wl.r, "s": wl.s},
+           "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+           "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+# --------------------------------------------------------------------------------------- CUDA arm
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2410_16029_b200 import workload as W
+    from paper_2410_16029_b200.ngalore import NGaLore
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    shapes = [(M, N) for _, M, N in wl.shapes]
+    n = len(shapes)
+    opt = NGaLore(shapes, wl.r, wl.s, wl.T, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
+                  wd=wl.wd, seed=1 + rank)
+    # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
+    wl_rank = W.Workload(**{**wl.__dict__, "index": wl.index + 100 * rank})
+    # With fewer than s + 1 distinct sets a gradient would sit twice in the history ring and the Gram matrix
+    # would be singular up to lambda; the optimizer never sees that in training.
+    pool_sets = args.pool if args.pool > 0 else wl.s + 1
+    pool = [[W.gradient_device(wl_rank, i, k, dev) for i in range(n)] for k in range(pool_sets)]
+    Wt = [W.initial_weight_device(wl_rank, i, dev) for i in range(n)]
+    Wp = NGaLore.pointer_array(Wt)
+    Gp = [NGaLore.pointer_array(g) for g in pool]
+    grad_bytes = sum(M * N * 2 for M, N in shapes)
+
+    def step(k):
+        opt.step_ptrs(Wp, Gp[k % pool_sets])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for k in range(args.warmup):
+        step(k)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    l0 = opt.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for k in range(args.steps):
+        step(args.warmup + k)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    launches = opt.launch_count - l0
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * 1e3 / ms_step
+
+    code, per = opt.poll_status()
+    if code != 0:
+        raise RuntimeError(f"device status {code}: {per[:8]}...")
+
+    # ---- per-phase kernel times (CUDA events on the launching stream, inside the library)
+    opt.set_profiling(True)
+    phase = np.zeros(3)
+    reps = 10
+    for k in range(reps):
+        step(args.warmup + args.steps + k)
+        phase += np.array([opt.last_phase_ms(p) for p in range(3)])
+    phase /= reps
+    opt.set_profiling(False)
+
+    # ---- refresh, timed alone
+    torch.cuda.synchronize()
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    r0.record()
+    opt.refresh_subspace(pool[0])
+    r1.record()
+    torch.cuda.synchronize()
+    refresh_ms = r0.elapsed_time(r1)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        Wh = [torch.empty((M, N), dtype=torch.float32).pin_memory() for M, N in shapes]
+        Gh = [torch.empty((M, N), dtype=torch.bfloat16).pin_memory() for M, N in shapes]
+        for i in range(n):
+            Wh[i].copy_(Wt[i])
+            Gh[i].copy_(pool[0][i])
+        opt.step_host(Wh, Gh)          # first call allocates the device staging
+        t0 = time.perf_counter()
+        e2e_steps = 3
+        for _ in range(e2e_steps):
+            opt.step_host(Wh, Gh)      # returns after the device-to-host copy of W has finished
+        dt = (time.perf_counter() - t0) / e2e_steps
+        w_bytes = sum(M * N * 4 for M, N in shapes)
+        e2e = {"value": 1.0 / dt, "unit": UNIT, "h2d_bytes_per_step": w_bytes + grad_bytes,
+               "d2h_bytes_per_step": w_bytes, "ms_per_step": dt * 1e3, "steps": e2e_steps}
+        del Wh, Gh
+
+    # ---- roofline of the dominant kernel and of the whole step
+    peak, peak_kind = measured_peak_hbm()
+    tot_bytes, stream_bytes = byte_model(wl)
+    names = ["tc_gemm_kernel<project>", "fused_stream_kernel", "tc_gemm_kernel<backproject>"]
+    proj_bytes = sum(2 * M * N + 2 * M * wl.rank_of(i) + 4 * wl.rank_of(i) * N for i, (M, N) in enumerate(shapes))
+    back_bytes = sum(8 * M * N + 2 * M * wl.rank_of(i) for i, (M, N) in enumerate(shapes))
+    alg = [proj_bytes, stream_bytes, back_bytes]
+    dom = int(np.argmax(phase))
+    achieved = alg[dom] / (phase[dom] * 1e-3) / 1e9
+    traffic = None
+    roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
+                "algorithmic_bytes_per_launch": alg[dom], "ms_per_launch": float(phase[dom]),
+                "phases_ms": {names[i]: float(phase[i]) for i in range(3)},
+                "phases_frac_of_peak": {names[i]: alg[i] / (phase[i] * 1e-3) / 1e9 / peak for i in range(3)}}
+    step_roofline_ms = max(tot_bytes / (peak * 1e9), flop_model(wl) / 1389.3e12) * 1e3
+    step_roof = {"bytes_per_step": tot_bytes, "flops_per_step": flop_model(wl), "roofline_ms": step_roofline_ms,
+                 "frac": step_roofline_ms / ms_step, "peak_kind": peak_kind}
+
+    # ---- the oracle on the host cores, bounded sample
+    cpu = None
+    if not args.no_cpu:
+        sec, desc, threads = oracle_sample(wl)
+        cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16 GEMM operands, f32 state/accumulation, f64 Gram+solve",
+           "data": "synthetic",
+           "config": {"workload": wl.name, "matrices": n, "r": wl.r, "s": wl.s, "T": wl.T,
+                      "l2": f"inputs larger than L2: {pool_sets} gradient sets of {grad_bytes / 1e9:.2f} GB cycled",
+                      "state_bytes": opt.device_bytes},
+           "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+           "step_roofline": step_roof,
+           "refresh": {"ms": refresh_ms, "T": wl.T, "amortised_ms_per_step": ms_step + refresh_ms / max(wl.T, 1),
+                       "amortised_steps_per_s": world * 1e3 / (ms_step + refresh_ms / max(wl.T, 1))},
+           "cpu_baseline": cpu}
+    print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--pool", type=int, default=0,
+                    help="gradient sets resident in HBM, cycled (default s + 1: no gradient repeats inside the history)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2410_16029_b200 import workload as W
+
+    wl = W.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        import __graft_entry__ as entry
+
+        entry.build()
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
