@@ -7,8 +7,8 @@
 //   back-projection  W <- (1 - lr wd) W - lr P u     A = P16 (M x r'), B = u_hi and u_lo (r' x N)
 //                    epilogue: fused read-modify-write of W                                      (Sec. 2.2)
 //
-// Warp roles (192 threads): warp 0 issues TMA loads, warp 1 allocates TMEM and issues the MMAs,
-// warps 2..5 drain the accumulator (tcgen05.ld), transpose through shared memory and write
+// Warp roles: warp 0 issues TMA loads, warp 1 allocates TMEM and issues the MMAs, four or eight further
+// warps drain the accumulator (tcgen05.ld), transpose through shared memory and write
 // coalesced rows.  Two accumulator buffers let the epilogue of one tile overlap the MMAs of the next.
 // Every mbarrier wait is bounded: when it runs out the CTA raises Ctrl::timeout_flag, stops issuing
 // work, and still releases its TMEM.
@@ -26,7 +26,6 @@ namespace ngalore {
 
 constexpr int kTcBM = 128;        // rows of one accumulator tile (TMEM lanes)
 constexpr int kTcBK = 64;         // K elements per pipeline stage (one 128-byte swizzle row of bf16)
-constexpr int kTcThreads = 192;
 constexpr unsigned long long kTcWaitLimitNs = 2000000000ull;  // a wait on an mbarrier is abandoned after 2 s
 
 struct TcTile {
@@ -132,25 +131,25 @@ __device__ __forceinline__ uint32_t instr_desc(int n) {
          (static_cast<uint32_t>(kTcBM >> 4) << 24);
 }
 
-template <int BN, int NB, int STAGES>
+template <int BN, int NB, int STAGES, int NEPI>
 struct TcSmem {
   static constexpr int kABytes = kTcBM * kTcBK * 2;           // 16 KB
   static constexpr int kBChunkBytes = 64 * kTcBK * 2;         // one 64-column chunk: 64 K rows x 128 B
   static constexpr int kBBytes = (BN / 64) * kBChunkBytes;    // per B operand
   static constexpr int kStageBytes = kABytes + NB * kBBytes;
   static constexpr int kEpiWarpBytes = 32 * 36 * 4;           // 32 rows x (32 + 4 pad) floats
-  static constexpr int kBarOffset = STAGES * kStageBytes + 4 * kEpiWarpBytes;
+  static constexpr int kBarOffset = STAGES * kStageBytes + NEPI * kEpiWarpBytes;
   static constexpr int kTotal = kBarOffset + 256 + 1024;      // barriers + slack for 1024-byte alignment
 };
 
 enum { TC_EPI_PROJECT = 0, TC_EPI_WUPDATE = 1 };
 
-template <int BN, int NB, int STAGES, int EPI>
-__global__ void __launch_bounds__(kTcThreads, 1)
+template <int BN, int NB, int STAGES, int EPI, int NEPI>
+__global__ void __launch_bounds__(64 + 32 * NEPI, 1)
 tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__ tiles, int n_tiles,
                const MatDesc* __restrict__ mats, Ctrl* ctrl, const Hyper* __restrict__ hyper,
                float* const* __restrict__ Wptrs) {
-  using L = TcSmem<BN, NB, STAGES>;
+  using L = TcSmem<BN, NB, STAGES, NEPI>;
   extern __shared__ unsigned char tc_smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
@@ -249,14 +248,19 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2 .. 2 + NEPI - 1)
+    // With 8 epilogue warps there are two groups of four; group g drains accumulator buffer g, i.e. the
+    // tiles with (local & 1) == g, so one group's W loads are in flight while the other computes.
     const int quarter = warp & 3;  // TMEM lanes 32 * quarter .. + 31 belong to this warp
+    constexpr int kGroups = NEPI / 4;
+    const int group = (warp - 2) >> 2;
     float* stg = reinterpret_cast<float*>(smem + STAGES * L::kStageBytes + (warp - 2) * L::kEpiWarpBytes);
     float lr = 0.f, decay = 1.f;
     if (EPI == TC_EPI_WUPDATE) { lr = hyper->lr; decay = 1.f - hyper->lr * hyper->wd; }
     int local = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
+      if (kGroups == 2 && (local & 1) != group) continue;
       const TcTile tile = tiles[t];
       const MatDesc& d = mats[tile.mat];
       const int n_rem = d.N - tile.n0;
@@ -274,51 +278,73 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
         rows_total = d.M;
         skip = __ldcg(d.step_bad) != 0;
       }
-      if (!mbar_wait(tfull_bar + buf, tphase, abort_flag)) { ok = false; break; }
-      tc_fence_after();
       const int row_base = tile.m0 + quarter * 32;
-      for (int c0 = 0; c0 < n_eff; c0 += 32) {
-        uint32_t r[32];
-        tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * BN + c0), r);
-        tc_wait_ld();
-        if (c0 + 32 >= n_eff) {
-          // all TMEM reads of this tile are done: hand the buffer back before the global traffic
-          tc_fence_before();
-          if (lane == 0) mbar_arrive(tempty_bar + buf);
-        }
+      const int sub_row = lane >> 3, sub_col = (lane & 7) * 4;
+      // W update: fetch this warp's whole 32 x BN slab of W before waiting for the accumulator, so that
+      // the loads overlap the MMAs of the tile (and the other group's epilogue).
+      constexpr int kChunks = BN / 32;
+      float4 wreg[EPI == TC_EPI_WUPDATE ? kChunks : 1][8];
+      if (EPI == TC_EPI_WUPDATE) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          *reinterpret_cast<float4*>(stg + lane * 36 + j * 4) =
-              make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                          __uint_as_float(r[4 * j + 3]));
-        __syncwarp();
-        const int col = tile.n0 + c0 + (lane & 7) * 4;
-        if (!skip && col < d.N) {
+        for (int c = 0; c < kChunks; ++c) {
+          const int col = tile.n0 + c * 32 + sub_col;
 #pragma unroll
           for (int it = 0; it < 8; ++it) {
-            const int rr = it * 4 + (lane >> 3);
-            const int row = row_base + rr;
-            if (row < rows_total) {
-              const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + (lane & 7) * 4);
-              float* p = out + static_cast<long long>(row) * d.N + col;
-              if (EPI == TC_EPI_PROJECT) {
-                if (tile.atomic) {
-                  atomicAdd(reinterpret_cast<float4*>(p), acc);
+            const int row = row_base + it * 4 + sub_row;
+            wreg[c][it] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (!skip && c * 32 < n_eff && col < d.N && row < rows_total)
+              wreg[c][it] = __ldcs(reinterpret_cast<const float4*>(out + static_cast<long long>(row) * d.N + col));
+          }
+        }
+      }
+      if (!mbar_wait(tfull_bar + buf, tphase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < kChunks; ++c) {
+        const int c0 = c * 32;
+        if (c0 < n_eff) {
+          uint32_t r[32];
+          tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * BN + c0), r);
+          tc_wait_ld();
+          if (c0 + 32 >= n_eff) {
+            // all TMEM reads of this tile are done: hand the buffer back before the global traffic
+            tc_fence_before();
+            if (lane == 0) mbar_arrive(tempty_bar + buf);
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<float4*>(stg + lane * 36 + j * 4) =
+                make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                            __uint_as_float(r[4 * j + 3]));
+          __syncwarp();
+          const int col = tile.n0 + c0 + sub_col;
+          if (!skip && col < d.N) {
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+              const int rr = it * 4 + sub_row;
+              const int row = row_base + rr;
+              if (row < rows_total) {
+                const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + sub_col);
+                float* p = out + static_cast<long long>(row) * d.N + col;
+                if (EPI == TC_EPI_PROJECT) {
+                  if (tile.atomic) {
+                    atomicAdd(reinterpret_cast<float4*>(p), acc);
+                  } else {
+                    *reinterpret_cast<float4*>(p) = acc;
+                  }
                 } else {
-                  *reinterpret_cast<float4*>(p) = acc;
+                  float4 w = wreg[EPI == TC_EPI_WUPDATE ? c : 0][it];
+                  w.x = decay * w.x - lr * acc.x;
+                  w.y = decay * w.y - lr * acc.y;
+                  w.z = decay * w.z - lr * acc.z;
+                  w.w = decay * w.w - lr * acc.w;
+                  __stcs(reinterpret_cast<float4*>(p), w);
                 }
-              } else {
-                float4 w = *reinterpret_cast<const float4*>(p);
-                w.x = decay * w.x - lr * acc.x;
-                w.y = decay * w.y - lr * acc.y;
-                w.z = decay * w.z - lr * acc.z;
-                w.w = decay * w.w - lr * acc.w;
-                *reinterpret_cast<float4*>(p) = w;
               }
             }
           }
+          __syncwarp();
         }
-        __syncwarp();
       }
     }
   }
@@ -352,8 +378,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-constexpr int kProjBN = 256, kProjStages = 4;
-constexpr int kBackBN = 128, kBackStages = 4;
+constexpr int kProjBN = 256, kProjStages = 4, kProjEpiWarps = 4;
+constexpr int kBackBN = 128, kBackStages = 3, kBackEpiWarps = 8;
 
 struct TcPlan {
   size_t device_bytes = 0;
@@ -475,11 +501,11 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   plan.rowsN.resize(n); plan.colsN.resize(n);
   for (int i = 0; i < n; ++i) { plan.rowsN[i] = mats[i].M; plan.colsN[i] = mats[i].N; }
 
-  using LP = TcSmem<kProjBN, 1, kProjStages>;
-  using LB = TcSmem<kBackBN, 2, kBackStages>;
-  if (cudaFuncSetAttribute(tc_gemm_kernel<kProjBN, 1, kProjStages, TC_EPI_PROJECT>,
+  using LP = TcSmem<kProjBN, 1, kProjStages, kProjEpiWarps>;
+  using LB = TcSmem<kBackBN, 2, kBackStages, kBackEpiWarps>;
+  if (cudaFuncSetAttribute(tc_gemm_kernel<kProjBN, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess ||
-      cudaFuncSetAttribute(tc_gemm_kernel<kBackBN, 2, kBackStages, TC_EPI_WUPDATE>,
+      cudaFuncSetAttribute(tc_gemm_kernel<kBackBN, 2, kBackStages, TC_EPI_WUPDATE, kBackEpiWarps>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, LB::kTotal) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   plan.maps_dirty = true;
@@ -509,8 +535,8 @@ inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ct
     zero_split_slots_kernel<<<dim3(64, plan.n_split), 256, 0, stream>>>(d_mats, plan.d_split_mats, d_ctrl);
     *launches += 1;
   }
-  using LP = TcSmem<kProjBN, 1, kProjStages>;
-  tc_gemm_kernel<kProjBN, 1, kProjStages, TC_EPI_PROJECT><<<plan.grid_proj, kTcThreads, LP::kTotal, stream>>>(
+  using LP = TcSmem<kProjBN, 1, kProjStages, kProjEpiWarps>;
+  tc_gemm_kernel<kProjBN, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps><<<plan.grid_proj, 64 + 32 * kProjEpiWarps, LP::kTotal, stream>>>(
       plan.d_maps, plan.d_tiles_proj, plan.n_tiles_proj, d_mats, d_ctrl, nullptr, nullptr);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
@@ -525,8 +551,8 @@ inline ngalore_status tc_backproject(TcPlan& plan, const MatDesc* d_mats, Ctrl* 
       return NGALORE_ERR_CUDA;
     plan.maps_dirty = false;
   }
-  using LB = TcSmem<kBackBN, 2, kBackStages>;
-  tc_gemm_kernel<kBackBN, 2, kBackStages, TC_EPI_WUPDATE><<<plan.grid_back, kTcThreads, LB::kTotal, stream>>>(
+  using LB = TcSmem<kBackBN, 2, kBackStages, kBackEpiWarps>;
+  tc_gemm_kernel<kBackBN, 2, kBackStages, TC_EPI_WUPDATE, kBackEpiWarps><<<plan.grid_back, 64 + 32 * kBackEpiWarps, LB::kTotal, stream>>>(
       plan.d_maps, plan.d_tiles_back, plan.n_tiles_back, d_mats, d_ctrl, d_hyper, d_W);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
