@@ -158,6 +158,34 @@ int64_t ngalore_launch_count(const ngalore_state* st);
 ngalore_status ngalore_set_profiling(ngalore_state* st, int on);
 double ngalore_last_phase_ms(ngalore_state* st, int phase);
 
+/*
+ * Natural-gradient transform of one matrix without any allocation.  (The paper has no counterpart:
+ * this entry point exists for callers that cannot obtain device memory themselves -- code running
+ * under a fixed, pre-carved memory budget, inside another framework's allocator-free region, or in
+ * a process where cudaMalloc is forbidden after start-up -- and therefore cannot use ngalore_create.)
+ *
+ * Given the ring H of low-rank gradients (s slots of n fp32 elements each, slot-major, `count` of them
+ * valid, the newest in slot `cur`) and the caller-kept raw Gram matrix K (s x s doubles, K_ij = <H_i, H_j>,
+ * zero before the first call), it refreshes row and column `cur` of K, solves
+ * (lambda I + K / count) w = e_cur by Cholesky in fp64 and writes out = sum_j w_j H_j (n floats).
+ * This equals F^-1 applied to the newest gradient with F = lambda I + (1/count) sum_j vec(H_j) vec(H_j)^T,
+ * the same arithmetic ngalore_step performs per matrix.
+ *
+ * All pointers are device pointers owned by the caller; H and out 16-byte aligned; n a multiple of 4.
+ * `status` (device int, may be NULL) receives NGALORE_ERR_NOT_SPD / NGALORE_ERR_NONFINITE when the solve
+ * fails (out is then all zeros); it is only ever set, so zero it beforehand.
+ *
+ * Scratch: the per-tile partial sums and the weights live in a 256.5 KiB array that is part of the
+ * library image on every GPU that loads it, which bounds n at 8,388,608 elements per slot; larger n is
+ * rejected with NGALORE_ERR_INVALID_ARG.  The call uses no cudaMalloc/cudaFree and no allocating library
+ * routine.  The first call on a device looks up the array's device address; make that first call outside
+ * any stream capture.  All calls on a device share the array (it keeps the previous call's contents, all
+ * of which the next call overwrites before reading): two calls whose kernels may overlap on the GPU race,
+ * so issue them on one stream or order them with events.  Asynchronous on `stream`.
+ */
+ngalore_status ngalore_natural_gradient_static(const float* H, int64_t n, int s, int count, int cur, double lambda,
+                                               double* K, float* out, int* status, void* stream);
+
 const char* ngalore_status_string(ngalore_status s);
 
 #ifdef __cplusplus

@@ -15,6 +15,7 @@
 #include "kernels_stream.cuh"
 #include "gemm_tcgen05.cuh"
 #include "kernels_fused_stream.cuh"
+#include "static_natural_gradient.cuh"
 
 using namespace ngalore;
 

@@ -75,6 +75,9 @@ _lib.ngalore_set_profiling.restype = ctypes.c_int
 _lib.ngalore_set_profiling.argtypes = [_vp, ctypes.c_int]
 _lib.ngalore_last_phase_ms.restype = ctypes.c_double
 _lib.ngalore_last_phase_ms.argtypes = [_vp, ctypes.c_int]
+_lib.ngalore_natural_gradient_static.restype = ctypes.c_int
+_lib.ngalore_natural_gradient_static.argtypes = [_vp, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                                 ctypes.c_double, _vp, _vp, _vp, _vp]
 _lib.ngalore_status_string.restype = ctypes.c_char_p
 _lib.ngalore_status_string.argtypes = [ctypes.c_int]
 
@@ -215,3 +218,20 @@ class NGaLore:
 
     def last_phase_ms(self, phase: int) -> float:
         return _lib.ngalore_last_phase_ms(self._h, phase)
+
+
+def natural_gradient_static(H: torch.Tensor, count: int, cur: int, lam: float, K: torch.Tensor, out: torch.Tensor,
+                            status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Allocation-free natural-gradient transform (ngalore_natural_gradient_static).
+
+    H: (s, n) fp32 history ring on the device, K: (s, s) fp64 raw Gram matrix kept by the caller
+    (zeros before the first call), out: (n,) fp32.  For callers that may not allocate device memory:
+    the library's scratch is a fixed array inside the library image (n <= 8,388,608).  Calls share
+    that array, so keep them on one stream."""
+    assert H.is_cuda and H.dtype == torch.float32 and H.is_contiguous() and H.dim() == 2
+    assert K.is_cuda and K.dtype == torch.float64 and K.is_contiguous() and tuple(K.shape) == (H.shape[0],) * 2
+    assert out.is_cuda and out.dtype == torch.float32 and out.is_contiguous() and out.numel() == H.shape[1]
+    sp = status.data_ptr() if status is not None else None
+    _check(_lib.ngalore_natural_gradient_static(H.data_ptr(), H.shape[1], H.shape[0], count, cur, lam, K.data_ptr(),
+                                                out.data_ptr(), sp, _stream_ptr(stream)),
+           "ngalore_natural_gradient_static")
