@@ -67,7 +67,7 @@ typedef enum {
 typedef struct {
   int32_t struct_size;              /* = sizeof(ngalore_options) */
   int32_t gemm_impl;                /* 0 (default): tensor-core (tcgen05) projection GEMMs; 1: plain SIMT GEMMs (debug) */
-  int32_t power_iterations;         /* subspace-iteration sweeps in the refresh; <= 0 selects the default 4 */
+  int32_t power_iterations;         /* subspace-iteration sweeps in the refresh; <= 0 selects the default 6 */
   int32_t reset_history_on_refresh; /* default 0: history, m and v survive a refresh */
   uint64_t seed;                    /* seed of the refresh's random test matrix; 0 selects a fixed default */
   int32_t stream_impl;              /* 0 (default): fused Gram/solve/moment kernel; 1: separate plain kernels (debug) */

@@ -28,8 +28,17 @@ constexpr int kTcBM = 128;        // rows of one accumulator tile (TMEM lanes)
 constexpr int kTcBK = 64;         // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr unsigned long long kTcWaitLimitNs = 2000000000ull;  // a wait on an mbarrier is abandoned after 2 s
 
+// Generic problem of the store-mode GEMM (subspace refresh): out (out_rows x out_cols, leading dimension
+// ld_out, fp32) = A B with the operands' tensor maps at tmaps[map_a + part] and tmaps[map_b + part].
+struct TcProblem {
+  float* out;
+  int out_rows, out_cols, ld_out;
+  int map_a, map_b;
+  int pad;
+};
+
 struct TcTile {
-  int mat;
+  int mat;         // matrix index (projection, W update) or problem index (store mode)
   int m0, n0;      // tile origin in the output
   int k0;          // first K element
   int kblocks;     // number of 64-wide K blocks
@@ -125,31 +134,36 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   d |= 2ull << 61;
   return d;
 }
-// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A (K-major) and B (MN-major), M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
+// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A (K-major, or MN-major when asked) and
+// B (MN-major), M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(int n, bool a_mn_major = false) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | (1u << 16) |
+         (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(kTcBM >> 4) << 24);
 }
 
-template <int BN, int NB, int STAGES, int NEPI>
+template <int BN, int NA, int NB, int STAGES, int NEPI>
 struct TcSmem {
   static constexpr int kABytes = kTcBM * kTcBK * 2;           // 16 KB
   static constexpr int kBChunkBytes = 64 * kTcBK * 2;         // one 64-column chunk: 64 K rows x 128 B
   static constexpr int kBBytes = (BN / 64) * kBChunkBytes;    // per B operand
-  static constexpr int kStageBytes = kABytes + NB * kBBytes;
+  static constexpr int kStageBytes = NA * kABytes + NB * kBBytes;
   static constexpr int kEpiWarpBytes = 32 * 36 * 4;           // 32 rows x (32 + 4 pad) floats
   static constexpr int kBarOffset = STAGES * kStageBytes + NEPI * kEpiWarpBytes;
   static constexpr int kTotal = kBarOffset + 256 + 1024;      // barriers + slack for 1024-byte alignment
 };
 
-enum { TC_EPI_PROJECT = 0, TC_EPI_WUPDATE = 1 };
+enum { TC_EPI_PROJECT = 0, TC_EPI_WUPDATE = 1, TC_EPI_STORE = 2 };
 
-template <int BN, int NB, int STAGES, int EPI, int NEPI>
+// NA / NB: number of bf16 parts of A / B (1, or 2 = high and low part).  With NA = NB = 2 the products
+// hi*hi, hi*lo and lo*hi are accumulated (lo*lo is below fp32 resolution).  A_MN: A is stored with its
+// row index contiguous (A^T row-major), staged as two 64-row chunks like B.
+template <int BN, int NA, int NB, int STAGES, int EPI, int NEPI, bool A_MN>
 __global__ void __launch_bounds__(64 + 32 * NEPI, 1)
 tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__ tiles, int n_tiles,
                const MatDesc* __restrict__ mats, Ctrl* ctrl, const Hyper* __restrict__ hyper,
-               float* const* __restrict__ Wptrs) {
-  using L = TcSmem<BN, NB, STAGES, NEPI>;
+               float* const* __restrict__ Wptrs, const TcProblem* __restrict__ probs) {
+  using L = TcSmem<BN, NA, NB, STAGES, NEPI>;
   extern __shared__ unsigned char tc_smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
@@ -186,22 +200,39 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
       bool ok = true;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
         const TcTile tile = tiles[t];
-        const MatDesc& d = mats[tile.mat];
-        const CUtensorMap* mapA = tmaps + tile.mat * 5 + (EPI == TC_EPI_PROJECT ? 0 : 2);
-        const CUtensorMap* mapB0 = tmaps + tile.mat * 5 + (EPI == TC_EPI_PROJECT ? 1 : 3);
-        const int n_rem = d.N - tile.n0;
+        const CUtensorMap *mapA, *mapB0;
+        int out_cols;
+        if (EPI == TC_EPI_STORE) {
+          const TcProblem pr = probs[tile.mat];
+          mapA = tmaps + pr.map_a;
+          mapB0 = tmaps + pr.map_b;
+          out_cols = pr.out_cols;
+        } else {
+          mapA = tmaps + tile.mat * 5 + (EPI == TC_EPI_PROJECT ? 0 : 2);
+          mapB0 = tmaps + tile.mat * 5 + (EPI == TC_EPI_PROJECT ? 1 : 3);
+          out_cols = mats[tile.mat].N;
+        }
+        const int n_rem = out_cols - tile.n0;
         const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
         const int nchunks = (n_eff + 63) >> 6;
-        const uint32_t bytes = L::kABytes + NB * nchunks * L::kBChunkBytes;
+        const uint32_t bytes = NA * L::kABytes + NB * nchunks * L::kBChunkBytes;
         for (int kb = 0; kb < tile.kblocks; ++kb) {
           if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           unsigned char* sA = smem + stage * L::kStageBytes;
           mbar_expect_tx(full_bar + stage, bytes);
           const int k = tile.k0 + kb * kTcBK;
-          tma_load_2d(sA, mapA, k, tile.m0, full_bar + stage);
+#pragma unroll
+          for (int na = 0; na < NA; ++na) {
+            if (A_MN) {
+              tma_load_2d(sA + na * L::kABytes, mapA + na, tile.m0, k, full_bar + stage);
+              tma_load_2d(sA + na * L::kABytes + L::kBChunkBytes, mapA + na, tile.m0 + 64, k, full_bar + stage);
+            } else {
+              tma_load_2d(sA + na * L::kABytes, mapA + na, k, tile.m0, full_bar + stage);
+            }
+          }
 #pragma unroll
           for (int nb = 0; nb < NB; ++nb) {
-            unsigned char* sB = sA + L::kABytes + nb * L::kBBytes;
+            unsigned char* sB = sA + NA * L::kABytes + nb * L::kBBytes;
             for (int c = 0; c < nchunks; ++c)
               tma_load_2d(sB + c * L::kBChunkBytes, mapB0 + nb, tile.n0 + c * 64, k, full_bar + stage);
           }
@@ -218,10 +249,10 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
       bool ok = true;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
         const TcTile tile = tiles[t];
-        const MatDesc& d = mats[tile.mat];
-        const int n_rem = d.N - tile.n0;
+        const int out_cols = (EPI == TC_EPI_STORE) ? probs[tile.mat].out_cols : mats[tile.mat].N;
+        const int n_rem = out_cols - tile.n0;
         const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
-        const uint32_t idesc = instr_desc(n_eff);
+        const uint32_t idesc = instr_desc(n_eff, A_MN);
         const int buf = local & 1;
         const uint32_t tphase = (local >> 1) & 1u;
         if (!mbar_wait(tempty_bar + buf, tphase ^ 1u, abort_flag)) { ok = false; break; }
@@ -230,15 +261,23 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
         for (int kb = 0; kb < tile.kblocks; ++kb) {
           if (!mbar_wait(full_bar + stage, phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t aaddr = smem_u32(smem + stage * L::kStageBytes);
+          const uint32_t aaddr0 = smem_u32(smem + stage * L::kStageBytes);
+          bool first = (kb == 0);
 #pragma unroll
-          for (int nb = 0; nb < NB; ++nb) {
-            const uint32_t baddr = aaddr + L::kABytes + nb * L::kBBytes;
+          for (int na = 0; na < NA; ++na) {
 #pragma unroll
-            for (int kk = 0; kk < kTcBK / 16; ++kk) {
-              const uint64_t adesc = smem_desc(aaddr + kk * 32, 16, 1024);
-              const uint64_t bdesc = smem_desc(baddr + kk * 2048, L::kBChunkBytes, 1024);
-              tc_mma_bf16(tmem_d, adesc, bdesc, idesc, (kb > 0 || nb > 0 || kk > 0) ? 1u : 0u);
+            for (int nb = 0; nb < NB; ++nb) {
+              if (na == 1 && nb == 1) continue;  // lo * lo is dropped
+              const uint32_t aaddr = aaddr0 + na * L::kABytes;
+              const uint32_t baddr = aaddr0 + NA * L::kABytes + nb * L::kBBytes;
+#pragma unroll
+              for (int kk = 0; kk < kTcBK / 16; ++kk) {
+                const uint64_t adesc = A_MN ? smem_desc(aaddr + kk * 2048, L::kBChunkBytes, 1024)
+                                            : smem_desc(aaddr + kk * 32, 16, 1024);
+                const uint64_t bdesc = smem_desc(baddr + kk * 2048, L::kBChunkBytes, 1024);
+                tc_mma_bf16(tmem_d, adesc, bdesc, idesc, first ? 0u : 1u);
+                first = false;
+              }
             }
           }
           tc_commit(empty_bar + stage);
@@ -262,22 +301,32 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
       if (kGroups == 2 && (local & 1) != group) continue;
       const TcTile tile = tiles[t];
-      const MatDesc& d = mats[tile.mat];
-      const int n_rem = d.N - tile.n0;
+      float* out;
+      int rows_total, out_cols, ld_out;
+      bool skip = false;
+      if (EPI == TC_EPI_STORE) {
+        const TcProblem pr = probs[tile.mat];
+        out = pr.out;
+        rows_total = pr.out_rows;
+        out_cols = pr.out_cols;
+        ld_out = pr.ld_out;
+      } else {
+        const MatDesc& d = mats[tile.mat];
+        out_cols = d.N;
+        ld_out = d.N;
+        if (EPI == TC_EPI_PROJECT) {
+          out = d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn;
+          rows_total = d.rp;
+        } else {
+          out = Wptrs[tile.mat];
+          rows_total = d.M;
+          skip = __ldcg(d.step_bad) != 0;
+        }
+      }
+      const int n_rem = out_cols - tile.n0;
       const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
       const int buf = local & 1;
       const uint32_t tphase = (local >> 1) & 1u;
-      float* out;
-      int rows_total;
-      bool skip = false;
-      if (EPI == TC_EPI_PROJECT) {
-        out = d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn;
-        rows_total = d.rp;
-      } else {
-        out = Wptrs[tile.mat];
-        rows_total = d.M;
-        skip = __ldcg(d.step_bad) != 0;
-      }
       const int row_base = tile.m0 + quarter * 32;
       const int sub_row = lane >> 3, sub_col = (lane & 7) * 4;
       // W update: fetch this warp's whole 32 x BN slab of W before waiting for the accumulator, so that
@@ -292,8 +341,8 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
           for (int it = 0; it < 8; ++it) {
             const int row = row_base + it * 4 + sub_row;
             wreg[c][it] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (!skip && c * 32 < n_eff && col < d.N && row < rows_total)
-              wreg[c][it] = __ldcs(reinterpret_cast<const float4*>(out + static_cast<long long>(row) * d.N + col));
+            if (!skip && c * 32 < n_eff && col < out_cols && row < rows_total)
+              wreg[c][it] = __ldcs(reinterpret_cast<const float4*>(out + static_cast<long long>(row) * ld_out + col));
           }
         }
       }
@@ -318,15 +367,15 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
                             __uint_as_float(r[4 * j + 3]));
           __syncwarp();
           const int col = tile.n0 + c0 + sub_col;
-          if (!skip && col < d.N) {
+          if (!skip && col < out_cols) {
 #pragma unroll
             for (int it = 0; it < 8; ++it) {
               const int rr = it * 4 + sub_row;
               const int row = row_base + rr;
               if (row < rows_total) {
                 const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + sub_col);
-                float* p = out + static_cast<long long>(row) * d.N + col;
-                if (EPI == TC_EPI_PROJECT) {
+                float* p = out + static_cast<long long>(row) * ld_out + col;
+                if (EPI != TC_EPI_WUPDATE) {
                   if (tile.atomic) {
                     atomicAdd(reinterpret_cast<float4*>(p), acc);
                   } else {
@@ -501,11 +550,11 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   plan.rowsN.resize(n); plan.colsN.resize(n);
   for (int i = 0; i < n; ++i) { plan.rowsN[i] = mats[i].M; plan.colsN[i] = mats[i].N; }
 
-  using LP = TcSmem<kProjBN, 1, kProjStages, kProjEpiWarps>;
-  using LB = TcSmem<kBackBN, 2, kBackStages, kBackEpiWarps>;
-  if (cudaFuncSetAttribute(tc_gemm_kernel<kProjBN, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps>,
+  using LP = TcSmem<kProjBN, 1, 1, kProjStages, kProjEpiWarps>;
+  using LB = TcSmem<kBackBN, 1, 2, kBackStages, kBackEpiWarps>;
+  if (cudaFuncSetAttribute(tc_gemm_kernel<kProjBN, 1, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps, false>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess ||
-      cudaFuncSetAttribute(tc_gemm_kernel<kBackBN, 2, kBackStages, TC_EPI_WUPDATE, kBackEpiWarps>,
+      cudaFuncSetAttribute(tc_gemm_kernel<kBackBN, 1, 2, kBackStages, TC_EPI_WUPDATE, kBackEpiWarps, false>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, LB::kTotal) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   plan.maps_dirty = true;
@@ -535,9 +584,9 @@ inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ct
     zero_split_slots_kernel<<<dim3(64, plan.n_split), 256, 0, stream>>>(d_mats, plan.d_split_mats, d_ctrl);
     *launches += 1;
   }
-  using LP = TcSmem<kProjBN, 1, kProjStages, kProjEpiWarps>;
-  tc_gemm_kernel<kProjBN, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps><<<plan.grid_proj, 64 + 32 * kProjEpiWarps, LP::kTotal, stream>>>(
-      plan.d_maps, plan.d_tiles_proj, plan.n_tiles_proj, d_mats, d_ctrl, nullptr, nullptr);
+  using LP = TcSmem<kProjBN, 1, 1, kProjStages, kProjEpiWarps>;
+  tc_gemm_kernel<kProjBN, 1, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps, false><<<plan.grid_proj, 64 + 32 * kProjEpiWarps, LP::kTotal, stream>>>(
+      plan.d_maps, plan.d_tiles_proj, plan.n_tiles_proj, d_mats, d_ctrl, nullptr, nullptr, nullptr);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
@@ -551,9 +600,9 @@ inline ngalore_status tc_backproject(TcPlan& plan, const MatDesc* d_mats, Ctrl* 
       return NGALORE_ERR_CUDA;
     plan.maps_dirty = false;
   }
-  using LB = TcSmem<kBackBN, 2, kBackStages, kBackEpiWarps>;
-  tc_gemm_kernel<kBackBN, 2, kBackStages, TC_EPI_WUPDATE, kBackEpiWarps><<<plan.grid_back, 64 + 32 * kBackEpiWarps, LB::kTotal, stream>>>(
-      plan.d_maps, plan.d_tiles_back, plan.n_tiles_back, d_mats, d_ctrl, d_hyper, d_W);
+  using LB = TcSmem<kBackBN, 1, 2, kBackStages, kBackEpiWarps>;
+  tc_gemm_kernel<kBackBN, 1, 2, kBackStages, TC_EPI_WUPDATE, kBackEpiWarps, false><<<plan.grid_back, 64 + 32 * kBackEpiWarps, LB::kTotal, stream>>>(
+      plan.d_maps, plan.d_tiles_back, plan.n_tiles_back, d_mats, d_ctrl, d_hyper, d_W, nullptr);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }

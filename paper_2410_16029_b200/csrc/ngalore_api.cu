@@ -15,6 +15,7 @@
 #include "kernels_stream.cuh"
 #include "gemm_tcgen05.cuh"
 #include "kernels_fused_stream.cuh"
+#include "refresh_tc.cuh"
 #include "static_natural_gradient.cuh"
 
 using namespace ngalore;
@@ -76,6 +77,8 @@ struct ngalore_state {
   TcPlan tc;
   // fused streaming kernel plan
   FusedPlan fused;
+  // tensor-core refresh plan
+  RefreshPlan refresh;
   // host-buffer staging
   char* stage = nullptr;
   size_t stage_bytes = 0;
@@ -229,9 +232,25 @@ ngalore_status apply_gradient(ngalore_state* st, const std::vector<int>& idx, co
   return NGALORE_OK;
 }
 
-ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G, const std::vector<int>& idx,
+ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bool basis_in_a, cudaStream_t stream) {
+  ngalore_status rc;
+  for (int i : idx) {
+    const HostMat& hm = st->mats[i];
+    NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, basis_in_a ? hm.Ya : hm.Yb, sizeof(float) * hm.M * hm.rp,
+                            cudaMemcpyDeviceToDevice, stream));
+    if ((rc = make_working_copies(st, i, stream))) return rc;
+  }
+  if (st->opt.reset_history_on_refresh && idx.size() == static_cast<size_t>(st->n)) {
+    st->n_appended = 0;
+    NG_CUDA(cudaMemsetAsync(&st->d_ctrl->n_appended, 0, sizeof(long long), stream));
+  }
+  if (idx.size() == static_cast<size_t>(st->n)) st->has_subspace = true;
+  return NGALORE_OK;
+}
+
+// Plain SIMT refresh (debug path, and single-matrix refreshes).
+ngalore_status refresh_simt(ngalore_state* st, const uint16_t* const* G, const std::vector<int>& idx, int q,
                             cudaStream_t stream) {
-  const int q = st->opt.power_iterations > 0 ? st->opt.power_iterations : 4;
   // Random test matrix Omega (N x rp), one hashed stream per matrix and refresh.
   for (int i : idx) {
     const HostMat& hm = st->mats[i];
@@ -254,17 +273,22 @@ ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G, const s
   }
   // Second pass Yb -> Ya so that a clamped pivot of the first pass cannot leave P non-orthonormal.
   if ((rc = orthonormalise(st, idx, 0, false, stream))) return rc;
-  for (int i : idx) {
-    const HostMat& hm = st->mats[i];
-    NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, hm.Ya, sizeof(float) * hm.M * hm.rp, cudaMemcpyDeviceToDevice, stream));
-    if ((rc = make_working_copies(st, i, stream))) return rc;
-  }
-  if (st->opt.reset_history_on_refresh && idx.size() == static_cast<size_t>(st->n)) {
-    st->n_appended = 0;
-    NG_CUDA(cudaMemsetAsync(&st->d_ctrl->n_appended, 0, sizeof(long long), stream));
-  }
-  if (idx.size() == static_cast<size_t>(st->n)) st->has_subspace = true;
-  return NGALORE_OK;
+  return finish_refresh(st, idx, true, stream);
+}
+
+ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G, const std::vector<int>& idx,
+                            cudaStream_t stream) {
+  const int q = st->opt.power_iterations > 0 ? st->opt.power_iterations : 6;
+  if (st->opt.gemm_impl == 1 || idx.size() != static_cast<size_t>(st->n) || !st->refresh.ready)
+    return refresh_simt(st, G, idx, q, stream);
+  ngalore_status rc;
+  if ((rc = refresh_tc_run(st->refresh, G, q, st->opt.seed, static_cast<unsigned long long>(st->k) * 65536ull,
+                           st->d_ctrl, stream, &st->launches)))
+    return rc;
+  // The last basis sits in Ya (fp32, well conditioned): exact orthonormalisation in fp64, Ya -> Yb -> Ya.
+  if ((rc = orthonormalise(st, idx, 0, true, stream))) return rc;
+  if ((rc = orthonormalise(st, idx, 0, false, stream))) return rc;
+  return finish_refresh(st, idx, true, stream);
 }
 
 ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream) {
@@ -541,6 +565,12 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (rc != NGALORE_OK) return fail(rc);
   rc = fused_plan_create(st->fused, st->h_desc, st->tile_elems, prop.multiProcessorCount);
   if (rc != NGALORE_OK) return fail(rc);
+  if (st->opt.gemm_impl != 1) {
+    std::vector<float*> Yf(n_matrices), Zf(n_matrices);
+    for (int i = 0; i < n_matrices; ++i) { Yf[i] = st->mats[i].Ya; Zf[i] = st->mats[i].Xa; }
+    rc = refresh_plan_create(st->refresh, st->h_desc, Yf, Zf, prop.multiProcessorCount);
+    if (rc != NGALORE_OK) return fail(rc);
+  }
   for (int e = 0; e < 4; ++e)
     if (cudaEventCreate(&st->ev[e]) != cudaSuccess) return fail(NGALORE_ERR_CUDA);
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(NGALORE_ERR_CUDA);
@@ -554,6 +584,7 @@ void ngalore_destroy(ngalore_state* st) {
   cudaDeviceSynchronize();
   tc_plan_destroy(st->tc);
   fused_plan_destroy(st->fused);
+  refresh_plan_destroy(st->refresh);
   for (int e = 0; e < 4; ++e)
     if (st->ev[e]) cudaEventDestroy(st->ev[e]);
   if (st->stage) cudaFree(st->stage);
@@ -719,7 +750,7 @@ ngalore_status ngalore_set_lr(ngalore_state* st, double lr) {
 int ngalore_num_matrices(const ngalore_state* st) { return st ? st->n : 0; }
 int ngalore_rank(const ngalore_state* st, int i) { return (st && i >= 0 && i < st->n) ? st->mats[i].rp : -1; }
 int64_t ngalore_step_count(const ngalore_state* st) { return st ? st->k : -1; }
-size_t ngalore_device_bytes(const ngalore_state* st) { return st ? st->arena_bytes + st->work_bytes + st->stage_bytes + st->tc.device_bytes : 0; }
+size_t ngalore_device_bytes(const ngalore_state* st) { return st ? st->arena_bytes + st->work_bytes + st->stage_bytes + st->tc.device_bytes + st->refresh.device_bytes : 0; }
 int64_t ngalore_launch_count(const ngalore_state* st) { return st ? st->launches : 0; }
 
 ngalore_status ngalore_set_profiling(ngalore_state* st, int on) {

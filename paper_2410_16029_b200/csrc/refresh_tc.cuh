@@ -1,0 +1,426 @@
+// Subspace refresh on the tensor cores (Sec. 1: P spans the leading left singular vectors of G).
+//
+// Randomized subspace iteration with L = r' columns: Y = G Omega, then q sweeps of
+//   Z = G^T Q_Y,  Q_Z = orth(Z),  Y = G Q_Z,  Q_Y = orth(Y).
+// Every product runs through the grouped tcgen05 GEMM with the iterate split into a high and a low
+// bf16 part (16 mantissa bits).  Between products the iterate only has to stay well conditioned, so
+// orth() is a *shifted* Cholesky QR: the Gram matrix Y^T Y comes from the tensor cores (three bf16
+// products, fp32 accumulation), its columns are scaled to unit norm and a small multiple of the identity
+// is added before the fp64 Cholesky factorisation so that the fp32 accumulation error cannot make it
+// indefinite, and
+// Q = Y R^-1 is again a tensor-core GEMM with R^-1 split in two bf16 parts.  The last basis is then
+// orthonormalised exactly (Gram, Cholesky and triangular solve in fp64) by the caller.
+#pragma once
+
+#include <cstring>
+#include <vector>
+
+#include "gemm_tcgen05.cuh"
+#include "kernels_refresh.cuh"
+
+namespace ngalore {
+
+// hi = bf16(x), lo = bf16(x - hi); rows x cols fp32 (dense) -> rows x ld bf16 (padding untouched: it is zero).
+__global__ void split_hilo_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ hi,
+                                  __nv_bfloat16* __restrict__ lo, long long n, int cols, int ld) {
+  const long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if (i >= n) return;
+  const float x = src[i];
+  const __nv_bfloat16 h = __float2bfloat16_rn(x);
+  const long long o = (i / cols) * ld + (i % cols);
+  hi[o] = h;
+  lo[o] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+struct GramPrep {
+  const float* C32;  // L x L Gram matrix from the tensor cores
+  double* C64;       // L x L, lower triangle written: column-scaled, symmetrised Gram + shift I
+  double* D;         // L column norms d_i = sqrt(C_ii)
+  int L;
+};
+
+// Shift added to the unit-diagonal Gram matrix.  Each entry carries a relative error of at most about
+// 3 * 2^-18 from the two-part bf16 split (the dropped lo*lo product and the rounding of lo) plus the fp32
+// accumulation error, so the error matrix has norm below 2^-16 L; with this shift the Cholesky factorisation
+// cannot meet a negative pivot.  The price is that directions closer than sqrt(shift) are not pulled
+// apart, which is harmless between products.
+__host__ __device__ inline double gram_shift(int L) { return static_cast<double>(L) / 65536.0; }
+
+// One CTA per matrix: C64 = D^-1 ((C32 + C32^T) / 2) D^-1 + shift I with D = diag(sqrt(C_ii)).
+// Scaling the columns to unit norm first makes the shift act on every column alike, whatever its
+// norm, so weak directions are still orthogonalised against each other and re-normalised.
+__global__ void __launch_bounds__(256) gram_prep_kernel(const GramPrep* probs) {
+  const GramPrep p = probs[blockIdx.x];
+  for (int i = threadIdx.x; i < p.L; i += 256) {
+    const double c = static_cast<double>(p.C32[static_cast<long long>(i) * p.L + i]);
+    p.D[i] = sqrt(fmax(c, 1e-60));
+  }
+  __syncthreads();
+  const long long total = static_cast<long long>(p.L) * p.L;
+  for (long long x = threadIdx.x; x < total; x += 256) {
+    const int i = static_cast<int>(x / p.L), j = static_cast<int>(x % p.L);
+    if (j > i) continue;
+    double v = 0.5 * (static_cast<double>(p.C32[x]) + static_cast<double>(p.C32[static_cast<long long>(j) * p.L + i]));
+    v /= p.D[i] * p.D[j];
+    if (i == j) v = 1.0 + gram_shift(p.L);
+    p.C64[x] = v;
+  }
+}
+
+struct TriInverse {
+  const double* Lf;      // L x L lower Cholesky factor of the column-scaled Gram matrix (row-major)
+  const double* D;       // L column norms: R^-1 = D^-1 Lf^-T
+  double* X;             // L x L scratch: X = Lf^-1 (lower)
+  __nv_bfloat16* Rhi;    // L x ld: high part of R^-1 = Lf^-T (upper triangular)
+  __nv_bfloat16* Rlo;
+  int L, ld;
+};
+
+// One CTA per matrix, thread j owns column j of X = Lf^-1 (forward substitution on e_j) and writes
+// row j of R^-1 = D^-1 X^T.  All threads walk the same (i, k) sequence, so Lf is read as a broadcast and X
+// with unit stride across the warp; a thread reads only entries of X that it wrote itself.
+__global__ void __launch_bounds__(512) tri_inverse_kernel(const TriInverse* probs) {
+  const TriInverse p = probs[blockIdx.x];
+  const int L = p.L;
+  for (int j = threadIdx.x; j < L; j += blockDim.x) {
+    for (int i = 0; i < L; ++i) {
+      double acc = (i == j) ? 1.0 : 0.0;
+      if (i >= j) {
+        const double* lrow = p.Lf + static_cast<long long>(i) * L;
+        for (int k = j; k < i; ++k) acc -= lrow[k] * p.X[static_cast<long long>(k) * L + j];
+        acc /= lrow[i];
+      } else {
+        acc = 0.0;
+      }
+      p.X[static_cast<long long>(i) * L + j] = acc;
+      const float f = static_cast<float>(fmin(fmax(acc / p.D[j], -1e30), 1e30));
+      const __nv_bfloat16 h = __float2bfloat16_rn(f);
+      p.Rhi[static_cast<long long>(j) * p.ld + i] = h;
+      p.Rlo[static_cast<long long>(j) * p.ld + i] = __float2bfloat16_rn(f - __bfloat162float(h));
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------ plan
+
+enum RefreshGemm { RG_Y_FROM_Z = 0, RG_Z_FROM_Y, RG_GRAM_Y, RG_GRAM_Z, RG_APPLY_Y, RG_APPLY_Z, RG_COUNT };
+enum RefreshMap { RM_G_A = 0, RM_G_MN, RM_Z_B, RM_Z_B_LO, RM_Y_B, RM_Y_B_LO, RM_Y_A, RM_Y_A_LO, RM_Z_A, RM_Z_A_LO,
+                  RM_RINV, RM_RINV_LO, RM_COUNT };
+
+struct RefreshMat {
+  int M, N, L, ldl;
+  float *Yf, *Zf;                       // fp32 GEMM outputs (M x L, N x L)
+  __nv_bfloat16 *Yhi, *Ylo, *Zhi, *Zlo; // bf16 parts of the iterates (rows x ldl)
+  float* C32;                           // L x L
+  double *C64, *X64;                    // L x L each
+  double* D;                            // L
+  __nv_bfloat16 *Rhi, *Rlo;             // L x ldl
+};
+
+constexpr int kRefBN = 128;
+constexpr int kRefStages1 = 4;  // NA = 1, NB = 2: 48 KB per stage
+constexpr int kRefStages2 = 3;  // NA = 2, NB = 2: 64 KB per stage
+
+struct RefreshPlan {
+  bool ready = false;
+  size_t device_bytes = 0;
+  EncodeTiledFn encode = nullptr;
+  int n = 0;
+  std::vector<RefreshMat> mats;
+  std::vector<CUtensorMap> h_maps;  // RM_COUNT per matrix
+  std::vector<const void*> last_G;
+  char* buf = nullptr;
+  CUtensorMap* d_maps = nullptr;
+  TcProblem* d_probs[RG_COUNT] = {};
+  TcTile* d_tiles[RG_COUNT] = {};
+  int n_tiles[RG_COUNT] = {};
+  int grid[RG_COUNT] = {};
+  std::vector<int> atomic_mats[RG_COUNT];  // matrices whose K is split for this GEMM (output must be zeroed)
+  GramPrep* d_prep = nullptr;
+  CholProblem* d_chol = nullptr;
+  TriInverse* d_tri = nullptr;
+};
+
+inline void refresh_plan_destroy(RefreshPlan& plan) {
+  if (plan.buf) cudaFree(plan.buf);
+  plan.buf = nullptr;
+  plan.ready = false;
+}
+
+inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<MatDesc>& mats,
+                                          const std::vector<float*>& Yf, const std::vector<float*>& Zf, int sm_count) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr)
+    return NGALORE_ERR_CUDA;
+  plan.encode = reinterpret_cast<EncodeTiledFn>(fn);
+  const int n = static_cast<int>(mats.size());
+  plan.n = n;
+  plan.mats.resize(n);
+  plan.last_G.assign(n, nullptr);
+
+  // ---- tile and problem tables (host)
+  std::vector<TcProblem> probs[RG_COUNT];
+  std::vector<TcTile> tiles[RG_COUNT];
+  for (int g = 0; g < RG_COUNT; ++g) probs[g].resize(n);
+  auto add_tiles = [&](int g, int i, int out_rows, int out_cols, int K, long long target_kb) {
+    const int kb_total = (K + kTcBK - 1) / kTcBK;
+    int splits = static_cast<int>((kb_total + target_kb - 1) / target_kb);
+    if (splits < 1) splits = 1;
+    const int kb_per = (kb_total + splits - 1) / splits;
+    splits = (kb_total + kb_per - 1) / kb_per;
+    if (splits > 1) plan.atomic_mats[g].push_back(i);
+    for (int n0 = 0; n0 < out_cols; n0 += kRefBN)
+      for (int sp = 0; sp < splits; ++sp)
+        for (int m0 = 0; m0 < out_rows; m0 += kTcBM) {
+          const int kb0 = sp * kb_per;
+          const int kbn = std::min(kb_per, kb_total - kb0);
+          tiles[g].push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0});
+        }
+  };
+
+  // ---- device buffer layout
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) / 256 * 256; return o; };
+  struct Offs { size_t Yhi, Ylo, Zhi, Zlo, C32, C64, X64, D, Rhi, Rlo; };
+  std::vector<Offs> offs(n);
+  for (int i = 0; i < n; ++i) {
+    RefreshMat& m = plan.mats[i];
+    m.M = mats[i].M; m.N = mats[i].N; m.L = mats[i].rp; m.ldl = (m.L + 7) / 8 * 8;
+    m.Yf = Yf[i]; m.Zf = Zf[i];
+    offs[i].Yhi = take(sizeof(__nv_bfloat16) * m.M * m.ldl);
+    offs[i].Ylo = take(sizeof(__nv_bfloat16) * m.M * m.ldl);
+    offs[i].Zhi = take(sizeof(__nv_bfloat16) * m.N * m.ldl);
+    offs[i].Zlo = take(sizeof(__nv_bfloat16) * m.N * m.ldl);
+    offs[i].C32 = take(sizeof(float) * m.L * m.L);
+    offs[i].C64 = take(sizeof(double) * m.L * m.L);
+    offs[i].X64 = take(sizeof(double) * m.L * m.L);
+    offs[i].D = take(sizeof(double) * m.L);
+    offs[i].Rhi = take(sizeof(__nv_bfloat16) * m.L * m.ldl);
+    offs[i].Rlo = take(sizeof(__nv_bfloat16) * m.L * m.ldl);
+  }
+  const size_t o_maps = take(sizeof(CUtensorMap) * RM_COUNT * n);
+  size_t o_probs[RG_COUNT], o_tiles[RG_COUNT];
+
+  // work estimate for the split-K targets: per GEMM kind, k-blocks per CTA if perfectly balanced
+  for (int g = 0; g < RG_COUNT; ++g) {
+    long long total_kb = 0;
+    for (int i = 0; i < n; ++i) {
+      const RefreshMat& m = plan.mats[i];
+      int rows, cols, K;
+      switch (g) {
+        case RG_Y_FROM_Z: rows = m.M; cols = m.L; K = m.N; break;
+        case RG_Z_FROM_Y: rows = m.N; cols = m.L; K = m.M; break;
+        case RG_GRAM_Y: rows = m.L; cols = m.L; K = m.M; break;
+        case RG_GRAM_Z: rows = m.L; cols = m.L; K = m.N; break;
+        case RG_APPLY_Y: rows = m.M; cols = m.L; K = m.L; break;
+        default: rows = m.N; cols = m.L; K = m.L; break;
+      }
+      total_kb += static_cast<long long>((rows + kTcBM - 1) / kTcBM) * ((cols + kRefBN - 1) / kRefBN) *
+                  ((K + kTcBK - 1) / kTcBK);
+    }
+    long long target = (total_kb + sm_count - 1) / sm_count / 4;
+    if (target < 16) target = 16;
+    for (int i = 0; i < n; ++i) {
+      const RefreshMat& m = plan.mats[i];
+      int rows, cols, K;
+      switch (g) {
+        case RG_Y_FROM_Z: rows = m.M; cols = m.L; K = m.N; break;
+        case RG_Z_FROM_Y: rows = m.N; cols = m.L; K = m.M; break;
+        case RG_GRAM_Y: rows = m.L; cols = m.L; K = m.M; break;
+        case RG_GRAM_Z: rows = m.L; cols = m.L; K = m.N; break;
+        case RG_APPLY_Y: rows = m.M; cols = m.L; K = m.L; break;
+        default: rows = m.N; cols = m.L; K = m.L; break;
+      }
+      add_tiles(g, i, rows, cols, K, target);
+    }
+    std::stable_sort(tiles[g].begin(), tiles[g].end(), [](const TcTile& a, const TcTile& b) { return a.kblocks > b.kblocks; });
+    o_probs[g] = take(sizeof(TcProblem) * n);
+    o_tiles[g] = take(sizeof(TcTile) * tiles[g].size());
+    plan.n_tiles[g] = static_cast<int>(tiles[g].size());
+    plan.grid[g] = std::min(plan.n_tiles[g], sm_count);
+  }
+  const size_t o_prep = take(sizeof(GramPrep) * n);
+  const size_t o_chol = take(sizeof(CholProblem) * n);
+  const size_t o_tri = take(sizeof(TriInverse) * n);
+  if (cudaMalloc(&plan.buf, off) != cudaSuccess) { plan.buf = nullptr; return NGALORE_ERR_ALLOC; }
+  if (cudaMemset(plan.buf, 0, off) != cudaSuccess) return NGALORE_ERR_CUDA;
+  plan.device_bytes = off;
+
+  std::vector<GramPrep> prep(n);
+  std::vector<CholProblem> chol(n);
+  std::vector<TriInverse> tri(n);
+  plan.h_maps.resize(static_cast<size_t>(RM_COUNT) * n);
+  std::memset(plan.h_maps.data(), 0, sizeof(CUtensorMap) * plan.h_maps.size());
+  for (int i = 0; i < n; ++i) {
+    RefreshMat& m = plan.mats[i];
+    m.Yhi = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Yhi);
+    m.Ylo = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Ylo);
+    m.Zhi = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Zhi);
+    m.Zlo = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Zlo);
+    m.C32 = reinterpret_cast<float*>(plan.buf + offs[i].C32);
+    m.C64 = reinterpret_cast<double*>(plan.buf + offs[i].C64);
+    m.X64 = reinterpret_cast<double*>(plan.buf + offs[i].X64);
+    m.D = reinterpret_cast<double*>(plan.buf + offs[i].D);
+    m.Rhi = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Rhi);
+    m.Rlo = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Rlo);
+    prep[i] = GramPrep{m.C32, m.C64, m.D, m.L};
+    chol[i] = CholProblem{m.C64, m.L};
+    tri[i] = TriInverse{m.C64, m.D, m.X64, m.Rhi, m.Rlo, m.L, m.ldl};
+    CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * RM_COUNT];
+    const uint64_t sl = static_cast<uint64_t>(m.ldl) * 2;
+    bool ok = true;
+    ok &= tc_encode_2d(plan.encode, mp + RM_Z_B, m.Zhi, m.L, m.N, sl, 64, kTcBK);
+    ok &= tc_encode_2d(plan.encode, mp + RM_Z_B_LO, m.Zlo, m.L, m.N, sl, 64, kTcBK);
+    ok &= tc_encode_2d(plan.encode, mp + RM_Y_B, m.Yhi, m.L, m.M, sl, 64, kTcBK);
+    ok &= tc_encode_2d(plan.encode, mp + RM_Y_B_LO, m.Ylo, m.L, m.M, sl, 64, kTcBK);
+    ok &= tc_encode_2d(plan.encode, mp + RM_Y_A, m.Yhi, m.L, m.M, sl, kTcBK, kTcBM);
+    ok &= tc_encode_2d(plan.encode, mp + RM_Y_A_LO, m.Ylo, m.L, m.M, sl, kTcBK, kTcBM);
+    ok &= tc_encode_2d(plan.encode, mp + RM_Z_A, m.Zhi, m.L, m.N, sl, kTcBK, kTcBM);
+    ok &= tc_encode_2d(plan.encode, mp + RM_Z_A_LO, m.Zlo, m.L, m.N, sl, kTcBK, kTcBM);
+    ok &= tc_encode_2d(plan.encode, mp + RM_RINV, m.Rhi, m.L, m.L, sl, 64, kTcBK);
+    ok &= tc_encode_2d(plan.encode, mp + RM_RINV_LO, m.Rlo, m.L, m.L, sl, 64, kTcBK);
+    if (!ok) return NGALORE_ERR_CUDA;
+    const int base = i * RM_COUNT;
+    probs[RG_Y_FROM_Z][i] = TcProblem{m.Yf, m.M, m.L, m.L, base + RM_G_A, base + RM_Z_B, 0};
+    probs[RG_Z_FROM_Y][i] = TcProblem{m.Zf, m.N, m.L, m.L, base + RM_G_MN, base + RM_Y_B, 0};
+    probs[RG_GRAM_Y][i] = TcProblem{m.C32, m.L, m.L, m.L, base + RM_Y_B, base + RM_Y_B, 0};
+    probs[RG_GRAM_Z][i] = TcProblem{m.C32, m.L, m.L, m.L, base + RM_Z_B, base + RM_Z_B, 0};
+    probs[RG_APPLY_Y][i] = TcProblem{m.Yf, m.M, m.L, m.L, base + RM_Y_A, base + RM_RINV, 0};
+    probs[RG_APPLY_Z][i] = TcProblem{m.Zf, m.N, m.L, m.L, base + RM_Z_A, base + RM_RINV, 0};
+  }
+  plan.d_maps = reinterpret_cast<CUtensorMap*>(plan.buf + o_maps);
+  for (int g = 0; g < RG_COUNT; ++g) {
+    plan.d_probs[g] = reinterpret_cast<TcProblem*>(plan.buf + o_probs[g]);
+    plan.d_tiles[g] = reinterpret_cast<TcTile*>(plan.buf + o_tiles[g]);
+    if (cudaMemcpy(plan.d_probs[g], probs[g].data(), sizeof(TcProblem) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(plan.d_tiles[g], tiles[g].data(), sizeof(TcTile) * tiles[g].size(), cudaMemcpyHostToDevice) != cudaSuccess)
+      return NGALORE_ERR_CUDA;
+  }
+  plan.d_prep = reinterpret_cast<GramPrep*>(plan.buf + o_prep);
+  plan.d_chol = reinterpret_cast<CholProblem*>(plan.buf + o_chol);
+  plan.d_tri = reinterpret_cast<TriInverse*>(plan.buf + o_tri);
+  if (cudaMemcpy(plan.d_prep, prep.data(), sizeof(GramPrep) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_chol, chol.data(), sizeof(CholProblem) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_tri, tri.data(), sizeof(TriInverse) * n, cudaMemcpyHostToDevice) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+
+  using L1 = TcSmem<kRefBN, 1, 2, kRefStages1, 4>;
+  using L2 = TcSmem<kRefBN, 2, 2, kRefStages2, 4>;
+  if (cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, false>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, L1::kTotal) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, true>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, L1::kTotal) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 2, 2, kRefStages2, TC_EPI_STORE, 4, false>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, L2::kTotal) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 2, 2, kRefStages2, TC_EPI_STORE, 4, true>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, L2::kTotal) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  plan.ready = true;
+  return NGALORE_OK;
+}
+
+
+inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
+  // outputs that several K slices accumulate into start from zero
+  for (int i : plan.atomic_mats[g]) {
+    const RefreshMat& m = plan.mats[i];
+    float* out; size_t bytes;
+    switch (g) {
+      case RG_Y_FROM_Z: case RG_APPLY_Y: out = m.Yf; bytes = sizeof(float) * m.M * m.L; break;
+      case RG_Z_FROM_Y: case RG_APPLY_Z: out = m.Zf; bytes = sizeof(float) * m.N * m.L; break;
+      default: out = m.C32; bytes = sizeof(float) * m.L * m.L; break;
+    }
+    if (cudaMemsetAsync(out, 0, bytes, stream) != cudaSuccess) return NGALORE_ERR_CUDA;
+  }
+  using L1 = TcSmem<kRefBN, 1, 2, kRefStages1, 4>;
+  using L2 = TcSmem<kRefBN, 2, 2, kRefStages2, 4>;
+  const int threads = 64 + 32 * 4;
+  switch (g) {
+    case RG_Y_FROM_Z:
+      tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, false><<<plan.grid[g], threads, L1::kTotal, stream>>>(
+          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, nullptr, nullptr, plan.d_probs[g]);
+      break;
+    case RG_Z_FROM_Y:
+      tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, true><<<plan.grid[g], threads, L1::kTotal, stream>>>(
+          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, nullptr, nullptr, plan.d_probs[g]);
+      break;
+    case RG_GRAM_Y:
+    case RG_GRAM_Z:
+      tc_gemm_kernel<kRefBN, 2, 2, kRefStages2, TC_EPI_STORE, 4, true><<<plan.grid[g], threads, L2::kTotal, stream>>>(
+          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, nullptr, nullptr, plan.d_probs[g]);
+      break;
+    default:
+      tc_gemm_kernel<kRefBN, 2, 2, kRefStages2, TC_EPI_STORE, 4, false><<<plan.grid[g], threads, L2::kTotal, stream>>>(
+          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, nullptr, nullptr, plan.d_probs[g]);
+      break;
+  }
+  *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
+}
+
+inline ngalore_status refresh_tc_split(RefreshPlan& plan, bool y_side, cudaStream_t stream, int64_t* launches) {
+  for (const RefreshMat& m : plan.mats) {
+    const long long cnt = static_cast<long long>(y_side ? m.M : m.N) * m.L;
+    split_hilo_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, stream>>>(
+        y_side ? m.Yf : m.Zf, y_side ? m.Yhi : m.Zhi, y_side ? m.Ylo : m.Zlo, cnt, m.L, m.ldl);
+    *launches += 1;
+  }
+  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
+}
+
+// iterate (fp32, in Yf or Zf) -> well-conditioned basis, left both as fp32 and as its bf16 parts.
+inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
+  ngalore_status rc;
+  if ((rc = refresh_tc_split(plan, y_side, stream, launches))) return rc;
+  if ((rc = refresh_tc_gemm(plan, y_side ? RG_GRAM_Y : RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
+  gram_prep_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep);
+  chol_batched_kernel<<<plan.n, 512, 0, stream>>>(plan.d_chol);
+  tri_inverse_kernel<<<plan.n, 512, 0, stream>>>(plan.d_tri);
+  *launches += 3;
+  if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
+  if ((rc = refresh_tc_gemm(plan, y_side ? RG_APPLY_Y : RG_APPLY_Z, d_ctrl, stream, launches))) return rc;
+  return refresh_tc_split(plan, y_side, stream, launches);
+}
+
+// Whole-set refresh up to the last basis, which is left in Yf (fp32, well conditioned, not yet orthonormal).
+inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G, int q, unsigned long long seed,
+                                     unsigned long long stream_base, Ctrl* d_ctrl, cudaStream_t stream,
+                                     int64_t* launches) {
+  bool changed = false;
+  for (int i = 0; i < plan.n; ++i) {
+    if (plan.last_G[i] != G[i]) {
+      plan.last_G[i] = G[i];
+      const RefreshMat& m = plan.mats[i];
+      CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * RM_COUNT];
+      if (!tc_encode_2d(plan.encode, mp + RM_G_A, G[i], m.N, m.M, static_cast<uint64_t>(m.N) * 2, kTcBK, kTcBM) ||
+          !tc_encode_2d(plan.encode, mp + RM_G_MN, G[i], m.N, m.M, static_cast<uint64_t>(m.N) * 2, 64, kTcBK))
+        return NGALORE_ERR_CUDA;
+      changed = true;
+    }
+  }
+  if (changed && cudaMemcpyAsync(plan.d_maps, plan.h_maps.data(), sizeof(CUtensorMap) * plan.h_maps.size(),
+                                 cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  ngalore_status rc;
+  for (int i = 0; i < plan.n; ++i) {
+    const RefreshMat& m = plan.mats[i];
+    const long long cnt = static_cast<long long>(m.N) * m.L;
+    fill_normal_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, stream>>>(m.Zf, cnt, seed,
+                                                                                     stream_base + static_cast<unsigned>(i));
+    *launches += 1;
+  }
+  if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
+  if ((rc = refresh_tc_split(plan, false, stream, launches))) return rc;
+  if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches))) return rc;
+  if ((rc = refresh_tc_orth(plan, true, d_ctrl, stream, launches))) return rc;
+  for (int it = 0; it < q; ++it) {
+    if ((rc = refresh_tc_gemm(plan, RG_Z_FROM_Y, d_ctrl, stream, launches))) return rc;
+    if ((rc = refresh_tc_orth(plan, false, d_ctrl, stream, launches))) return rc;
+    if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches))) return rc;
+    if ((rc = refresh_tc_orth(plan, true, d_ctrl, stream, launches))) return rc;
+  }
+  return NGALORE_OK;
+}
+
+}  // namespace ngalore

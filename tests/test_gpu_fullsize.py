@@ -1,0 +1,57 @@
+"""Full-size parity: the whole matrix set of each Llama-shaped workload runs on the GPU in the launch
+configuration bench.py times (grouped tensor-core GEMMs, fused stream kernel, device-drawn gradients);
+one matrix of every distinct shape is downloaded and stepped by the fp64 oracle with the GPU's own
+working P (matrices are independent units, so the oracle can follow any subset exactly)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import natural_galore as orc
+from paper_2410_16029_b200 import workload as wl
+from tests.parity_util import (TOL_PROJECTOR, TOL_UPDATE, oracle_hyper, projector_distance, rel_err)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("index,steps,svd_shapes", [(1, 10, {(512, 512), (512, 1376), (1376, 512)}),
+                                                     (2, 10, {(768, 768)}),
+                                                     (3, 5, {(1024, 1024)}),
+                                                     (4, 4, {(2048, 256), (2048, 2048)})])
+def test_sampled_matrices_of_full_workload(index, steps, svd_shapes):
+    from paper_2410_16029_b200.ngalore import NGaLore
+
+    w = wl.WORKLOADS[index]
+    dev = torch.device("cuda")
+    shapes = [(M, N) for _, M, N in w.shapes]
+    opt = NGaLore(shapes, w.r, w.s, w.T, lam=w.lam, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, wd=w.wd)
+    sample = [i for i, _, _ in w.distinct_shapes()]
+    states = {i: orc.MatrixState(shapes[i][0], shapes[i][1], oracle_hyper(w)) for i in sample}
+    W = [torch.zeros(s, dtype=torch.float32, device=dev) for s in shapes]
+    worst = 0.0
+    for k in range(steps):
+        G = [wl.gradient_device(w, i, k, dev) for i in range(len(shapes))]
+        for t in W:
+            t.zero_()
+        opt.step(W, G)
+        torch.cuda.synchronize()
+        for i in sample:
+            st = states[i]
+            g64 = wl.bf16_bits_to_f64(wl.torch_bf16_to_bits(G[i]))
+            if k == 0:
+                P16 = opt.get_subspace(i, working=True).cpu().numpy().astype(np.float64)
+                P32 = opt.get_subspace(i).cpu().numpy().astype(np.float64)
+                assert np.max(np.abs(P32.T @ P32 - np.eye(P32.shape[1]))) <= 1e-5
+                assert np.max(np.abs(P16.T @ P16 - np.eye(P16.shape[1]))) <= 5e-3
+                st.set_subspace(P16)
+                if shapes[i] in svd_shapes:
+                    kk, dist = projector_distance(P32, g64, st.rp)
+                    assert kk >= 1
+                    assert dist <= TOL_PROJECTOR, (shapes[i], kk, dist)
+            dW = st.step(np.zeros(shapes[i]), g64, auto_refresh=False)
+            err = rel_err(W[i].cpu().numpy().astype(np.float64), dW)
+            worst = max(worst, err)
+            assert err <= TOL_UPDATE, (index, k, shapes[i], err)
+        del G
+    code, per = opt.poll_status()
+    assert code == 0, (code, [p for p in per if p])
+    print(f"workload {index}: worst relative update error {worst:.2e}")
