@@ -333,6 +333,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--pool", type=int, default=0,
                     help="gradient sets resident in HBM, cycled (default s + 1: no gradient repeats inside the history)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="keep only the first LAYERS transformer layers of the workload (small case for profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
@@ -340,6 +342,8 @@ def main():
     from paper_2410_16029_b200 import workload as W
 
     wl = W.WORKLOADS[args.workload]
+    if args.layers > 0:
+        wl = W.truncated(wl, args.layers)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -285,10 +285,10 @@ ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G, const s
   if ((rc = refresh_tc_run(st->refresh, G, q, st->opt.seed, static_cast<unsigned long long>(st->k) * 65536ull,
                            st->d_ctrl, stream, &st->launches)))
     return rc;
-  // The last basis sits in Ya (fp32, well conditioned): exact orthonormalisation in fp64, Ya -> Yb -> Ya.
+  // The last basis sits in Ya (fp32, well conditioned after the sweeps): one Cholesky QR pass with the Gram
+  // matrix, the factorisation and the triangular solve in fp64 makes it orthonormal to fp32 accuracy: Ya -> Yb.
   if ((rc = orthonormalise(st, idx, 0, true, stream))) return rc;
-  if ((rc = orthonormalise(st, idx, 0, false, stream))) return rc;
-  return finish_refresh(st, idx, true, stream);
+  return finish_refresh(st, idx, false, stream);
 }
 
 ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream) {

@@ -103,6 +103,14 @@ WORKLOADS = {
 }
 
 
+def truncated(wl: "Workload", layers: int) -> "Workload":
+    """The same workload with only its first `layers` transformer layers (embedding and lm_head kept):
+    a small case with the full-size shapes, for profiler captures."""
+    keep = tuple(sh for sh in wl.shapes if not sh[0].startswith("l") or sh[0] == "lm_head"
+                 or int(sh[0][1:].split(".")[0]) < layers)
+    return dataclasses.replace(wl, name=f"{wl.name}[{layers} layers]", shapes=keep)
+
+
 def tiny_workload(shapes, r, s, T, generator="lowrank_noise", inner_rank=4, index=90, **kw) -> Workload:
     """A small ad-hoc workload for tests; same recipes, caller-chosen shapes."""
     shp = tuple((f"t{i}", int(M), int(N)) for i, (M, N) in enumerate(shapes))
