@@ -31,6 +31,7 @@ struct MatDesc {
   int* gram_done;             // fused kernel: count of finished Gram tiles of this step
   int* w_ready;               // fused kernel: set to the step epoch once wsol is valid
   int tile0, ntiles;          // range of streaming tiles owned by this matrix
+  int te;                     // elements of one streaming tile of this matrix (multiple of 1024)
 };
 
 struct Ctrl {

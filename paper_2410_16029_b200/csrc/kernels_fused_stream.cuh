@@ -1,18 +1,26 @@
 // One persistent kernel for the whole history phase of a step: the Gram row of every matrix,
 // the s x s solves, and the natural-gradient combination with the Adam moments (Sec. 2.4, 2.2).
 //
-// Work items are fetched in order from a global counter.  Gram items never wait; the CTA that
-// finishes a matrix's last Gram tile solves its s x s system and publishes the weights; combination
-// items wait (bounded) for that flag.  Every item a combination item depends on sits earlier in
-// the list and has therefore been fetched by a running CTA, so the kernel cannot deadlock whatever
-// the grid size.  The list interleaves matrices so that the combination pass of a matrix starts
-// while its history is still in L2 and the wait is hidden behind the next matrix's Gram tiles.
+// Structure: one CTA per SM; a producer warp streams the history (and m, v) through a ring of
+// shared-memory stages with bulk asynchronous copies (cp.async.bulk + mbarrier), eight consumer
+// warps compute from shared memory.  The producer runs ahead of the consumers across tile and
+// matrix boundaries, so the SM always has several stages of loads in flight.
+//
+// Work items (Gram tiles and combination tiles of all matrices) are fetched in order from a global
+// counter by the producer.  Gram items never wait; the CTA that finishes a matrix's last Gram tile
+// solves its s x s system and publishes the weights; the consumers of a combination item wait
+// (bounded) for that flag.  Every item a combination item depends on sits earlier in the list and
+// has been fetched by a CTA that consumes its items in order, so the kernel cannot deadlock.
+// Tiles are small enough that all SMs sweep one matrix together; its combination pass then runs in
+// reverse order right behind its Gram pass, while part of the history is still in L2.
 #pragma once
 
+#include <cstdlib>
 #include <vector>
 
 #include "../../include/ngalore.h"
 #include "common.cuh"
+#include "gemm_tcgen05.cuh"  // mbarrier wrappers
 #include "kernels_stream.cuh"
 
 namespace ngalore {
@@ -28,80 +36,292 @@ struct FusedPlan {
   FusedItem* d_items = nullptr;
   int n_items = 0;
   int grid = 0;
-  int tile_elems = 0;
 };
 
-constexpr long long kSpinLimit = 4000000;  // polls of ~100 ns each before a wait is abandoned
+constexpr long long kSpinLimit = 4000000;  // polls of ~100 ns each before a flag wait is abandoned
+constexpr int kConsumerThreads = 256;
+constexpr int kFusedThreads = kConsumerThreads + 32;
+
+struct StageMeta {
+  int mat, kind, local, first, last, count;
+  long long e0;
+};
 
 template <int SMAX>
-__global__ void __launch_bounds__(kStreamThreads, 2)
+struct FusedCfg {
+  static constexpr int CE = SMAX <= 16 ? 1024 : 512;  // elements per stage and slot
+  static constexpr int kSlots = SMAX + 2;             // history slots + m + v
+  static constexpr int kStageBytes = kSlots * CE * 4;
+  static constexpr int kStages = SMAX <= 8 ? 5 : 3;
+  static constexpr int kBase = kStages * kStageBytes;
+  static constexpr int kFullOff = kBase, kEmptyOff = kBase + 64, kMetaOff = kBase + 128, kFlagOff = kBase + 384;
+  static constexpr int kWOff = kBase + 512, kRedOff = kBase + 640;
+  static constexpr int kAOff = kRedOff + (kConsumerThreads / 32) * SMAX * 8;
+  static constexpr int kTotal = kAOff + kMaxHistory * (kMaxHistory + 1) * 8;
+  static_assert(kStages * sizeof(StageMeta) <= 256, "stage metadata overflows its slot");
+  static_assert(kTotal <= 232448, "shared memory budget of one CTA exceeded");
+};
+
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void consumer_sync() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+}
+
+template <int SMAX>
+__global__ void __launch_bounds__(kFusedThreads, 1)
 fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restrict__ items, int n_items, Ctrl* ctrl,
-                    const Hyper* __restrict__ hyper, int tile_elems) {
-  __shared__ double red[(kStreamThreads / 32) * SMAX];
-  __shared__ double A[kMaxHistory * (kMaxHistory + 1)];
-  __shared__ float wsm[kMaxHistory];
-  __shared__ int s_item, s_flag;
+                    const Hyper* __restrict__ hyper) {
+  using C = FusedCfg<SMAX>;
+  constexpr int CE = C::CE;
+  constexpr int VEC = CE / kConsumerThreads;  // 4 or 2 elements per thread and stage
+  extern __shared__ __align__(128) unsigned char fs_smem[];
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(fs_smem + C::kFullOff);
+  uint64_t* empty_bar = reinterpret_cast<uint64_t*>(fs_smem + C::kEmptyOff);
+  StageMeta* meta = reinterpret_cast<StageMeta*>(fs_smem + C::kMetaOff);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(fs_smem + C::kFlagOff);
+  volatile int* s_flag = abort_flag + 1;
+  float* wsm = reinterpret_cast<float*>(fs_smem + C::kWOff);
+  double* red = reinterpret_cast<double*>(fs_smem + C::kRedOff);
+  double* Amat = reinterpret_cast<double*>(fs_smem + C::kAOff);
+
   const int tid = threadIdx.x;
-  const int tag = ctrl->epoch + 1;
-  const Hyper hp = *hyper;
-  while (true) {
-    if (tid == 0) s_item = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
-    __syncthreads();
-    const int it = s_item;
-    __syncthreads();
-    if (it >= n_items) break;
-    const FusedItem item = items[it];
-    const MatDesc& d = mats[item.mat];
-    const int cur = ring_cur(ctrl, d.s), c = ring_count(ctrl, d.s);
-    if (item.kind == 0) {
-      gram_tile<SMAX>(d, item.local, cur, c, tile_elems, red);
-      if (tid == 0) {
-        __threadfence();
-        const int done = atomicAdd(d.gram_done, 1);
-        s_flag = (done == d.ntiles - 1) ? 1 : 0;
-      }
-      __syncthreads();
-      if (s_flag && tid < 32) {
-        __threadfence();
-        solve_matrix(d, cur, c, hp.lambda, A);
-        if (tid == 0) {
-          *d.gram_done = 0;
-          __threadfence();
-          atomicExch(d.w_ready, tag);
-        }
-      }
-      __syncthreads();
-    } else {
-      if (d.s > 0) {
-        if (tid == 0) {
-          const volatile int* flag = d.w_ready;
-          long long spins = 0;
-          int ok = 1;
-          while (*flag != tag) {
-            if (++spins > kSpinLimit) { ok = 0; break; }
-            __nanosleep(100);
-          }
-          if (!ok) atomicExch(&ctrl->timeout_flag, 1);
-          s_flag = ok;
-        }
-        __syncthreads();
-        const int ok = s_flag;
-        __syncthreads();
-        if (!ok) continue;
-        __threadfence();
-      }
-      if (tid < kMaxHistory) wsm[tid] = __ldcg(d.wsol + tid);
-      __syncthreads();
-      combine_tile<SMAX>(d, item.local, cur, c, tile_elems, hp, wsm);
-      __syncthreads();
+  if (tid == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(full_bar + s, 1);
+      mbar_init(empty_bar + s, kConsumerThreads / 32);
     }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  const int tag = ctrl->epoch + 1;
+
+  if (tid >= kConsumerThreads) {
+    // ------------------------------------------------------------------ producer (one elected thread)
+    if (tid == kConsumerThreads) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      while (ok) {
+        const int it = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
+        if (it >= n_items) {
+          if (mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) {
+            meta[stage].kind = -1;
+            mbar_arrive(full_bar + stage);
+          }
+          break;
+        }
+        const FusedItem item = items[it];
+        const MatDesc& d = mats[item.mat];
+        const int c = ring_count(ctrl, d.s);
+        const long long e0 = static_cast<long long>(item.local) * d.te;
+        const long long e1 = (e0 + d.te < d.rn) ? e0 + d.te : d.rn;
+        for (long long e = e0; e < e1; e += CE) {
+          const int cnt = (e1 - e < CE) ? static_cast<int>(e1 - e) : CE;
+          if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          StageMeta mt;
+          mt.mat = item.mat; mt.kind = item.kind; mt.local = item.local;
+          mt.first = (e == e0) ? 1 : 0; mt.last = (e + CE >= e1) ? 1 : 0; mt.count = cnt; mt.e0 = e;
+          meta[stage] = mt;
+          unsigned char* sb = fs_smem + stage * C::kStageBytes;
+          const uint32_t bytes = static_cast<uint32_t>(cnt) * 4u;
+          mbar_expect_tx(full_bar + stage, bytes * static_cast<uint32_t>(c + (item.kind == 1 ? 2 : 0)));
+          for (int j = 0; j < c; ++j)
+            bulk_load(sb + j * CE * 4, d.H + static_cast<long long>(j) * d.rn + e, bytes, full_bar + stage);
+          if (item.kind == 1) {
+            bulk_load(sb + SMAX * CE * 4, d.m + e, bytes, full_bar + stage);
+            bulk_load(sb + (SMAX + 1) * CE * 4, d.v + e, bytes, full_bar + stage);
+          }
+          if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ consumers (256 threads)
+    const int warp = tid >> 5, lane = tid & 31;
+    const Hyper hp = *hyper;
+    int stage = 0;
+    uint32_t phase = 0;
+    float acc[SMAX];
+    float w[SMAX];
+#pragma unroll
+    for (int j = 0; j < SMAX; ++j) { acc[j] = 0.f; w[j] = 0.f; }
+    bool item_bad = false, item_ok = true;
+    while (true) {
+      if (!mbar_wait(full_bar + stage, phase, abort_flag)) break;
+      const StageMeta mt = meta[stage];
+      if (mt.kind < 0) break;
+      const MatDesc& d = mats[mt.mat];
+      const int cur = ring_cur(ctrl, d.s), c = ring_count(ctrl, d.s);
+      const float* sb = reinterpret_cast<const float*>(fs_smem + stage * C::kStageBytes);
+      const int idx = tid * VEC;
+      if (mt.kind == 0) {
+        if (mt.first) {
+#pragma unroll
+          for (int j = 0; j < SMAX; ++j) acc[j] = 0.f;
+        }
+        if (idx < mt.count) {
+          float x[VEC];
+#pragma unroll
+          for (int q = 0; q < VEC; ++q) x[q] = sb[cur * CE + idx + q];
+#pragma unroll
+          for (int j = 0; j < SMAX; ++j) {
+            if (j < c) {
+              float t = 0.f;
+#pragma unroll
+              for (int q = 0; q < VEC; ++q) t += x[q] * sb[j * CE + idx + q];
+              acc[j] += t;
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar + stage);
+        if (mt.last) {
+#pragma unroll
+          for (int j = 0; j < SMAX; ++j) {
+            const double t = warp_sum(static_cast<double>(acc[j]));
+            if (lane == 0) red[warp * SMAX + j] = t;
+          }
+          consumer_sync();
+          if (tid < SMAX && tid < d.s) {
+            double t = 0.0;
+#pragma unroll
+            for (int ww = 0; ww < kConsumerThreads / 32; ++ww) t += red[ww * SMAX + tid];
+            d.gpart[static_cast<long long>(mt.local) * d.s + tid] = t;
+            __threadfence();
+          }
+          consumer_sync();
+          if (tid == 0) {
+            const int done = atomicAdd(d.gram_done, 1);
+            *s_flag = (done == d.ntiles - 1) ? 1 : 0;
+          }
+          consumer_sync();
+          if (*s_flag) {
+            // last Gram tile of this matrix: all consumers pre-sum the per-tile partials (fixed partition,
+            // so the result is reproducible), then one warp factors and solves
+            __threadfence();
+            const int j = tid & 31, g = tid >> 5;
+            if (j < SMAX) {
+              double t0 = 0.0, t1 = 0.0;
+              if (j < d.s) {
+                int t = g;
+                for (; t + 8 < d.ntiles; t += 16) {
+                  t0 += __ldcg(d.gpart + static_cast<long long>(t) * d.s + j);
+                  t1 += __ldcg(d.gpart + static_cast<long long>(t + 8) * d.s + j);
+                }
+                if (t < d.ntiles) t0 += __ldcg(d.gpart + static_cast<long long>(t) * d.s + j);
+              }
+              red[g * SMAX + j] = t0 + t1;
+            }
+            consumer_sync();
+            if (tid < 32) {
+              solve_matrix(d, cur, c, hp.lambda, Amat, red, kConsumerThreads / 32, SMAX);
+              if (tid == 0) {
+                *d.gram_done = 0;
+                __threadfence();
+                atomicExch(d.w_ready, tag);
+              }
+            }
+          }
+          consumer_sync();
+        }
+      } else {
+        if (mt.first) {
+          item_ok = true;
+          if (d.s > 0) {
+            if (tid == 0) {
+              const volatile int* flag = d.w_ready;
+              long long spins = 0;
+              int ok = 1;
+              while (*flag != tag) {
+                if (++spins > kSpinLimit) { ok = 0; break; }
+                __nanosleep(100);
+              }
+              if (!ok) atomicExch(&ctrl->timeout_flag, 1);
+              *s_flag = ok;
+            }
+            consumer_sync();
+            item_ok = *s_flag != 0;
+            __threadfence();
+          }
+          if (tid < kMaxHistory) wsm[tid] = __ldcg(d.wsol + tid);
+          item_bad = __ldcg(d.step_bad) != 0;
+          consumer_sync();
+#pragma unroll
+          for (int j = 0; j < SMAX; ++j) w[j] = wsm[j];
+        }
+        if (item_ok && idx < mt.count) {
+          const long long e = mt.e0 + idx;
+          if (item_bad) {
+            // The poisoned slot becomes a zero gradient; m, v are left alone and the update is zero.
+            float* Hc = d.H + static_cast<long long>(cur) * d.rn + e;
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) {
+              Hc[q] = 0.f;
+              d.u_hi[e + q] = __float2bfloat16_rn(0.f);
+              d.u_lo[e + q] = __float2bfloat16_rn(0.f);
+            }
+          } else {
+            float n[VEC], mm[VEC], vv[VEC], uu[VEC];
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) n[q] = 0.f;
+#pragma unroll
+            for (int j = 0; j < SMAX; ++j) {
+              if (j < c) {
+#pragma unroll
+                for (int q = 0; q < VEC; ++q) n[q] = fmaf(w[j], sb[j * CE + idx + q], n[q]);
+              }
+            }
+#pragma unroll
+            for (int q = 0; q < VEC; ++q) {
+              mm[q] = hp.beta1 * sb[SMAX * CE + idx + q] + (1.f - hp.beta1) * n[q];
+              vv[q] = hp.beta2 * sb[(SMAX + 1) * CE + idx + q] + (1.f - hp.beta2) * n[q] * n[q];
+              uu[q] = mm[q] / sqrtf(vv[q] + hp.eps);
+            }
+            if (VEC == 4) {
+              *reinterpret_cast<float4*>(d.m + e) = make_float4(mm[0], mm[1], mm[2 % VEC], mm[3 % VEC]);
+              *reinterpret_cast<float4*>(d.v + e) = make_float4(vv[0], vv[1], vv[2 % VEC], vv[3 % VEC]);
+              const uint2 hi = pack_bf16x4(uu[0], uu[1], uu[2 % VEC], uu[3 % VEC]);
+              const __nv_bfloat162 h01 = *reinterpret_cast<const __nv_bfloat162*>(&hi.x);
+              const __nv_bfloat162 h23 = *reinterpret_cast<const __nv_bfloat162*>(&hi.y);
+              const uint2 lo = pack_bf16x4(uu[0] - __low2float(h01), uu[1] - __high2float(h01),
+                                           uu[2 % VEC] - __low2float(h23), uu[3 % VEC] - __high2float(h23));
+              *reinterpret_cast<uint2*>(d.u_hi + e) = hi;
+              *reinterpret_cast<uint2*>(d.u_lo + e) = lo;
+            } else {
+              *reinterpret_cast<float2*>(d.m + e) = make_float2(mm[0], mm[1]);
+              *reinterpret_cast<float2*>(d.v + e) = make_float2(vv[0], vv[1]);
+              const __nv_bfloat162 h = __floats2bfloat162_rn(uu[0], uu[1]);
+              const __nv_bfloat162 l = __floats2bfloat162_rn(uu[0] - __low2float(h), uu[1] - __high2float(h));
+              *reinterpret_cast<__nv_bfloat162*>(d.u_hi + e) = h;
+              *reinterpret_cast<__nv_bfloat162*>(d.u_lo + e) = l;
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar + stage);
+      }
+      if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
+    }
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    // a wait ran out: give bulk copies that may still be in flight time to land before the CTA retires
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    if (tid == 0) atomicExch(&ctrl->timeout_flag, 1);
   }
 }
 
-inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDesc>& mats, int tile_elems, int sm_count) {
-  plan.tile_elems = tile_elems;
-  plan.grid = sm_count * 2;
-  const int head = plan.grid * 2;  // Gram tiles of the next matrix issued before a matrix's combination pass
+inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDesc>& mats, int s, int sm_count) {
+  plan.grid = sm_count;
+  int head = plan.grid * 2;  // Gram tiles of the next matrix issued before a matrix's combination pass
+  if (const char* e = getenv("NGALORE_HEAD")) head = atoi(e);  // TUNING-ONLY
   std::vector<FusedItem> items;
   const int n = static_cast<int>(mats.size());
   auto gram_range = [&](int i, int t0, int t1) {
@@ -131,7 +351,14 @@ inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDe
   }
   if (cudaMemcpy(plan.d_items, items.data(), sizeof(FusedItem) * items.size(), cudaMemcpyHostToDevice) != cudaSuccess)
     return NGALORE_ERR_CUDA;
-  return NGALORE_OK;
+  cudaError_t e;
+  if (s <= 8)
+    e = cudaFuncSetAttribute(fused_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedCfg<8>::kTotal);
+  else if (s <= 16)
+    e = cudaFuncSetAttribute(fused_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedCfg<16>::kTotal);
+  else
+    e = cudaFuncSetAttribute(fused_stream_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedCfg<32>::kTotal);
+  return e == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
 inline void fused_plan_destroy(FusedPlan& plan) {
@@ -142,11 +369,11 @@ inline void fused_plan_destroy(FusedPlan& plan) {
 inline ngalore_status fused_stream_launch(FusedPlan& plan, const MatDesc* d_mats, int /*n_mats*/, Ctrl* d_ctrl,
                                           const Hyper* d_hyper, int s, cudaStream_t stream, int64_t* launches) {
   if (s <= 8)
-    fused_stream_kernel<8><<<plan.grid, kStreamThreads, 0, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper, plan.tile_elems);
+    fused_stream_kernel<8><<<plan.grid, kFusedThreads, FusedCfg<8>::kTotal, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper);
   else if (s <= 16)
-    fused_stream_kernel<16><<<plan.grid, kStreamThreads, 0, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper, plan.tile_elems);
+    fused_stream_kernel<16><<<plan.grid, kFusedThreads, FusedCfg<16>::kTotal, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper);
   else
-    fused_stream_kernel<32><<<plan.grid, kStreamThreads, 0, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper, plan.tile_elems);
+    fused_stream_kernel<32><<<plan.grid, kFusedThreads, FusedCfg<32>::kTotal, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }

@@ -62,7 +62,10 @@ __device__ __forceinline__ void gram_tile(const MatDesc& d, int local, int cur, 
 // current gradient by the Woodbury identity, written for the case where the current gradient is a
 // column of the stacked matrix; it avoids the cancellation of the two-term form.
 // A is warp-private shared memory of kMaxHistory x (kMaxHistory + 1) doubles.
-__device__ __forceinline__ void solve_matrix(const MatDesc& d, int cur, int c, double lambda, double* A) {
+// presum (optional, shared memory): groups x stride partial sums of the Gram row, already reduced over
+// disjoint subsets of the tiles by the caller.
+__device__ __forceinline__ void solve_matrix(const MatDesc& d, int cur, int c, double lambda, double* A,
+                                             const double* presum = nullptr, int groups = 0, int stride = 0) {
   const int lane = threadIdx.x & 31;
   constexpr int LD = kMaxHistory + 1;
   bool finite = true;
@@ -70,7 +73,11 @@ __device__ __forceinline__ void solve_matrix(const MatDesc& d, int cur, int c, d
   if (d.s > 0) {
     double row = 0.0;
     if (lane < c) {
-      for (int t = 0; t < d.ntiles; ++t) row += __ldcg(d.gpart + static_cast<long long>(t) * d.s + lane);
+      if (presum != nullptr) {
+        for (int g = 0; g < groups; ++g) row += presum[g * stride + lane];
+      } else {
+        for (int t = 0; t < d.ntiles; ++t) row += __ldcg(d.gpart + static_cast<long long>(t) * d.s + lane);
+      }
       if (!isfinite(row)) finite = false;
     }
     finite = __all_sync(0xffffffffu, finite);
@@ -207,12 +214,12 @@ __device__ __forceinline__ void combine_tile(const MatDesc& d, int local, int cu
 
 template <int SMAX>
 __global__ void __launch_bounds__(kStreamThreads) gram_kernel(const MatDesc* mats, const StreamTile* tiles,
-                                                              const Ctrl* ctrl, int tile_elems) {
+                                                              const Ctrl* ctrl) {
   __shared__ double red[(kStreamThreads / 32) * SMAX];
   const StreamTile t = tiles[blockIdx.x];
   const MatDesc& d = mats[t.mat];
   if (d.s == 0) return;
-  gram_tile<SMAX>(d, t.local, ring_cur(ctrl, d.s), ring_count(ctrl, d.s), tile_elems, red);
+  gram_tile<SMAX>(d, t.local, ring_cur(ctrl, d.s), ring_count(ctrl, d.s), d.te, red);
 }
 
 __global__ void __launch_bounds__(128) solve_kernel(const MatDesc* mats, int n_mats, const Ctrl* ctrl,
@@ -228,14 +235,13 @@ __global__ void __launch_bounds__(128) solve_kernel(const MatDesc* mats, int n_m
 
 template <int SMAX>
 __global__ void __launch_bounds__(kStreamThreads) combine_kernel(const MatDesc* mats, const StreamTile* tiles,
-                                                                 const Ctrl* ctrl, const Hyper* hyper,
-                                                                 int tile_elems) {
+                                                                 const Ctrl* ctrl, const Hyper* hyper) {
   __shared__ float wsm[kMaxHistory];
   const StreamTile t = tiles[blockIdx.x];
   const MatDesc& d = mats[t.mat];
   if (threadIdx.x < kMaxHistory) wsm[threadIdx.x] = d.wsol[threadIdx.x];
   __syncthreads();
-  combine_tile<SMAX>(d, t.local, ring_cur(ctrl, d.s), ring_count(ctrl, d.s), tile_elems, *hyper, wsm);
+  combine_tile<SMAX>(d, t.local, ring_cur(ctrl, d.s), ring_count(ctrl, d.s), d.te, *hyper, wsm);
 }
 
 __global__ void advance_kernel(Ctrl* ctrl) {

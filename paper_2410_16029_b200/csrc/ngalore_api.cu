@@ -6,6 +6,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <cstdlib>
 #include <new>
 #include <vector>
 
@@ -63,7 +64,7 @@ struct ngalore_state {
   int* d_status = nullptr;
   int* d_step_bad = nullptr;
   StreamTile* d_tiles = nullptr;
-  int n_tiles = 0, tile_elems = 0;
+  int n_tiles = 0;
   float** d_W = nullptr;
   const __nv_bfloat16** d_G = nullptr;
   std::vector<const void*> last_W, last_G;
@@ -114,12 +115,11 @@ struct DeviceGuard {
 template <int SMAX>
 void launch_plain_stream(ngalore_state* st, cudaStream_t stream) {
   if (st->s > 0) {
-    gram_kernel<SMAX><<<st->n_tiles, kStreamThreads, 0, stream>>>(st->d_desc, st->d_tiles, st->d_ctrl, st->tile_elems);
+    gram_kernel<SMAX><<<st->n_tiles, kStreamThreads, 0, stream>>>(st->d_desc, st->d_tiles, st->d_ctrl);
     solve_kernel<<<(st->n + 3) / 4, 128, 0, stream>>>(st->d_desc, st->n, st->d_ctrl, st->d_hyper);
     st->launches += 2;
   }
-  combine_kernel<SMAX><<<st->n_tiles, kStreamThreads, 0, stream>>>(st->d_desc, st->d_tiles, st->d_ctrl, st->d_hyper,
-                                                                   st->tile_elems);
+  combine_kernel<SMAX><<<st->n_tiles, kStreamThreads, 0, stream>>>(st->d_desc, st->d_tiles, st->d_ctrl, st->d_hyper);
   st->launches += 1;
 }
 
@@ -416,25 +416,26 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   st->opt.struct_size = sizeof(ngalore_options);
   if (st->opt.seed == 0) st->opt.seed = 0x9E3779B97F4A7C15ull;
 
-  // ---- streaming tile size: large tiles amortise the per-item latency of the persistent kernel (measured:
-  // 32768 elements is 12 % faster than 8192 on the 1.1B shapes); shrink only to keep ~8 tiles per SM
-  long long total_rn = 0;
-  st->mats.resize(n_matrices);
+  // ---- streaming tile size, per matrix: small enough that every SM works on the same matrix at the same time
+  // (at least two tiles per SM), so that the second pass over a matrix's history finds part of it in L2.
   uint64_t hash = 1469598103934665603ull;
+  st->mats.resize(n_matrices);
+  std::vector<int> tile_elems(n_matrices);
   for (int i = 0; i < n_matrices; ++i) {
     HostMat& hm = st->mats[i];
     hm.M = static_cast<int>(shapes[i].rows); hm.N = static_cast<int>(shapes[i].cols);
     hm.rp = r < hm.M ? r : hm.M;
     if (hm.N < hm.rp) hm.rp = hm.N;
     hm.rn = static_cast<long long>(hm.rp) * hm.N;
-    total_rn += hm.rn;
     hash = (hash ^ static_cast<uint64_t>(hm.M)) * 1099511628211ull;
     hash = (hash ^ static_cast<uint64_t>(hm.N)) * 1099511628211ull;
+    long long te = hm.rn / (2ll * prop.multiProcessorCount) / 1024 * 1024;
+    if (const char* e = getenv("NGALORE_TE")) te = atoi(e);  // TUNING-ONLY
+    if (te < 1024) te = 1024;
+    if (te > 32768) te = 32768;
+    tile_elems[i] = static_cast<int>(te);
   }
   st->shape_hash = hash;
-  int te = 32768;
-  while (te > 2048 && total_rn / te < static_cast<long long>(prop.multiProcessorCount) * 8) te >>= 1;
-  st->tile_elems = te;
 
   // ---- arena layout
   const int slots = s > 0 ? s : 1;
@@ -473,6 +474,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   std::vector<int> tile0(n_matrices), ntl(n_matrices);
   for (int i = 0; i < n_matrices; ++i) {
     const HostMat& hm = st->mats[i];
+    const int te = tile_elems[i];
     ntl[i] = static_cast<int>((hm.rn + te - 1) / te);
     tile0[i] = n_tiles;
     for (int t = 0; t < ntl[i]; ++t) tiles.push_back(StreamTile{i, t});
@@ -534,7 +536,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     d.step_bad = st->d_step_bad + i;
     d.gram_done = flags + 2 * i;
     d.w_ready = flags + 2 * i + 1;
-    d.tile0 = tile0[i]; d.ntiles = ntl[i];
+    d.tile0 = tile0[i]; d.ntiles = ntl[i]; d.te = tile_elems[i];
     hm.Ya = reinterpret_cast<float*>(st->work + woffs[i].Ya);
     hm.Yb = reinterpret_cast<float*>(st->work + woffs[i].Yb);
     hm.Xa = reinterpret_cast<float*>(st->work + woffs[i].Xa);
@@ -563,7 +565,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
 
   ngalore_status rc = tc_plan_create(st->tc, st->h_desc, st->d_desc, s, prop.multiProcessorCount);
   if (rc != NGALORE_OK) return fail(rc);
-  rc = fused_plan_create(st->fused, st->h_desc, st->tile_elems, prop.multiProcessorCount);
+  rc = fused_plan_create(st->fused, st->h_desc, s, prop.multiProcessorCount);
   if (rc != NGALORE_OK) return fail(rc);
   if (st->opt.gemm_impl != 1) {
     std::vector<float*> Yf(n_matrices), Zf(n_matrices);
