@@ -56,7 +56,8 @@ struct FusedCfg {
   static constexpr int kBase = kStages * kStageBytes;
   static constexpr int kFullOff = kBase, kEmptyOff = kBase + 64, kMetaOff = kBase + 128, kFlagOff = kBase + 384;
   static constexpr int kWOff = kBase + 512, kRedOff = kBase + 640;
-  static constexpr int kAOff = kRedOff + (kConsumerThreads / 32) * SMAX * 8;
+  static constexpr int kAOff = kRedOff + 2 * (kConsumerThreads / 32) * SMAX * 8;  // red is double-buffered
+  static constexpr int kPreOff = kAOff;  // the pre-summed Gram row is consumed before the solve fills its matrix
   static constexpr int kTotal = kAOff + kMaxHistory * (kMaxHistory + 1) * 8;
   static_assert(kStages * sizeof(StageMeta) <= 256, "stage metadata overflows its slot");
   static_assert(kTotal <= 232448, "shared memory budget of one CTA exceeded");
@@ -87,6 +88,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
   volatile int* s_flag = abort_flag + 1;
   float* wsm = reinterpret_cast<float*>(fs_smem + C::kWOff);
   double* red = reinterpret_cast<double*>(fs_smem + C::kRedOff);
+  double* presum = reinterpret_cast<double*>(fs_smem + C::kPreOff);
   double* Amat = reinterpret_cast<double*>(fs_smem + C::kAOff);
 
   const int tid = threadIdx.x;
@@ -153,6 +155,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
 #pragma unroll
     for (int j = 0; j < SMAX; ++j) { acc[j] = 0.f; w[j] = 0.f; }
     bool item_bad = false, item_ok = true;
+    int red_buf = 0;
     while (true) {
       if (!mbar_wait(full_bar + stage, phase, abort_flag)) break;
       const StageMeta mt = meta[stage];
@@ -183,53 +186,56 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar + stage);
         if (mt.last) {
+          // End of a Gram tile.  Every warp leaves its partial sums in shared memory and moves on; warp 0
+          // alone finishes the tile (fixed summation order), publishes it and, if it was the matrix's
+          // last tile, solves the s x s system.  `red` is double-buffered because warp 0 may still be
+          // reading one half while the other warps reach the end of the next tile.
+          double* redb = red + red_buf * (kConsumerThreads / 32) * SMAX;
+          red_buf ^= 1;
 #pragma unroll
           for (int j = 0; j < SMAX; ++j) {
             const double t = warp_sum(static_cast<double>(acc[j]));
-            if (lane == 0) red[warp * SMAX + j] = t;
+            if (lane == 0) redb[warp * SMAX + j] = t;
           }
           consumer_sync();
-          if (tid < SMAX && tid < d.s) {
-            double t = 0.0;
+          if (warp == 0) {
+            if (lane < SMAX && lane < d.s) {
+              double t = 0.0;
 #pragma unroll
-            for (int ww = 0; ww < kConsumerThreads / 32; ++ww) t += red[ww * SMAX + tid];
-            d.gpart[static_cast<long long>(mt.local) * d.s + tid] = t;
-            __threadfence();
-          }
-          consumer_sync();
-          if (tid == 0) {
-            const int done = atomicAdd(d.gram_done, 1);
-            *s_flag = (done == d.ntiles - 1) ? 1 : 0;
-          }
-          consumer_sync();
-          if (*s_flag) {
-            // last Gram tile of this matrix: all consumers pre-sum the per-tile partials (fixed partition,
-            // so the result is reproducible), then one warp factors and solves
-            __threadfence();
-            const int j = tid & 31, g = tid >> 5;
-            if (j < SMAX) {
-              double t0 = 0.0, t1 = 0.0;
-              if (j < d.s) {
-                int t = g;
-                for (; t + 8 < d.ntiles; t += 16) {
-                  t0 += __ldcg(d.gpart + static_cast<long long>(t) * d.s + j);
-                  t1 += __ldcg(d.gpart + static_cast<long long>(t + 8) * d.s + j);
-                }
-                if (t < d.ntiles) t0 += __ldcg(d.gpart + static_cast<long long>(t) * d.s + j);
-              }
-              red[g * SMAX + j] = t0 + t1;
+              for (int ww = 0; ww < kConsumerThreads / 32; ++ww) t += redb[ww * SMAX + lane];
+              d.gpart[static_cast<long long>(mt.local) * d.s + lane] = t;
+              __threadfence();
             }
-            consumer_sync();
-            if (tid < 32) {
-              solve_matrix(d, cur, c, hp.lambda, Amat, red, kConsumerThreads / 32, SMAX);
-              if (tid == 0) {
+            __syncwarp();
+            int done = 0;
+            if (lane == 0) done = atomicAdd(d.gram_done, 1);
+            done = __shfl_sync(0xffffffffu, done, 0);
+            if (done == d.ntiles - 1) {
+              __threadfence();
+              // pre-sum the per-tile partials: lane j owns column j, eight loads in flight
+              double tsum = 0.0;
+              if (lane < d.s) {
+                double p[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) p[q] = 0.0;
+                int t = 0;
+                for (; t + 8 <= d.ntiles; t += 8) {
+#pragma unroll
+                  for (int q = 0; q < 8; ++q) p[q] += __ldcg(d.gpart + static_cast<long long>(t + q) * d.s + lane);
+                }
+                for (; t < d.ntiles; ++t) p[0] += __ldcg(d.gpart + static_cast<long long>(t) * d.s + lane);
+                tsum = ((p[0] + p[1]) + (p[2] + p[3])) + ((p[4] + p[5]) + (p[6] + p[7]));
+              }
+              presum[lane] = tsum;
+              __syncwarp();
+              solve_matrix(d, cur, c, hp.lambda, Amat, presum, 1, kMaxHistory);
+              if (lane == 0) {
                 *d.gram_done = 0;
                 __threadfence();
                 atomicExch(d.w_ready, tag);
               }
             }
           }
-          consumer_sync();
         }
       } else {
         if (mt.first) {
