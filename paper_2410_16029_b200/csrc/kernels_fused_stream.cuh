@@ -107,20 +107,40 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
   if (tid >= kConsumerThreads) {
     // ------------------------------------------------------------------ producer (one elected thread)
     if (tid == kConsumerThreads) {
+      // The producer claims work items three ahead: while it issues the copies of item k, the descriptor of
+      // item k+1, the table entry of item k+2 and the counter value of item k+3 are already on their way,
+      // so no global-memory latency sits between two items.
+      struct Desc { const float* H; const float* m; const float* v; long long rn; int te, s; };
+      auto load_desc = [&](const FusedItem& item) {
+        Desc x;
+        const MatDesc& d = mats[item.mat];
+        x.H = d.H; x.m = d.m; x.v = d.v; x.rn = d.rn; x.te = d.te; x.s = d.s;
+        return x;
+      };
+      const FusedItem none{0, 0, -1, 0};
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      int it0 = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
+      int it1 = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
+      int it2 = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
+      FusedItem item0 = it0 < n_items ? items[it0] : none;
+      FusedItem item1 = it1 < n_items ? items[it1] : none;
+      Desc d0 = load_desc(item0);
       while (ok) {
-        const int it = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
-        if (it >= n_items) {
+        if (item0.kind < 0) {
           if (mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) {
             meta[stage].kind = -1;
             mbar_arrive(full_bar + stage);
           }
           break;
         }
-        const FusedItem item = items[it];
-        const MatDesc& d = mats[item.mat];
+        // prefetch: descriptor of the next item, table entry of the one after, counter for the third
+        const Desc d1 = load_desc(item1);
+        const FusedItem item2 = it2 < n_items ? items[it2] : none;
+        const int it3 = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
+        const FusedItem item = item0;
+        const Desc d = d0;
         const int c = ring_count(ctrl, d.s);
         const long long e0 = static_cast<long long>(item.local) * d.te;
         const long long e1 = (e0 + d.te < d.rn) ? e0 + d.te : d.rn;
@@ -142,6 +162,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
           }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
+        item0 = item1; d0 = d1; item1 = item2; it2 = it3;
       }
     }
   } else {
