@@ -11,11 +11,10 @@
 // solves its s x s system and publishes the weights; the consumers of a combination item wait
 // (bounded) for that flag.  Every item a combination item depends on sits earlier in the list and
 // has been fetched by a CTA that consumes its items in order, so the kernel cannot deadlock.
-// Tiles are small enough that all SMs sweep one matrix together; its combination pass then runs in
-// reverse order right behind its Gram pass, while part of the history is still in L2.
+// The combination pass of a matrix runs in reverse tile order right behind its Gram pass, so that what
+// is left of its history in L2 is used first.
 #pragma once
 
-#include <cstdlib>
 #include <vector>
 
 #include "../../include/ngalore.h"
@@ -56,8 +55,7 @@ struct FusedCfg {
   static constexpr int kBase = kStages * kStageBytes;
   static constexpr int kFullOff = kBase, kEmptyOff = kBase + 64, kMetaOff = kBase + 128, kFlagOff = kBase + 384;
   static constexpr int kWOff = kBase + 512, kRedOff = kBase + 640;
-  static constexpr int kAOff = kRedOff + 2 * (kConsumerThreads / 32) * SMAX * 8;  // red is double-buffered
-  static constexpr int kPreOff = kAOff;  // the pre-summed Gram row is consumed before the solve fills its matrix
+  static constexpr int kAOff = kRedOff + (kConsumerThreads / 32) * SMAX * 8;
   static constexpr int kTotal = kAOff + kMaxHistory * (kMaxHistory + 1) * 8;
   static_assert(kStages * sizeof(StageMeta) <= 256, "stage metadata overflows its slot");
   static_assert(kTotal <= 232448, "shared memory budget of one CTA exceeded");
@@ -88,7 +86,6 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
   volatile int* s_flag = abort_flag + 1;
   float* wsm = reinterpret_cast<float*>(fs_smem + C::kWOff);
   double* red = reinterpret_cast<double*>(fs_smem + C::kRedOff);
-  double* presum = reinterpret_cast<double*>(fs_smem + C::kPreOff);
   double* Amat = reinterpret_cast<double*>(fs_smem + C::kAOff);
 
   const int tid = threadIdx.x;
@@ -107,40 +104,20 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
   if (tid >= kConsumerThreads) {
     // ------------------------------------------------------------------ producer (one elected thread)
     if (tid == kConsumerThreads) {
-      // The producer claims work items three ahead: while it issues the copies of item k, the descriptor of
-      // item k+1, the table entry of item k+2 and the counter value of item k+3 are already on their way,
-      // so no global-memory latency sits between two items.
-      struct Desc { const float* H; const float* m; const float* v; long long rn; int te, s; };
-      auto load_desc = [&](const FusedItem& item) {
-        Desc x;
-        const MatDesc& d = mats[item.mat];
-        x.H = d.H; x.m = d.m; x.v = d.v; x.rn = d.rn; x.te = d.te; x.s = d.s;
-        return x;
-      };
-      const FusedItem none{0, 0, -1, 0};
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      int it0 = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
-      int it1 = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
-      int it2 = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
-      FusedItem item0 = it0 < n_items ? items[it0] : none;
-      FusedItem item1 = it1 < n_items ? items[it1] : none;
-      Desc d0 = load_desc(item0);
       while (ok) {
-        if (item0.kind < 0) {
+        const int it = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
+        if (it >= n_items) {
           if (mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) {
             meta[stage].kind = -1;
             mbar_arrive(full_bar + stage);
           }
           break;
         }
-        // prefetch: descriptor of the next item, table entry of the one after, counter for the third
-        const Desc d1 = load_desc(item1);
-        const FusedItem item2 = it2 < n_items ? items[it2] : none;
-        const int it3 = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
-        const FusedItem item = item0;
-        const Desc d = d0;
+        const FusedItem item = items[it];
+        const MatDesc& d = mats[item.mat];
         const int c = ring_count(ctrl, d.s);
         const long long e0 = static_cast<long long>(item.local) * d.te;
         const long long e1 = (e0 + d.te < d.rn) ? e0 + d.te : d.rn;
@@ -162,7 +139,6 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
           }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
-        item0 = item1; d0 = d1; item1 = item2; it2 = it3;
       }
     }
   } else {
@@ -176,7 +152,6 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
 #pragma unroll
     for (int j = 0; j < SMAX; ++j) { acc[j] = 0.f; w[j] = 0.f; }
     bool item_bad = false, item_ok = true;
-    int red_buf = 0;
     while (true) {
       if (!mbar_wait(full_bar + stage, phase, abort_flag)) break;
       const StageMeta mt = meta[stage];
@@ -207,56 +182,53 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar + stage);
         if (mt.last) {
-          // End of a Gram tile.  Every warp leaves its partial sums in shared memory and moves on; warp 0
-          // alone finishes the tile (fixed summation order), publishes it and, if it was the matrix's
-          // last tile, solves the s x s system.  `red` is double-buffered because warp 0 may still be
-          // reading one half while the other warps reach the end of the next tile.
-          double* redb = red + red_buf * (kConsumerThreads / 32) * SMAX;
-          red_buf ^= 1;
 #pragma unroll
           for (int j = 0; j < SMAX; ++j) {
             const double t = warp_sum(static_cast<double>(acc[j]));
-            if (lane == 0) redb[warp * SMAX + j] = t;
+            if (lane == 0) red[warp * SMAX + j] = t;
           }
           consumer_sync();
-          if (warp == 0) {
-            if (lane < SMAX && lane < d.s) {
-              double t = 0.0;
+          if (tid < SMAX && tid < d.s) {
+            double t = 0.0;
 #pragma unroll
-              for (int ww = 0; ww < kConsumerThreads / 32; ++ww) t += redb[ww * SMAX + lane];
-              d.gpart[static_cast<long long>(mt.local) * d.s + lane] = t;
-              __threadfence();
-            }
-            __syncwarp();
-            int done = 0;
-            if (lane == 0) done = atomicAdd(d.gram_done, 1);
-            done = __shfl_sync(0xffffffffu, done, 0);
-            if (done == d.ntiles - 1) {
-              __threadfence();
-              // pre-sum the per-tile partials: lane j owns column j, eight loads in flight
-              double tsum = 0.0;
-              if (lane < d.s) {
-                double p[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) p[q] = 0.0;
-                int t = 0;
-                for (; t + 8 <= d.ntiles; t += 8) {
-#pragma unroll
-                  for (int q = 0; q < 8; ++q) p[q] += __ldcg(d.gpart + static_cast<long long>(t + q) * d.s + lane);
+            for (int ww = 0; ww < kConsumerThreads / 32; ++ww) t += red[ww * SMAX + tid];
+            d.gpart[static_cast<long long>(mt.local) * d.s + tid] = t;
+            __threadfence();
+          }
+          consumer_sync();
+          if (tid == 0) {
+            const int done = atomicAdd(d.gram_done, 1);
+            *s_flag = (done == d.ntiles - 1) ? 1 : 0;
+          }
+          consumer_sync();
+          if (*s_flag) {
+            // last Gram tile of this matrix: all consumers pre-sum the per-tile partials (fixed partition,
+            // so the result is reproducible), then one warp factors and solves
+            __threadfence();
+            const int j = tid & 31, g = tid >> 5;
+            if (j < SMAX) {
+              double t0 = 0.0, t1 = 0.0;
+              if (j < d.s) {
+                int t = g;
+                for (; t + 8 < d.ntiles; t += 16) {
+                  t0 += __ldcg(d.gpart + static_cast<long long>(t) * d.s + j);
+                  t1 += __ldcg(d.gpart + static_cast<long long>(t + 8) * d.s + j);
                 }
-                for (; t < d.ntiles; ++t) p[0] += __ldcg(d.gpart + static_cast<long long>(t) * d.s + lane);
-                tsum = ((p[0] + p[1]) + (p[2] + p[3])) + ((p[4] + p[5]) + (p[6] + p[7]));
+                if (t < d.ntiles) t0 += __ldcg(d.gpart + static_cast<long long>(t) * d.s + j);
               }
-              presum[lane] = tsum;
-              __syncwarp();
-              solve_matrix(d, cur, c, hp.lambda, Amat, presum, 1, kMaxHistory);
-              if (lane == 0) {
+              red[g * SMAX + j] = t0 + t1;
+            }
+            consumer_sync();
+            if (tid < 32) {
+              solve_matrix(d, cur, c, hp.lambda, Amat, red, kConsumerThreads / 32, SMAX);
+              if (tid == 0) {
                 *d.gram_done = 0;
                 __threadfence();
                 atomicExch(d.w_ready, tag);
               }
             }
           }
+          consumer_sync();
         }
       } else {
         if (mt.first) {
@@ -347,8 +319,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
 
 inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDesc>& mats, int s, int sm_count) {
   plan.grid = sm_count;
-  int head = plan.grid * 2;  // Gram tiles of the next matrix issued before a matrix's combination pass
-  if (const char* e = getenv("NGALORE_HEAD")) head = atoi(e);  // TUNING-ONLY
+  const int head = plan.grid * 2;  // Gram tiles of the next matrix issued before a matrix's combination pass
   std::vector<FusedItem> items;
   const int n = static_cast<int>(mats.size());
   auto gram_range = [&](int i, int t0, int t1) {
