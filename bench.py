@@ -167,6 +167,32 @@ def run_reference(args, wl):
     print(json.dumps(out))
 
 
+# --------------------------------------------------------------------------------------- multi-rank helpers
+
+def rank_workload(wl, rank):
+    """Every rank steps its own replica: same shapes and hyper-parameters, its own seed stream."""
+    import dataclasses
+
+    return dataclasses.replace(wl, index=wl.index + 100 * rank)
+
+
+def max_over_ranks(value, device, world):
+    """The slowest rank's time: the job is as fast as its slowest replica."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world, steps, ms_total):
+    """Whole-job steps/s: all ranks' steps over the slowest rank's time."""
+    return world * steps * 1e3 / ms_total
+
+
 # --------------------------------------------------------------------------------------- CUDA arm
 
 def run_ours(args, wl):
@@ -189,7 +215,7 @@ def run_ours(args, wl):
     opt = NGaLore(shapes, wl.r, wl.s, wl.T, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
                   wd=wl.wd, seed=1 + rank)
     # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
-    wl_rank = W.Workload(**{**wl.__dict__, "index": wl.index + 100 * rank})
+    wl_rank = rank_workload(wl, rank)
     # With fewer than s + 1 distinct sets a gradient would sit twice in the history ring and the Gram matrix
     # would be singular up to lambda; the optimizer never sees that in training.
     pool_sets = args.pool if args.pool > 0 else wl.s + 1
@@ -226,12 +252,9 @@ def run_ours(args, wl):
     ms_total = e0.elapsed_time(e1)
     launches = opt.launch_count - l0
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dev, world)
     ms_step = ms_total / args.steps
-    value = world * 1e3 / ms_step
+    value = job_throughput(world, args.steps, ms_total)
 
     code, per = opt.poll_status()
     if code != 0:
