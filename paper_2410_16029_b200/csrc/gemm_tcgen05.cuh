@@ -329,70 +329,77 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
       const uint32_t tphase = (local >> 1) & 1u;
       const int row_base = tile.m0 + quarter * 32;
       const int sub_row = lane >> 3, sub_col = (lane & 7) * 4;
-      // W update: fetch this warp's whole 32 x BN slab of W before waiting for the accumulator, so that
-      // the loads overlap the MMAs of the tile (and the other group's epilogue).
+      // W update: fetch this warp's 32-row slab of W (at most four 32-column chunks at a time, 128 registers)
+      // before waiting for the accumulator, so that the loads overlap the MMAs of the tile and the other
+      // group's epilogue; a 256-wide tile fetches its second half after draining the first.
       constexpr int kChunks = BN / 32;
-      float4 wreg[EPI == TC_EPI_WUPDATE ? kChunks : 1][8];
-      if (EPI == TC_EPI_WUPDATE) {
+      constexpr int kBatch = (EPI == TC_EPI_WUPDATE && kChunks > 4) ? 4 : kChunks;
+      float4 wreg[EPI == TC_EPI_WUPDATE ? kBatch : 1][8];
 #pragma unroll
-        for (int c = 0; c < kChunks; ++c) {
-          const int col = tile.n0 + c * 32 + sub_col;
+      for (int cb = 0; cb < kChunks; cb += kBatch) {
+        if (EPI == TC_EPI_WUPDATE) {
 #pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int row = row_base + it * 4 + sub_row;
-            wreg[c][it] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (!skip && c * 32 < n_eff && col < out_cols && row < rows_total)
-              wreg[c][it] = __ldcs(reinterpret_cast<const float4*>(out + static_cast<long long>(row) * ld_out + col));
-          }
-        }
-      }
-      if (!mbar_wait(tfull_bar + buf, tphase, abort_flag)) { ok = false; break; }
-      tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < kChunks; ++c) {
-        const int c0 = c * 32;
-        if (c0 < n_eff) {
-          uint32_t r[32];
-          tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * BN + c0), r);
-          tc_wait_ld();
-          if (c0 + 32 >= n_eff) {
-            // all TMEM reads of this tile are done: hand the buffer back before the global traffic
-            tc_fence_before();
-            if (lane == 0) mbar_arrive(tempty_bar + buf);
-          }
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<float4*>(stg + lane * 36 + j * 4) =
-                make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                            __uint_as_float(r[4 * j + 3]));
-          __syncwarp();
-          const int col = tile.n0 + c0 + sub_col;
-          if (!skip && col < out_cols) {
+          for (int c = 0; c < kBatch; ++c) {
+            const int col = tile.n0 + (cb + c) * 32 + sub_col;
 #pragma unroll
             for (int it = 0; it < 8; ++it) {
-              const int rr = it * 4 + sub_row;
-              const int row = row_base + rr;
-              if (row < rows_total) {
-                const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + sub_col);
-                float* p = out + static_cast<long long>(row) * ld_out + col;
-                if (EPI != TC_EPI_WUPDATE) {
-                  if (tile.atomic) {
-                    atomicAdd(reinterpret_cast<float4*>(p), acc);
+              const int row = row_base + it * 4 + sub_row;
+              wreg[c][it] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (!skip && (cb + c) * 32 < n_eff && col < out_cols && row < rows_total)
+                wreg[c][it] = __ldcs(reinterpret_cast<const float4*>(out + static_cast<long long>(row) * ld_out + col));
+            }
+          }
+        }
+        if (cb == 0) {
+          if (!mbar_wait(tfull_bar + buf, tphase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+        }
+#pragma unroll
+        for (int c = 0; c < kBatch; ++c) {
+          const int c0 = (cb + c) * 32;
+          if (c0 < n_eff) {
+            uint32_t r[32];
+            tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * BN + c0), r);
+            tc_wait_ld();
+            if (c0 + 32 >= n_eff) {
+              // all TMEM reads of this tile are done: hand the buffer back before the global traffic
+              tc_fence_before();
+              if (lane == 0) mbar_arrive(tempty_bar + buf);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              *reinterpret_cast<float4*>(stg + lane * 36 + j * 4) =
+                  make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                              __uint_as_float(r[4 * j + 3]));
+            __syncwarp();
+            const int col = tile.n0 + c0 + sub_col;
+            if (!skip && col < out_cols) {
+#pragma unroll
+              for (int it = 0; it < 8; ++it) {
+                const int rr = it * 4 + sub_row;
+                const int row = row_base + rr;
+                if (row < rows_total) {
+                  const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + sub_col);
+                  float* p = out + static_cast<long long>(row) * ld_out + col;
+                  if (EPI != TC_EPI_WUPDATE) {
+                    if (tile.atomic) {
+                      atomicAdd(reinterpret_cast<float4*>(p), acc);
+                    } else {
+                      *reinterpret_cast<float4*>(p) = acc;
+                    }
                   } else {
-                    *reinterpret_cast<float4*>(p) = acc;
+                    float4 w = wreg[EPI == TC_EPI_WUPDATE ? c : 0][it];
+                    w.x = decay * w.x - lr * acc.x;
+                    w.y = decay * w.y - lr * acc.y;
+                    w.z = decay * w.z - lr * acc.z;
+                    w.w = decay * w.w - lr * acc.w;
+                    __stcs(reinterpret_cast<float4*>(p), w);
                   }
-                } else {
-                  float4 w = wreg[EPI == TC_EPI_WUPDATE ? c : 0][it];
-                  w.x = decay * w.x - lr * acc.x;
-                  w.y = decay * w.y - lr * acc.y;
-                  w.z = decay * w.z - lr * acc.z;
-                  w.w = decay * w.w - lr * acc.w;
-                  __stcs(reinterpret_cast<float4*>(p), w);
                 }
               }
             }
+            __syncwarp();
           }
-          __syncwarp();
         }
       }
     }
