@@ -284,10 +284,19 @@ ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G, const s
   if ((rc = refresh_tc_run(st->refresh, G, q, st->opt.seed, static_cast<unsigned long long>(st->k) * 65536ull,
                            st->d_ctrl, stream, &st->launches)))
     return rc;
-  // The last basis sits in Ya (fp32, well conditioned after the sweeps): one Cholesky QR pass with the Gram
-  // matrix, the factorisation and the triangular solve in fp64 makes it orthonormal to fp32 accuracy: Ya -> Yb.
-  if ((rc = orthonormalise(st, idx, 0, true, stream))) return rc;
-  return finish_refresh(st, idx, false, stream);
+  // The basis sits in Ya, orthonormal to about 1e-6 where the matrix has enough rows for the bf16-pair rounding
+  // of the last product to average out.  Short matrices get one exact pass (Gram, Cholesky and triangular solve in fp64): Ya -> Yb -> Ya.
+  std::vector<int> small;
+  for (int i : idx)
+    if (st->mats[i].M < 512) small.push_back(i);
+  if (!small.empty()) {
+    if ((rc = orthonormalise(st, small, 0, true, stream))) return rc;
+    for (int i : small) {
+      const HostMat& hm = st->mats[i];
+      NG_CUDA(cudaMemcpyAsync(hm.Ya, hm.Yb, sizeof(float) * hm.M * hm.rp, cudaMemcpyDeviceToDevice, stream));
+    }
+  }
+  return finish_refresh(st, idx, true, stream);
 }
 
 ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream) {

@@ -32,6 +32,26 @@ __global__ void split_hilo_kernel(const float* __restrict__ src, __nv_bfloat16* 
   lo[o] = __float2bfloat16_rn(x - __bfloat162float(h));
 }
 
+struct SplitJob {
+  const float* src;
+  __nv_bfloat16 *hi, *lo;
+  long long n;
+  int cols, ld;
+};
+
+// All matrices in one launch: blockIdx.y selects the matrix, blockIdx.x strides over its elements.
+__global__ void split_hilo_grouped_kernel(const SplitJob* jobs) {
+  const SplitJob jb = jobs[blockIdx.y];
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < jb.n;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const float x = jb.src[i];
+    const __nv_bfloat16 h = __float2bfloat16_rn(x);
+    const long long o = (i / jb.cols) * jb.ld + (i % jb.cols);
+    jb.hi[o] = h;
+    jb.lo[o] = __float2bfloat16_rn(x - __bfloat162float(h));
+  }
+}
+
 struct GramPrep {
   const float* C32;  // L x L Gram matrix from the tensor cores
   double* C64;       // L x L, lower triangle written: column-scaled, symmetrised Gram + shift I
@@ -49,7 +69,7 @@ __host__ __device__ inline double gram_shift(int L) { return static_cast<double>
 // One CTA per matrix: C64 = D^-1 ((C32 + C32^T) / 2) D^-1 + shift I with D = diag(sqrt(C_ii)).
 // Scaling the columns to unit norm first makes the shift act on every column alike, whatever its
 // norm, so weak directions are still orthogonalised against each other and re-normalised.
-__global__ void __launch_bounds__(256) gram_prep_kernel(const GramPrep* probs) {
+__global__ void __launch_bounds__(256) gram_prep_kernel(const GramPrep* probs, double shift_scale) {
   const GramPrep p = probs[blockIdx.x];
   for (int i = threadIdx.x; i < p.L; i += 256) {
     const double c = static_cast<double>(p.C32[static_cast<long long>(i) * p.L + i]);
@@ -62,8 +82,87 @@ __global__ void __launch_bounds__(256) gram_prep_kernel(const GramPrep* probs) {
     if (j > i) continue;
     double v = 0.5 * (static_cast<double>(p.C32[x]) + static_cast<double>(p.C32[static_cast<long long>(j) * p.L + i]));
     v /= p.D[i] * p.D[j];
-    if (i == j) v = 1.0 + gram_shift(p.L);
+    if (i == j) v = 1.0 + shift_scale * gram_shift(p.L);
     p.C64[x] = v;
+  }
+}
+
+struct SyrkTile {
+  int mat, ti, tj, k0;  // output tile (ti, tj <= ti) of 64 x 64, rows k0 .. k0 + kSyrkRows of Y
+};
+constexpr int kSyrkRows = 1024;
+
+struct SyrkMat {
+  const float* Y;  // rows x L fp32
+  double* C;       // L x L fp64 accumulator (zeroed before the launch); lower tiles are written
+  int rows, L;
+};
+
+// Exact Gram matrix C += Y^T Y in fp64 (products of fp32 values are exact in fp64), grouped over all
+// matrices: one CTA per 64 x 64 lower tile and slab of rows, partial sums added with fp64 atomics.
+__global__ void __launch_bounds__(256) syrk_f64_kernel(const SyrkMat* mats, const SyrkTile* tiles) {
+  __shared__ float As[16][64 + 4];
+  __shared__ float Bs[16][64 + 4];
+  const SyrkTile t = tiles[blockIdx.x];
+  const SyrkMat m = mats[t.mat];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int i0 = t.ti * 64, j0 = t.tj * 64;
+  const int k1 = (t.k0 + kSyrkRows < m.rows) ? t.k0 + kSyrkRows : m.rows;
+  double acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+  for (int k0 = t.k0; k0 < k1; k0 += 16) {
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      const int kk = (threadIdx.x >> 6) + 4 * p, c = threadIdx.x & 63;
+      const int k = k0 + kk;
+      As[kk][c] = (k < k1 && i0 + c < m.L) ? m.Y[static_cast<long long>(k) * m.L + i0 + c] : 0.f;
+      Bs[kk][c] = (k < k1 && j0 + c < m.L) ? m.Y[static_cast<long long>(k) * m.L + j0 + c] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      double a[4], b[4];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) { a[x] = static_cast<double>(As[kk][ty * 4 + x]); b[x] = static_cast<double>(Bs[kk][tx * 4 + x]); }
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+#pragma unroll
+        for (int y = 0; y < 4; ++y) acc[x][y] += a[x] * b[y];
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    const int i = i0 + ty * 4 + x;
+    if (i >= m.L) continue;
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const int j = j0 + tx * 4 + y;
+      if (j <= i) atomicAdd(m.C + static_cast<long long>(i) * m.L + j, acc[x][y]);
+    }
+  }
+}
+
+struct GramPrep64 {
+  const double* G;  // L x L exact Gram matrix, lower triangle valid
+  double* C64;      // L x L out: column-scaled Gram + tiny shift, lower triangle
+  double* D;
+  int L;
+};
+
+// Column scaling for the exact pass; the shift only keeps a numerically rank-deficient basis factorisable.
+__global__ void __launch_bounds__(256) gram_prep64_kernel(const GramPrep64* probs) {
+  const GramPrep64 p = probs[blockIdx.x];
+  for (int i = threadIdx.x; i < p.L; i += 256) p.D[i] = sqrt(fmax(p.G[static_cast<long long>(i) * p.L + i], 1e-60));
+  __syncthreads();
+  const long long total = static_cast<long long>(p.L) * p.L;
+  for (long long x = threadIdx.x; x < total; x += 256) {
+    const int i = static_cast<int>(x / p.L), j = static_cast<int>(x % p.L);
+    if (j > i) continue;
+    p.C64[x] = (i == j) ? 1.0 + 1e-12 : p.G[x] / (p.D[i] * p.D[j]);
   }
 }
 
@@ -87,7 +186,17 @@ __global__ void __launch_bounds__(512) tri_inverse_kernel(const TriInverse* prob
       double acc = (i == j) ? 1.0 : 0.0;
       if (i >= j) {
         const double* lrow = p.Lf + static_cast<long long>(i) * L;
-        for (int k = j; k < i; ++k) acc -= lrow[k] * p.X[static_cast<long long>(k) * L + j];
+        const double* xcol = p.X + j;
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;  // independent chains keep four loads in flight
+        int k = j;
+        for (; k + 4 <= i; k += 4) {
+          a0 += lrow[k] * xcol[static_cast<long long>(k) * L];
+          a1 += lrow[k + 1] * xcol[static_cast<long long>(k + 1) * L];
+          a2 += lrow[k + 2] * xcol[static_cast<long long>(k + 2) * L];
+          a3 += lrow[k + 3] * xcol[static_cast<long long>(k + 3) * L];
+        }
+        for (; k < i; ++k) a0 += lrow[k] * xcol[static_cast<long long>(k) * L];
+        acc -= (a0 + a1) + (a2 + a3);
         acc /= lrow[i];
       } else {
         acc = 0.0;
@@ -139,6 +248,12 @@ struct RefreshPlan {
   GramPrep* d_prep = nullptr;
   CholProblem* d_chol = nullptr;
   TriInverse* d_tri = nullptr;
+  SplitJob* d_split_y = nullptr;
+  SyrkMat* d_syrk_mats = nullptr;
+  SyrkTile* d_syrk_tiles = nullptr;
+  int n_syrk_tiles = 0;
+  GramPrep64* d_prep64 = nullptr;
+  SplitJob* d_split_z = nullptr;
 };
 
 inline void refresh_plan_destroy(RefreshPlan& plan) {
@@ -243,6 +358,19 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   const size_t o_prep = take(sizeof(GramPrep) * n);
   const size_t o_chol = take(sizeof(CholProblem) * n);
   const size_t o_tri = take(sizeof(TriInverse) * n);
+  std::vector<SyrkTile> syrk_tiles;
+  for (int i = 0; i < n; ++i) {
+    const int nt = (plan.mats[i].L + 63) / 64;
+    for (int k0 = 0; k0 < plan.mats[i].M; k0 += kSyrkRows)
+      for (int ti = 0; ti < nt; ++ti)
+        for (int tj = 0; tj <= ti; ++tj) syrk_tiles.push_back(SyrkTile{i, ti, tj, k0});
+  }
+  plan.n_syrk_tiles = static_cast<int>(syrk_tiles.size());
+  const size_t o_syrk_m = take(sizeof(SyrkMat) * n);
+  const size_t o_syrk_t = take(sizeof(SyrkTile) * syrk_tiles.size());
+  const size_t o_prep64 = take(sizeof(GramPrep64) * n);
+  const size_t o_sy = take(sizeof(SplitJob) * n);
+  const size_t o_sz = take(sizeof(SplitJob) * n);
   if (cudaMalloc(&plan.buf, off) != cudaSuccess) { plan.buf = nullptr; return NGALORE_ERR_ALLOC; }
   if (cudaMemset(plan.buf, 0, off) != cudaSuccess) return NGALORE_ERR_CUDA;
   plan.device_bytes = off;
@@ -250,6 +378,9 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   std::vector<GramPrep> prep(n);
   std::vector<CholProblem> chol(n);
   std::vector<TriInverse> tri(n);
+  std::vector<SplitJob> sy(n), sz(n);
+  std::vector<SyrkMat> syrk_m(n);
+  std::vector<GramPrep64> prep64(n);
   plan.h_maps.resize(static_cast<size_t>(RM_COUNT) * n);
   std::memset(plan.h_maps.data(), 0, sizeof(CUtensorMap) * plan.h_maps.size());
   for (int i = 0; i < n; ++i) {
@@ -267,6 +398,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     prep[i] = GramPrep{m.C32, m.C64, m.D, m.L};
     chol[i] = CholProblem{m.C64, m.L};
     tri[i] = TriInverse{m.C64, m.D, m.X64, m.Rhi, m.Rlo, m.L, m.ldl};
+    syrk_m[i] = SyrkMat{m.Yf, m.X64, m.M, m.L};
+    prep64[i] = GramPrep64{m.X64, m.C64, m.D, m.L};
+    sy[i] = SplitJob{m.Yf, m.Yhi, m.Ylo, static_cast<long long>(m.M) * m.L, m.L, m.ldl};
+    sz[i] = SplitJob{m.Zf, m.Zhi, m.Zlo, static_cast<long long>(m.N) * m.L, m.L, m.ldl};
     CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * RM_COUNT];
     const uint64_t sl = static_cast<uint64_t>(m.ldl) * 2;
     bool ok = true;
@@ -300,9 +435,19 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   plan.d_prep = reinterpret_cast<GramPrep*>(plan.buf + o_prep);
   plan.d_chol = reinterpret_cast<CholProblem*>(plan.buf + o_chol);
   plan.d_tri = reinterpret_cast<TriInverse*>(plan.buf + o_tri);
+  plan.d_split_y = reinterpret_cast<SplitJob*>(plan.buf + o_sy);
+  plan.d_syrk_mats = reinterpret_cast<SyrkMat*>(plan.buf + o_syrk_m);
+  plan.d_syrk_tiles = reinterpret_cast<SyrkTile*>(plan.buf + o_syrk_t);
+  plan.d_prep64 = reinterpret_cast<GramPrep64*>(plan.buf + o_prep64);
+  plan.d_split_z = reinterpret_cast<SplitJob*>(plan.buf + o_sz);
   if (cudaMemcpy(plan.d_prep, prep.data(), sizeof(GramPrep) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_chol, chol.data(), sizeof(CholProblem) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemcpy(plan.d_tri, tri.data(), sizeof(TriInverse) * n, cudaMemcpyHostToDevice) != cudaSuccess)
+      cudaMemcpy(plan.d_tri, tri.data(), sizeof(TriInverse) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_syrk_mats, syrk_m.data(), sizeof(SyrkMat) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_syrk_tiles, syrk_tiles.data(), sizeof(SyrkTile) * syrk_tiles.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_prep64, prep64.data(), sizeof(GramPrep64) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_split_y, sy.data(), sizeof(SplitJob) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_split_z, sz.data(), sizeof(SplitJob) * n, cudaMemcpyHostToDevice) != cudaSuccess)
     return NGALORE_ERR_CUDA;
 
   using L1 = TcSmem<kRefBN, 1, 2, kRefStages1, 4>;
@@ -360,21 +505,18 @@ inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cu
 }
 
 inline ngalore_status refresh_tc_split(RefreshPlan& plan, bool y_side, cudaStream_t stream, int64_t* launches) {
-  for (const RefreshMat& m : plan.mats) {
-    const long long cnt = static_cast<long long>(y_side ? m.M : m.N) * m.L;
-    split_hilo_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, stream>>>(
-        y_side ? m.Yf : m.Zf, y_side ? m.Yhi : m.Zhi, y_side ? m.Ylo : m.Zlo, cnt, m.L, m.ldl);
-    *launches += 1;
-  }
+  split_hilo_grouped_kernel<<<dim3(64, plan.n), 256, 0, stream>>>(y_side ? plan.d_split_y : plan.d_split_z);
+  *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
 // iterate (fp32, in Yf or Zf) -> well-conditioned basis, left both as fp32 and as its bf16 parts.
-inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
+inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches,
+                                      double shift_scale = 1.0) {
   ngalore_status rc;
   if ((rc = refresh_tc_split(plan, y_side, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, y_side ? RG_GRAM_Y : RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
-  gram_prep_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep);
+  gram_prep_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep, shift_scale);
   chol_batched_kernel<<<plan.n, 512, 0, stream>>>(plan.d_chol);
   tri_inverse_kernel<<<plan.n, 512, 0, stream>>>(plan.d_tri);
   *launches += 3;
@@ -383,7 +525,25 @@ inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ct
   return refresh_tc_split(plan, y_side, stream, launches);
 }
 
-// Whole-set refresh up to the last basis, which is left in Yf (fp32, well conditioned, not yet orthonormal).
+// Final pass: Cholesky QR of the last basis with the Gram matrix accumulated exactly in fp64 (no shift beyond
+// 1e-12), Cholesky and triangular inverse in fp64; only Q = Y R^-1 goes through the tensor cores in two bf16
+// parts, whose rounding averages out over the rows.  Matrices with few rows are re-done entirely in fp64 by
+// the caller.
+inline ngalore_status refresh_tc_final(RefreshPlan& plan, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
+  ngalore_status rc;
+  if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;  // bf16 parts of the basis for the apply
+  for (const RefreshMat& m : plan.mats)
+    if (cudaMemsetAsync(m.X64, 0, sizeof(double) * m.L * m.L, stream) != cudaSuccess) return NGALORE_ERR_CUDA;
+  syrk_f64_kernel<<<plan.n_syrk_tiles, 256, 0, stream>>>(plan.d_syrk_mats, plan.d_syrk_tiles);
+  gram_prep64_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep64);
+  chol_batched_kernel<<<plan.n, 512, 0, stream>>>(plan.d_chol);
+  tri_inverse_kernel<<<plan.n, 512, 0, stream>>>(plan.d_tri);
+  *launches += 4;
+  if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
+  return refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches);
+}
+
+// Whole-set refresh; leaves the basis in Yf.
 inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G, int q, unsigned long long seed,
                                      unsigned long long stream_base, Ctrl* d_ctrl, cudaStream_t stream,
                                      int64_t* launches) {
@@ -420,7 +580,11 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
     if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches))) return rc;
     if ((rc = refresh_tc_orth(plan, true, d_ctrl, stream, launches))) return rc;
   }
-  return NGALORE_OK;
+  // twice: the basis that leaves the sweeps can be ill conditioned in its weak directions, and the bf16-pair
+  // product then carries its rounding amplified by that condition number; the second pass starts from a
+  // nearly orthonormal basis
+  if ((rc = refresh_tc_final(plan, d_ctrl, stream, launches))) return rc;
+  return refresh_tc_final(plan, d_ctrl, stream, launches);
 }
 
 }  // namespace ngalore
