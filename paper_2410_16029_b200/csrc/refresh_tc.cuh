@@ -169,46 +169,119 @@ __global__ void __launch_bounds__(256) gram_prep64_kernel(const GramPrep64* prob
 struct TriInverse {
   const double* Lf;      // L x L lower Cholesky factor of the column-scaled Gram matrix (row-major)
   const double* D;       // L column norms: R^-1 = D^-1 Lf^-T
-  double* X;             // L x L scratch: X = Lf^-1 (lower)
+  double* X;             // L x L: X = Lf^-1 (lower triangular, upper part zero)
   __nv_bfloat16* Rhi;    // L x ld: high part of R^-1 = Lf^-T (upper triangular)
   __nv_bfloat16* Rlo;
   int L, ld;
 };
 
-// One CTA per matrix, thread j owns column j of X = Lf^-1 (forward substitution on e_j) and writes
-// row j of R^-1 = D^-1 X^T.  All threads walk the same (i, k) sequence, so Lf is read as a broadcast and X
-// with unit stride across the warp; a thread reads only entries of X that it wrote itself.
-__global__ void __launch_bounds__(512) tri_inverse_kernel(const TriInverse* probs) {
-  const TriInverse p = probs[blockIdx.x];
-  const int L = p.L;
-  for (int j = threadIdx.x; j < L; j += blockDim.x) {
-    for (int i = 0; i < L; ++i) {
-      double acc = (i == j) ? 1.0 : 0.0;
-      if (i >= j) {
-        const double* lrow = p.Lf + static_cast<long long>(i) * L;
-        const double* xcol = p.X + j;
-        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;  // independent chains keep four loads in flight
-        int k = j;
-        for (; k + 4 <= i; k += 4) {
-          a0 += lrow[k] * xcol[static_cast<long long>(k) * L];
-          a1 += lrow[k + 1] * xcol[static_cast<long long>(k + 1) * L];
-          a2 += lrow[k + 2] * xcol[static_cast<long long>(k + 2) * L];
-          a3 += lrow[k + 3] * xcol[static_cast<long long>(k + 3) * L];
-        }
-        for (; k < i; ++k) a0 += lrow[k] * xcol[static_cast<long long>(k) * L];
-        acc -= (a0 + a1) + (a2 + a3);
-        acc /= lrow[i];
+// ---- blocked inverse of the lower Cholesky factor: X = Lf^-1 by recursive halving,
+//   [[A, 0], [C, B]]^-1 = [[A^-1, 0], [-B^-1 C A^-1, B^-1]],
+// leaves (<= 32 x 32) by forward substitution, inner nodes by two small batched fp64 GEMMs per level.
+
+struct TriLeaf {
+  const double* Lf;  // top-left element of the diagonal block inside the L x L factor
+  double* X;         // same position inside X
+  int ld, size;
+};
+
+// One warp per leaf; lane j solves column j of the block by forward substitution in shared memory.
+__global__ void __launch_bounds__(128) tri_leaf_kernel(const TriLeaf* leaves, int n_leaves) {
+  __shared__ double blk[4][32][33];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int id = blockIdx.x * 4 + warp;
+  if (id >= n_leaves) return;
+  const TriLeaf lf = leaves[id];
+  for (int i = 0; i < lf.size; ++i)
+    if (lane < lf.size) blk[warp][i][lane] = lf.Lf[static_cast<long long>(i) * lf.ld + lane];
+  __syncwarp();
+  if (lane < lf.size) {
+    double x[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      double acc = (i == lane) ? 1.0 : 0.0;
+      if (i < lf.size && i >= lane) {
+#pragma unroll
+        for (int k = 0; k < 32; ++k)
+          if (k < i && k >= lane) acc -= blk[warp][i][k] * x[k];
+        acc /= blk[warp][i][i];
       } else {
         acc = 0.0;
       }
-      p.X[static_cast<long long>(i) * L + j] = acc;
-      const float f = static_cast<float>(fmin(fmax(acc / p.D[j], -1e30), 1e30));
-      const __nv_bfloat16 h = __float2bfloat16_rn(f);
-      p.Rhi[static_cast<long long>(j) * p.ld + i] = h;
-      p.Rlo[static_cast<long long>(j) * p.ld + i] = __float2bfloat16_rn(f - __bfloat162float(h));
+      x[i] = acc;
+      if (i < lf.size) lf.X[static_cast<long long>(i) * lf.ld + lane] = acc;
     }
   }
 }
+
+struct TriGemm {
+  const double* A;  // m x k
+  const double* B;  // k x n
+  double* C;        // m x n = (negate ? -1 : 1) * A B
+  int lda, ldb, ldc, m, n, k, negate;
+};
+
+// Batched small fp64 GEMM: blockIdx.z selects the problem, (blockIdx.y, blockIdx.x) a 64 x 64 tile of it.
+__global__ void __launch_bounds__(256) tri_gemm_kernel(const TriGemm* probs) {
+  __shared__ double As[16][64 + 1];
+  __shared__ double Bs[16][64 + 1];
+  const TriGemm g = probs[blockIdx.z];
+  const int i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+  if (i0 >= g.m || j0 >= g.n) return;
+  const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+  double acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+  for (int k0 = 0; k0 < g.k; k0 += 16) {
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      const int kk = t & 15, i = (t >> 4) + 16 * p;  // A: k contiguous
+      As[kk][i] = (i0 + i < g.m && k0 + kk < g.k) ? g.A[static_cast<long long>(i0 + i) * g.lda + k0 + kk] : 0.0;
+      const int j = t & 63, kb = (t >> 6) + 4 * p;   // B: n contiguous
+      Bs[kb][j] = (j0 + j < g.n && k0 + kb < g.k) ? g.B[static_cast<long long>(k0 + kb) * g.ldb + j0 + j] : 0.0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      double a[4], b[4];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) { a[x] = As[kk][ty * 4 + x]; b[x] = Bs[kk][tx * 4 + x]; }
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+#pragma unroll
+        for (int y = 0; y < 4; ++y) acc[x][y] += a[x] * b[y];
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    const int i = i0 + ty * 4 + x;
+    if (i >= g.m) continue;
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const int j = j0 + tx * 4 + y;
+      if (j < g.n) g.C[static_cast<long long>(i) * g.ldc + j] = g.negate ? -acc[x][y] : acc[x][y];
+    }
+  }
+}
+
+// R^-1 = D^-1 X^T (upper triangular) split into two bf16 parts; one CTA per matrix.
+__global__ void __launch_bounds__(256) tri_convert_kernel(const TriInverse* probs) {
+  const TriInverse p = probs[blockIdx.x];
+  const long long total = static_cast<long long>(p.L) * p.L;
+  for (long long x = threadIdx.x; x < total; x += 256) {
+    const int j = static_cast<int>(x / p.L), i = static_cast<int>(x % p.L);  // entry (j, i) of R^-1
+    const double v = (i >= j) ? p.X[static_cast<long long>(i) * p.L + j] / p.D[j] : 0.0;
+    const float f = static_cast<float>(fmin(fmax(v, -1e30), 1e30));
+    const __nv_bfloat16 h = __float2bfloat16_rn(f);
+    p.Rhi[static_cast<long long>(j) * p.ld + i] = h;
+    p.Rlo[static_cast<long long>(j) * p.ld + i] = __float2bfloat16_rn(f - __bfloat162float(h));
+  }
+}
+
+constexpr int kTriMaxLevels = 12;
 
 // ------------------------------------------------------------------------------------------ plan
 
@@ -221,7 +294,7 @@ struct RefreshMat {
   float *Yf, *Zf;                       // fp32 GEMM outputs (M x L, N x L)
   __nv_bfloat16 *Yhi, *Ylo, *Zhi, *Zlo; // bf16 parts of the iterates (rows x ldl)
   float* C32;                           // L x L
-  double *C64, *X64;                    // L x L each
+  double *C64, *X64, *T64;              // L x L each
   double* D;                            // L
   __nv_bfloat16 *Rhi, *Rlo;             // L x ldl
 };
@@ -239,6 +312,7 @@ struct RefreshPlan {
   std::vector<CUtensorMap> h_maps;  // RM_COUNT per matrix
   std::vector<const void*> last_G;
   char* buf = nullptr;
+  char* tri_tables = nullptr;
   CUtensorMap* d_maps = nullptr;
   TcProblem* d_probs[RG_COUNT] = {};
   TcTile* d_tiles[RG_COUNT] = {};
@@ -248,6 +322,13 @@ struct RefreshPlan {
   GramPrep* d_prep = nullptr;
   CholProblem* d_chol = nullptr;
   TriInverse* d_tri = nullptr;
+  TriLeaf* d_leaves = nullptr;
+  int n_leaves = 0;
+  TriGemm* d_tg1[kTriMaxLevels] = {};
+  TriGemm* d_tg2[kTriMaxLevels] = {};
+  int n_tg[kTriMaxLevels] = {};
+  int tg_max[kTriMaxLevels] = {};
+  int tri_levels = 0;
   SplitJob* d_split_y = nullptr;
   SyrkMat* d_syrk_mats = nullptr;
   SyrkTile* d_syrk_tiles = nullptr;
@@ -258,7 +339,9 @@ struct RefreshPlan {
 
 inline void refresh_plan_destroy(RefreshPlan& plan) {
   if (plan.buf) cudaFree(plan.buf);
+  if (plan.tri_tables) cudaFree(plan.tri_tables);
   plan.buf = nullptr;
+  plan.tri_tables = nullptr;
   plan.ready = false;
 }
 
@@ -297,7 +380,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   // ---- device buffer layout
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) / 256 * 256; return o; };
-  struct Offs { size_t Yhi, Ylo, Zhi, Zlo, C32, C64, X64, D, Rhi, Rlo; };
+  struct Offs { size_t Yhi, Ylo, Zhi, Zlo, C32, C64, X64, T64, D, Rhi, Rlo; };
   std::vector<Offs> offs(n);
   for (int i = 0; i < n; ++i) {
     RefreshMat& m = plan.mats[i];
@@ -310,6 +393,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     offs[i].C32 = take(sizeof(float) * m.L * m.L);
     offs[i].C64 = take(sizeof(double) * m.L * m.L);
     offs[i].X64 = take(sizeof(double) * m.L * m.L);
+    offs[i].T64 = take(sizeof(double) * m.L * m.L);
     offs[i].D = take(sizeof(double) * m.L);
     offs[i].Rhi = take(sizeof(__nv_bfloat16) * m.L * m.ldl);
     offs[i].Rlo = take(sizeof(__nv_bfloat16) * m.L * m.ldl);
@@ -392,6 +476,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     m.C32 = reinterpret_cast<float*>(plan.buf + offs[i].C32);
     m.C64 = reinterpret_cast<double*>(plan.buf + offs[i].C64);
     m.X64 = reinterpret_cast<double*>(plan.buf + offs[i].X64);
+    m.T64 = reinterpret_cast<double*>(plan.buf + offs[i].T64);
     m.D = reinterpret_cast<double*>(plan.buf + offs[i].D);
     m.Rhi = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Rhi);
     m.Rlo = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Rlo);
@@ -423,6 +508,65 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     probs[RG_GRAM_Z][i] = TcProblem{m.C32, m.L, m.L, m.L, base + RM_Z_B, base + RM_Z_B, 0};
     probs[RG_APPLY_Y][i] = TcProblem{m.Yf, m.M, m.L, m.L, base + RM_Y_A, base + RM_RINV, 0};
     probs[RG_APPLY_Z][i] = TcProblem{m.Zf, m.N, m.L, m.L, base + RM_Z_A, base + RM_RINV, 0};
+  }
+  // ---- tables of the blocked triangular inverse
+  {
+    std::vector<TriLeaf> leaves;
+    std::vector<TriGemm> g1[kTriMaxLevels], g2[kTriMaxLevels];
+    int max_level = 0;
+    for (int i = 0; i < n; ++i) {
+      const RefreshMat& m = plan.mats[i];
+      // returns the height of the node covering [lo, hi)
+      struct Rec {
+        static int go(const RefreshMat& m, int lo, int hi, std::vector<TriLeaf>& leaves, std::vector<TriGemm>* g1,
+                      std::vector<TriGemm>* g2) {
+          const int len = hi - lo;
+          if (len <= 32) {
+            leaves.push_back(TriLeaf{m.C64 + static_cast<long long>(lo) * m.L + lo, m.X64 + static_cast<long long>(lo) * m.L + lo, m.L, len});
+            return 0;
+          }
+          const int mid = lo + ((len / 2 + 31) / 32) * 32;
+          const int ha = go(m, lo, mid, leaves, g1, g2), hb = go(m, mid, hi, leaves, g1, g2);
+          const int h = (ha > hb ? ha : hb) + 1;
+          // T = C A^-1 with C = Lf[mid:hi, lo:mid];  X[mid:hi, lo:mid] = -B^-1 T
+          double* T = m.T64 + static_cast<long long>(mid) * m.L + lo;
+          g1[h].push_back(TriGemm{m.C64 + static_cast<long long>(mid) * m.L + lo, m.X64 + static_cast<long long>(lo) * m.L + lo, T,
+                                  m.L, m.L, m.L, hi - mid, mid - lo, mid - lo, 0});
+          g2[h].push_back(TriGemm{m.X64 + static_cast<long long>(mid) * m.L + mid, T, m.X64 + static_cast<long long>(mid) * m.L + lo,
+                                  m.L, m.L, m.L, hi - mid, mid - lo, hi - mid, 1});
+          return h;
+        }
+      };
+      const int h = Rec::go(m, 0, m.L, leaves, g1, g2);
+      if (h > max_level) max_level = h;
+    }
+    if (max_level >= kTriMaxLevels) return NGALORE_ERR_INVALID_ARG;
+    plan.tri_levels = max_level;
+    plan.n_leaves = static_cast<int>(leaves.size());
+    size_t bytes = sizeof(TriLeaf) * leaves.size();
+    for (int h = 1; h <= max_level; ++h) bytes += 2 * ((sizeof(TriGemm) * g1[h].size() + 255) / 256 * 256);
+    bytes = (bytes + 255) / 256 * 256 + 256;
+    char* tb = nullptr;
+    if (cudaMalloc(&tb, bytes) != cudaSuccess) return NGALORE_ERR_ALLOC;
+    plan.tri_tables = tb;
+    plan.device_bytes += bytes;
+    size_t o = 0;
+    plan.d_leaves = reinterpret_cast<TriLeaf*>(tb);
+    if (cudaMemcpy(tb, leaves.data(), sizeof(TriLeaf) * leaves.size(), cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
+    o = (sizeof(TriLeaf) * leaves.size() + 255) / 256 * 256;
+    for (int h = 1; h <= max_level; ++h) {
+      const size_t sz = sizeof(TriGemm) * g1[h].size();
+      plan.n_tg[h] = static_cast<int>(g1[h].size());
+      int mx = 1;
+      for (const TriGemm& g : g1[h]) { if (g.m > mx) mx = g.m; if (g.n > mx) mx = g.n; }
+      plan.tg_max[h] = mx;
+      plan.d_tg1[h] = reinterpret_cast<TriGemm*>(tb + o);
+      if (sz && cudaMemcpy(tb + o, g1[h].data(), sz, cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
+      o += (sz + 255) / 256 * 256;
+      plan.d_tg2[h] = reinterpret_cast<TriGemm*>(tb + o);
+      if (sz && cudaMemcpy(tb + o, g2[h].data(), sz, cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
+      o += (sz + 255) / 256 * 256;
+    }
   }
   plan.d_maps = reinterpret_cast<CUtensorMap*>(plan.buf + o_maps);
   for (int g = 0; g < RG_COUNT; ++g) {
@@ -504,6 +648,24 @@ inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cu
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
+// X = Lf^-1 for every matrix (blocked), then R^-1 = D^-1 X^T in two bf16 parts.
+inline ngalore_status refresh_tc_tri_inverse(RefreshPlan& plan, cudaStream_t stream, int64_t* launches) {
+  for (const RefreshMat& m : plan.mats)
+    if (cudaMemsetAsync(m.X64, 0, sizeof(double) * m.L * m.L, stream) != cudaSuccess) return NGALORE_ERR_CUDA;
+  tri_leaf_kernel<<<(plan.n_leaves + 3) / 4, 128, 0, stream>>>(plan.d_leaves, plan.n_leaves);
+  *launches += 1;
+  for (int h = 1; h <= plan.tri_levels; ++h) {
+    if (plan.n_tg[h] == 0) continue;
+    const int tiles = (plan.tg_max[h] + 63) / 64;
+    tri_gemm_kernel<<<dim3(tiles, tiles, plan.n_tg[h]), 256, 0, stream>>>(plan.d_tg1[h]);
+    tri_gemm_kernel<<<dim3(tiles, tiles, plan.n_tg[h]), 256, 0, stream>>>(plan.d_tg2[h]);
+    *launches += 2;
+  }
+  tri_convert_kernel<<<plan.n, 256, 0, stream>>>(plan.d_tri);
+  *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
+}
+
 inline ngalore_status refresh_tc_split(RefreshPlan& plan, bool y_side, cudaStream_t stream, int64_t* launches) {
   split_hilo_grouped_kernel<<<dim3(64, plan.n), 256, 0, stream>>>(y_side ? plan.d_split_y : plan.d_split_z);
   *launches += 1;
@@ -518,9 +680,9 @@ inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ct
   if ((rc = refresh_tc_gemm(plan, y_side ? RG_GRAM_Y : RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
   gram_prep_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep, shift_scale);
   chol_batched_kernel<<<plan.n, 512, 0, stream>>>(plan.d_chol);
-  tri_inverse_kernel<<<plan.n, 512, 0, stream>>>(plan.d_tri);
-  *launches += 3;
+  *launches += 2;
   if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
+  if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, y_side ? RG_APPLY_Y : RG_APPLY_Z, d_ctrl, stream, launches))) return rc;
   return refresh_tc_split(plan, y_side, stream, launches);
 }
@@ -537,9 +699,9 @@ inline ngalore_status refresh_tc_final(RefreshPlan& plan, Ctrl* d_ctrl, cudaStre
   syrk_f64_kernel<<<plan.n_syrk_tiles, 256, 0, stream>>>(plan.d_syrk_mats, plan.d_syrk_tiles);
   gram_prep64_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep64);
   chol_batched_kernel<<<plan.n, 512, 0, stream>>>(plan.d_chol);
-  tri_inverse_kernel<<<plan.n, 512, 0, stream>>>(plan.d_tri);
-  *launches += 4;
+  *launches += 3;
   if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
+  if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
   return refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches);
 }
 
