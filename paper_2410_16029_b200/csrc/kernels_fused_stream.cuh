@@ -102,15 +102,20 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
   const int tag = ctrl->epoch + 1;
 
   if (tid >= kConsumerThreads) {
-    // ------------------------------------------------------------------ producer (one elected thread)
-    if (tid == kConsumerThreads) {
+    // ------------------------------------------------------------------ producer warp
+    // Lane 0 claims items and arms the barriers; every lane issues the bulk copy of "its" slot (lane j copies
+    // history slot j, the next two lanes m and v), so a stage's copies are issued in parallel.
+    {
+      const int lane = tid & 31;
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       while (ok) {
-        const int it = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
+        int it = 0;
+        if (lane == 0) it = static_cast<int>(atomicAdd(&ctrl->work_counter, 1u));
+        it = __shfl_sync(0xffffffffu, it, 0);
         if (it >= n_items) {
-          if (mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) {
+          if (lane == 0 && mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) {
             meta[stage].kind = -1;
             mbar_arrive(full_bar + stage);
           }
@@ -119,23 +124,32 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
         const FusedItem item = items[it];
         const MatDesc& d = mats[item.mat];
         const int c = ring_count(ctrl, d.s);
+        const int ncopies = c + (item.kind == 1 ? 2 : 0);
         const long long e0 = static_cast<long long>(item.local) * d.te;
         const long long e1 = (e0 + d.te < d.rn) ? e0 + d.te : d.rn;
         for (long long e = e0; e < e1; e += CE) {
           const int cnt = (e1 - e < CE) ? static_cast<int>(e1 - e) : CE;
-          if (!mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          StageMeta mt;
-          mt.mat = item.mat; mt.kind = item.kind; mt.local = item.local;
-          mt.first = (e == e0) ? 1 : 0; mt.last = (e + CE >= e1) ? 1 : 0; mt.count = cnt; mt.e0 = e;
-          meta[stage] = mt;
+          int good = 1;
+          if (lane == 0) good = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag) ? 1 : 0;
+          good = __shfl_sync(0xffffffffu, good, 0);
+          if (!good) { ok = false; break; }
           unsigned char* sb = fs_smem + stage * C::kStageBytes;
           const uint32_t bytes = static_cast<uint32_t>(cnt) * 4u;
-          mbar_expect_tx(full_bar + stage, bytes * static_cast<uint32_t>(c + (item.kind == 1 ? 2 : 0)));
-          for (int j = 0; j < c; ++j)
-            bulk_load(sb + j * CE * 4, d.H + static_cast<long long>(j) * d.rn + e, bytes, full_bar + stage);
-          if (item.kind == 1) {
-            bulk_load(sb + SMAX * CE * 4, d.m + e, bytes, full_bar + stage);
-            bulk_load(sb + (SMAX + 1) * CE * 4, d.v + e, bytes, full_bar + stage);
+          if (lane == 0) {
+            StageMeta mt;
+            mt.mat = item.mat; mt.kind = item.kind; mt.local = item.local;
+            mt.first = (e == e0) ? 1 : 0; mt.last = (e + CE >= e1) ? 1 : 0; mt.count = cnt; mt.e0 = e;
+            meta[stage] = mt;
+            mbar_expect_tx(full_bar + stage, bytes * static_cast<uint32_t>(ncopies));
+          }
+          __syncwarp();
+          for (int j = lane; j < ncopies; j += 32) {
+            if (j < c) {
+              bulk_load(sb + j * CE * 4, d.H + static_cast<long long>(j) * d.rn + e, bytes, full_bar + stage);
+            } else {
+              const int k = j - c;  // 0: m, 1: v
+              bulk_load(sb + (SMAX + k) * CE * 4, (k == 0 ? d.m : d.v) + e, bytes, full_bar + stage);
+            }
           }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
         }
