@@ -24,6 +24,14 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes per launch of the step kernels from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
+# taken on the 1.1B shapes cut to 2 layers with a full history (profiles/step_kernels_llama-1.1b-2layers_ncu_full.md)
+# and expressed per unit of work so that it scales to the full workload: the stream kernel's traffic grows with
+# the low-rank elements sum(r' N), the GEMMs' with sum(M N).  Valid for r = 512, s = 16 only; set an entry to None
+# when its kernel changes.
+NCU_TRAFFIC_PER_UNIT = {"fused_stream_kernel": ("rn", 146.93), "tc_gemm_kernel<backproject>": ("mn", 8.621),
+                        "tc_gemm_kernel<project>": ("mn", 3.064)}
+
 METRIC = "optimizer steps/sec over all matrices (device-timed)"
 UNIT = "steps/s"
 
@@ -314,6 +322,10 @@ def run_ours(args, wl):
     dom = int(np.argmax(phase))
     achieved = alg[dom] / (phase[dom] * 1e-3) / 1e9
     traffic = None
+    per_unit = NCU_TRAFFIC_PER_UNIT.get(names[dom])
+    if per_unit is not None and wl.r == 512 and wl.s == 16:
+        units = sum(wl.rank_of(i) * N for i, (M, N) in enumerate(shapes)) if per_unit[0] == "rn" else sum(M * N for M, N in shapes)
+        traffic = per_unit[1] * units
     roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": alg[dom], "ms_per_launch": float(phase[dom]),
