@@ -426,7 +426,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
 
   // ---- streaming tile size.  Measured on the 1.1B shapes: the persistent stream kernel pays a fixed latency per
   // work item (table and descriptor loads, the end-of-tile reduction, the completion counter), so large tiles win
-  // (131072 elements: 5.0 ms, 32768: 5.6 ms, 4096: 9.5 ms per step); tiles shrink only to keep about eight
+  // (131072 elements: 5.0 ms, 32768: 5.6 ms, 4096: 9.5 ms per step); tiles shrink only to keep about two
   // items per SM and pass on small models.  The price: the combination pass finds little of a big matrix's
   // history still in L2, so the history is read from HBM twice per step.
   uint64_t hash = 1469598103934665603ull;
@@ -443,7 +443,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     hash = (hash ^ static_cast<uint64_t>(hm.N)) * 1099511628211ull;
   }
   st->shape_hash = hash;
-  long long te_all = total_rn / (8ll * prop.multiProcessorCount) / 1024 * 1024;
+  long long te_all = total_rn / (2ll * prop.multiProcessorCount) / 1024 * 1024;
   if (te_all < 2048) te_all = 2048;
   if (te_all > 131072) te_all = 131072;
   std::vector<int> tile_elems(n_matrices, static_cast<int>(te_all));
