@@ -100,6 +100,9 @@ void ngalore_destroy(ngalore_state* st);
  *   G  host array of n_matrices device pointers, bf16 bit patterns M x N, read only
  * If T > 0 and the step index k satisfies k mod T == 0, the subspace of every
  * matrix is refreshed from G first.  Increments k.
+ * After one call with the same W and G pointers a further call enqueues kernels only (no copies), so it can
+ * be captured in a CUDA graph.  A replay advances the device-side ring position but not the host-side k:
+ * create the state with T = 0 when replaying from a graph and call ngalore_refresh_subspace yourself.
  */
 ngalore_status ngalore_step(ngalore_state* st, float* const* W, const uint16_t* const* G, void* stream);
 

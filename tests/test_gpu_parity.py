@@ -172,3 +172,36 @@ def test_invalid_arguments_are_rejected():
     with pytest.raises(NGaLoreError) as e:
         opt.step(W, G)                            # T == 0 and no subspace yet
     assert e.value.code == 5
+
+
+def test_step_replays_from_a_cuda_graph():
+    """A step enqueues only kernels once its pointer tables are warm (same W and G buffers, T = 0), so it can
+    be captured in a CUDA graph; replays must match eager steps (ring position and counters live on the device)."""
+    w = wl.tiny_workload([(256, 520), (520, 256)], r=32, s=4, T=0, inner_rank=4, index=99)
+    dev = torch.device("cuda")
+    shapes = [(M, N) for _, M, N in w.shapes]
+    G0 = [to_device_bf16(wl.gradient_bits(w, i, 0), dev) for i in range(2)]
+    eager, graphed = _make(w), _make(w)
+    for opt in (eager, graphed):
+        opt.refresh_subspace(G0)
+    Wa = [torch.zeros(s, device=dev) for s in shapes]
+    Wb = [torch.zeros(s, device=dev) for s in shapes]
+    Gs = [g.clone() for g in G0]                     # static gradient buffers, refilled in place
+    for k in range(2):
+        for i in range(2):
+            Gs[i].copy_(to_device_bf16(wl.gradient_bits(w, i, k), dev))
+        eager.step(Wa, Gs)
+        graphed.step(Wb, Gs)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        graphed.step(Wb, Gs)
+    for k in range(2, 7):
+        for i in range(2):
+            Gs[i].copy_(to_device_bf16(wl.gradient_bits(w, i, k), dev))
+        eager.step(Wa, Gs)
+        graph.replay()
+        torch.cuda.synchronize()
+        for a, b in zip(Wa, Wb):
+            assert rel_err(b.cpu().numpy(), a.cpu().numpy()) <= 1e-6
+    assert eager.poll_status()[0] == 0 and graphed.poll_status()[0] == 0
