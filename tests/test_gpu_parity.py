@@ -174,6 +174,16 @@ def test_invalid_arguments_are_rejected():
     assert e.value.code == 5
 
 
+@pytest.mark.parametrize("impl", IMPLS[:2])
+def test_long_history_uses_the_32_slot_kernels(impl):
+    """s = 20 exercises the 32-slot instantiation of the stream kernels; 24 steps fill and wrap the ring."""
+    w = wl.tiny_workload([(200, 264), (136, 96), (64, 1032)], r=24, s=20, T=12, inner_rank=4, index=89)
+    opt = _make(w, **impl)
+    errs, _, _ = run_side_by_side(opt, w, 24, "B")
+    _assert_errs(errs)
+    assert opt.poll_status()[0] == 0
+
+
 def test_step_replays_from_a_cuda_graph():
     """A step enqueues only kernels once its pointer tables are warm (same W and G buffers, T = 0), so it can
     be captured in a CUDA graph; replays must match eager steps (ring position and counters live on the device)."""
