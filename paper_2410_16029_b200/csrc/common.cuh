@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -18,9 +19,9 @@ struct MatDesc {
   float* H;                   // history ring: s slots of rp x N fp32 (one slot when s == 0)
   float* m;                   // first moment, rp x N
   float* v;                   // second moment, rp x N
-  __nv_bfloat16* u_hi;        // direction u = m / sqrt(v + eps), high bf16 part, rp x N
-  __nv_bfloat16* u_lo;        // low part: bf16(u - hi)
-  __nv_bfloat16* P16;         // working copy of P, M x ldp row-major (padding is zero)
+  __half* u16;                // direction u = m / sqrt(v + eps) rounded to fp16, rp x N
+  __half* P16;                // working copy of P for the back-projection: the bf16-rounded values held as
+                              // fp16 (same numbers as Pt16), M x ldp row-major (padding is zero)
   __nv_bfloat16* Pt16;        // working copy of P^T, rp x ldpt row-major
   float* P32;                 // fp32 master of P, M x rp row-major
   double* Kraw;               // s x s raw inner products <H_i, H_j>
@@ -54,6 +55,17 @@ struct StreamTile {
   int mat;    // matrix index
   int local;  // tile index inside the matrix
 };
+
+// Four floats to four fp16 values (round to nearest even, clamped to the largest finite fp16).
+__device__ __forceinline__ uint2 pack_f16x4(float a, float b, float c, float d) {
+  constexpr float kMax = 65504.f;
+  const __half2 lo = __floats2half2_rn(fminf(fmaxf(a, -kMax), kMax), fminf(fmaxf(b, -kMax), kMax));
+  const __half2 hi = __floats2half2_rn(fminf(fmaxf(c, -kMax), kMax), fminf(fmaxf(d, -kMax), kMax));
+  uint2 r;
+  r.x = *reinterpret_cast<const uint32_t*>(&lo);
+  r.y = *reinterpret_cast<const uint32_t*>(&hi);
+  return r;
+}
 
 __device__ __forceinline__ int ring_cur(const Ctrl* c, int s) {
   return s > 0 ? static_cast<int>(c->n_appended % s) : 0;

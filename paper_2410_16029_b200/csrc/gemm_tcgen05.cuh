@@ -4,8 +4,9 @@
 //
 //   projection       R = P^T G          A = Pt16 (r' x M, K-major), B = G (M x N, N contiguous)
 //                    epilogue: store (or atomically add, when K is split) into ring slot `cur`   (Sec. 1)
-//   back-projection  W <- (1 - lr wd) W - lr P u     A = P16 (M x r'), B = u_hi and u_lo (r' x N)
-//                    epilogue: fused read-modify-write of W                                      (Sec. 2.2)
+//   store mode       out = A B for a table of problems (subspace refresh)
+//
+// The back-projection has a kernel of its own (backproject_tcgen05.cuh) built from the same wrappers.
 //
 // Warp roles: warp 0 issues TMA loads, warp 1 allocates TMEM and issues the MMAs, four or eight further
 // warps drain the accumulator (tcgen05.ld), transpose through shared memory and write
@@ -43,6 +44,18 @@ struct TcTile {
   int k0;          // first K element
   int kblocks;     // number of 64-wide K blocks
   int atomic;      // 1: K is split, accumulate into the output with atomics
+  int rows, cols;  // extent of the output the tile belongs to
+};
+
+// Tensor maps of the step GEMMs, kTcMapsPerMat consecutive entries per matrix.
+enum {
+  TC_MAP_A_PROJ = 0,   // Pt16: r' rows x M (K), box 64 x 128
+  TC_MAP_B_PROJ = 1,   // G: M (K) rows x N, box 64 x 64
+  TC_MAP_A_BACK = 2,   // P16: M rows x r' (K), box 64 x 128
+  TC_MAP_B_BACK = 3,   // u16: r' (K) rows x N, box 64 x 64
+  TC_MAP_W_LOAD = 4,   // W (fp32): M rows x N, box 32 columns x 128 rows
+  TC_MAP_W_STORE = 5,  // W (fp32): box 32 x 32
+  kTcMapsPerMat = 6
 };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
@@ -101,7 +114,7 @@ __device__ __forceinline__ void tc_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                             uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
@@ -134,10 +147,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   d |= 2ull << 61;
   return d;
 }
-// Instruction descriptor of kind::f16: fp32 accumulator, bf16 A (K-major, or MN-major when asked) and
-// B (MN-major), M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc(int n, bool a_mn_major = false) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | (1u << 16) |
+// Instruction descriptor of kind::f16: fp32 accumulator, A (K-major, or MN-major when asked) and
+// B (MN-major) both bf16 or both fp16, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc(int n, bool a_mn_major, bool fp16_operands) {
+  const uint32_t fmt = fp16_operands ? 0u : 1u;  // operand format field: 0 = fp16, 1 = bf16
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((a_mn_major ? 1u : 0u) << 15) | (1u << 16) |
          (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(kTcBM >> 4) << 24);
 }
@@ -153,16 +167,16 @@ struct TcSmem {
   static constexpr int kTotal = kBarOffset + 256 + 1024;      // barriers + slack for 1024-byte alignment
 };
 
-enum { TC_EPI_PROJECT = 0, TC_EPI_WUPDATE = 1, TC_EPI_STORE = 2 };
+enum { TC_EPI_PROJECT = 0, TC_EPI_STORE = 2 };
 
-// NA / NB: number of bf16 parts of A / B (1, or 2 = high and low part).  With NA = NB = 2 the products
+// NA / NB: number of 16-bit parts of A / B (1, or 2 = high and low part).  With NA = NB = 2 the products
 // hi*hi, hi*lo and lo*hi are accumulated (lo*lo is below fp32 resolution).  A_MN: A is stored with its
-// row index contiguous (A^T row-major), staged as two 64-row chunks like B.
-template <int BN, int NA, int NB, int STAGES, int EPI, int NEPI, bool A_MN>
+// row index contiguous (A^T row-major), staged as two 64-row chunks like B.  F16: the operands are fp16
+// (otherwise bf16); TMA moves either as opaque 16-bit elements.
+template <int BN, int NA, int NB, int STAGES, int EPI, int NEPI, bool A_MN, bool F16 = false>
 __global__ void __launch_bounds__(64 + 32 * NEPI, 1)
 tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__ tiles, int n_tiles,
-               const MatDesc* __restrict__ mats, Ctrl* ctrl, const Hyper* __restrict__ hyper,
-               float* const* __restrict__ Wptrs, const TcProblem* __restrict__ probs) {
+               const MatDesc* __restrict__ mats, Ctrl* ctrl, const TcProblem* __restrict__ probs) {
   using L = TcSmem<BN, NA, NB, STAGES, NEPI>;
   extern __shared__ unsigned char tc_smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
@@ -208,8 +222,8 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
           mapB0 = tmaps + pr.map_b;
           out_cols = pr.out_cols;
         } else {
-          mapA = tmaps + tile.mat * 5 + (EPI == TC_EPI_PROJECT ? 0 : 2);
-          mapB0 = tmaps + tile.mat * 5 + (EPI == TC_EPI_PROJECT ? 1 : 3);
+          mapA = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_A_PROJ;
+          mapB0 = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_B_PROJ;
           out_cols = mats[tile.mat].N;
         }
         const int n_rem = out_cols - tile.n0;
@@ -252,7 +266,7 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
         const int out_cols = (EPI == TC_EPI_STORE) ? probs[tile.mat].out_cols : mats[tile.mat].N;
         const int n_rem = out_cols - tile.n0;
         const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
-        const uint32_t idesc = instr_desc(n_eff, A_MN);
+        const uint32_t idesc = instr_desc(n_eff, A_MN, F16);
         const int buf = local & 1;
         const uint32_t tphase = (local >> 1) & 1u;
         if (!mbar_wait(tempty_bar + buf, tphase ^ 1u, abort_flag)) { ok = false; break; }
@@ -275,7 +289,7 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
                 const uint64_t adesc = A_MN ? smem_desc(aaddr + kk * 2048, L::kBChunkBytes, 1024)
                                             : smem_desc(aaddr + kk * 32, 16, 1024);
                 const uint64_t bdesc = smem_desc(baddr + kk * 2048, L::kBChunkBytes, 1024);
-                tc_mma_bf16(tmem_d, adesc, bdesc, idesc, first ? 0u : 1u);
+                tc_mma(tmem_d, adesc, bdesc, idesc, first ? 0u : 1u);
                 first = false;
               }
             }
@@ -289,13 +303,11 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2 .. 2 + NEPI - 1)
     // With 8 epilogue warps there are two groups of four; group g drains accumulator buffer g, i.e. the
-    // tiles with (local & 1) == g, so one group's W loads are in flight while the other computes.
+    // tiles with (local & 1) == g.
     const int quarter = warp & 3;  // TMEM lanes 32 * quarter .. + 31 belong to this warp
     constexpr int kGroups = NEPI / 4;
     const int group = (warp - 2) >> 2;
     float* stg = reinterpret_cast<float*>(smem + STAGES * L::kStageBytes + (warp - 2) * L::kEpiWarpBytes);
-    float lr = 0.f, decay = 1.f;
-    if (EPI == TC_EPI_WUPDATE) { lr = hyper->lr; decay = 1.f - hyper->lr * hyper->wd; }
     int local = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
@@ -303,7 +315,6 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
       const TcTile tile = tiles[t];
       float* out;
       int rows_total, out_cols, ld_out;
-      bool skip = false;
       if (EPI == TC_EPI_STORE) {
         const TcProblem pr = probs[tile.mat];
         out = pr.out;
@@ -314,14 +325,8 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
         const MatDesc& d = mats[tile.mat];
         out_cols = d.N;
         ld_out = d.N;
-        if (EPI == TC_EPI_PROJECT) {
-          out = d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn;
-          rows_total = d.rp;
-        } else {
-          out = Wptrs[tile.mat];
-          rows_total = d.M;
-          skip = __ldcg(d.step_bad) != 0;
-        }
+        out = d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn;
+        rows_total = d.rp;
       }
       const int n_rem = out_cols - tile.n0;
       const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
@@ -329,77 +334,43 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
       const uint32_t tphase = (local >> 1) & 1u;
       const int row_base = tile.m0 + quarter * 32;
       const int sub_row = lane >> 3, sub_col = (lane & 7) * 4;
-      // W update: fetch this warp's 32-row slab of W (at most four 32-column chunks at a time, 128 registers)
-      // before waiting for the accumulator, so that the loads overlap the MMAs of the tile and the other
-      // group's epilogue; a 256-wide tile fetches its second half after draining the first.
-      constexpr int kChunks = BN / 32;
-      constexpr int kBatch = (EPI == TC_EPI_WUPDATE && kChunks > 4) ? 4 : kChunks;
-      float4 wreg[EPI == TC_EPI_WUPDATE ? kBatch : 1][8];
+      if (!mbar_wait(tfull_bar + buf, tphase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
 #pragma unroll
-      for (int cb = 0; cb < kChunks; cb += kBatch) {
-        if (EPI == TC_EPI_WUPDATE) {
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (c0 < n_eff) {
+          uint32_t r[32];
+          tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * BN + c0), r);
+          tc_wait_ld();
+          if (c0 + 32 >= n_eff) {
+            // all TMEM reads of this tile are done: hand the buffer back before the global traffic
+            tc_fence_before();
+            if (lane == 0) mbar_arrive(tempty_bar + buf);
+          }
 #pragma unroll
-          for (int c = 0; c < kBatch; ++c) {
-            const int col = tile.n0 + (cb + c) * 32 + sub_col;
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<float4*>(stg + lane * 36 + j * 4) =
+                make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                            __uint_as_float(r[4 * j + 3]));
+          __syncwarp();
+          const int col = tile.n0 + c0 + sub_col;
+          if (col < out_cols) {
 #pragma unroll
             for (int it = 0; it < 8; ++it) {
-              const int row = row_base + it * 4 + sub_row;
-              wreg[c][it] = make_float4(0.f, 0.f, 0.f, 0.f);
-              if (!skip && (cb + c) * 32 < n_eff && col < out_cols && row < rows_total)
-                wreg[c][it] = __ldcs(reinterpret_cast<const float4*>(out + static_cast<long long>(row) * ld_out + col));
-            }
-          }
-        }
-        if (cb == 0) {
-          if (!mbar_wait(tfull_bar + buf, tphase, abort_flag)) { ok = false; break; }
-          tc_fence_after();
-        }
-#pragma unroll
-        for (int c = 0; c < kBatch; ++c) {
-          const int c0 = (cb + c) * 32;
-          if (c0 < n_eff) {
-            uint32_t r[32];
-            tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * BN + c0), r);
-            tc_wait_ld();
-            if (c0 + 32 >= n_eff) {
-              // all TMEM reads of this tile are done: hand the buffer back before the global traffic
-              tc_fence_before();
-              if (lane == 0) mbar_arrive(tempty_bar + buf);
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-              *reinterpret_cast<float4*>(stg + lane * 36 + j * 4) =
-                  make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                              __uint_as_float(r[4 * j + 3]));
-            __syncwarp();
-            const int col = tile.n0 + c0 + sub_col;
-            if (!skip && col < out_cols) {
-#pragma unroll
-              for (int it = 0; it < 8; ++it) {
-                const int rr = it * 4 + sub_row;
-                const int row = row_base + rr;
-                if (row < rows_total) {
-                  const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + sub_col);
-                  float* p = out + static_cast<long long>(row) * ld_out + col;
-                  if (EPI != TC_EPI_WUPDATE) {
-                    if (tile.atomic) {
-                      atomicAdd(reinterpret_cast<float4*>(p), acc);
-                    } else {
-                      *reinterpret_cast<float4*>(p) = acc;
-                    }
-                  } else {
-                    float4 w = wreg[EPI == TC_EPI_WUPDATE ? c : 0][it];
-                    w.x = decay * w.x - lr * acc.x;
-                    w.y = decay * w.y - lr * acc.y;
-                    w.z = decay * w.z - lr * acc.z;
-                    w.w = decay * w.w - lr * acc.w;
-                    __stcs(reinterpret_cast<float4*>(p), w);
-                  }
+              const int rr = it * 4 + sub_row;
+              const int row = row_base + rr;
+              if (row < rows_total) {
+                const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + sub_col);
+                float* p = out + static_cast<long long>(row) * ld_out + col;
+                if (tile.atomic) {
+                  atomicAdd(reinterpret_cast<float4*>(p), acc);
+                } else {
+                  *reinterpret_cast<float4*>(p) = acc;
                 }
               }
             }
-            __syncwarp();
           }
+          __syncwarp();
         }
       }
     }
@@ -435,16 +406,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kProjBN = 256, kProjStages = 4, kProjEpiWarps = 4;
-constexpr int kBackBN = 128, kBackStages = 3, kBackEpiWarps = 8;
 
 struct TcPlan {
   size_t device_bytes = 0;
   EncodeTiledFn encode = nullptr;
   int n_mats = 0;
-  std::vector<CUtensorMap> h_maps;  // 5 per matrix: A_proj, B_proj (G), A_back, B_hi, B_lo
-  std::vector<int> rowsN;           // per matrix: M, N for re-encoding G maps
+  std::vector<CUtensorMap> h_maps;  // kTcMapsPerMat per matrix (TC_MAP_*)
+  std::vector<int> rowsN;           // per matrix: M, N for re-encoding the maps of G and W
   std::vector<int> colsN;
   std::vector<const void*> last_G;
+  std::vector<const void*> last_W;
   CUtensorMap* d_maps = nullptr;
   TcTile* d_tiles_proj = nullptr;
   TcTile* d_tiles_back = nullptr;
@@ -455,13 +426,14 @@ struct TcPlan {
   bool maps_dirty = true;
 };
 
+// 16-bit elements unless fp32 is asked for (TMA moves fp16 and bf16 alike).
 inline bool tc_encode_2d(EncodeTiledFn fn, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer,
-                         uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer) {
+                         uint64_t row_stride_bytes, uint32_t box_inner, uint32_t box_outer, bool fp32 = false) {
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {row_stride_bytes};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -483,21 +455,20 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   plan.encode = reinterpret_cast<EncodeTiledFn>(fn);
   const int n = static_cast<int>(mats.size());
   plan.n_mats = n;
-  plan.h_maps.resize(static_cast<size_t>(n) * 5);
+  plan.h_maps.resize(static_cast<size_t>(n) * kTcMapsPerMat);
   plan.last_G.assign(n, nullptr);
+  plan.last_W.assign(n, nullptr);
   std::memset(plan.h_maps.data(), 0, sizeof(CUtensorMap) * plan.h_maps.size());
   for (int i = 0; i < n; ++i) {
     const MatDesc& d = mats[i];
     // A_proj: Pt16, r' rows x M (K) columns, row stride ldpt
-    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 0], d.Pt16, d.M, d.rp, static_cast<uint64_t>(d.ldpt) * 2, kTcBK, kTcBM))
+    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * kTcMapsPerMat + TC_MAP_A_PROJ], d.Pt16, d.M, d.rp, static_cast<uint64_t>(d.ldpt) * 2, kTcBK, kTcBM))
       return NGALORE_ERR_CUDA;
     // A_back: P16, M rows x r' (K) columns, row stride ldp
-    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 2], d.P16, d.rp, d.M, static_cast<uint64_t>(d.ldp) * 2, kTcBK, kTcBM))
+    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * kTcMapsPerMat + TC_MAP_A_BACK], d.P16, d.rp, d.M, static_cast<uint64_t>(d.ldp) * 2, kTcBK, kTcBM))
       return NGALORE_ERR_CUDA;
-    // B_hi / B_lo: r' (K) rows x N columns
-    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 3], d.u_hi, d.N, d.rp, static_cast<uint64_t>(d.N) * 2, 64, kTcBK))
-      return NGALORE_ERR_CUDA;
-    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 4], d.u_lo, d.N, d.rp, static_cast<uint64_t>(d.N) * 2, 64, kTcBK))
+    // B_back: u16, r' (K) rows x N columns
+    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * kTcMapsPerMat + TC_MAP_B_BACK], d.u16, d.N, d.rp, static_cast<uint64_t>(d.N) * 2, 64, kTcBK))
       return NGALORE_ERR_CUDA;
   }
 
@@ -526,7 +497,7 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
         for (int m0 = 0; m0 < d.rp; m0 += kTcBM) {
           const int kb0 = sp * kb_per;
           const int kbn = std::min(kb_per, kb_total - kb0);
-          proj.push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0});
+          proj.push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0, d.rp, d.N});
         }
   }
   std::stable_sort(proj.begin(), proj.end(), [](const TcTile& a, const TcTile& b) { return a.kblocks > b.kblocks; });
@@ -534,7 +505,7 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
     const MatDesc& d = mats[i];
     const int kbn = (d.rp + kTcBK - 1) / kTcBK;
     for (int m0 = 0; m0 < d.M; m0 += kTcBM)
-      for (int n0 = 0; n0 < d.N; n0 += kBackBN) back.push_back(TcTile{i, m0, n0, 0, kbn, 0});
+      for (int n0 = 0; n0 < d.N; n0 += 128) back.push_back(TcTile{i, m0, n0, 0, kbn, 0, d.M, d.N});
   }
   plan.n_tiles_proj = static_cast<int>(proj.size());
   plan.n_tiles_back = static_cast<int>(back.size());
@@ -558,25 +529,32 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   for (int i = 0; i < n; ++i) { plan.rowsN[i] = mats[i].M; plan.colsN[i] = mats[i].N; }
 
   using LP = TcSmem<kProjBN, 1, 1, kProjStages, kProjEpiWarps>;
-  using LB = TcSmem<kBackBN, 1, 2, kBackStages, kBackEpiWarps>;
   if (cudaFuncSetAttribute(tc_gemm_kernel<kProjBN, 1, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps, false>,
-                           cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess ||
-      cudaFuncSetAttribute(tc_gemm_kernel<kBackBN, 1, 2, kBackStages, TC_EPI_WUPDATE, kBackEpiWarps, false>,
-                           cudaFuncAttributeMaxDynamicSharedMemorySize, LB::kTotal) != cudaSuccess)
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   plan.maps_dirty = true;
   return NGALORE_OK;
 }
 
-// R = P^T G for every matrix, into ring slot `cur` (read on the device from Ctrl).
-inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const uint16_t* const* G,
-                                 cudaStream_t stream, int64_t* launches) {
+// Point the tensor maps of the step at this call's gradients and weights (host arrays of device pointers,
+// 16-byte aligned, row-major M x N).  Maps are rebuilt and uploaded only when a pointer differs from the
+// last call's, so a step with unchanged buffers enqueues kernels only.
+inline ngalore_status tc_bind_buffers(TcPlan& plan, const uint16_t* const* G, float* const* W, cudaStream_t stream) {
   bool changed = plan.maps_dirty;
   for (int i = 0; i < plan.n_mats; ++i) {
+    CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * kTcMapsPerMat];
     if (plan.last_G[i] != G[i]) {
       plan.last_G[i] = G[i];
-      if (!tc_encode_2d(plan.encode, &plan.h_maps[i * 5 + 1], G[i], plan.colsN[i], plan.rowsN[i],
+      if (!tc_encode_2d(plan.encode, mp + TC_MAP_B_PROJ, G[i], plan.colsN[i], plan.rowsN[i],
                         static_cast<uint64_t>(plan.colsN[i]) * 2, 64, kTcBK))
+        return NGALORE_ERR_CUDA;
+      changed = true;
+    }
+    if (plan.last_W[i] != W[i]) {
+      plan.last_W[i] = W[i];
+      const uint64_t row_bytes = static_cast<uint64_t>(plan.colsN[i]) * 4;
+      if (!tc_encode_2d(plan.encode, mp + TC_MAP_W_LOAD, W[i], plan.colsN[i], plan.rowsN[i], row_bytes, 32, kTcBM, true) ||
+          !tc_encode_2d(plan.encode, mp + TC_MAP_W_STORE, W[i], plan.colsN[i], plan.rowsN[i], row_bytes, 32, 32, true))
         return NGALORE_ERR_CUDA;
       changed = true;
     }
@@ -587,29 +565,19 @@ inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ct
       return NGALORE_ERR_CUDA;
     plan.maps_dirty = false;
   }
+  return NGALORE_OK;
+}
+
+// R = P^T G for every matrix, into ring slot `cur` (read on the device from Ctrl).
+inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, cudaStream_t stream,
+                                 int64_t* launches) {
   if (plan.n_split > 0) {
     zero_split_slots_kernel<<<dim3(64, plan.n_split), 256, 0, stream>>>(d_mats, plan.d_split_mats, d_ctrl);
     *launches += 1;
   }
   using LP = TcSmem<kProjBN, 1, 1, kProjStages, kProjEpiWarps>;
   tc_gemm_kernel<kProjBN, 1, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps, false><<<plan.grid_proj, 64 + 32 * kProjEpiWarps, LP::kTotal, stream>>>(
-      plan.d_maps, plan.d_tiles_proj, plan.n_tiles_proj, d_mats, d_ctrl, nullptr, nullptr, nullptr);
-  *launches += 1;
-  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
-}
-
-// W <- (1 - lr wd) W - lr P (u_hi + u_lo) for every matrix; d_W is the device array of W pointers.
-inline ngalore_status tc_backproject(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const Hyper* d_hyper,
-                                     float* const* d_W, cudaStream_t stream, int64_t* launches) {
-  if (plan.maps_dirty) {
-    if (cudaMemcpyAsync(plan.d_maps, plan.h_maps.data(), sizeof(CUtensorMap) * plan.h_maps.size(),
-                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
-      return NGALORE_ERR_CUDA;
-    plan.maps_dirty = false;
-  }
-  using LB = TcSmem<kBackBN, 1, 2, kBackStages, kBackEpiWarps>;
-  tc_gemm_kernel<kBackBN, 1, 2, kBackStages, TC_EPI_WUPDATE, kBackEpiWarps, false><<<plan.grid_back, 64 + 32 * kBackEpiWarps, LB::kTotal, stream>>>(
-      plan.d_maps, plan.d_tiles_back, plan.n_tiles_back, d_mats, d_ctrl, d_hyper, d_W, nullptr);
+      plan.d_maps, plan.d_tiles_proj, plan.n_tiles_proj, d_mats, d_ctrl, nullptr);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }

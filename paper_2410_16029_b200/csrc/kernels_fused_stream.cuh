@@ -277,8 +277,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
 #pragma unroll
             for (int q = 0; q < VEC; ++q) {
               Hc[q] = 0.f;
-              d.u_hi[e + q] = __float2bfloat16_rn(0.f);
-              d.u_lo[e + q] = __float2bfloat16_rn(0.f);
+              d.u16[e + q] = __float2half_rn(0.f);
             }
           } else {
             float n[VEC], mm[VEC], vv[VEC], uu[VEC];
@@ -300,20 +299,11 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
             if (VEC == 4) {
               *reinterpret_cast<float4*>(d.m + e) = make_float4(mm[0], mm[1], mm[2 % VEC], mm[3 % VEC]);
               *reinterpret_cast<float4*>(d.v + e) = make_float4(vv[0], vv[1], vv[2 % VEC], vv[3 % VEC]);
-              const uint2 hi = pack_bf16x4(uu[0], uu[1], uu[2 % VEC], uu[3 % VEC]);
-              const __nv_bfloat162 h01 = *reinterpret_cast<const __nv_bfloat162*>(&hi.x);
-              const __nv_bfloat162 h23 = *reinterpret_cast<const __nv_bfloat162*>(&hi.y);
-              const uint2 lo = pack_bf16x4(uu[0] - __low2float(h01), uu[1] - __high2float(h01),
-                                           uu[2 % VEC] - __low2float(h23), uu[3 % VEC] - __high2float(h23));
-              *reinterpret_cast<uint2*>(d.u_hi + e) = hi;
-              *reinterpret_cast<uint2*>(d.u_lo + e) = lo;
+              *reinterpret_cast<uint2*>(d.u16 + e) = pack_f16x4(uu[0], uu[1], uu[2 % VEC], uu[3 % VEC]);
             } else {
               *reinterpret_cast<float2*>(d.m + e) = make_float2(mm[0], mm[1]);
               *reinterpret_cast<float2*>(d.v + e) = make_float2(vv[0], vv[1]);
-              const __nv_bfloat162 h = __floats2bfloat162_rn(uu[0], uu[1]);
-              const __nv_bfloat162 l = __floats2bfloat162_rn(uu[0] - __low2float(h), uu[1] - __high2float(h));
-              *reinterpret_cast<__nv_bfloat162*>(d.u_hi + e) = h;
-              *reinterpret_cast<__nv_bfloat162*>(d.u_lo + e) = l;
+              *reinterpret_cast<uint32_t*>(d.u16 + e) = pack_f16x4(uu[0], uu[1], 0.f, 0.f).x;
             }
           }
         }

@@ -219,9 +219,12 @@ __global__ void __launch_bounds__(256) orth_apply_kernel(OrthApply p) {
 
 // ---------------------------------------------------------------- working copies of P
 
-// P16 = bf16(P32) (M x rp, leading dimension ldp) and Pt16 = its transpose (rp x M, leading dimension ldpt).
+// Pt16 = bf16(P32)^T (rp x M, leading dimension ldpt) for the projection, and P16 = the same rounded values
+// stored as fp16 (M x rp, leading dimension ldp) for the back-projection, whose other operand is fp16.  A
+// bf16 number converts to fp16 without error unless it is below 2^-17 in magnitude, where the error is at
+// most 2^-25: far below the resolution of an orthonormal column's entries.
 // Block (32, 8).
-__global__ void working_copies_kernel(const float* P32, __nv_bfloat16* P16, __nv_bfloat16* Pt16, int M, int rp,
+__global__ void working_copies_kernel(const float* P32, __half* P16, __nv_bfloat16* Pt16, int M, int rp,
                                       int ldp, int ldpt) {
   __shared__ float tile[32][33];
   const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
@@ -230,7 +233,7 @@ __global__ void working_copies_kernel(const float* P32, __nv_bfloat16* P16, __nv
     float val = 0.f;
     if (i < M && j < rp) {
       val = P32[static_cast<long long>(i) * rp + j];
-      P16[static_cast<long long>(i) * ldp + j] = __float2bfloat16_rn(val);
+      P16[static_cast<long long>(i) * ldp + j] = __float2half_rn(__bfloat162float(__float2bfloat16_rn(val)));
     }
     tile[a][threadIdx.x] = val;
   }
@@ -241,10 +244,10 @@ __global__ void working_copies_kernel(const float* P32, __nv_bfloat16* P16, __nv
   }
 }
 
-// dst (rows x cols, dense fp32) = src (rows x cols, leading dimension ld, bf16)
-__global__ void widen_bf16_kernel(const __nv_bfloat16* src, float* dst, long long n, int cols, int ld) {
+// dst (rows x cols, dense fp32) = src (rows x cols, leading dimension ld, fp16)
+__global__ void widen_f16_kernel(const __half* src, float* dst, long long n, int cols, int ld) {
   const long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  if (i < n) dst[i] = __bfloat162float(src[(i / cols) * ld + (i % cols)]);
+  if (i < n) dst[i] = __half2float(src[(i / cols) * ld + (i % cols)]);
 }
 
 }  // namespace ngalore

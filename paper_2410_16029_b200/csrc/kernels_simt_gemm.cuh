@@ -6,7 +6,7 @@
 
 namespace ngalore {
 
-enum SimtDtype { DT_BF16 = 0, DT_F32 = 1, DT_F64 = 2 };
+enum SimtDtype { DT_BF16 = 0, DT_F32 = 1, DT_F64 = 2, DT_F16 = 3 };
 enum SimtEpilogue {
   EPI_STORE = 0,      // C = acc
   EPI_W_UPDATE = 1,   // C = (1 - lr wd) C - lr acc          (Sec. 2.2 update; decoupled decay)
@@ -34,6 +34,7 @@ struct SimtGemm {
 template <typename Acc>
 __device__ __forceinline__ Acc simt_load(const void* p, int dt, long long idx) {
   if (dt == DT_BF16) return static_cast<Acc>(__bfloat162float(static_cast<const __nv_bfloat16*>(p)[idx]));
+  if (dt == DT_F16) return static_cast<Acc>(__half2float(static_cast<const __half*>(p)[idx]));
   if (dt == DT_F32) return static_cast<Acc>(static_cast<const float*>(p)[idx]);
   return static_cast<Acc>(static_cast<const double*>(p)[idx]);
 }

@@ -146,17 +146,9 @@ __device__ __forceinline__ void solve_matrix(const MatDesc& d, int cur, int c, d
   __syncwarp();
 }
 
-__device__ __forceinline__ uint2 pack_bf16x4(float a, float b, float c, float d) {
-  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b);
-  __nv_bfloat162 hi = __floats2bfloat162_rn(c, d);
-  uint2 r;
-  r.x = *reinterpret_cast<unsigned int*>(&lo);
-  r.y = *reinterpret_cast<unsigned int*>(&hi);
-  return r;
-}
 
 // N~ = sum_j w_j H_j, then the Adam moments as printed in Sec. 2.2 (eps inside the root, no bias
-// correction), then u split into a high and a low bf16 part for the back-projection GEMM.
+// correction), then u rounded to fp16 for the back-projection GEMM.
 template <int SMAX>
 __device__ __forceinline__ void combine_tile(const MatDesc& d, int local, int cur, int c, int tile_elems,
                                              const Hyper& hp, const float* wsm /* smem weights */) {
@@ -166,8 +158,7 @@ __device__ __forceinline__ void combine_tile(const MatDesc& d, int local, int cu
     float* Hc = d.H + static_cast<long long>(cur) * d.rn;
     for (long long e = e0 + threadIdx.x * 4; e < e1; e += kStreamThreads * 4) {
       *reinterpret_cast<float4*>(Hc + e) = make_float4(0.f, 0.f, 0.f, 0.f);
-      *reinterpret_cast<uint2*>(d.u_hi + e) = make_uint2(0u, 0u);
-      *reinterpret_cast<uint2*>(d.u_lo + e) = make_uint2(0u, 0u);
+      *reinterpret_cast<uint2*>(d.u16 + e) = make_uint2(0u, 0u);
     }
     return;
   }
@@ -200,13 +191,7 @@ __device__ __forceinline__ void combine_tile(const MatDesc& d, int local, int cu
     *reinterpret_cast<float4*>(d.v + e) = v;
     const float u0 = m.x / sqrtf(v.x + eps), u1 = m.y / sqrtf(v.y + eps);
     const float u2 = m.z / sqrtf(v.z + eps), u3 = m.w / sqrtf(v.w + eps);
-    const uint2 hi = pack_bf16x4(u0, u1, u2, u3);
-    const __nv_bfloat162 h01 = *reinterpret_cast<const __nv_bfloat162*>(&hi.x);
-    const __nv_bfloat162 h23 = *reinterpret_cast<const __nv_bfloat162*>(&hi.y);
-    const uint2 lo = pack_bf16x4(u0 - __low2float(h01), u1 - __high2float(h01),
-                                 u2 - __low2float(h23), u3 - __high2float(h23));
-    *reinterpret_cast<uint2*>(d.u_hi + e) = hi;
-    *reinterpret_cast<uint2*>(d.u_lo + e) = lo;
+    *reinterpret_cast<uint2*>(d.u16 + e) = pack_f16x4(u0, u1, u2, u3);
   }
 }
 

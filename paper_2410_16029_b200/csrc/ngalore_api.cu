@@ -14,6 +14,7 @@
 #include "kernels_simt_gemm.cuh"
 #include "kernels_stream.cuh"
 #include "gemm_tcgen05.cuh"
+#include "backproject_tcgen05.cuh"
 #include "kernels_fused_stream.cuh"
 #include "refresh_tc.cuh"
 #include "static_natural_gradient.cuh"
@@ -310,6 +311,7 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
   bool ptr_changed = false;
   if ((rc = upload_pointers(st, W, G, stream, &ptr_changed))) return rc;
   if ((rc = upload_hyper(st, stream))) return rc;
+  if (st->opt.gemm_impl != 1 && (rc = tc_bind_buffers(st->tc, G, W, stream))) return rc;
   const int cur = st->s > 0 ? static_cast<int>(st->n_appended % st->s) : 0;
 
   if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[0], stream));
@@ -328,7 +330,7 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       st->launches += 1;
     }
   } else {
-    if ((rc = tc_project(st->tc, st->d_desc, st->d_ctrl, G, stream, &st->launches))) return rc;
+    if ((rc = tc_project(st->tc, st->d_desc, st->d_ctrl, stream, &st->launches))) return rc;
   }
   if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[1], stream));
   // ---- phase 1: Gram row, solve, natural gradient + moments
@@ -348,8 +350,8 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       const MatDesc& d = st->h_desc[i];
       SimtGemm g{};
       g.m = hm.M; g.n = hm.N; g.k = hm.rp;
-      g.A = d.P16; g.a_rs = d.ldp; g.a_cs = 1; g.a_dt = DT_BF16;
-      g.B = d.u_hi; g.B2 = d.u_lo; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_BF16;
+      g.A = d.P16; g.a_rs = d.ldp; g.a_cs = 1; g.a_dt = DT_F16;
+      g.B = d.u16; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_F16;
       g.C = W[i]; g.c_rs = hm.N; g.c_cs = 1; g.c_dt = DT_F32;
       g.epilogue = EPI_W_UPDATE;
       g.hyper = st->d_hyper;
@@ -358,7 +360,7 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       st->launches += 1;
     }
   } else {
-    if ((rc = tc_backproject(st->tc, st->d_desc, st->d_ctrl, st->d_hyper, st->d_W, stream, &st->launches))) return rc;
+    if ((rc = tc_backproject(st->tc, st->d_desc, st->d_ctrl, st->d_hyper, stream, &st->launches))) return rc;
   }
   advance_kernel<<<1, 1, 0, stream>>>(st->d_ctrl);
   st->launches += 1;
@@ -472,7 +474,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
 
   // ---- work layout
   off = 0;
-  struct WOffs { size_t uhi, ulo, gpart, Ya, Yb, Xa, Xb, C; };
+  struct WOffs { size_t u16, gpart, Ya, Yb, Xa, Xb, C; };
   std::vector<WOffs> woffs(n_matrices);
   const size_t o_hyper = take(sizeof(Hyper));
   const size_t o_desc = take(sizeof(MatDesc) * n_matrices);
@@ -490,8 +492,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     tile0[i] = n_tiles;
     for (int t = 0; t < ntl[i]; ++t) tiles.push_back(StreamTile{i, t});
     n_tiles += ntl[i];
-    woffs[i].uhi = take(sizeof(__nv_bfloat16) * hm.rn);
-    woffs[i].ulo = take(sizeof(__nv_bfloat16) * hm.rn);
+    woffs[i].u16 = take(sizeof(__half) * hm.rn);
     woffs[i].gpart = take(sizeof(double) * ntl[i] * slots);
     woffs[i].Ya = take(sizeof(float) * hm.M * hm.rp);
     woffs[i].Yb = take(sizeof(float) * hm.M * hm.rp);
@@ -536,12 +537,11 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     d.m = reinterpret_cast<float*>(st->arena + offs[i].m);
     d.v = reinterpret_cast<float*>(st->arena + offs[i].v);
     d.P32 = reinterpret_cast<float*>(st->arena + offs[i].P32);
-    d.P16 = reinterpret_cast<__nv_bfloat16*>(st->arena + offs[i].P16);
+    d.P16 = reinterpret_cast<__half*>(st->arena + offs[i].P16);
     d.Pt16 = reinterpret_cast<__nv_bfloat16*>(st->arena + offs[i].Pt16);
     d.Kraw = reinterpret_cast<double*>(st->arena + offs[i].Kraw);
     d.wsol = reinterpret_cast<float*>(st->arena + offs[i].wsol);
-    d.u_hi = reinterpret_cast<__nv_bfloat16*>(st->work + woffs[i].uhi);
-    d.u_lo = reinterpret_cast<__nv_bfloat16*>(st->work + woffs[i].ulo);
+    d.u16 = reinterpret_cast<__half*>(st->work + woffs[i].u16);
     d.gpart = reinterpret_cast<double*>(st->work + woffs[i].gpart);
     d.status = st->d_status + i;
     d.step_bad = st->d_step_bad + i;
@@ -576,6 +576,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
 
   ngalore_status rc = tc_plan_create(st->tc, st->h_desc, st->d_desc, s, prop.multiProcessorCount);
   if (rc != NGALORE_OK) return fail(rc);
+  if ((rc = tc_backproject_init()) != NGALORE_OK) return fail(rc);
   rc = fused_plan_create(st->fused, st->h_desc, s, prop.multiProcessorCount);
   if (rc != NGALORE_OK) return fail(rc);
   if (st->opt.gemm_impl != 1) {
@@ -704,7 +705,7 @@ ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, 
   DeviceGuard guard(st->device);
   const HostMat& hm = st->mats[i];
   const long long cnt = static_cast<long long>(hm.M) * hm.rp;
-  widen_bf16_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+  widen_f16_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
       st->h_desc[i].P16, P, cnt, hm.rp, st->h_desc[i].ldp);
   st->launches += 1;
   NG_CUDA(cudaGetLastError());

@@ -373,7 +373,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
         for (int m0 = 0; m0 < out_rows; m0 += kTcBM) {
           const int kb0 = sp * kb_per;
           const int kbn = std::min(kb_per, kb_total - kb0);
-          tiles[g].push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0});
+          tiles[g].push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0, out_rows, out_cols});
         }
   };
 
@@ -628,20 +628,20 @@ inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cu
   switch (g) {
     case RG_Y_FROM_Z:
       tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, false><<<plan.grid[g], threads, L1::kTotal, stream>>>(
-          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, nullptr, nullptr, plan.d_probs[g]);
+          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
       break;
     case RG_Z_FROM_Y:
       tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, true><<<plan.grid[g], threads, L1::kTotal, stream>>>(
-          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, nullptr, nullptr, plan.d_probs[g]);
+          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
       break;
     case RG_GRAM_Y:
     case RG_GRAM_Z:
       tc_gemm_kernel<kRefBN, 2, 2, kRefStages2, TC_EPI_STORE, 4, true><<<plan.grid[g], threads, L2::kTotal, stream>>>(
-          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, nullptr, nullptr, plan.d_probs[g]);
+          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
       break;
     default:
       tc_gemm_kernel<kRefBN, 2, 2, kRefStages2, TC_EPI_STORE, 4, false><<<plan.grid[g], threads, L2::kTotal, stream>>>(
-          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, nullptr, nullptr, plan.d_probs[g]);
+          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
       break;
   }
   *launches += 1;
