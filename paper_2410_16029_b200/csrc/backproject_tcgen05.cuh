@@ -8,9 +8,10 @@
 // with TMA stores.  The 128-byte swizzle of the W boxes makes the row-per-lane float4 accesses free of
 // bank conflicts, so no transposition is needed between the TMEM layout and shared memory.
 //
-// Warp roles: warp 0 TMA producer (W tile, then the K blocks of the operands), warp 1 TMEM owner and MMA
-// issuer, warps 2..9 epilogue in two groups of four; group g owns accumulator buffer g and W buffer g,
-// i.e. every second tile of the CTA.  Every mbarrier wait is bounded (see mbar_wait).
+// Warp roles: warp 0 TMA producer of the operands' K blocks, warp 1 TMEM owner and MMA issuer, warps 2..9
+// epilogue in two groups of four (group g owns accumulator buffer g and W buffer g, i.e. every second tile
+// of the CTA), warp 10 TMA producer of the W tiles, so that a wait for a W buffer never holds up the
+// operand pipeline.  Every mbarrier wait is bounded (see mbar_wait).
 #pragma once
 
 #include "gemm_tcgen05.cuh"
@@ -19,7 +20,8 @@ namespace ngalore {
 
 constexpr int kBpBN = 128;      // tile columns
 constexpr int kBpStages = 3;    // operand pipeline depth
-constexpr int kBpThreads = 64 + 32 * 8;
+constexpr int kBpWProducerWarp = 10;  // warps 0, 1: operand producer and MMA issuer; 2..9: epilogue; 10: W producer
+constexpr int kBpThreads = 32 * 11;
 
 struct BpSmem {
   static constexpr int kABytes = kTcBM * kTcBK * 2;                 // 16 KB
@@ -81,25 +83,16 @@ tc_backproject_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __res
   const int stride = gridDim.x;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer of the operands
     if (lane == 0 && static_cast<int>(blockIdx.x) < n_tiles) {
       int stage = 0;
       uint32_t phase = 0;
-      int local = 0;
       TcTile tile = tiles[blockIdx.x];
-      for (int t = blockIdx.x; t < n_tiles; t += stride, ++local) {
+      for (int t = blockIdx.x; t < n_tiles; t += stride) {
         const int tn = t + stride;
         const TcTile next = tiles[tn < n_tiles ? tn : t];  // fetched early: its latency hides behind this tile
         const CUtensorMap* maps = tmaps + tile.mat * kTcMapsPerMat;
-        const int buf = local & 1;
-        const uint32_t wphase = (local >> 1) & 1u;
         const int n_rem = tile.cols - tile.n0;
-        const int wchunks = n_rem >= kBpBN ? kBpBN / 32 : (n_rem + 31) >> 5;
-        if (!mbar_wait(wempty_bar + buf, wphase ^ 1u, abort_flag)) break;
-        mbar_expect_tx(wfull_bar + buf, static_cast<uint32_t>(wchunks) * L::kWChunkBytes);
-        unsigned char* sW = smem + L::kWOffset + buf * L::kWBufBytes;
-        for (int c = 0; c < wchunks; ++c)
-          tma_load_2d(sW + c * L::kWChunkBytes, maps + TC_MAP_W_LOAD, tile.n0 + c * 32, tile.m0, wfull_bar + buf);
         const int n_eff = n_rem >= kBpBN ? kBpBN : ((n_rem + 15) & ~15);
         const int nchunks = (n_eff + 63) >> 6;
         const uint32_t bytes = L::kABytes + nchunks * L::kBChunkBytes;
@@ -115,6 +108,27 @@ tc_backproject_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __res
           if (++stage == kBpStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
+        tile = next;
+      }
+    }
+  } else if (warp == kBpWProducerWarp) {
+    // ------------------------------------------------------------------ TMA producer of the W tiles
+    if (lane == 0 && static_cast<int>(blockIdx.x) < n_tiles) {
+      int local = 0;
+      TcTile tile = tiles[blockIdx.x];
+      for (int t = blockIdx.x; t < n_tiles; t += stride, ++local) {
+        const int tn = t + stride;
+        const TcTile next = tiles[tn < n_tiles ? tn : t];
+        const int buf = local & 1;
+        const uint32_t wphase = (local >> 1) & 1u;
+        const int n_rem = tile.cols - tile.n0;
+        const int wchunks = n_rem >= kBpBN ? kBpBN / 32 : (n_rem + 31) >> 5;
+        if (!mbar_wait(wempty_bar + buf, wphase ^ 1u, abort_flag)) break;
+        mbar_expect_tx(wfull_bar + buf, static_cast<uint32_t>(wchunks) * L::kWChunkBytes);
+        unsigned char* sW = smem + L::kWOffset + buf * L::kWBufBytes;
+        const CUtensorMap* mapW = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_W_LOAD;
+        for (int c = 0; c < wchunks; ++c)
+          tma_load_2d(sW + c * L::kWChunkBytes, mapW, tile.n0 + c * 32, tile.m0, wfull_bar + buf);
         tile = next;
       }
     }
