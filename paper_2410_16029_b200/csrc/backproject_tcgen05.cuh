@@ -1,45 +1,53 @@
 // Back-projection with the weight update fused in (Sec. 2.2):  W <- (1 - lr wd) W - lr P u  for every matrix.
 //
-// One persistent warp-specialised CTA per SM walks 128 x 128 tiles of W.  A = P16 (M x r', fp16, K-major),
-// B = u16 (r' x N, fp16), fp32 accumulator in TMEM (two buffers).  W never passes through registers as
-// global traffic: the producer warp brings the W tile into shared memory with TMA while the MMAs of the
-// tile (and the epilogue of the previous one) run, the epilogue warps update it in place, row per lane,
-// against the accumulator they read with tcgen05.ld, and one lane per warp sends the 32 x 32 boxes back
-// with TMA stores.  The 128-byte swizzle of the W boxes makes the row-per-lane float4 accesses free of
-// bank conflicts, so no transposition is needed between the TMEM layout and shared memory.
+// One persistent warp-specialised CTA per SM walks 128 x 256 tiles of W.  A = P16 (M x r', fp16, K-major),
+// B = u16 (r' x N, fp16), fp32 accumulator in TMEM (two buffers of 256 columns).  W never passes through
+// registers as global traffic: a producer warp streams the tile into shared memory with TMA, 32 columns
+// (one 16 KB slot of a ring) at a time, while the MMAs of the tile run; the epilogue warps update each slot
+// in place, row per lane, against the accumulator they read with tcgen05.ld, and one lane per warp sends
+// its 32 x 32 box back with a TMA store.  The 128-byte swizzle of the W boxes makes the row-per-lane float4
+// accesses free of bank conflicts, so no transposition is needed between the TMEM layout and shared memory.
+// The wide tile is what keeps the operand traffic from L2 (A once per 256 columns) below the W traffic.
 //
 // Warp roles: warp 0 TMA producer of the operands' K blocks, warp 1 TMEM owner and MMA issuer, warps 2..9
-// epilogue in two groups of four (group g owns accumulator buffer g and W buffer g, i.e. every second tile
-// of the CTA), warp 10 TMA producer of the W tiles, so that a wait for a W buffer never holds up the
-// operand pipeline.  Every mbarrier wait is bounded (see mbar_wait).
+// epilogue (warp quarter q = warp % 4 owns rows 32 q .. 32 q + 31 of the tile, the two warps of a quarter
+// take the even and the odd 32-column chunks), warp 10 TMA producer of the W slots.  Every mbarrier wait is
+// bounded (see mbar_wait).
 #pragma once
 
 #include "gemm_tcgen05.cuh"
 
 namespace ngalore {
 
-constexpr int kBpBN = 128;      // tile columns
-constexpr int kBpStages = 3;    // operand pipeline depth
-constexpr int kBpWProducerWarp = 10;  // warps 0, 1: operand producer and MMA issuer; 2..9: epilogue; 10: W producer
+constexpr int kBpBN = kTcBackBN;        // tile columns
+constexpr int kBpStages = 2;            // operand pipeline depth (48 KB per stage)
+constexpr int kBpSlots = 8;             // W ring: slots of 128 rows x 32 columns
+constexpr int kBpWProducerWarp = 10;    // warps 0, 1: operand producer and MMA issuer; 2..9: epilogue; 10: W producer
 constexpr int kBpThreads = 32 * 11;
 
 struct BpSmem {
   static constexpr int kABytes = kTcBM * kTcBK * 2;                 // 16 KB
   static constexpr int kBChunkBytes = 64 * kTcBK * 2;               // 8 KB: 64 columns x 64 K rows
-  static constexpr int kStageBytes = kABytes + (kBpBN / 64) * kBChunkBytes;  // 32 KB
+  static constexpr int kStageBytes = kABytes + (kBpBN / 64) * kBChunkBytes;  // 48 KB
   static constexpr int kWBoxBytes = 32 * 32 * 4;                    // 4 KB: 32 rows x 128 B
-  static constexpr int kWChunkBytes = 4 * kWBoxBytes;               // 128 rows x 32 columns
-  static constexpr int kWBufBytes = (kBpBN / 32) * kWChunkBytes;    // 64 KB
+  static constexpr int kWSlotBytes = 4 * kWBoxBytes;                // 128 rows x 32 columns
   static constexpr int kWOffset = kBpStages * kStageBytes;
-  static constexpr int kBarOffset = kWOffset + 2 * kWBufBytes;
+  static constexpr int kBarOffset = kWOffset + kBpSlots * kWSlotBytes;
   static constexpr int kTotal = kBarOffset + 256 + 1024;            // barriers + slack for 1024-byte alignment
 };
 static_assert(BpSmem::kTotal <= 232448, "shared memory budget of one CTA");
+static_assert((2 * kBpStages + 4 + 2 * kBpSlots) * 8 + 8 <= 256, "barrier block");
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
                ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(src))
                : "memory");
+}
+
+// 32-column chunks of W a tile covers.
+__device__ __forceinline__ int bp_wchunks(const TcTile& tile) {
+  const int n_rem = tile.cols - tile.n0;
+  return n_rem >= kBpBN ? kBpBN / 32 : (n_rem + 31) >> 5;
 }
 
 __global__ void __launch_bounds__(kBpThreads, 1)
@@ -53,26 +61,22 @@ tc_backproject_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __res
   uint64_t* empty_bar = bars + kBpStages;           // [kBpStages] operands consumed
   uint64_t* tfull_bar = bars + 2 * kBpStages;       // [2] accumulator complete
   uint64_t* tempty_bar = bars + 2 * kBpStages + 2;  // [2] accumulator drained
-  uint64_t* wfull_bar = bars + 2 * kBpStages + 4;   // [2] W tile landed
-  uint64_t* wempty_bar = bars + 2 * kBpStages + 6;  // [2] W tile sent back (its shared memory is free)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kBpStages + 8);
+  uint64_t* wfull_bar = bars + 2 * kBpStages + 4;   // [kBpSlots] W slot landed
+  uint64_t* wempty_bar = wfull_bar + kBpSlots;      // [kBpSlots] W slot sent back (its shared memory is free)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wempty_bar + kBpSlots);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kBpStages; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(tfull_bar + b, 1);
-      mbar_init(tempty_bar + b, 4);
-      mbar_init(wfull_bar + b, 1);
-      mbar_init(wempty_bar + b, 4);
-    }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, 8); }
+    for (int s = 0; s < kBpSlots; ++s) { mbar_init(wfull_bar + s, 1); mbar_init(wempty_bar + s, 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -112,23 +116,25 @@ tc_backproject_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __res
       }
     }
   } else if (warp == kBpWProducerWarp) {
-    // ------------------------------------------------------------------ TMA producer of the W tiles
+    // ------------------------------------------------------------------ TMA producer of the W slots
+    // The slots are used in the order (tile, chunk); slot and barrier phase follow from the running count.
     if (lane == 0 && static_cast<int>(blockIdx.x) < n_tiles) {
-      int local = 0;
+      int slot = 0;
+      uint32_t phase = 0;
       TcTile tile = tiles[blockIdx.x];
-      for (int t = blockIdx.x; t < n_tiles; t += stride, ++local) {
+      for (int t = blockIdx.x; t < n_tiles; t += stride) {
         const int tn = t + stride;
         const TcTile next = tiles[tn < n_tiles ? tn : t];
-        const int buf = local & 1;
-        const uint32_t wphase = (local >> 1) & 1u;
-        const int n_rem = tile.cols - tile.n0;
-        const int wchunks = n_rem >= kBpBN ? kBpBN / 32 : (n_rem + 31) >> 5;
-        if (!mbar_wait(wempty_bar + buf, wphase ^ 1u, abort_flag)) break;
-        mbar_expect_tx(wfull_bar + buf, static_cast<uint32_t>(wchunks) * L::kWChunkBytes);
-        unsigned char* sW = smem + L::kWOffset + buf * L::kWBufBytes;
+        const int wchunks = bp_wchunks(tile);
         const CUtensorMap* mapW = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_W_LOAD;
-        for (int c = 0; c < wchunks; ++c)
-          tma_load_2d(sW + c * L::kWChunkBytes, mapW, tile.n0 + c * 32, tile.m0, wfull_bar + buf);
+        bool ok = true;
+        for (int c = 0; c < wchunks; ++c) {
+          if (!mbar_wait(wempty_bar + slot, phase ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(wfull_bar + slot, L::kWSlotBytes);
+          tma_load_2d(smem + L::kWOffset + slot * L::kWSlotBytes, mapW, tile.n0 + c * 32, tile.m0, wfull_bar + slot);
+          if (++slot == kBpSlots) { slot = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
         tile = next;
       }
     }
@@ -173,62 +179,87 @@ tc_backproject_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __res
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2 .. 9)
     const int quarter = warp & 3;        // TMEM lanes 32 * quarter .. + 31 belong to this warp
-    const int group = (warp - 2) >> 2;   // accumulator / W buffer this warp's group owns
+    const int parity = (warp - 2) >> 2;  // this warp takes the chunks with (c & 1) == parity
     const float lr = hyper->lr, decay = 1.f - hyper->lr * hyper->wd;
-    unsigned char* sW = smem + L::kWOffset + group * L::kWBufBytes + quarter * L::kWBoxBytes;
-    const int first = blockIdx.x + group * stride;
-    if (first < n_tiles) {
-      TcTile tile = tiles[first];
+    int slot = 0;                        // ring position of the tile's chunk 0, advanced over all chunks
+    uint32_t phase = 0;
+    int pending_slot = -1;               // slot whose store was issued last and is not yet released
+    if (static_cast<int>(blockIdx.x) < n_tiles) {
+      TcTile tile = tiles[blockIdx.x];
       int bad = __ldcg(mats[tile.mat].step_bad);
-      int it = 0;
-      for (int t = first; t < n_tiles; t += 2 * stride, ++it) {
-        const int tn = t + 2 * stride;
+      int local = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += stride, ++local) {
+        const int tn = t + stride;
         const TcTile next = tiles[tn < n_tiles ? tn : t];
         const int bad_next = __ldcg(mats[next.mat].step_bad);
-        const uint32_t ph = it & 1u;
-        const int n_rem = tile.cols - tile.n0;
-        const int wchunks = n_rem >= kBpBN ? kBpBN / 32 : (n_rem + 31) >> 5;
-        // every lane polls; the warp goes on only if all of them saw both barriers complete
-        bool ready = mbar_wait(wfull_bar + group, ph, abort_flag);
-        ready = ready && mbar_wait(tfull_bar + group, ph, abort_flag);
-        if (!__all_sync(0xffffffffu, ready)) break;
+        const int buf = local & 1;
+        const uint32_t tphase = (local >> 1) & 1u;
+        const int wchunks = bp_wchunks(tile);
+        const int row0 = tile.m0 + quarter * 32;
+        const bool store = !bad && row0 < tile.rows;
+        const CUtensorMap* mapW = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_W_STORE;
+        // every lane polls; the warp goes on only if all of them saw the barrier complete
+        if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar + buf, tphase, abort_flag))) break;
         tc_fence_after();
+        const int last_own = ((wchunks - 1 - parity) & ~1) + parity;  // this warp's last chunk (< parity: none)
+        if (last_own < parity) {
+          tc_fence_before();
+          if (lane == 0) mbar_arrive(tempty_bar + buf);
+        }
         for (int c = 0; c < wchunks; ++c) {
-          uint32_t r[32];
-          tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(group * kBpBN + c * 32), r);
-          tc_wait_ld();
-          if (c == wchunks - 1) {
-            // all TMEM reads of this tile are done: the MMAs of the group's next tile may start
-            tc_fence_before();
-            if (lane == 0) mbar_arrive(tempty_bar + group);
-          }
-          // this lane's row of the 32 x 32 box: 16-byte piece j sits at piece (j ^ (row & 7)) of the 128-byte row
-          unsigned char* rowp = sW + c * L::kWChunkBytes + lane * 128;
+          if ((c & 1) == parity) {
+            if (!__all_sync(0xffffffffu, mbar_wait(wfull_bar + slot, phase, abort_flag))) { ok = false; break; }
+            uint32_t r[32];
+            tc_ld32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * kBpBN + c * 32), r);
+            tc_wait_ld();
+            if (c == last_own) {
+              // this warp's TMEM reads of the tile are done; with all eight arrivals the next MMAs may start
+              tc_fence_before();
+              if (lane == 0) mbar_arrive(tempty_bar + buf);
+            }
+            // this lane's row of the 32 x 32 box: 16-byte piece j sits at piece (j ^ (row & 7)) of the 128-byte row
+            unsigned char* box = smem + L::kWOffset + slot * L::kWSlotBytes + quarter * L::kWBoxBytes;
+            unsigned char* rowp = box + lane * 128;
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            float4* p = reinterpret_cast<float4*>(rowp + ((j ^ (lane & 7)) << 4));
-            float4 w = *p;
-            w.x = decay * w.x - lr * __uint_as_float(r[4 * j]);
-            w.y = decay * w.y - lr * __uint_as_float(r[4 * j + 1]);
-            w.z = decay * w.z - lr * __uint_as_float(r[4 * j + 2]);
-            w.w = decay * w.w - lr * __uint_as_float(r[4 * j + 3]);
-            *p = w;
+            for (int j = 0; j < 8; ++j) {
+              float4* p = reinterpret_cast<float4*>(rowp + ((j ^ (lane & 7)) << 4));
+              float4 w = *p;
+              w.x = decay * w.x - lr * __uint_as_float(r[4 * j]);
+              w.y = decay * w.y - lr * __uint_as_float(r[4 * j + 1]);
+              w.z = decay * w.z - lr * __uint_as_float(r[4 * j + 2]);
+              w.w = decay * w.w - lr * __uint_as_float(r[4 * j + 3]);
+              *p = w;
+            }
+            // hand the updated rows to the async proxy, then one lane stores the box; the slot is released
+            // once the store has read it, which inside a tile is checked one chunk later so that the warp
+            // does not idle
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+              if (store) {
+                tma_store_2d(mapW, tile.n0 + c * 32, row0, box);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                if (pending_slot >= 0) {
+                  asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                  mbar_arrive(wempty_bar + pending_slot);
+                }
+                pending_slot = slot;
+              } else {
+                mbar_arrive(wempty_bar + slot);
+              }
+            }
+            __syncwarp();
           }
+          if (++slot == kBpSlots) { slot = 0; phase ^= 1u; }
         }
-        // hand the updated rows to the async proxy, then one lane stores the warp's boxes
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) {
-          const int row0 = tile.m0 + quarter * 32;
-          if (!bad && row0 < tile.rows) {
-            const CUtensorMap* mapW = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_W_STORE;
-            for (int c = 0; c < wchunks; ++c) tma_store_2d(mapW, tile.n0 + c * 32, row0, sW + c * L::kWChunkBytes);
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-          }
-          mbar_arrive(wempty_bar + group);
+        // No release stays pending across tiles: the W producer may need the slot before this warp's next
+        // chunk comes up (a narrow tile can leave a warp without a chunk of its own).
+        if (lane == 0 && pending_slot >= 0) {
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          mbar_arrive(wempty_bar + pending_slot);
+          pending_slot = -1;
         }
-        __syncwarp();
         tile = next;
         bad = bad_next;
       }
@@ -246,7 +277,7 @@ tc_backproject_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __res
   }
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 

@@ -406,6 +406,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 constexpr int kProjBN = 256, kProjStages = 4, kProjEpiWarps = 4;
+constexpr int kTcBackBN = 256;  // tile width of the back-projection kernel
 
 struct TcPlan {
   size_t device_bytes = 0;
@@ -505,7 +506,7 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
     const MatDesc& d = mats[i];
     const int kbn = (d.rp + kTcBK - 1) / kTcBK;
     for (int m0 = 0; m0 < d.M; m0 += kTcBM)
-      for (int n0 = 0; n0 < d.N; n0 += 128) back.push_back(TcTile{i, m0, n0, 0, kbn, 0, d.M, d.N});
+      for (int n0 = 0; n0 < d.N; n0 += kTcBackBN) back.push_back(TcTile{i, m0, n0, 0, kbn, 0, d.M, d.N});
   }
   plan.n_tiles_proj = static_cast<int>(proj.size());
   plan.n_tiles_back = static_cast<int>(back.size());
