@@ -29,8 +29,8 @@ if ROOT not in sys.path:
 # and expressed per unit of work so that it scales to the full workload: the stream kernel's traffic grows with
 # the low-rank elements sum(r' N), the GEMMs' with sum(M N).  Valid for r = 512, s = 16 only; set an entry to None
 # when its kernel changes.
-NCU_TRAFFIC_PER_UNIT = {"fused_stream_kernel": ("rn", 146.93), "tc_gemm_kernel<backproject>": ("mn", 8.621),
-                        "tc_gemm_kernel<project>": ("mn", 3.064)}
+NCU_TRAFFIC_PER_UNIT = {"fused_stream_kernel": ("rn", 145.04), "tc_backproject_kernel": ("mn", 8.382),
+                        "tc_gemm_kernel<project>": ("mn", 3.075)}
 
 METRIC = "optimizer steps/sec over all matrices (device-timed)"
 UNIT = "steps/s"
@@ -315,7 +315,7 @@ def run_ours(args, wl):
     # ---- roofline of the dominant kernel and of the whole step
     peak, peak_kind = measured_peak_hbm()
     tot_bytes, stream_bytes = byte_model(wl)
-    names = ["tc_gemm_kernel<project>", "fused_stream_kernel", "tc_gemm_kernel<backproject>"]
+    names = ["tc_gemm_kernel<project>", "fused_stream_kernel", "tc_backproject_kernel"]
     proj_bytes = sum(2 * M * N + 2 * M * wl.rank_of(i) + 4 * wl.rank_of(i) * N for i, (M, N) in enumerate(shapes))
     back_bytes = sum(8 * M * N + 2 * M * wl.rank_of(i) for i, (M, N) in enumerate(shapes))
     alg = [proj_bytes, stream_bytes, back_bytes]
@@ -343,7 +343,7 @@ def run_ours(args, wl):
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-           "vs_baseline": None, "dtype": "bf16 GEMM operands, f32 state/accumulation, f64 Gram+solve",
+           "vs_baseline": None, "dtype": "bf16 (projection) and fp16 (back-projection) GEMM operands, f32 state/accumulation, f64 Gram+solve",
            "data": "synthetic",
            "config": {"workload": wl.name, "matrices": n, "r": wl.r, "s": wl.s, "T": wl.T,
                       "l2": f"inputs larger than L2: {pool_sets} gradient sets of {grad_bytes / 1e9:.2f} GB cycled",
