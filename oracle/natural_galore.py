@@ -21,7 +21,11 @@ paper gives:
 with U = [vec(H_1) ... vec(H_c)] / sqrt(c) and c the number of gradients held.
 
 Readings taken where the paper is silent or inconsistent (each is listed in the
-design notes): left projection only; r' = min(r, M, N); the empirical Fisher is
+design notes): left projection only (the default; ``Hyper.projection =
+"short_side"`` selects the GaLore convention the paper inherits when it says, at
+the start of Sec. 2.4, that most steps are those of GaLore: project on the
+right, R = G Q with Q the first r' right singular vectors, when M >= N);
+r' = min(r, M, N); the empirical Fisher is
 the *mean* of outer products plus lambda I (the 1/h of the Sec. 2.2 definition
 carried into Sec. 2.4); exactly s columns, the current gradient among them;
 divide by the number of gradients actually held while the history fills; eps
@@ -63,6 +67,15 @@ def left_singular_basis(G: np.ndarray, r: int) -> np.ndarray:
     rp = min(r, G.shape[0], G.shape[1])
     U, _, _ = np.linalg.svd(G, full_matrices=False)
     return np.ascontiguousarray(U[:, :rp])
+
+
+def right_singular_basis(G: np.ndarray, r: int) -> np.ndarray:
+    """First r' = min(r, M, N) right singular vectors of G, as the columns of an N x r' matrix
+    (compact SVD G = P Sigma Q^T, Sec. 1; used by the short-side projection rule)."""
+    G = np.asarray(G, dtype=np.float64)
+    rp = min(r, G.shape[0], G.shape[1])
+    _, _, Vt = np.linalg.svd(G, full_matrices=False)
+    return np.ascontiguousarray(Vt[:rp, :].T)
 
 
 def project(P: np.ndarray, G: np.ndarray) -> np.ndarray:
@@ -157,6 +170,7 @@ class Hyper:
     eps_outside: bool = False
     reset_history_on_refresh: bool = False
     store_P_as_bf16: bool = True
+    projection: str = "left"        # "left": always R = P^T G; "short_side": R = G Q when M >= N
 
 
 class MatrixState:
@@ -165,9 +179,15 @@ class MatrixState:
     def __init__(self, M: int, N: int, hp: Hyper):
         self.M, self.N, self.hp = M, N, hp
         self.rp = min(hp.r, M, N)
-        self.P: Optional[np.ndarray] = None
-        self.m = np.zeros((self.rp, N), dtype=np.float64)
-        self.v = np.zeros((self.rp, N), dtype=np.float64)
+        if hp.projection not in ("left", "short_side"):
+            raise ValueError(hp.projection)
+        # Short-side rule: the projector lives on the shorter side of the matrix; a square matrix
+        # takes the right projection, as in GaLore.
+        self.right = hp.projection == "short_side" and M >= N
+        self.P: Optional[np.ndarray] = None      # M x r' (left) or the N x r' matrix Q (right)
+        low_rank_shape = (M, self.rp) if self.right else (self.rp, N)
+        self.m = np.zeros(low_rank_shape, dtype=np.float64)
+        self.v = np.zeros(low_rank_shape, dtype=np.float64)
         self.slots: List[Optional[np.ndarray]] = [None] * max(hp.s, 0)
         self.head = 0
         self.count = 0
@@ -178,11 +198,13 @@ class MatrixState:
     # -- subspace -------------------------------------------------------------
     def set_subspace(self, P: np.ndarray) -> None:
         P = np.asarray(P, dtype=np.float64)
-        assert P.shape == (self.M, self.rp), (P.shape, (self.M, self.rp))
+        want = (self.N if self.right else self.M, self.rp)
+        assert P.shape == want, (P.shape, want)
         self.P = round_to_bf16(P) if self.hp.store_P_as_bf16 else P.copy()
 
     def refresh(self, G: np.ndarray) -> None:
-        self.set_subspace(left_singular_basis(G, self.hp.r))
+        basis = right_singular_basis if self.right else left_singular_basis
+        self.set_subspace(basis(G, self.hp.r))
         if self.hp.reset_history_on_refresh:
             self.slots = [None] * max(self.hp.s, 0)
             self.head = 0
@@ -200,7 +222,7 @@ class MatrixState:
             self.refresh(G)
         if self.P is None:
             raise RuntimeError("no subspace: refresh first")
-        R = project(self.P, G)                                          # O1
+        R = G @ self.P if self.right else project(self.P, G)            # O1
         if hp.s > 0:
             self.slots[self.head] = R                                   # O2
             self.head = (self.head + 1) % hp.s
@@ -211,7 +233,8 @@ class MatrixState:
         self.m, self.v, u = adam_moments(self.m, self.v, Nt, hp.beta1, hp.beta2, hp.eps,
                                          step_index=self.k, bias_correction=hp.bias_correction,
                                          eps_outside=hp.eps_outside)    # O6
-        dW = -hp.lr * (self.P @ u) - hp.lr * hp.wd * W                  # O7
+        back = u @ self.P.T if self.right else self.P @ u
+        dW = -hp.lr * back - hp.lr * hp.wd * W                          # O7
         W += dW
         self.k += 1
         self.last_natural_gradient = Nt

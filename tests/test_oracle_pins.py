@@ -353,3 +353,75 @@ def test_adam_moments_as_printed():
     m, v, u = orc.adam_moments(np.array([0.0]), np.array([0.0]), np.array([2.0]), 0.9, 0.999, 1e-8)
     assert m[0] == pytest.approx(0.2) and v[0] == pytest.approx(0.004)
     assert u[0] == pytest.approx(0.2 / math.sqrt(0.004 + 1e-8), rel=1e-14)
+
+
+# ----------------------------------------------------------------------------- short-side projection rule
+
+def test_right_singular_basis_recovers_planted_right_factor():
+    """Eckart-Young on the right: G = A diag(sigma) B^T with orthonormal A, B has B[:, :r] as its
+    leading right singular subspace."""
+    rng = np.random.default_rng(41)
+    M, N, r = 40, 24, 5
+    A, _ = np.linalg.qr(rng.standard_normal((M, N)))
+    B, _ = np.linalg.qr(rng.standard_normal((N, N)))
+    sigma = np.array([10.0, 7.0, 5.0, 3.0, 2.0] + [0.1] * (N - 5))
+    G = (A * sigma) @ B.T
+    Q = orc.right_singular_basis(G, r)
+    assert Q.shape == (N, r)
+    assert np.max(np.abs(Q.T @ Q - np.eye(r))) <= 1e-12
+    assert np.linalg.norm(Q @ Q.T - B[:, :r] @ B[:, :r].T, 2) <= 1e-10
+
+
+@pytest.mark.parametrize("M,N", [(24, 16), (16, 16)])
+def test_right_projection_is_the_left_projection_of_the_transposed_problem(M, N):
+    """Projecting G on the right with Q is projecting G^T on the left with the same Q; every later
+    step acts on vec() of the low-rank gradient, whose element order the mathematics ignores.  So
+    the updates of a tall matrix under the short-side rule are the transposed updates of its
+    transpose under the left rule."""
+    rng = np.random.default_rng(43)
+    hp_short = orc.Hyper(r=4, s=3, T=4, lr=1e-2, wd=0.1, projection="short_side", store_P_as_bf16=False)
+    hp_left = orc.Hyper(r=4, s=3, T=4, lr=1e-2, wd=0.1, projection="left", store_P_as_bf16=False)
+    a = orc.MatrixState(M, N, hp_short)
+    b = orc.MatrixState(N, M, hp_left)
+    assert a.right and not b.right
+    Wa = rng.standard_normal((M, N))
+    Wb = Wa.T.copy()
+    for k in range(9):
+        G = sum((0.5 ** i) * np.outer(rng.standard_normal(M), rng.standard_normal(N)) for i in range(6))
+        if k % 4 == 0:
+            # one basis for both: signs of singular vectors are not unique, and the moments kept across
+            # a refresh make the update depend on them
+            Q = orc.right_singular_basis(G, 4)
+            a.set_subspace(Q)
+            b.set_subspace(Q)
+        da = a.step(Wa, G, auto_refresh=False)
+        db = b.step(Wb, G.T.copy(), auto_refresh=False)
+        assert np.linalg.norm(da - db.T) <= 1e-9 * np.linalg.norm(db), k
+    assert np.linalg.norm(Wa - Wb.T) <= 1e-9 * np.linalg.norm(Wb)
+    assert a.m.shape == (M, 4) and b.m.shape == (4, M)
+
+
+def test_short_side_rule_picks_the_side_and_leaves_wide_matrices_alone():
+    """M < N keeps the left projection (identical numbers to the default rule); M >= N projects on the right."""
+    rng = np.random.default_rng(47)
+    hp_short = orc.Hyper(r=3, s=2, T=3, projection="short_side")
+    hp_left = orc.Hyper(r=3, s=2, T=3)
+    wide_s, wide_l = orc.MatrixState(8, 16, hp_short), orc.MatrixState(8, 16, hp_left)
+    assert not wide_s.right
+    assert orc.MatrixState(16, 8, hp_short).right and orc.MatrixState(8, 8, hp_short).right
+    Ws, Wl = np.zeros((8, 16)), np.zeros((8, 16))
+    for k in range(5):
+        G = rng.standard_normal((8, 16))
+        assert np.array_equal(wide_s.step(Ws, G), wide_l.step(Wl, G))
+
+
+def test_right_projected_update_lies_in_the_row_space_of_Q():
+    """Delta W = -lr u Q^T (Sec. 2.2 update with the projector on the right): its rows are combinations of Q's columns."""
+    rng = np.random.default_rng(53)
+    st = orc.MatrixState(20, 12, orc.Hyper(r=3, s=2, T=100, projection="short_side", store_P_as_bf16=False))
+    W = np.zeros((20, 12))
+    dW = st.step(W, rng.standard_normal((20, 12)))
+    Q = st.P
+    assert Q.shape == (12, 3)
+    assert np.linalg.norm(dW - dW @ Q @ Q.T) <= 1e-12 * np.linalg.norm(dW)
+    assert np.linalg.matrix_rank(dW, tol=1e-10) <= 3
