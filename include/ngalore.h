@@ -16,6 +16,9 @@
  * and, every T steps, first refreshes P to an orthonormal basis of the
  * dominant r'-dimensional left singular subspace of G, r' = min(r, M, N)
  * (Sec. 1: P from the compact SVD of the gradient, "updated periodically").
+ * With ngalore_options.projection_rule = 1 a matrix with M >= N uses the mirrored
+ * form instead: R = G Q, W <- (1 - lr wd) W - lr u Q^T, Q (N x r') from the
+ * right singular vectors; everything between projection and update is the same.
  *
  * Conventions
  *  - All matrix pointers are DEVICE pointers unless a parameter says "host".
@@ -71,7 +74,11 @@ typedef struct {
   int32_t reset_history_on_refresh; /* default 0: history, m and v survive a refresh */
   uint64_t seed;                    /* seed of the refresh's random test matrix; 0 selects a fixed default */
   int32_t stream_impl;              /* 0 (default): fused Gram/solve/moment kernel; 1: separate plain kernels (debug) */
-  int32_t reserved;
+  int32_t projection_rule;          /* 0 (default): every matrix is projected on the left, R = P^T G, as the paper
+                                       writes it; 1: the short-side rule of GaLore, which the paper's "most steps are
+                                       similar to GaLore" (start of Sec. 2.4) inherits: a matrix with rows >= cols is
+                                       projected on the right, R = G Q (rows x r'), W <- (1 - lr wd) W - lr u Q^T, with
+                                       Q (cols x r') spanning the leading right singular vectors of G */
 } ngalore_options;
 
 /*
@@ -130,7 +137,8 @@ ngalore_status ngalore_step_host(ngalore_state* st, float* const* W_host, const 
  * Returns NGALORE_OK when all are OK, else the first non-OK status. */
 ngalore_status ngalore_poll_status(ngalore_state* st, int* per_matrix);
 
-/* Copy the fp32 master of P (rows x r', row-major) of matrix i to / from the device buffer P.
+/* Copy the fp32 master of the projector of matrix i (ngalore_subspace_rows(i) x r', row-major: P, or Q for a
+ * matrix projected on the right) to / from the device buffer P.
  * set also rebuilds the bf16 working copies; the step uses the bf16 values. */
 ngalore_status ngalore_get_subspace(ngalore_state* st, int i, float* P, void* stream);
 ngalore_status ngalore_set_subspace(ngalore_state* st, int i, const float* P, void* stream);
@@ -149,6 +157,8 @@ ngalore_status ngalore_set_lr(ngalore_state* st, double lr);
 /* Introspection (host values, no device work). */
 int ngalore_num_matrices(const ngalore_state* st);
 int ngalore_rank(const ngalore_state* st, int i);          /* r' of matrix i, -1 if i is out of range */
+int ngalore_projects_right(const ngalore_state* st, int i); /* 1 if matrix i is projected on the right, 0 if on the left, -1 if out of range */
+int ngalore_subspace_rows(const ngalore_state* st, int i);  /* rows of its projector: M (left) or N (right), -1 if out of range */
 int64_t ngalore_step_count(const ngalore_state* st);        /* k */
 size_t ngalore_device_bytes(const ngalore_state* st);       /* device memory held by the state */
 /* Kernels launched by the library on behalf of this state since creation. */

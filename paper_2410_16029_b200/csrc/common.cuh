@@ -14,16 +14,22 @@ constexpr int kStreamThreads = 256;   // threads per CTA of the streaming kernel
 // Per-matrix device descriptor (array in device memory, one entry per weight matrix).
 struct MatDesc {
   int M, N, rp, s;            // rows, cols, r' = min(r, M, N), history length
-  long long rn;               // rp * N, elements of one low-rank matrix
-  int ldp, ldpt;              // leading dimensions of P16 (>= rp) and Pt16 (>= M), multiples of 8 for TMA
+  int right;                  // 0: left projection R = P^T G (r' x N); 1: right projection R = G Q (M x r')
+  int pr;                     // rows of the projector: M (left) or N (right)
+  int lr_rows, lr_cols;       // layout of one low-rank matrix: r' x N (left) or M x ldp (right; columns >= r' stay zero)
+  long long rn;               // lr_rows * lr_cols, elements of one low-rank matrix
+  int ldp, ldpt;              // leading dimensions of P16 (>= rp) and Pt16 (>= pr), multiples of 8 for TMA
   float* H;                   // history ring: s slots of rp x N fp32 (one slot when s == 0)
   float* m;                   // first moment, rp x N
   float* v;                   // second moment, rp x N
-  __half* u16;                // direction u = m / sqrt(v + eps) rounded to fp16, rp x N
-  __half* P16;                // working copy of P for the back-projection: the bf16-rounded values held as
-                              // fp16 (same numbers as Pt16), M x ldp row-major (padding is zero)
-  __nv_bfloat16* Pt16;        // working copy of P^T, rp x ldpt row-major
-  float* P32;                 // fp32 master of P, M x rp row-major
+  __half* u16;                // direction u = m / sqrt(v + eps) rounded to fp16, lr_rows x lr_cols
+  // Working copies of the projector, both holding the bf16-rounded values of P32 (padding is zero).  The
+  // projection GEMM reads bf16 (its other operand G is bf16), the back-projection fp16 (its other operand u is):
+  //   left:  P16 (pr x ldp) as fp16 = A of the back-projection;  Pt16 (rp x ldpt) as bf16 = A of the projection
+  //   right: P16 (pr x ldp) as bf16 = B of the projection;       Pt16 (rp x ldpt) as fp16 = B of the back-projection
+  uint16_t* P16;
+  uint16_t* Pt16;
+  float* P32;                 // fp32 master of the projector, pr x rp row-major
   double* Kraw;               // s x s raw inner products <H_i, H_j>
   float* wsol;                // kMaxHistory solution weights of (lambda I + K) w = e_cur
   double* gpart;              // per-tile partial Gram rows: ntiles x s

@@ -3,6 +3,7 @@
 // warp-specialised CTA per SM.
 //
 //   projection       R = P^T G          A = Pt16 (r' x M, K-major), B = G (M x N, N contiguous)
+//                    or, for a matrix projected on the right, R = G Q:  A = G (M x N, K = N), B = Q (N x r')
 //                    epilogue: store (or atomically add, when K is split) into ring slot `cur`   (Sec. 1)
 //   store mode       out = A B for a table of problems (subspace refresh)
 //
@@ -49,10 +50,11 @@ struct TcTile {
 
 // Tensor maps of the step GEMMs, kTcMapsPerMat consecutive entries per matrix.
 enum {
-  TC_MAP_A_PROJ = 0,   // Pt16: r' rows x M (K), box 64 x 128
-  TC_MAP_B_PROJ = 1,   // G: M (K) rows x N, box 64 x 64
-  TC_MAP_A_BACK = 2,   // P16: M rows x r' (K), box 64 x 128
-  TC_MAP_B_BACK = 3,   // u16: r' (K) rows x N, box 64 x 64
+  // left projection                                        right projection
+  TC_MAP_A_PROJ = 0,   // Pt16: r' rows x M (K), box 64 x 128      G: M rows x N (K)
+  TC_MAP_B_PROJ = 1,   // G: M (K) rows x N, box 64 x 64           P16 = Q (bf16): N (K) rows x r'
+  TC_MAP_A_BACK = 2,   // P16: M rows x r' (K), box 64 x 128       u16: M rows x r' (K)
+  TC_MAP_B_BACK = 3,   // u16: r' (K) rows x N, box 64 x 64        Pt16 = Q^T (fp16): r' (K) rows x N
   TC_MAP_W_LOAD = 4,   // W (fp32): M rows x N, box 32 columns x 128 rows
   TC_MAP_W_STORE = 5,  // W (fp32): box 32 x 32
   kTcMapsPerMat = 6
@@ -224,7 +226,7 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
         } else {
           mapA = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_A_PROJ;
           mapB0 = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_B_PROJ;
-          out_cols = mats[tile.mat].N;
+          out_cols = tile.cols;
         }
         const int n_rem = out_cols - tile.n0;
         const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
@@ -263,7 +265,7 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
       bool ok = true;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
         const TcTile tile = tiles[t];
-        const int out_cols = (EPI == TC_EPI_STORE) ? probs[tile.mat].out_cols : mats[tile.mat].N;
+        const int out_cols = (EPI == TC_EPI_STORE) ? probs[tile.mat].out_cols : tile.cols;
         const int n_rem = out_cols - tile.n0;
         const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
         const uint32_t idesc = instr_desc(n_eff, A_MN, F16);
@@ -323,10 +325,10 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
         ld_out = pr.ld_out;
       } else {
         const MatDesc& d = mats[tile.mat];
-        out_cols = d.N;
-        ld_out = d.N;
+        out_cols = tile.cols;
+        ld_out = tile.cols;
         out = d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn;
-        rows_total = d.rp;
+        rows_total = tile.rows;
       }
       const int n_rem = out_cols - tile.n0;
       const int n_eff = n_rem >= BN ? BN : ((n_rem + 15) & ~15);
@@ -415,6 +417,7 @@ struct TcPlan {
   std::vector<CUtensorMap> h_maps;  // kTcMapsPerMat per matrix (TC_MAP_*)
   std::vector<int> rowsN;           // per matrix: M, N for re-encoding the maps of G and W
   std::vector<int> colsN;
+  std::vector<int> right;           // per matrix: projected on the right
   std::vector<const void*> last_G;
   std::vector<const void*> last_W;
   CUtensorMap* d_maps = nullptr;
@@ -462,24 +465,34 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   std::memset(plan.h_maps.data(), 0, sizeof(CUtensorMap) * plan.h_maps.size());
   for (int i = 0; i < n; ++i) {
     const MatDesc& d = mats[i];
-    // A_proj: Pt16, r' rows x M (K) columns, row stride ldpt
-    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * kTcMapsPerMat + TC_MAP_A_PROJ], d.Pt16, d.M, d.rp, static_cast<uint64_t>(d.ldpt) * 2, kTcBK, kTcBM))
-      return NGALORE_ERR_CUDA;
-    // A_back: P16, M rows x r' (K) columns, row stride ldp
-    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * kTcMapsPerMat + TC_MAP_A_BACK], d.P16, d.rp, d.M, static_cast<uint64_t>(d.ldp) * 2, kTcBK, kTcBM))
-      return NGALORE_ERR_CUDA;
-    // B_back: u16, r' (K) rows x N columns
-    if (!tc_encode_2d(plan.encode, &plan.h_maps[i * kTcMapsPerMat + TC_MAP_B_BACK], d.u16, d.N, d.rp, static_cast<uint64_t>(d.N) * 2, 64, kTcBK))
-      return NGALORE_ERR_CUDA;
+    CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * kTcMapsPerMat];
+    bool ok = true;
+    if (!d.right) {
+      // A_proj: Pt16, r' rows x M (K) columns, row stride ldpt
+      ok &= tc_encode_2d(plan.encode, mp + TC_MAP_A_PROJ, d.Pt16, d.M, d.rp, static_cast<uint64_t>(d.ldpt) * 2, kTcBK, kTcBM);
+      // A_back: P16, M rows x r' (K) columns, row stride ldp
+      ok &= tc_encode_2d(plan.encode, mp + TC_MAP_A_BACK, d.P16, d.rp, d.M, static_cast<uint64_t>(d.ldp) * 2, kTcBK, kTcBM);
+      // B_back: u16, r' (K) rows x N columns
+      ok &= tc_encode_2d(plan.encode, mp + TC_MAP_B_BACK, d.u16, d.N, d.rp, static_cast<uint64_t>(d.N) * 2, 64, kTcBK);
+    } else {
+      // B_proj: Q as bf16 (P16), N (K) rows x ldp columns (those beyond r' are zero), row stride ldp
+      ok &= tc_encode_2d(plan.encode, mp + TC_MAP_B_PROJ, d.P16, d.ldp, d.N, static_cast<uint64_t>(d.ldp) * 2, 64, kTcBK);
+      // A_back: u16, M rows x lr_cols (K) columns (those beyond r' are zero)
+      ok &= tc_encode_2d(plan.encode, mp + TC_MAP_A_BACK, d.u16, d.lr_cols, d.M, static_cast<uint64_t>(d.lr_cols) * 2, kTcBK, kTcBM);
+      // B_back: Q^T as fp16 (Pt16), r' (K) rows x N columns, row stride ldpt
+      ok &= tc_encode_2d(plan.encode, mp + TC_MAP_B_BACK, d.Pt16, d.N, d.rp, static_cast<uint64_t>(d.ldpt) * 2, 64, kTcBK);
+    }
+    if (!ok) return NGALORE_ERR_CUDA;
   }
 
-  // ---- projection tiles: output r' x N, K = M; split K so that no tile dominates the schedule
+  // ---- projection tiles: output lr_rows x lr_cols (r' x N with K = M, or M x r' with K = N when the matrix is
+  // projected on the right); split K so that no tile dominates the schedule
   std::vector<TcTile> proj, back;
   long long total_kb = 0;
   for (int i = 0; i < n; ++i) {
     const MatDesc& d = mats[i];
-    const long long tiles_i = static_cast<long long>((d.rp + kTcBM - 1) / kTcBM) * ((d.N + kProjBN - 1) / kProjBN);
-    total_kb += tiles_i * ((d.M + kTcBK - 1) / kTcBK);
+    const long long tiles_i = static_cast<long long>((d.lr_rows + kTcBM - 1) / kTcBM) * ((d.lr_cols + kProjBN - 1) / kProjBN);
+    total_kb += tiles_i * (((d.right ? d.N : d.M) + kTcBK - 1) / kTcBK);
   }
   const long long per_cta = (total_kb + sm_count - 1) / sm_count;
   long long target_kb = per_cta / 4;
@@ -487,18 +500,18 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   std::vector<int> split_mats;
   for (int i = 0; i < n; ++i) {
     const MatDesc& d = mats[i];
-    const int kb_total = (d.M + kTcBK - 1) / kTcBK;
+    const int kb_total = ((d.right ? d.N : d.M) + kTcBK - 1) / kTcBK;
     int splits = static_cast<int>((kb_total + target_kb - 1) / target_kb);
     if (splits < 1) splits = 1;
     const int kb_per = (kb_total + splits - 1) / splits;
     splits = (kb_total + kb_per - 1) / kb_per;
     if (splits > 1) split_mats.push_back(i);
-    for (int n0 = 0; n0 < d.N; n0 += kProjBN)
+    for (int n0 = 0; n0 < d.lr_cols; n0 += kProjBN)
       for (int sp = 0; sp < splits; ++sp)
-        for (int m0 = 0; m0 < d.rp; m0 += kTcBM) {
+        for (int m0 = 0; m0 < d.lr_rows; m0 += kTcBM) {
           const int kb0 = sp * kb_per;
           const int kbn = std::min(kb_per, kb_total - kb0);
-          proj.push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0, d.rp, d.N});
+          proj.push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0, d.lr_rows, d.lr_cols});
         }
   }
   std::stable_sort(proj.begin(), proj.end(), [](const TcTile& a, const TcTile& b) { return a.kblocks > b.kblocks; });
@@ -526,8 +539,8 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   if (!split_mats.empty() &&
       cudaMemcpy(plan.d_split_mats, split_mats.data(), sizeof(int) * split_mats.size(), cudaMemcpyHostToDevice) != cudaSuccess)
     return NGALORE_ERR_CUDA;
-  plan.rowsN.resize(n); plan.colsN.resize(n);
-  for (int i = 0; i < n; ++i) { plan.rowsN[i] = mats[i].M; plan.colsN[i] = mats[i].N; }
+  plan.rowsN.resize(n); plan.colsN.resize(n); plan.right.resize(n);
+  for (int i = 0; i < n; ++i) { plan.rowsN[i] = mats[i].M; plan.colsN[i] = mats[i].N; plan.right[i] = mats[i].right; }
 
   using LP = TcSmem<kProjBN, 1, 1, kProjStages, kProjEpiWarps>;
   if (cudaFuncSetAttribute(tc_gemm_kernel<kProjBN, 1, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps, false>,
@@ -546,9 +559,13 @@ inline ngalore_status tc_bind_buffers(TcPlan& plan, const uint16_t* const* G, fl
     CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * kTcMapsPerMat];
     if (plan.last_G[i] != G[i]) {
       plan.last_G[i] = G[i];
-      if (!tc_encode_2d(plan.encode, mp + TC_MAP_B_PROJ, G[i], plan.colsN[i], plan.rowsN[i],
-                        static_cast<uint64_t>(plan.colsN[i]) * 2, 64, kTcBK))
-        return NGALORE_ERR_CUDA;
+      // G is the B operand of a left projection (K = M rows) and the A operand of a right one (K = N columns)
+      const bool enc = plan.right[i]
+                           ? tc_encode_2d(plan.encode, mp + TC_MAP_A_PROJ, G[i], plan.colsN[i], plan.rowsN[i],
+                                          static_cast<uint64_t>(plan.colsN[i]) * 2, kTcBK, kTcBM)
+                           : tc_encode_2d(plan.encode, mp + TC_MAP_B_PROJ, G[i], plan.colsN[i], plan.rowsN[i],
+                                          static_cast<uint64_t>(plan.colsN[i]) * 2, 64, kTcBK);
+      if (!enc) return NGALORE_ERR_CUDA;
       changed = true;
     }
     if (plan.last_W[i] != W[i]) {

@@ -219,35 +219,58 @@ __global__ void __launch_bounds__(256) orth_apply_kernel(OrthApply p) {
 
 // ---------------------------------------------------------------- working copies of P
 
-// Pt16 = bf16(P32)^T (rp x M, leading dimension ldpt) for the projection, and P16 = the same rounded values
-// stored as fp16 (M x rp, leading dimension ldp) for the back-projection, whose other operand is fp16.  A
-// bf16 number converts to fp16 without error unless it is below 2^-17 in magnitude, where the error is at
-// most 2^-25: far below the resolution of an orthonormal column's entries.
+// Working copies of a projector P32 (rows x rp): P16 (rows x ldp) and its transpose Pt16 (rp x ldpt), both
+// holding the bf16-rounded values.  One of the two is stored as bf16 and the other as fp16 (p16_is_half says
+// which): a bf16 number converts to fp16 without error unless it is below 2^-17 in magnitude, where the error is
+// at most 2^-25, far below the resolution of an orthonormal column's entries.
 // Block (32, 8).
-__global__ void working_copies_kernel(const float* P32, __half* P16, __nv_bfloat16* Pt16, int M, int rp,
-                                      int ldp, int ldpt) {
+__device__ __forceinline__ uint16_t working_bits(float val, bool as_half) {
+  const __nv_bfloat16 b = __float2bfloat16_rn(val);
+  if (!as_half) return __bfloat16_as_ushort(b);
+  return __half_as_ushort(__float2half_rn(__bfloat162float(b)));
+}
+
+__global__ void working_copies_kernel(const float* P32, uint16_t* P16, uint16_t* Pt16, int rows, int rp, int ldp,
+                                      int ldpt, int p16_is_half) {
   __shared__ float tile[32][33];
   const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
   for (int a = threadIdx.y; a < 32; a += blockDim.y) {
     const int i = i0 + a, j = j0 + threadIdx.x;
     float val = 0.f;
-    if (i < M && j < rp) {
+    if (i < rows && j < rp) {
       val = P32[static_cast<long long>(i) * rp + j];
-      P16[static_cast<long long>(i) * ldp + j] = __float2half_rn(__bfloat162float(__float2bfloat16_rn(val)));
+      P16[static_cast<long long>(i) * ldp + j] = working_bits(val, p16_is_half != 0);
     }
     tile[a][threadIdx.x] = val;
   }
   __syncthreads();
   for (int a = threadIdx.y; a < 32; a += blockDim.y) {
     const int j = j0 + a, i = i0 + threadIdx.x;
-    if (i < M && j < rp) Pt16[static_cast<long long>(j) * ldpt + i] = __float2bfloat16_rn(tile[threadIdx.x][a]);
+    if (i < rows && j < rp) Pt16[static_cast<long long>(j) * ldpt + i] = working_bits(tile[threadIdx.x][a], p16_is_half == 0);
   }
 }
 
-// dst (rows x cols, dense fp32) = src (rows x cols, leading dimension ld, fp16)
-__global__ void widen_f16_kernel(const __half* src, float* dst, long long n, int cols, int ld) {
+// dst (rows x cols, dense fp32) = src (rows x cols, leading dimension ld; fp16 or bf16 bits)
+__global__ void widen_16_kernel(const uint16_t* src, float* dst, long long n, int cols, int ld, int is_half) {
   const long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-  if (i < n) dst[i] = __half2float(src[(i / cols) * ld + (i % cols)]);
+  if (i >= n) return;
+  const uint16_t bits = src[(i / cols) * ld + (i % cols)];
+  dst[i] = is_half ? __half2float(__ushort_as_half(bits)) : __bfloat162float(__ushort_as_bfloat16(bits));
+}
+
+// dst (cols x ld_dst, bf16, padding columns left untouched) = src^T for src (rows x cols, bf16).  Block (32, 8).
+__global__ void transpose_bf16_kernel(const uint16_t* src, uint16_t* dst, int rows, int cols, int ld_dst) {
+  __shared__ uint16_t tile[32][33];
+  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
+  for (int a = threadIdx.y; a < 32; a += blockDim.y) {
+    const int i = i0 + a, j = j0 + threadIdx.x;
+    tile[a][threadIdx.x] = (i < rows && j < cols) ? src[static_cast<long long>(i) * cols + j] : uint16_t(0);
+  }
+  __syncthreads();
+  for (int a = threadIdx.y; a < 32; a += blockDim.y) {
+    const int j = j0 + a, i = i0 + threadIdx.x;
+    if (i < rows && j < cols) dst[static_cast<long long>(j) * ld_dst + i] = tile[threadIdx.x][a];
+  }
 }
 
 }  // namespace ngalore

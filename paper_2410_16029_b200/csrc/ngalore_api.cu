@@ -28,10 +28,15 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct HostMat {
   int M, N, rp;
+  bool right;        // projected on the right (short-side rule, M >= N)
+  int eM, eN;        // the matrix the refresh sees: G itself (M x N), or G^T with its rows padded to a multiple
+                     // of 8 columns (N x eN, eN >= M) when the matrix is projected on the right
+  int lr_rows, lr_cols;
   long long rn;
   // refresh scratch (device)
   float *Ya, *Yb, *Xa, *Xb;
   double* C;
+  uint16_t* Gt;      // right-projected matrices: G^T as bf16, N x eN (padding columns stay zero)
 };
 
 struct BlobHeader {
@@ -68,6 +73,7 @@ struct ngalore_state {
   float** d_W = nullptr;
   const __nv_bfloat16** d_G = nullptr;
   std::vector<const void*> last_W, last_G;
+  std::vector<const uint16_t*> refresh_G;  // the gradients as the refresh reads them (G, or its transposed copy)
   CholProblem* d_chol = nullptr;
   int64_t k = 0;
   int64_t n_appended = 0;
@@ -149,8 +155,8 @@ ngalore_status upload_hyper(ngalore_state* st, cudaStream_t stream) {
 ngalore_status make_working_copies(ngalore_state* st, int i, cudaStream_t stream) {
   const HostMat& hm = st->mats[i];
   const MatDesc& d = st->h_desc[i];
-  dim3 grid((hm.rp + 31) / 32, (hm.M + 31) / 32), block(32, 8);
-  working_copies_kernel<<<grid, block, 0, stream>>>(d.P32, d.P16, d.Pt16, hm.M, hm.rp, d.ldp, d.ldpt);
+  dim3 grid((hm.rp + 31) / 32, (hm.eM + 31) / 32), block(32, 8);
+  working_copies_kernel<<<grid, block, 0, stream>>>(d.P32, d.P16, d.Pt16, hm.eM, hm.rp, d.ldp, d.ldpt, hm.right ? 0 : 1);
   st->launches += 1;
   NG_CUDA(cudaGetLastError());
   return NGALORE_OK;
@@ -163,7 +169,7 @@ ngalore_status orthonormalise(ngalore_state* st, const std::vector<int>& idx, in
   for (int i : idx) {
     const HostMat& hm = st->mats[i];
     const float* Y = side == 0 ? (from_a ? hm.Ya : hm.Yb) : (from_a ? hm.Xa : hm.Xb);
-    const int rows = side == 0 ? hm.M : hm.N;
+    const int rows = side == 0 ? hm.eM : hm.eN;
     SimtGemm g{};
     g.m = hm.rp; g.n = hm.rp; g.k = rows;
     g.A = Y; g.a_rs = 1; g.a_cs = hm.rp; g.a_dt = DT_F32;
@@ -190,7 +196,7 @@ ngalore_status orthonormalise(ngalore_state* st, const std::vector<int>& idx, in
     p.Y = side == 0 ? (from_a ? hm.Ya : hm.Yb) : (from_a ? hm.Xa : hm.Xb);
     p.Q = side == 0 ? (from_a ? hm.Yb : hm.Ya) : (from_a ? hm.Xb : hm.Xa);
     p.Lf = hm.C;
-    p.rows = side == 0 ? hm.M : hm.N;
+    p.rows = side == 0 ? hm.eM : hm.eN;
     p.L = hm.rp;
     orth_apply_kernel<<<(p.rows + 31) / 32, 256, orth_apply_smem_bytes(p.L), stream>>>(p);
     st->launches += 1;
@@ -216,11 +222,11 @@ ngalore_status apply_gradient(ngalore_state* st, const std::vector<int>& idx, co
     const HostMat& hm = st->mats[i];
     SimtGemm g{};
     if (side == 0) {
-      g.m = hm.M; g.n = hm.rp; g.k = hm.N;
-      g.A = G[i]; g.a_rs = hm.N; g.a_cs = 1;
+      g.m = hm.eM; g.n = hm.rp; g.k = hm.eN;
+      g.A = G[i]; g.a_rs = hm.eN; g.a_cs = 1;
     } else {
-      g.m = hm.N; g.n = hm.rp; g.k = hm.M;
-      g.A = G[i]; g.a_rs = 1; g.a_cs = hm.N;
+      g.m = hm.eN; g.n = hm.rp; g.k = hm.eM;
+      g.A = G[i]; g.a_rs = 1; g.a_cs = hm.eN;
     }
     g.a_dt = DT_BF16;
     g.B = refresh_buf(hm, src); g.b_rs = hm.rp; g.b_cs = 1; g.b_dt = DT_F32;
@@ -236,7 +242,7 @@ ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bo
   ngalore_status rc;
   for (int i : idx) {
     const HostMat& hm = st->mats[i];
-    NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, basis_in_a ? hm.Ya : hm.Yb, sizeof(float) * hm.M * hm.rp,
+    NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, basis_in_a ? hm.Ya : hm.Yb, sizeof(float) * hm.eM * hm.rp,
                             cudaMemcpyDeviceToDevice, stream));
     if ((rc = make_working_copies(st, i, stream))) return rc;
   }
@@ -254,7 +260,7 @@ ngalore_status refresh_simt(ngalore_state* st, const uint16_t* const* G, const s
   // Random test matrix Omega (N x rp), one hashed stream per matrix and refresh.
   for (int i : idx) {
     const HostMat& hm = st->mats[i];
-    const long long cnt = static_cast<long long>(hm.N) * hm.rp;
+    const long long cnt = static_cast<long long>(hm.eN) * hm.rp;
     fill_normal_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, stream>>>(
         hm.Xa, cnt, st->opt.seed, static_cast<unsigned long long>(st->k) * 65536ull + static_cast<unsigned>(i));
     st->launches += 1;
@@ -276,9 +282,23 @@ ngalore_status refresh_simt(ngalore_state* st, const uint16_t* const* G, const s
   return finish_refresh(st, idx, true, stream);
 }
 
-ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G, const std::vector<int>& idx,
+// The subspace a matrix needs is the leading left one of G (left projection) or the leading right one, i.e. the
+// left one of G^T (right projection).  Right-projected matrices get G^T written out once per refresh, so that
+// every product below sees a plain row-major matrix of eM x eN.
+ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G_in, const std::vector<int>& idx,
                             cudaStream_t stream) {
   const int q = st->opt.power_iterations > 0 ? st->opt.power_iterations : 6;
+  st->refresh_G.assign(G_in, G_in + st->n);
+  for (int i : idx) {
+    const HostMat& hm = st->mats[i];
+    if (!hm.right) continue;
+    dim3 grid((hm.N + 31) / 32, (hm.M + 31) / 32), block(32, 8);
+    transpose_bf16_kernel<<<grid, block, 0, stream>>>(G_in[i], hm.Gt, hm.M, hm.N, hm.eN);
+    st->launches += 1;
+    st->refresh_G[i] = hm.Gt;
+  }
+  NG_CUDA(cudaGetLastError());
+  const uint16_t* const* G = st->refresh_G.data();
   if (st->opt.gemm_impl == 1 || idx.size() != static_cast<size_t>(st->n) || !st->refresh.ready)
     return refresh_simt(st, G, idx, q, stream);
   ngalore_status rc;
@@ -289,12 +309,12 @@ ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G, const s
   // of the last product to average out.  Short matrices get one exact pass (Gram, Cholesky and triangular solve in fp64): Ya -> Yb -> Ya.
   std::vector<int> small;
   for (int i : idx)
-    if (st->mats[i].M < 512) small.push_back(i);
+    if (st->mats[i].eM < 512) small.push_back(i);
   if (!small.empty()) {
     if ((rc = orthonormalise(st, small, 0, true, stream))) return rc;
     for (int i : small) {
       const HostMat& hm = st->mats[i];
-      NG_CUDA(cudaMemcpyAsync(hm.Ya, hm.Yb, sizeof(float) * hm.M * hm.rp, cudaMemcpyDeviceToDevice, stream));
+      NG_CUDA(cudaMemcpyAsync(hm.Ya, hm.Yb, sizeof(float) * hm.eM * hm.rp, cudaMemcpyDeviceToDevice, stream));
     }
   }
   return finish_refresh(st, idx, true, stream);
@@ -321,10 +341,16 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       const HostMat& hm = st->mats[i];
       const MatDesc& d = st->h_desc[i];
       SimtGemm g{};
-      g.m = hm.rp; g.n = hm.N; g.k = hm.M;
-      g.A = d.Pt16; g.a_rs = d.ldpt; g.a_cs = 1; g.a_dt = DT_BF16;
-      g.B = G[i]; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_BF16;
-      g.C = d.H + static_cast<long long>(cur) * hm.rn; g.c_rs = hm.N; g.c_cs = 1; g.c_dt = DT_F32;
+      if (!hm.right) {
+        g.m = hm.rp; g.n = hm.N; g.k = hm.M;
+        g.A = d.Pt16; g.a_rs = d.ldpt; g.a_cs = 1; g.a_dt = DT_BF16;
+        g.B = G[i]; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_BF16;
+      } else {
+        g.m = hm.M; g.n = hm.rp; g.k = hm.N;
+        g.A = G[i]; g.a_rs = hm.N; g.a_cs = 1; g.a_dt = DT_BF16;
+        g.B = d.P16; g.b_rs = d.ldp; g.b_cs = 1; g.b_dt = DT_BF16;
+      }
+      g.C = d.H + static_cast<long long>(cur) * hm.rn; g.c_rs = hm.lr_cols; g.c_cs = 1; g.c_dt = DT_F32;
       g.epilogue = EPI_STORE;
       NG_CUDA(launch_simt_gemm<float>(g, stream));
       st->launches += 1;
@@ -350,8 +376,13 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       const MatDesc& d = st->h_desc[i];
       SimtGemm g{};
       g.m = hm.M; g.n = hm.N; g.k = hm.rp;
-      g.A = d.P16; g.a_rs = d.ldp; g.a_cs = 1; g.a_dt = DT_F16;
-      g.B = d.u16; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_F16;
+      if (!hm.right) {
+        g.A = d.P16; g.a_rs = d.ldp; g.a_cs = 1; g.a_dt = DT_F16;
+        g.B = d.u16; g.b_rs = hm.N; g.b_cs = 1; g.b_dt = DT_F16;
+      } else {
+        g.A = d.u16; g.a_rs = hm.lr_cols; g.a_cs = 1; g.a_dt = DT_F16;
+        g.B = d.Pt16; g.b_rs = d.ldpt; g.b_cs = 1; g.b_dt = DT_F16;
+      }
       g.C = W[i]; g.c_rs = hm.N; g.c_cs = 1; g.c_dt = DT_F32;
       g.epilogue = EPI_W_UPDATE;
       g.hyper = st->d_hyper;
@@ -408,6 +439,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     if (shapes[i].rows > (1 << 24) || shapes[i].cols > (1 << 24)) return NGALORE_ERR_INVALID_ARG;
   }
   if (opt != nullptr && opt->struct_size != static_cast<int32_t>(sizeof(ngalore_options))) return NGALORE_ERR_INVALID_ARG;
+  if (opt != nullptr && (opt->projection_rule < 0 || opt->projection_rule > 1)) return NGALORE_ERR_INVALID_ARG;
 
   int dev = 0;
   NG_CUDA(cudaGetDevice(&dev));
@@ -439,10 +471,18 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     hm.M = static_cast<int>(shapes[i].rows); hm.N = static_cast<int>(shapes[i].cols);
     hm.rp = r < hm.M ? r : hm.M;
     if (hm.N < hm.rp) hm.rp = hm.N;
-    hm.rn = static_cast<long long>(hm.rp) * hm.N;
+    hm.right = st->opt.projection_rule == 1 && hm.M >= hm.N;
+    const int ldr = (hm.rp + 7) / 8 * 8;
+    hm.eM = hm.right ? hm.N : hm.M;
+    hm.eN = hm.right ? (hm.M + 7) / 8 * 8 : hm.N;
+    hm.lr_rows = hm.right ? hm.M : hm.rp;
+    hm.lr_cols = hm.right ? ldr : hm.N;
+    hm.rn = static_cast<long long>(hm.lr_rows) * hm.lr_cols;
+    hm.Gt = nullptr;
     total_rn += hm.rn;
     hash = (hash ^ static_cast<uint64_t>(hm.M)) * 1099511628211ull;
     hash = (hash ^ static_cast<uint64_t>(hm.N)) * 1099511628211ull;
+    hash = (hash ^ static_cast<uint64_t>(hm.right ? 2 : 1)) * 1099511628211ull;
   }
   st->shape_hash = hash;
   long long te_all = total_rn / (2ll * prop.multiProcessorCount) / 1024 * 1024;
@@ -464,9 +504,9 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     offs[i].H = take(sizeof(float) * hm.rn * slots);
     offs[i].m = take(sizeof(float) * hm.rn);
     offs[i].v = take(sizeof(float) * hm.rn);
-    offs[i].P32 = take(sizeof(float) * hm.M * hm.rp);
-    offs[i].P16 = take(sizeof(__nv_bfloat16) * hm.M * ((hm.rp + 7) / 8 * 8));
-    offs[i].Pt16 = take(sizeof(__nv_bfloat16) * hm.rp * ((hm.M + 7) / 8 * 8));
+    offs[i].P32 = take(sizeof(float) * hm.eM * hm.rp);
+    offs[i].P16 = take(sizeof(uint16_t) * hm.eM * ((hm.rp + 7) / 8 * 8));
+    offs[i].Pt16 = take(sizeof(uint16_t) * hm.rp * ((hm.eM + 7) / 8 * 8));
     offs[i].Kraw = take(sizeof(double) * slots * slots);
     offs[i].wsol = take(sizeof(float) * kMaxHistory);
   }
@@ -474,7 +514,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
 
   // ---- work layout
   off = 0;
-  struct WOffs { size_t u16, gpart, Ya, Yb, Xa, Xb, C; };
+  struct WOffs { size_t u16, gpart, Ya, Yb, Xa, Xb, C, Gt; };
   std::vector<WOffs> woffs(n_matrices);
   const size_t o_hyper = take(sizeof(Hyper));
   const size_t o_desc = take(sizeof(MatDesc) * n_matrices);
@@ -494,11 +534,12 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     n_tiles += ntl[i];
     woffs[i].u16 = take(sizeof(__half) * hm.rn);
     woffs[i].gpart = take(sizeof(double) * ntl[i] * slots);
-    woffs[i].Ya = take(sizeof(float) * hm.M * hm.rp);
-    woffs[i].Yb = take(sizeof(float) * hm.M * hm.rp);
-    woffs[i].Xa = take(sizeof(float) * hm.N * hm.rp);
-    woffs[i].Xb = take(sizeof(float) * hm.N * hm.rp);
+    woffs[i].Ya = take(sizeof(float) * hm.eM * hm.rp);
+    woffs[i].Yb = take(sizeof(float) * hm.eM * hm.rp);
+    woffs[i].Xa = take(sizeof(float) * hm.eN * hm.rp);
+    woffs[i].Xb = take(sizeof(float) * hm.eN * hm.rp);
     woffs[i].C = take(sizeof(double) * hm.rp * hm.rp);
+    woffs[i].Gt = hm.right ? take(sizeof(uint16_t) * hm.N * hm.eN) : 0;
   }
   st->n_tiles = n_tiles;
   const size_t o_tiles = take(sizeof(StreamTile) * n_tiles);
@@ -532,13 +573,14 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     HostMat& hm = st->mats[i];
     MatDesc& d = st->h_desc[i];
     d.M = hm.M; d.N = hm.N; d.rp = hm.rp; d.s = s; d.rn = hm.rn;
-    d.ldp = (hm.rp + 7) / 8 * 8; d.ldpt = (hm.M + 7) / 8 * 8;
+    d.right = hm.right ? 1 : 0; d.pr = hm.eM; d.lr_rows = hm.lr_rows; d.lr_cols = hm.lr_cols;
+    d.ldp = (hm.rp + 7) / 8 * 8; d.ldpt = (hm.eM + 7) / 8 * 8;
     d.H = reinterpret_cast<float*>(st->arena + offs[i].H);
     d.m = reinterpret_cast<float*>(st->arena + offs[i].m);
     d.v = reinterpret_cast<float*>(st->arena + offs[i].v);
     d.P32 = reinterpret_cast<float*>(st->arena + offs[i].P32);
-    d.P16 = reinterpret_cast<__half*>(st->arena + offs[i].P16);
-    d.Pt16 = reinterpret_cast<__nv_bfloat16*>(st->arena + offs[i].Pt16);
+    d.P16 = reinterpret_cast<uint16_t*>(st->arena + offs[i].P16);
+    d.Pt16 = reinterpret_cast<uint16_t*>(st->arena + offs[i].Pt16);
     d.Kraw = reinterpret_cast<double*>(st->arena + offs[i].Kraw);
     d.wsol = reinterpret_cast<float*>(st->arena + offs[i].wsol);
     d.u16 = reinterpret_cast<__half*>(st->work + woffs[i].u16);
@@ -553,6 +595,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     hm.Xa = reinterpret_cast<float*>(st->work + woffs[i].Xa);
     hm.Xb = reinterpret_cast<float*>(st->work + woffs[i].Xb);
     hm.C = reinterpret_cast<double*>(st->work + woffs[i].C);
+    if (hm.right) hm.Gt = reinterpret_cast<uint16_t*>(st->work + woffs[i].Gt);
     chol[i].C = hm.C; chol[i].L = hm.rp;
     if (s == 0 && cudaMemcpy(d.wsol, w_init.data(), sizeof(float) * kMaxHistory, cudaMemcpyHostToDevice) != cudaSuccess)
       return fail(NGALORE_ERR_CUDA);
@@ -582,7 +625,10 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (st->opt.gemm_impl != 1) {
     std::vector<float*> Yf(n_matrices), Zf(n_matrices);
     for (int i = 0; i < n_matrices; ++i) { Yf[i] = st->mats[i].Ya; Zf[i] = st->mats[i].Xa; }
-    rc = refresh_plan_create(st->refresh, st->h_desc, Yf, Zf, prop.multiProcessorCount);
+    // the refresh plan sees every matrix in the orientation whose left subspace is wanted
+    std::vector<MatDesc> eff(st->h_desc);
+    for (int i = 0; i < n_matrices; ++i) { eff[i].M = st->mats[i].eM; eff[i].N = st->mats[i].eN; }
+    rc = refresh_plan_create(st->refresh, eff, Yf, Zf, prop.multiProcessorCount);
     if (rc != NGALORE_OK) return fail(rc);
   }
   for (int e = 0; e < 4; ++e)
@@ -695,7 +741,7 @@ ngalore_status ngalore_get_subspace(ngalore_state* st, int i, float* P, void* st
   if (st == nullptr || i < 0 || i >= st->n || P == nullptr) return NGALORE_ERR_INVALID_ARG;
   DeviceGuard guard(st->device);
   const HostMat& hm = st->mats[i];
-  NG_CUDA(cudaMemcpyAsync(P, st->h_desc[i].P32, sizeof(float) * hm.M * hm.rp, cudaMemcpyDeviceToDevice,
+  NG_CUDA(cudaMemcpyAsync(P, st->h_desc[i].P32, sizeof(float) * hm.eM * hm.rp, cudaMemcpyDeviceToDevice,
                           static_cast<cudaStream_t>(stream)));
   return NGALORE_OK;
 }
@@ -704,9 +750,9 @@ ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, 
   if (st == nullptr || i < 0 || i >= st->n || P == nullptr) return NGALORE_ERR_INVALID_ARG;
   DeviceGuard guard(st->device);
   const HostMat& hm = st->mats[i];
-  const long long cnt = static_cast<long long>(hm.M) * hm.rp;
-  widen_f16_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      st->h_desc[i].P16, P, cnt, hm.rp, st->h_desc[i].ldp);
+  const long long cnt = static_cast<long long>(hm.eM) * hm.rp;
+  widen_16_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      st->h_desc[i].P16, P, cnt, hm.rp, st->h_desc[i].ldp, hm.right ? 0 : 1);
   st->launches += 1;
   NG_CUDA(cudaGetLastError());
   return NGALORE_OK;
@@ -717,7 +763,7 @@ ngalore_status ngalore_set_subspace(ngalore_state* st, int i, const float* P, vo
   DeviceGuard guard(st->device);
   const HostMat& hm = st->mats[i];
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, P, sizeof(float) * hm.M * hm.rp, cudaMemcpyDeviceToDevice, s));
+  NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, P, sizeof(float) * hm.eM * hm.rp, cudaMemcpyDeviceToDevice, s));
   ngalore_status rc = make_working_copies(st, i, s);
   if (rc != NGALORE_OK) return rc;
   st->has_subspace = true;  // the caller is responsible for setting every matrix before stepping
@@ -763,6 +809,8 @@ ngalore_status ngalore_set_lr(ngalore_state* st, double lr) {
 
 int ngalore_num_matrices(const ngalore_state* st) { return st ? st->n : 0; }
 int ngalore_rank(const ngalore_state* st, int i) { return (st && i >= 0 && i < st->n) ? st->mats[i].rp : -1; }
+int ngalore_projects_right(const ngalore_state* st, int i) { return (st && i >= 0 && i < st->n) ? (st->mats[i].right ? 1 : 0) : -1; }
+int ngalore_subspace_rows(const ngalore_state* st, int i) { return (st && i >= 0 && i < st->n) ? st->mats[i].eM : -1; }
 int64_t ngalore_step_count(const ngalore_state* st) { return st ? st->k : -1; }
 size_t ngalore_device_bytes(const ngalore_state* st) { return st ? st->arena_bytes + st->work_bytes + st->stage_bytes + st->tc.device_bytes + st->refresh.device_bytes : 0; }
 int64_t ngalore_launch_count(const ngalore_state* st) { return st ? st->launches : 0; }

@@ -34,7 +34,7 @@ class Shape(ctypes.Structure):
 class Options(ctypes.Structure):
     _fields_ = [("struct_size", ctypes.c_int32), ("gemm_impl", ctypes.c_int32),
                 ("power_iterations", ctypes.c_int32), ("reset_history_on_refresh", ctypes.c_int32),
-                ("seed", ctypes.c_uint64), ("stream_impl", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("seed", ctypes.c_uint64), ("stream_impl", ctypes.c_int32), ("projection_rule", ctypes.c_int32)]
 
 
 _vp = ctypes.c_void_p
@@ -63,8 +63,9 @@ _lib.ngalore_set_lr.restype = ctypes.c_int
 _lib.ngalore_set_lr.argtypes = [_vp, ctypes.c_double]
 _lib.ngalore_num_matrices.restype = ctypes.c_int
 _lib.ngalore_num_matrices.argtypes = [_vp]
-_lib.ngalore_rank.restype = ctypes.c_int
-_lib.ngalore_rank.argtypes = [_vp, ctypes.c_int]
+for _name in ("ngalore_rank", "ngalore_projects_right", "ngalore_subspace_rows"):
+    getattr(_lib, _name).restype = ctypes.c_int
+    getattr(_lib, _name).argtypes = [_vp, ctypes.c_int]
 _lib.ngalore_step_count.restype = ctypes.c_int64
 _lib.ngalore_step_count.argtypes = [_vp]
 _lib.ngalore_device_bytes.restype = ctypes.c_size_t
@@ -110,11 +111,13 @@ class NGaLore:
     """Optimizer state for a list of (rows, cols) weight matrices on the current CUDA device."""
 
     def __init__(self, shapes, r, s, T, lam=1e-3, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, wd=0.0, *,
-                 gemm_impl=0, stream_impl=0, power_iterations=0, reset_history_on_refresh=False, seed=0):
+                 gemm_impl=0, stream_impl=0, power_iterations=0, reset_history_on_refresh=False, seed=0,
+                 projection="left"):
         self.shapes = [(int(M), int(N)) for M, N in shapes]
         arr = (Shape * len(self.shapes))(*[Shape(M, N) for M, N in self.shapes])
+        rule = {"left": 0, "short_side": 1}[projection]
         opt = Options(ctypes.sizeof(Options), gemm_impl, power_iterations, int(reset_history_on_refresh), seed,
-                      stream_impl, 0)
+                      stream_impl, rule)
         handle = _vp()
         _check(_lib.ngalore_create(arr, len(self.shapes), r, s, T, lam, lr, beta1, beta2, eps, wd,
                                    ctypes.byref(opt), ctypes.byref(handle)), "ngalore_create")
@@ -174,17 +177,21 @@ class NGaLore:
     def rank(self, i):
         return _lib.ngalore_rank(self._h, i)
 
+    def projects_right(self, i) -> bool:
+        return _lib.ngalore_projects_right(self._h, i) == 1
+
+    def subspace_rows(self, i):
+        return _lib.ngalore_subspace_rows(self._h, i)
+
     def get_subspace(self, i, working=False) -> torch.Tensor:
-        M, _ = self.shapes[i]
-        out = torch.empty((M, self.rank(i)), dtype=torch.float32, device=self.device)
+        out = torch.empty((self.subspace_rows(i), self.rank(i)), dtype=torch.float32, device=self.device)
         fn = _lib.ngalore_get_working_subspace if working else _lib.ngalore_get_subspace
         _check(fn(self._h, i, out.data_ptr(), _stream_ptr(None)), "ngalore_get_subspace")
         return out
 
     def set_subspace(self, i, P: torch.Tensor):
-        M, _ = self.shapes[i]
         P = P.to(device=self.device, dtype=torch.float32).contiguous()
-        assert tuple(P.shape) == (M, self.rank(i))
+        assert tuple(P.shape) == (self.subspace_rows(i), self.rank(i))
         _check(_lib.ngalore_set_subspace(self._h, i, P.data_ptr(), _stream_ptr(None)), "ngalore_set_subspace")
         torch.cuda.current_stream().synchronize()  # P may be freed by the caller
 
