@@ -45,22 +45,30 @@ def measured_peak_hbm():
         return 6650.0, "fallback"
 
 
-def byte_model(wl):
+def low_rank_dims(wl, i, projection):
+    """(r', rows of the projector, elements of one low-rank matrix) of matrix i: the low-rank gradient is
+    r' x N under a left projection and M x r' under a right one (short-side rule, M >= N)."""
+    _, M, N = wl.shapes[i]
+    rp = wl.rank_of(i)
+    right = projection == "short_side" and M >= N
+    return rp, (N if right else M), rp * (M if right else N)
+
+
+def byte_model(wl, projection="left"):
     """Algorithmic bytes per step: every datum moved once (G bf16, W fp32, P bf16, history/m/v fp32)."""
     tot = stream = 0
     for i, (_, M, N) in enumerate(wl.shapes):
-        rp = wl.rank_of(i)
-        rn = rp * N
-        tot += 10 * M * N + 2 * M * rp + (4 * wl.s + 20) * rn
+        rp, pr, rn = low_rank_dims(wl, i, projection)
+        tot += 10 * M * N + 2 * pr * rp + (4 * wl.s + 20) * rn
         stream += (4 * wl.s + 16) * rn          # history read once + m, v read and written
     return tot, stream
 
 
-def flop_model(wl):
+def flop_model(wl, projection="left"):
     f = 0
     for i, (_, M, N) in enumerate(wl.shapes):
-        rp = wl.rank_of(i)
-        f += 4 * M * N * rp + 4 * wl.s * rp * N + 12 * rp * N
+        rp, _, rn = low_rank_dims(wl, i, projection)
+        f += 4 * M * N * rp + 4 * wl.s * rn + 12 * rn
     return f
 
 
@@ -117,7 +125,7 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------------------- oracle arm
 
-def oracle_sample(wl, seed_shift=0, P_by_shape=None):
+def oracle_sample(wl, seed_shift=0, P_by_shape=None, projection="left"):
     """Time the fp64 oracle on one matrix per distinct shape (history pre-filled to s slots) and scale by
     the shape counts to one full step.  Returns (seconds per full step, description, threads)."""
     from oracle import natural_galore as orc
@@ -129,15 +137,16 @@ def oracle_sample(wl, seed_shift=0, P_by_shape=None):
     total = 0.0
     rng = np.random.default_rng(1234 + seed_shift)
     for i, M, N in wl.distinct_shapes():
-        hp = orc.Hyper(r=wl.r, s=wl.s, T=0, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps)
+        hp = orc.Hyper(r=wl.r, s=wl.s, T=0, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
+                       projection=projection)
         st = orc.MatrixState(M, N, hp)
         if P_by_shape is not None and (M, N) in P_by_shape:
             P = P_by_shape[(M, N)]
         else:
-            P, _ = np.linalg.qr(rng.standard_normal((M, st.rp)))
+            P, _ = np.linalg.qr(rng.standard_normal((N if st.right else M, st.rp)))
         st.set_subspace(P)
         for j in range(wl.s):                       # steady state: a full history
-            st.slots[j] = rng.standard_normal((st.rp, N))
+            st.slots[j] = rng.standard_normal(st.m.shape)
         st.count, st.head = wl.s, 0
         G = W.bf16_bits_to_f64(W.gradient_bits(wl, i, 1))
         Wm = np.zeros((M, N))
@@ -161,7 +170,7 @@ def run_reference(args, wl):
     times = []
     desc, threads = "", 0
     for k in range(args.warmup + args.steps):
-        t, desc, threads = oracle_sample(wl, seed_shift=k)
+        t, desc, threads = oracle_sample(wl, seed_shift=k, projection=args.projection)
         if k >= args.warmup:
             times.append(t)
     sec = float(np.mean(times))
@@ -169,7 +178,7 @@ def run_reference(args, wl):
     out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": wl.name, "matrices": wl.n_matrices, "r": wl.r, "s": wl.s},
+           "config": {"workload": wl.name, "matrices": wl.n_matrices, "r": wl.r, "s": wl.s, "projection": args.projection},
            "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out))
@@ -221,7 +230,7 @@ def run_ours(args, wl):
     shapes = [(M, N) for _, M, N in wl.shapes]
     n = len(shapes)
     opt = NGaLore(shapes, wl.r, wl.s, wl.T, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
-                  wd=wl.wd, seed=1 + rank)
+                  wd=wl.wd, seed=1 + rank, projection=args.projection)
     # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
     wl_rank = rank_workload(wl, rank)
     # With fewer than s + 1 distinct sets a gradient would sit twice in the history ring and the Gram matrix
@@ -314,31 +323,33 @@ def run_ours(args, wl):
 
     # ---- roofline of the dominant kernel and of the whole step
     peak, peak_kind = measured_peak_hbm()
-    tot_bytes, stream_bytes = byte_model(wl)
+    tot_bytes, stream_bytes = byte_model(wl, args.projection)
+    dims = [low_rank_dims(wl, i, args.projection) for i in range(n)]
     names = ["tc_gemm_kernel<project>", "fused_stream_kernel", "tc_backproject_kernel"]
-    proj_bytes = sum(2 * M * N + 2 * M * wl.rank_of(i) + 4 * wl.rank_of(i) * N for i, (M, N) in enumerate(shapes))
-    back_bytes = sum(8 * M * N + 2 * M * wl.rank_of(i) for i, (M, N) in enumerate(shapes))
+    proj_bytes = sum(2 * M * N + 2 * dims[i][1] * dims[i][0] + 4 * dims[i][2] for i, (M, N) in enumerate(shapes))
+    back_bytes = sum(8 * M * N + 2 * dims[i][1] * dims[i][0] for i, (M, N) in enumerate(shapes))
     alg = [proj_bytes, stream_bytes, back_bytes]
     dom = int(np.argmax(phase))
     achieved = alg[dom] / (phase[dom] * 1e-3) / 1e9
     traffic = None
     per_unit = NCU_TRAFFIC_PER_UNIT.get(names[dom])
-    if per_unit is not None and wl.r == 512 and wl.s == 16:
-        units = sum(wl.rank_of(i) * N for i, (M, N) in enumerate(shapes)) if per_unit[0] == "rn" else sum(M * N for M, N in shapes)
+    if per_unit is not None and wl.r == 512 and wl.s == 16 and args.projection == "left":
+        units = sum(d[2] for d in dims) if per_unit[0] == "rn" else sum(M * N for M, N in shapes)
         traffic = per_unit[1] * units
     roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": alg[dom], "ms_per_launch": float(phase[dom]),
                 "phases_ms": {names[i]: float(phase[i]) for i in range(3)},
                 "phases_frac_of_peak": {names[i]: alg[i] / (phase[i] * 1e-3) / 1e9 / peak for i in range(3)}}
-    step_roofline_ms = max(tot_bytes / (peak * 1e9), flop_model(wl) / 1389.3e12) * 1e3
-    step_roof = {"bytes_per_step": tot_bytes, "flops_per_step": flop_model(wl), "roofline_ms": step_roofline_ms,
+    flops = flop_model(wl, args.projection)
+    step_roofline_ms = max(tot_bytes / (peak * 1e9), flops / 1389.3e12) * 1e3
+    step_roof = {"bytes_per_step": tot_bytes, "flops_per_step": flops, "roofline_ms": step_roofline_ms,
                  "frac": step_roofline_ms / ms_step, "peak_kind": peak_kind}
 
     # ---- the oracle on the host cores, bounded sample
     cpu = None
     if not args.no_cpu:
-        sec, desc, threads = oracle_sample(wl)
+        sec, desc, threads = oracle_sample(wl, projection=args.projection)
         cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -346,6 +357,7 @@ def run_ours(args, wl):
            "vs_baseline": None, "dtype": "bf16 (projection) and fp16 (back-projection) GEMM operands, f32 state/accumulation, f64 Gram+solve",
            "data": "synthetic",
            "config": {"workload": wl.name, "matrices": n, "r": wl.r, "s": wl.s, "T": wl.T,
+                      "projection": args.projection,
                       "l2": f"inputs larger than L2: {pool_sets} gradient sets of {grad_bytes / 1e9:.2f} GB cycled",
                       "state_bytes": opt.device_bytes},
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
@@ -370,6 +382,9 @@ def main():
                     help="gradient sets resident in HBM, cycled (default s + 1: no gradient repeats inside the history)")
     ap.add_argument("--layers", type=int, default=0,
                     help="keep only the first LAYERS transformer layers of the workload (small case for profiling)")
+    ap.add_argument("--projection", default="left", choices=["left", "short_side"],
+                    help="left: R = P^T G for every matrix (the paper's form, the headline configuration); "
+                         "short_side: matrices with rows >= cols are projected on the right")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
