@@ -1,7 +1,8 @@
 """Seeded synthetic workloads: matrix shapes, hyper-parameters and gradient generators.
 
-This module holds no optimizer arithmetic.  It only describes the five
-Llama-shaped matrix sets (shapes, rank r, history length s, refresh period T)
+This module holds no optimizer arithmetic.  It only describes the matrix sets
+(five Llama-shaped pre-training sets and three small-rank fine-tuning sets:
+shapes, rank r, history length s, refresh period T)
 and draws the synthetic gradients and initial weights that stand in for the
 paper's C4 pre-training gradients (Sec. 4.1, Table 1 gives the model sizes and
 ranks).  Both the CUDA path and the CPU oracle consume its outputs; neither
@@ -88,6 +89,20 @@ def _llama_shapes(layers: int, hidden: int, mlp: int, vocab: int, kv_dim: int | 
     return tuple(shapes)
 
 
+def _encoder_shapes(layers: int, hidden: int, ffn: int):
+    shapes = []
+    for l in range(layers):
+        shapes += [
+            (f"l{l}.q", hidden, hidden),
+            (f"l{l}.k", hidden, hidden),
+            (f"l{l}.v", hidden, hidden),
+            (f"l{l}.o", hidden, hidden),
+            (f"l{l}.ffn_in", hidden, ffn),
+            (f"l{l}.ffn_out", ffn, hidden),
+        ]
+    return tuple(shapes)
+
+
 WORKLOADS = {
     0: Workload(0, "single-512x1376", r=128, s=8, T=10, steps=20, inner_rank=32,
                 generator="lowrank_noise", shapes=(("w", 512, 1376),)),
@@ -100,6 +115,15 @@ WORKLOADS = {
     4: Workload(4, "llama-1.1b", r=512, s=16, T=200, steps=100, inner_rank=POWERLAW_TERMS,
                 generator="powerlaw_noise",
                 shapes=_llama_shapes(22, 2048, 5632, 32000, kv_dim=256)),
+    # Small-rank fine-tuning regime (Sec. 4.2: ranks 4 and 8 on RoBERTa-Base; Sec. 4.3: TinyLlama 1.1B): the
+    # attention and feed-forward matrices of the encoder blocks, and the 1.1B shapes again at rank 8.  The
+    # planted signal has rank 4, so that the rank-4 and rank-8 subspaces both hold all of it.
+    5: Workload(5, "roberta-base-r8", r=8, s=8, T=200, steps=100, inner_rank=4,
+                generator="lowrank_noise", shapes=_encoder_shapes(12, 768, 3072), lr=2e-5),
+    6: Workload(6, "roberta-base-r4", r=4, s=8, T=200, steps=100, inner_rank=4,
+                generator="lowrank_noise", shapes=_encoder_shapes(12, 768, 3072), lr=2e-5),
+    7: Workload(7, "tinyllama-1.1b-r8", r=8, s=8, T=200, steps=100, inner_rank=4,
+                generator="lowrank_noise", shapes=_llama_shapes(22, 2048, 5632, 32000, kv_dim=256), lr=7e-5),
 }
 
 

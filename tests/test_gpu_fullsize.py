@@ -16,7 +16,10 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("index,steps,svd_shapes", [(1, 10, {(512, 512), (512, 1376), (1376, 512)}),
                                                      (2, 10, {(768, 768)}),
                                                      (3, 5, {(1024, 1024)}),
-                                                     (4, 4, {(2048, 256), (2048, 2048)})])
+                                                     (4, 4, {(2048, 256), (2048, 2048)}),
+                                                     (5, 10, {(768, 768), (768, 3072), (3072, 768)}),
+                                                     (6, 10, {(768, 768), (768, 3072), (3072, 768)}),
+                                                     (7, 4, {(2048, 2048), (2048, 5632)})])
 def test_sampled_matrices_of_full_workload(index, steps, svd_shapes):
     from paper_2410_16029_b200.ngalore import NGaLore
 

@@ -6,7 +6,8 @@ from paper_2410_16029_b200 import workload as wl
 
 
 @pytest.mark.parametrize("idx,n_mat,sum_mn", [(0, 1, 704512), (1, 58, 58.1e6), (2, 86, 134.1e6),
-                                                (3, 170, 367.9e6), (4, 156, 1100.0e6)])
+                                                (3, 170, 367.9e6), (4, 156, 1100.0e6), (5, 72, 84.9e6),
+                                                (6, 72, 84.9e6), (7, 156, 1100.0e6)])
 def test_matrix_sets(idx, n_mat, sum_mn):
     w = wl.WORKLOADS[idx]
     assert w.n_matrices == n_mat
