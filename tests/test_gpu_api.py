@@ -1,0 +1,140 @@
+"""The entry points around the step: host-buffer stepping, learning-rate changes, single-matrix refresh,
+history reset on refresh, and checkpoints under the short-side rule."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import natural_galore as orc
+from paper_2410_16029_b200 import workload as wl
+from tests.parity_util import (TOL_PROJECTOR, TOL_UPDATE, oracle_hyper, projector_distance, rel_err,
+                               to_device_bf16)
+
+pytestmark = pytest.mark.gpu
+
+
+def _make(w, T=None, **kw):
+    from paper_2410_16029_b200.ngalore import NGaLore
+
+    return NGaLore([(M, N) for _, M, N in w.shapes], w.r, w.s, w.T if T is None else T, lam=w.lam, lr=w.lr,
+                   beta1=w.beta1, beta2=w.beta2, eps=w.eps, wd=w.wd, **kw)
+
+
+def _grads(w, steps, dev):
+    return [[to_device_bf16(wl.gradient_bits(w, i, k), dev) for i in range(w.n_matrices)] for k in range(steps)]
+
+
+def test_step_host_equals_device_step():
+    """ngalore_step_host moves W and G through its own staging and must give the bits ngalore_step gives."""
+    w = wl.tiny_workload([(136, 264), (264, 136), (72, 40)], r=16, s=3, T=3, inner_rank=4, index=81, wd=0.05)
+    dev = torch.device("cuda")
+    grads = _grads(w, 7, dev)
+    a, b = _make(w), _make(w)
+    Wd = [wl.initial_weight_device(w, i, dev) for i in range(w.n_matrices)]
+    Wh = [t.cpu().pin_memory() for t in Wd]
+    for k in range(7):
+        a.step(Wd, grads[k])
+        Gh = [g.cpu().pin_memory() for g in grads[k]]
+        b.step_host(Wh, Gh)
+    torch.cuda.synchronize()
+    for x, y in zip(Wd, Wh):
+        assert torch.equal(x.cpu(), y)
+    assert a.poll_status()[0] == 0 and b.poll_status()[0] == 0
+
+
+def test_set_lr_scales_the_next_update_exactly():
+    """W <- W - lr P u with W = 0 and wd = 0: doubling lr doubles every element (a power of two is exact in fp32),
+    and the oracle with the new rate agrees."""
+    w = wl.tiny_workload([(96, 160)], r=16, s=2, T=100, inner_rank=4, index=82)
+    dev = torch.device("cuda")
+    grads = _grads(w, 3, dev)
+    a, b = _make(w), _make(w)
+    Wa = [torch.zeros((96, 160), device=dev)]
+    Wb = [torch.zeros((96, 160), device=dev)]
+    for k in range(2):
+        a.step(Wa, grads[k])
+        b.step(Wb, grads[k])
+    b.set_lr(2.0 * w.lr)
+    Wa[0].zero_()
+    Wb[0].zero_()
+    a.step(Wa, grads[2])
+    b.step(Wb, grads[2])
+    torch.cuda.synchronize()
+    assert torch.equal(Wb[0], 2.0 * Wa[0])
+    st = orc.MatrixState(96, 160, oracle_hyper(w))
+    st.set_subspace(a.get_subspace(0, working=True).cpu().numpy().astype(np.float64))
+    Wo = np.zeros((96, 160))
+    for k in range(2):
+        st.step(Wo, wl.bf16_bits_to_f64(wl.gradient_bits(w, 0, k)), auto_refresh=False)
+    st.hp.lr = 2.0 * w.lr
+    dW = st.step(np.zeros((96, 160)), wl.bf16_bits_to_f64(wl.gradient_bits(w, 0, 2)), auto_refresh=False)
+    assert rel_err(Wb[0].cpu().numpy().astype(np.float64), dW) <= TOL_UPDATE
+
+
+@pytest.mark.parametrize("impl", [dict(gemm_impl=0), dict(gemm_impl=1)])
+def test_single_matrix_refresh_touches_only_that_matrix(impl):
+    w = wl.tiny_workload([(512, 264), (264, 512)], r=32, s=2, T=0, inner_rank=8, index=83)
+    dev = torch.device("cuda")
+    opt = _make(w, **impl)
+    G0 = _grads(w, 1, dev)[0]
+    opt.refresh_subspace(G0)
+    torch.cuda.synchronize()
+    P0 = opt.get_subspace(0).clone()
+    P1 = opt.get_subspace(1).clone()
+    bits = wl.gradient_bits(w, 1, 5)
+    G1 = [G0[0], to_device_bf16(bits, dev)]
+    opt.refresh_subspace(G1, matrix_index=1)
+    torch.cuda.synchronize()
+    assert torch.equal(opt.get_subspace(0), P0)
+    Q = opt.get_subspace(1)
+    assert not torch.equal(Q, P1)
+    Qn = Q.cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(Qn.T @ Qn - np.eye(32))) <= 1e-5
+    kk, dist = projector_distance(Qn, wl.bf16_bits_to_f64(bits), opt.rank(1))
+    assert kk == 8 and dist <= TOL_PROJECTOR, (kk, dist)
+
+
+def test_reset_history_on_refresh_matches_the_oracle_option():
+    w = wl.tiny_workload([(136, 200), (200, 136)], r=16, s=4, T=3, inner_rank=4, index=84)
+    dev = torch.device("cuda")
+    opt = _make(w, reset_history_on_refresh=True)
+    hp = oracle_hyper(w, reset_history_on_refresh=True)
+    states = [orc.MatrixState(M, N, hp) for _, M, N in w.shapes]
+    W = [torch.zeros((M, N), device=dev) for _, M, N in w.shapes]
+    for k in range(8):
+        bits = [wl.gradient_bits(w, i, k) for i in range(2)]
+        for t in W:
+            t.zero_()
+        opt.step(W, [to_device_bf16(b, dev) for b in bits])
+        torch.cuda.synchronize()
+        for i, st in enumerate(states):
+            if k % w.T == 0:
+                st.set_subspace(opt.get_subspace(i, working=True).cpu().numpy().astype(np.float64))
+                st.slots, st.head, st.count = [None] * w.s, 0, 0
+            dW = st.step(np.zeros(W[i].shape), wl.bf16_bits_to_f64(bits[i]), auto_refresh=False)
+            assert rel_err(W[i].cpu().numpy().astype(np.float64), dW) <= TOL_UPDATE, (k, i)
+    assert opt.poll_status()[0] == 0
+
+
+def test_checkpoint_roundtrip_under_the_short_side_rule():
+    w = wl.tiny_workload([(200, 104), (104, 200)], r=16, s=3, T=4, inner_rank=4, index=85)
+    dev = torch.device("cuda")
+    grads = _grads(w, 9, dev)
+
+    def run(split):
+        opt = _make(w, projection="short_side")
+        W = [torch.zeros((M, N), device=dev) for _, M, N in w.shapes]
+        for k in range(9):
+            if k == split:
+                blob = opt.export_state()
+                opt.close()
+                opt = _make(w, projection="short_side")
+                opt.import_state(blob)
+            opt.step(W, grads[k])
+        torch.cuda.synchronize()
+        return W
+
+    a, b = run(-1), run(5)
+    assert all(torch.equal(x, y) for x, y in zip(a, b))
+    left = _make(w)
+    with pytest.raises(Exception):
+        left.import_state(_make(w, projection="short_side").export_state())
