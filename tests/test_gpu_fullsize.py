@@ -58,3 +58,38 @@ def test_sampled_matrices_of_full_workload(index, steps, svd_shapes):
     code, per = opt.poll_status()
     assert code == 0, (code, [p for p in per if p])
     print(f"workload {index}: worst relative update error {worst:.2e}")
+
+
+def test_long_run_across_three_refreshes():
+    """420 steps of the 60M shapes (T = 200: refreshes at steps 0, 200 and 400, the ring wraps 52 times):
+    two matrices are followed by the oracle at every step; nothing drifts, no status is raised."""
+    from paper_2410_16029_b200.ngalore import NGaLore
+
+    w = wl.WORKLOADS[1]
+    dev = torch.device("cuda")
+    shapes = [(M, N) for _, M, N in w.shapes]
+    opt = NGaLore(shapes, w.r, w.s, w.T, lam=w.lam, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, wd=w.wd)
+    sample = [1, 5]  # a 512 x 512 and a 512 x 1376 matrix of the first block
+    assert shapes[1] == (512, 512) and shapes[5] == (512, 1376)
+    states = {i: orc.MatrixState(shapes[i][0], shapes[i][1], oracle_hyper(w)) for i in sample}
+    W = [torch.zeros(s, dtype=torch.float32, device=dev) for s in shapes]
+    pool = [[wl.gradient_device(w, i, k, dev) for i in range(len(shapes))] for k in range(w.s + 3)]
+    bits = [{i: wl.bf16_bits_to_f64(wl.torch_bf16_to_bits(pool[k][i])) for i in sample} for k in range(len(pool))]
+    worst = 0.0
+    for k in range(420):
+        G = pool[k % len(pool)]
+        for i in sample:
+            W[i].zero_()
+        opt.step(W, G)
+        for i in sample:
+            st = states[i]
+            if k % w.T == 0:
+                st.set_subspace(opt.get_subspace(i, working=True).cpu().numpy().astype(np.float64))
+            dW = st.step(np.zeros(shapes[i]), bits[k % len(pool)][i], auto_refresh=False)
+            err = rel_err(W[i].cpu().numpy().astype(np.float64), dW)
+            worst = max(worst, err)
+            assert err <= TOL_UPDATE, (k, shapes[i], err)
+    code, per = opt.poll_status()
+    assert code == 0, (code, [p for p in per if p])
+    assert all(bool(torch.isfinite(t).all()) for t in W)
+    print(f"long run: worst relative update error {worst:.2e}")
