@@ -54,13 +54,19 @@ def low_rank_dims(wl, i, projection):
     return rp, (N if right else M), rp * (M if right else N)
 
 
-def byte_model(wl, projection="left"):
-    """Algorithmic bytes per step: every datum moved once (G bf16, W fp32, P bf16, history/m/v fp32)."""
+def byte_model(wl, projection="left", history="fp32"):
+    """Algorithmic bytes per step: every datum moved once (G bf16, W fp32, P bf16, history/m/v fp32).
+    With a bf16 history the s - 1 older gradients are 2 bytes each, the current one is written and read in
+    fp32, and its bf16 copy is written once."""
     tot = stream = 0
     for i, (_, M, N) in enumerate(wl.shapes):
         rp, pr, rn = low_rank_dims(wl, i, projection)
-        tot += 10 * M * N + 2 * pr * rp + (4 * wl.s + 20) * rn
-        stream += (4 * wl.s + 16) * rn          # history read once + m, v read and written
+        if history == "bf16":
+            tot += 10 * M * N + 2 * pr * rp + (2 * wl.s + 24) * rn
+            stream += (2 * wl.s + 20) * rn      # older slots (bf16) + current (fp32) once, bf16 copy, m and v
+        else:
+            tot += 10 * M * N + 2 * pr * rp + (4 * wl.s + 20) * rn
+            stream += (4 * wl.s + 16) * rn      # history read once + m, v read and written
     return tot, stream
 
 
@@ -125,7 +131,7 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------------------- oracle arm
 
-def oracle_sample(wl, seed_shift=0, P_by_shape=None, projection="left"):
+def oracle_sample(wl, seed_shift=0, P_by_shape=None, projection="left", history="fp32"):
     """Time the fp64 oracle on one matrix per distinct shape (history pre-filled to s slots) and scale by
     the shape counts to one full step.  Returns (seconds per full step, description, threads)."""
     from oracle import natural_galore as orc
@@ -138,7 +144,7 @@ def oracle_sample(wl, seed_shift=0, P_by_shape=None, projection="left"):
     rng = np.random.default_rng(1234 + seed_shift)
     for i, M, N in wl.distinct_shapes():
         hp = orc.Hyper(r=wl.r, s=wl.s, T=0, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
-                       projection=projection)
+                       projection=projection, history_bf16=history == "bf16")
         st = orc.MatrixState(M, N, hp)
         if P_by_shape is not None and (M, N) in P_by_shape:
             P = P_by_shape[(M, N)]
@@ -170,7 +176,7 @@ def run_reference(args, wl):
     times = []
     desc, threads = "", 0
     for k in range(args.warmup + args.steps):
-        t, desc, threads = oracle_sample(wl, seed_shift=k, projection=args.projection)
+        t, desc, threads = oracle_sample(wl, seed_shift=k, projection=args.projection, history=args.history)
         if k >= args.warmup:
             times.append(t)
     sec = float(np.mean(times))
@@ -178,7 +184,8 @@ def run_reference(args, wl):
     out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": wl.name, "matrices": wl.n_matrices, "r": wl.r, "s": wl.s, "projection": args.projection},
+           "config": {"workload": wl.name, "matrices": wl.n_matrices, "r": wl.r, "s": wl.s, "projection": args.projection,
+                      "history": args.history},
            "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out))
@@ -230,7 +237,7 @@ def run_ours(args, wl):
     shapes = [(M, N) for _, M, N in wl.shapes]
     n = len(shapes)
     opt = NGaLore(shapes, wl.r, wl.s, wl.T, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
-                  wd=wl.wd, seed=1 + rank, projection=args.projection)
+                  wd=wl.wd, seed=1 + rank, projection=args.projection, history_bf16=args.history == "bf16")
     # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
     wl_rank = rank_workload(wl, rank)
     # With fewer than s + 1 distinct sets a gradient would sit twice in the history ring and the Gram matrix
@@ -323,7 +330,7 @@ def run_ours(args, wl):
 
     # ---- roofline of the dominant kernel and of the whole step
     peak, peak_kind = measured_peak_hbm()
-    tot_bytes, stream_bytes = byte_model(wl, args.projection)
+    tot_bytes, stream_bytes = byte_model(wl, args.projection, args.history)
     dims = [low_rank_dims(wl, i, args.projection) for i in range(n)]
     names = ["tc_gemm_kernel<project>", "fused_stream_kernel", "tc_backproject_kernel"]
     proj_bytes = sum(2 * M * N + 2 * dims[i][1] * dims[i][0] + 4 * dims[i][2] for i, (M, N) in enumerate(shapes))
@@ -333,7 +340,7 @@ def run_ours(args, wl):
     achieved = alg[dom] / (phase[dom] * 1e-3) / 1e9
     traffic = None
     per_unit = NCU_TRAFFIC_PER_UNIT.get(names[dom])
-    if per_unit is not None and wl.r == 512 and wl.s == 16 and args.projection == "left":
+    if per_unit is not None and wl.r == 512 and wl.s == 16 and args.projection == "left" and args.history == "fp32":
         units = sum(d[2] for d in dims) if per_unit[0] == "rn" else sum(M * N for M, N in shapes)
         traffic = per_unit[1] * units
     roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -349,7 +356,7 @@ def run_ours(args, wl):
     # ---- the oracle on the host cores, bounded sample
     cpu = None
     if not args.no_cpu:
-        sec, desc, threads = oracle_sample(wl, projection=args.projection)
+        sec, desc, threads = oracle_sample(wl, projection=args.projection, history=args.history)
         cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -357,7 +364,7 @@ def run_ours(args, wl):
            "vs_baseline": None, "dtype": "bf16 (projection) and fp16 (back-projection) GEMM operands, f32 state/accumulation, f64 Gram+solve",
            "data": "synthetic",
            "config": {"workload": wl.name, "matrices": n, "r": wl.r, "s": wl.s, "T": wl.T,
-                      "projection": args.projection,
+                      "projection": args.projection, "history": args.history,
                       "l2": f"inputs larger than L2: {pool_sets} gradient sets of {grad_bytes / 1e9:.2f} GB cycled",
                       "state_bytes": opt.device_bytes},
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
@@ -385,6 +392,9 @@ def main():
     ap.add_argument("--projection", default="left", choices=["left", "short_side"],
                     help="left: R = P^T G for every matrix (the paper's form, the headline configuration); "
                          "short_side: matrices with rows >= cols are projected on the right")
+    ap.add_argument("--history", default="fp32", choices=["fp32", "bf16"],
+                    help="fp32: the ring of low-rank gradients in fp32 (the headline configuration); bf16: every "
+                         "stored gradient but the current one in bf16 (reduced-precision state option)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -79,6 +79,12 @@ typedef struct {
                                        similar to GaLore" (start of Sec. 2.4) inherits: a matrix with rows >= cols is
                                        projected on the right, R = G Q (rows x r'), W <- (1 - lr wd) W - lr u Q^T, with
                                        Q (cols x r') spanning the leading right singular vectors of G */
+  int32_t history_bf16;             /* 0 (default): the ring of low-rank gradients is fp32.  1: reduced-precision state
+                                       (the paper's conclusion names it as future work): the gradient of the current
+                                       step takes part in fp32, which the Woodbury form needs, and is stored as bf16
+                                       afterwards; the Gram matrix is kept that of the stored values.  Halves the
+                                       history traffic and memory.  Needs s >= 1 and the fused stream kernel. */
+  int32_t reserved;
 } ngalore_options;
 
 /*

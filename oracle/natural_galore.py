@@ -25,7 +25,9 @@ design notes): left projection only (the default; ``Hyper.projection =
 "short_side"`` selects the GaLore convention the paper inherits when it says, at
 the start of Sec. 2.4, that most steps are those of GaLore: project on the
 right, R = G Q with Q the first r' right singular vectors, when M >= N);
-r' = min(r, M, N); the empirical Fisher is
+r' = min(r, M, N); ``Hyper.history_bf16`` is the reduced-precision state the paper's
+conclusion names as future work: every stored gradient but the current one is
+rounded to bf16; the empirical Fisher is
 the *mean* of outer products plus lambda I (the 1/h of the Sec. 2.2 definition
 carried into Sec. 2.4); exactly s columns, the current gradient among them;
 divide by the number of gradients actually held while the history fills; eps
@@ -171,6 +173,7 @@ class Hyper:
     reset_history_on_refresh: bool = False
     store_P_as_bf16: bool = True
     projection: str = "left"        # "left": always R = P^T G; "short_side": R = G Q when M >= N
+    history_bf16: bool = False      # keep every low-rank gradient but the current one rounded to bf16
 
 
 class MatrixState:
@@ -230,6 +233,11 @@ class MatrixState:
             Nt = natural_gradient(R, self.history(), hp.lam)            # O3-O5
         else:
             Nt = R
+        if hp.s > 0 and hp.history_bf16:
+            # Reduced-precision history: the gradient of this step took part exactly (the Woodbury form
+            # needs it to lie in the span of the stacked matrix); from now on it is held as bf16.
+            slot = (self.head - 1) % hp.s
+            self.slots[slot] = round_to_bf16(self.slots[slot])
         self.m, self.v, u = adam_moments(self.m, self.v, Nt, hp.beta1, hp.beta2, hp.eps,
                                          step_index=self.k, bias_correction=hp.bias_correction,
                                          eps_outside=hp.eps_outside)    # O6

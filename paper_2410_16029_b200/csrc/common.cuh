@@ -19,7 +19,9 @@ struct MatDesc {
   int lr_rows, lr_cols;       // layout of one low-rank matrix: r' x N (left) or M x ldp (right; columns >= r' stay zero)
   long long rn;               // lr_rows * lr_cols, elements of one low-rank matrix
   int ldp, ldpt;              // leading dimensions of P16 (>= rp) and Pt16 (>= pr), multiples of 8 for TMA
-  float* H;                   // history ring: s slots of rp x N fp32 (one slot when s == 0)
+  float* H;                   // history ring: s slots of one low-rank matrix, fp32 (one slot when s == 0); with a
+                              // bf16 history only the gradient of the current step (one slot, fp32)
+  uint16_t* H16;              // bf16 history ring, s slots (null unless the state keeps its history in bf16)
   float* m;                   // first moment, rp x N
   float* v;                   // second moment, rp x N
   __half* u16;                // direction u = m / sqrt(v + eps) rounded to fp16, lr_rows x lr_cols
@@ -71,6 +73,11 @@ __device__ __forceinline__ uint2 pack_f16x4(float a, float b, float c, float d) 
   r.x = *reinterpret_cast<const uint32_t*>(&lo);
   r.y = *reinterpret_cast<const uint32_t*>(&hi);
   return r;
+}
+
+// Where the projection writes the low-rank gradient of the current step.
+__device__ __forceinline__ float* current_gradient(const MatDesc& d, int cur) {
+  return d.H16 != nullptr ? d.H : d.H + static_cast<long long>(cur) * d.rn;
 }
 
 __device__ __forceinline__ int ring_cur(const Ctrl* c, int s) {

@@ -327,7 +327,7 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
         const MatDesc& d = mats[tile.mat];
         out_cols = tile.cols;
         ld_out = tile.cols;
-        out = d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn;
+        out = current_gradient(d, ring_cur(ctrl, d.s));
         rows_total = tile.rows;
       }
       const int n_rem = out_cols - tile.n0;
@@ -394,7 +394,7 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
 // Zero the ring slot the projection is about to accumulate into, for the matrices whose K is split.
 __global__ void zero_split_slots_kernel(const MatDesc* mats, const int* split_mats, const Ctrl* ctrl) {
   const MatDesc& d = mats[split_mats[blockIdx.y]];
-  float4* p = reinterpret_cast<float4*>(d.H + static_cast<long long>(ring_cur(ctrl, d.s)) * d.rn);
+  float4* p = reinterpret_cast<float4*>(current_gradient(d, ring_cur(ctrl, d.s)));
   const long long n4 = d.rn / 4;
   for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n4;
        i += static_cast<long long>(gridDim.x) * blockDim.x)

@@ -34,29 +34,39 @@ struct FusedPlan {
   FusedItem* d_items = nullptr;
   int n_items = 0;
   int grid = 0;
+  bool hist16 = false;  // the state keeps its history ring in bf16
 };
 
 constexpr long long kSpinLimit = 4000000;  // polls of ~100 ns each before a flag wait is abandoned
-constexpr int kConsumerThreads = 256;
-constexpr int kFusedThreads = kConsumerThreads + 32;
 
 struct StageMeta {
   int mat, kind, local, first, last, count;
+  int cur, c;  // ring position and number of valid slots of this step (the same for every stage of a launch)
   long long e0;
 };
 
-template <int SMAX>
+// Stage layout.  fp32 history: SMAX slots of CE floats, then m, then v.  bf16 history (HIST16): SMAX slots of CE
+// bf16 values (the current slot's place stays unused), then the current gradient, m and v as floats.
+template <int SMAX, bool HIST16>
 struct FusedCfg {
   static constexpr int CE = SMAX <= 16 ? 1024 : 512;  // elements per stage and slot
-  static constexpr int kSlots = SMAX + 2;             // history slots + m + v
-  static constexpr int kStageBytes = kSlots * CE * 4;
-  static constexpr int kStages = SMAX <= 8 ? 5 : 3;
+  // consumer threads: the bf16 history costs more instructions per byte (conversion, two Gram rows), so it gets
+  // sixteen warps where the registers allow it
+  static constexpr int kConsumers = (HIST16 && SMAX <= 16) ? 512 : 256;
+  static constexpr int kThreads = kConsumers + 32;
+  static constexpr int kHistBytes = SMAX * CE * (HIST16 ? 2 : 4);
+  static constexpr int kCurOff = kHistBytes;                          // HIST16: fp32 gradient of this step
+  static constexpr int kMOff = kHistBytes + (HIST16 ? CE * 4 : 0);
+  static constexpr int kVOff = kMOff + CE * 4;
+  static constexpr int kStageBytes = kVOff + CE * 4;
+  static constexpr int kStages = HIST16 ? (SMAX <= 8 ? 7 : (SMAX <= 16 ? 4 : 5)) : (SMAX <= 8 ? 5 : 3);
   static constexpr int kBase = kStages * kStageBytes;
-  static constexpr int kFullOff = kBase, kEmptyOff = kBase + 64, kMetaOff = kBase + 128, kFlagOff = kBase + 384;
-  static constexpr int kWOff = kBase + 512, kRedOff = kBase + 640;
-  static constexpr int kAOff = kRedOff + (kConsumerThreads / 32) * SMAX * 8;
+  static constexpr int kFullOff = kBase, kEmptyOff = kBase + 64, kMetaOff = kBase + 128, kFlagOff = kBase + 512;
+  static constexpr int kWOff = kBase + 640, kRedOff = kBase + 768;
+  static constexpr int kRedDoubles = (kConsumers / 32) * SMAX;  // one Gram row per consumer warp
+  static constexpr int kAOff = kRedOff + (HIST16 ? 2 : 1) * kRedDoubles * 8;
   static constexpr int kTotal = kAOff + kMaxHistory * (kMaxHistory + 1) * 8;
-  static_assert(kStages * sizeof(StageMeta) <= 256, "stage metadata overflows its slot");
+  static_assert(kStages * sizeof(StageMeta) <= 384, "stage metadata overflows its slot");
   static_assert(kTotal <= 232448, "shared memory budget of one CTA exceeded");
 };
 
@@ -66,17 +76,30 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
       ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
       : "memory");
 }
+template <int THREADS>
 __device__ __forceinline__ void consumer_sync() {
-  asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+  asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");
 }
 
-template <int SMAX>
-__global__ void __launch_bounds__(kFusedThreads, 1)
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+__device__ __forceinline__ uint32_t float_to_bf16_bits(float x) {
+  return static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(x)));
+}
+
+// HIST16: the ring holds bf16 values; the gradient of the current step is read in fp32 from its own buffer
+// (MatDesc::H) and its bf16 rounding is written into ring slot `cur` by the combination pass.  The Gram pass
+// then also recomputes the row of the slot that was current one step ago, now that it is a rounded value, so
+// that Kraw stays the Gram matrix of exactly the values the combination uses.
+template <int SMAX, bool HIST16>
+__global__ void __launch_bounds__((FusedCfg<SMAX, HIST16>::kThreads), 1)
 fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restrict__ items, int n_items, Ctrl* ctrl,
                     const Hyper* __restrict__ hyper) {
-  using C = FusedCfg<SMAX>;
+  using C = FusedCfg<SMAX, HIST16>;
   constexpr int CE = C::CE;
+  constexpr int kConsumerThreads = C::kConsumers;
+  constexpr int kGroups = kConsumerThreads / 32;
   constexpr int VEC = CE / kConsumerThreads;  // 4 or 2 elements per thread and stage
+  static_assert(VEC == 2 || VEC == 4, "a thread handles two or four elements of a stage");
   extern __shared__ __align__(128) unsigned char fs_smem[];
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(fs_smem + C::kFullOff);
   uint64_t* empty_bar = reinterpret_cast<uint64_t*>(fs_smem + C::kEmptyOff);
@@ -85,6 +108,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
   volatile int* s_flag = abort_flag + 1;
   float* wsm = reinterpret_cast<float*>(fs_smem + C::kWOff);
   double* red = reinterpret_cast<double*>(fs_smem + C::kRedOff);
+  double* red2 = red + C::kRedDoubles;  // HIST16 only: the second Gram row
   double* Amat = reinterpret_cast<double*>(fs_smem + C::kAOff);
 
   const int tid = threadIdx.x;
@@ -123,6 +147,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
         const FusedItem item = items[it];
         const MatDesc& d = mats[item.mat];
         const int c = ring_count(ctrl, d.s);
+        const int cur_slot = ring_cur(ctrl, d.s);
         const int ncopies = c + (item.kind == 1 ? 2 : 0);
         const long long e0 = static_cast<long long>(item.local) * d.te;
         const long long e1 = (e0 + d.te < d.rn) ? e0 + d.te : d.rn;
@@ -138,16 +163,23 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
             StageMeta mt;
             mt.mat = item.mat; mt.kind = item.kind; mt.local = item.local;
             mt.first = (e == e0) ? 1 : 0; mt.last = (e + CE >= e1) ? 1 : 0; mt.count = cnt; mt.e0 = e;
+            mt.cur = cur_slot; mt.c = c;
             meta[stage] = mt;
-            mbar_expect_tx(full_bar + stage, bytes * static_cast<uint32_t>(ncopies));
+            mbar_expect_tx(full_bar + stage, HIST16 ? bytes * static_cast<uint32_t>(ncopies) - (bytes / 2) * static_cast<uint32_t>(c - 1)
+                                                    : bytes * static_cast<uint32_t>(ncopies));
           }
           __syncwarp();
           for (int j = lane; j < ncopies; j += 32) {
             if (j < c) {
-              bulk_load(sb + j * CE * 4, d.H + static_cast<long long>(j) * d.rn + e, bytes, full_bar + stage);
+              if (!HIST16)
+                bulk_load(sb + j * CE * 4, d.H + static_cast<long long>(j) * d.rn + e, bytes, full_bar + stage);
+              else if (j == cur_slot)
+                bulk_load(sb + C::kCurOff, d.H + e, bytes, full_bar + stage);
+              else
+                bulk_load(sb + j * CE * 2, d.H16 + static_cast<long long>(j) * d.rn + e, bytes / 2, full_bar + stage);
             } else {
               const int k = j - c;  // 0: m, 1: v
-              bulk_load(sb + (SMAX + k) * CE * 4, (k == 0 ? d.m : d.v) + e, bytes, full_bar + stage);
+              bulk_load(sb + (k == 0 ? C::kMOff : C::kVOff), (k == 0 ? d.m : d.v) + e, bytes, full_bar + stage);
             }
           }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
@@ -161,34 +193,75 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
     int stage = 0;
     uint32_t phase = 0;
     float acc[SMAX];
+    float acc2[HIST16 ? SMAX : 1];  // HIST16: inner products with the slot that was current one step ago
     float w[SMAX];
 #pragma unroll
     for (int j = 0; j < SMAX; ++j) { acc[j] = 0.f; w[j] = 0.f; }
+#pragma unroll
+    for (int j = 0; j < (HIST16 ? SMAX : 1); ++j) acc2[j] = 0.f;
     bool item_bad = false, item_ok = true;
+    // per-item pointers of the combination pass, fetched once at the item's first stage
+    float *it_m = nullptr, *it_v = nullptr, *it_cur = nullptr;
+    __half* it_u = nullptr;
+    uint16_t* it_h16 = nullptr;
     while (true) {
       if (!mbar_wait(full_bar + stage, phase, abort_flag)) break;
       const StageMeta mt = meta[stage];
       if (mt.kind < 0) break;
       const MatDesc& d = mats[mt.mat];
-      const int cur = ring_cur(ctrl, d.s), c = ring_count(ctrl, d.s);
-      const float* sb = reinterpret_cast<const float*>(fs_smem + stage * C::kStageBytes);
+      const int cur = mt.cur, c = mt.c;
+      const unsigned char* sbytes = fs_smem + stage * C::kStageBytes;
       const int idx = tid * VEC;
+      // this thread's VEC elements of history slot j in this stage
+      auto load_hist = [&](int j, float (&h)[VEC]) {
+        if (!HIST16) {
+          const float* p = reinterpret_cast<const float*>(sbytes) + j * CE + idx;
+#pragma unroll
+          for (int q = 0; q < VEC; ++q) h[q] = p[q];
+        } else if (j == cur) {
+          const float* p = reinterpret_cast<const float*>(sbytes + C::kCurOff) + idx;
+#pragma unroll
+          for (int q = 0; q < VEC; ++q) h[q] = p[q];
+        } else {
+          const uint32_t* p = reinterpret_cast<const uint32_t*>(sbytes + (j * CE + idx) * 2);
+#pragma unroll
+          for (int q = 0; q < VEC; q += 2) {
+            const uint32_t pair = p[q >> 1];
+            h[q] = bf16_bits_to_float(pair & 0xFFFFu);
+            h[q + 1] = bf16_bits_to_float(pair >> 16);
+          }
+        }
+      };
+      const float* sm_m = reinterpret_cast<const float*>(sbytes + C::kMOff);
+      const float* sm_v = reinterpret_cast<const float*>(sbytes + C::kVOff);
+      const bool two_rows = HIST16 && c >= 2;
+      const int prev = two_rows ? (cur == 0 ? d.s : cur) - 1 : 0;
       if (mt.kind == 0) {
         if (mt.first) {
 #pragma unroll
           for (int j = 0; j < SMAX; ++j) acc[j] = 0.f;
+#pragma unroll
+          for (int j = 0; j < (HIST16 ? SMAX : 1); ++j) acc2[j] = 0.f;
         }
         if (idx < mt.count) {
-          float x[VEC];
-#pragma unroll
-          for (int q = 0; q < VEC; ++q) x[q] = sb[cur * CE + idx + q];
+          float x[VEC], xp[VEC];
+          load_hist(cur, x);
+          if (two_rows) load_hist(prev, xp);
 #pragma unroll
           for (int j = 0; j < SMAX; ++j) {
             if (j < c) {
+              float h[VEC];
+              load_hist(j, h);
               float t = 0.f;
 #pragma unroll
-              for (int q = 0; q < VEC; ++q) t += x[q] * sb[j * CE + idx + q];
+              for (int q = 0; q < VEC; ++q) t += x[q] * h[q];
               acc[j] += t;
+              if (HIST16 && two_rows) {
+                float t2 = 0.f;
+#pragma unroll
+                for (int q = 0; q < VEC; ++q) t2 += xp[q] * h[q];
+                acc2[HIST16 ? j : 0] += t2;
+              }
             }
           }
         }
@@ -199,40 +272,66 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
           for (int j = 0; j < SMAX; ++j) {
             const double t = warp_sum(static_cast<double>(acc[j]));
             if (lane == 0) red[warp * SMAX + j] = t;
+            if (HIST16) {
+              const double t2 = warp_sum(static_cast<double>(acc2[HIST16 ? j : 0]));
+              if (lane == 0) red2[warp * SMAX + j] = t2;
+            }
           }
-          consumer_sync();
-          if (tid < SMAX && tid < d.s) {
+          consumer_sync<kConsumerThreads>();
+          // per-tile partial rows: [tile][s] (fp32 history) or [tile][2][s] (HIST16: row of `cur`, row of `prev`)
+          constexpr int kRows = HIST16 ? 2 : 1;
+          if (tid < kRows * 32 && (tid & 31) < SMAX && (tid & 31) < d.s) {
+            const int row = tid >> 5, j = tid & 31;
+            const double* src = row == 0 ? red : red2;
             double t = 0.0;
 #pragma unroll
-            for (int ww = 0; ww < kConsumerThreads / 32; ++ww) t += red[ww * SMAX + tid];
-            d.gpart[static_cast<long long>(mt.local) * d.s + tid] = t;
+            for (int ww = 0; ww < kConsumerThreads / 32; ++ww) t += src[ww * SMAX + j];
+            d.gpart[(static_cast<long long>(mt.local) * kRows + row) * d.s + j] = t;
             __threadfence();
           }
-          consumer_sync();
+          consumer_sync<kConsumerThreads>();
           if (tid == 0) {
             const int done = atomicAdd(d.gram_done, 1);
             *s_flag = (done == d.ntiles - 1) ? 1 : 0;
           }
-          consumer_sync();
+          consumer_sync<kConsumerThreads>();
           if (*s_flag) {
             // last Gram tile of this matrix: all consumers pre-sum the per-tile partials (fixed partition,
             // so the result is reproducible), then one warp factors and solves
             __threadfence();
             const int j = tid & 31, g = tid >> 5;
             if (j < SMAX) {
-              double t0 = 0.0, t1 = 0.0;
-              if (j < d.s) {
-                int t = g;
-                for (; t + 8 < d.ntiles; t += 16) {
-                  t0 += __ldcg(d.gpart + static_cast<long long>(t) * d.s + j);
-                  t1 += __ldcg(d.gpart + static_cast<long long>(t + 8) * d.s + j);
+#pragma unroll
+              for (int row = 0; row < kRows; ++row) {
+                double t0 = 0.0, t1 = 0.0;
+                if (j < d.s) {
+                  const double* gp = d.gpart + static_cast<long long>(row) * d.s + j;
+                  const long long tstride = static_cast<long long>(kRows) * d.s;
+                  int t = g;
+                  for (; t + kGroups < d.ntiles; t += 2 * kGroups) {
+                    t0 += __ldcg(gp + t * tstride);
+                    t1 += __ldcg(gp + (t + kGroups) * tstride);
+                  }
+                  if (t < d.ntiles) t0 += __ldcg(gp + t * tstride);
                 }
-                if (t < d.ntiles) t0 += __ldcg(d.gpart + static_cast<long long>(t) * d.s + j);
+                (row == 0 ? red : red2)[g * SMAX + j] = t0 + t1;
               }
-              red[g * SMAX + j] = t0 + t1;
             }
-            consumer_sync();
+            consumer_sync<kConsumerThreads>();
             if (tid < 32) {
+              if (two_rows) {
+                // row and column `prev` of Kraw against the stored (rounded) values; its entry with `cur`
+                // is written with the rest of row `cur` below, from the same products
+                double rowp = 0.0;
+                if (tid < c && tid != cur) {
+                  for (int gg = 0; gg < kConsumerThreads / 32; ++gg) rowp += red2[gg * SMAX + tid];
+                  if (isfinite(rowp)) {
+                    d.Kraw[prev * d.s + tid] = rowp;
+                    d.Kraw[tid * d.s + prev] = rowp;
+                  }
+                }
+                __syncwarp();
+              }
               solve_matrix(d, cur, c, hp.lambda, Amat, red, kConsumerThreads / 32, SMAX);
               if (tid == 0) {
                 *d.gram_done = 0;
@@ -241,7 +340,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
               }
             }
           }
-          consumer_sync();
+          consumer_sync<kConsumerThreads>();
         }
       } else {
         if (mt.first) {
@@ -258,13 +357,16 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
               if (!ok) atomicExch(&ctrl->timeout_flag, 1);
               *s_flag = ok;
             }
-            consumer_sync();
+            consumer_sync<kConsumerThreads>();
             item_ok = *s_flag != 0;
             __threadfence();
           }
           if (tid < kMaxHistory) wsm[tid] = __ldcg(d.wsol + tid);
           item_bad = __ldcg(d.step_bad) != 0;
-          consumer_sync();
+          it_m = d.m; it_v = d.v; it_u = d.u16;
+          it_cur = current_gradient(d, cur);
+          it_h16 = HIST16 ? d.H16 + static_cast<long long>(cur) * d.rn : nullptr;
+          consumer_sync<kConsumerThreads>();
 #pragma unroll
           for (int j = 0; j < SMAX; ++j) w[j] = wsm[j];
         }
@@ -272,11 +374,11 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
           const long long e = mt.e0 + idx;
           if (item_bad) {
             // The poisoned slot becomes a zero gradient; m, v are left alone and the update is zero.
-            float* Hc = d.H + static_cast<long long>(cur) * d.rn + e;
 #pragma unroll
             for (int q = 0; q < VEC; ++q) {
-              Hc[q] = 0.f;
-              d.u16[e + q] = __float2half_rn(0.f);
+              it_cur[e + q] = 0.f;
+              it_u[e + q] = __float2half_rn(0.f);
+              if (HIST16) it_h16[e + q] = 0;
             }
           } else {
             float n[VEC], mm[VEC], vv[VEC], uu[VEC];
@@ -285,24 +387,34 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
 #pragma unroll
             for (int j = 0; j < SMAX; ++j) {
               if (j < c) {
+                float h[VEC];
+                load_hist(j, h);
 #pragma unroll
-                for (int q = 0; q < VEC; ++q) n[q] = fmaf(w[j], sb[j * CE + idx + q], n[q]);
+                for (int q = 0; q < VEC; ++q) n[q] = fmaf(w[j], h[q], n[q]);
               }
+            }
+            if (HIST16) {
+              // from the next step on this gradient is an old one: store its bf16 rounding in the ring
+              float x[VEC];
+              load_hist(cur, x);
+              uint32_t* dst = reinterpret_cast<uint32_t*>(it_h16 + e);
+#pragma unroll
+              for (int q = 0; q < VEC; q += 2) dst[q >> 1] = float_to_bf16_bits(x[q]) | (float_to_bf16_bits(x[q + 1]) << 16);
             }
 #pragma unroll
             for (int q = 0; q < VEC; ++q) {
-              mm[q] = hp.beta1 * sb[SMAX * CE + idx + q] + (1.f - hp.beta1) * n[q];
-              vv[q] = hp.beta2 * sb[(SMAX + 1) * CE + idx + q] + (1.f - hp.beta2) * n[q] * n[q];
+              mm[q] = hp.beta1 * sm_m[idx + q] + (1.f - hp.beta1) * n[q];
+              vv[q] = hp.beta2 * sm_v[idx + q] + (1.f - hp.beta2) * n[q] * n[q];
               uu[q] = mm[q] / sqrtf(vv[q] + hp.eps);
             }
             if (VEC == 4) {
-              *reinterpret_cast<float4*>(d.m + e) = make_float4(mm[0], mm[1], mm[2 % VEC], mm[3 % VEC]);
-              *reinterpret_cast<float4*>(d.v + e) = make_float4(vv[0], vv[1], vv[2 % VEC], vv[3 % VEC]);
-              *reinterpret_cast<uint2*>(d.u16 + e) = pack_f16x4(uu[0], uu[1], uu[2 % VEC], uu[3 % VEC]);
+              *reinterpret_cast<float4*>(it_m + e) = make_float4(mm[0], mm[1], mm[2 % VEC], mm[3 % VEC]);
+              *reinterpret_cast<float4*>(it_v + e) = make_float4(vv[0], vv[1], vv[2 % VEC], vv[3 % VEC]);
+              *reinterpret_cast<uint2*>(it_u + e) = pack_f16x4(uu[0], uu[1], uu[2 % VEC], uu[3 % VEC]);
             } else {
-              *reinterpret_cast<float2*>(d.m + e) = make_float2(mm[0], mm[1]);
-              *reinterpret_cast<float2*>(d.v + e) = make_float2(vv[0], vv[1]);
-              *reinterpret_cast<uint32_t*>(d.u16 + e) = pack_f16x4(uu[0], uu[1], 0.f, 0.f).x;
+              *reinterpret_cast<float2*>(it_m + e) = make_float2(mm[0], mm[1]);
+              *reinterpret_cast<float2*>(it_v + e) = make_float2(vv[0], vv[1]);
+              *reinterpret_cast<uint32_t*>(it_u + e) = pack_f16x4(uu[0], uu[1], 0.f, 0.f).x;
             }
           }
         }
@@ -318,6 +430,12 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
     for (int i = 0; i < 200; ++i) __nanosleep(1000);
     if (tid == 0) atomicExch(&ctrl->timeout_flag, 1);
   }
+}
+
+template <int SMAX, bool HIST16>
+inline cudaError_t fused_set_smem() {
+  return cudaFuncSetAttribute(fused_stream_kernel<SMAX, HIST16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              FusedCfg<SMAX, HIST16>::kTotal);
 }
 
 inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDesc>& mats, int s, int sm_count) {
@@ -343,13 +461,12 @@ inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDe
   }
   if (cudaMemcpy(plan.d_items, items.data(), sizeof(FusedItem) * items.size(), cudaMemcpyHostToDevice) != cudaSuccess)
     return NGALORE_ERR_CUDA;
+  plan.hist16 = !mats.empty() && mats[0].H16 != nullptr;
   cudaError_t e;
-  if (s <= 8)
-    e = cudaFuncSetAttribute(fused_stream_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedCfg<8>::kTotal);
-  else if (s <= 16)
-    e = cudaFuncSetAttribute(fused_stream_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedCfg<16>::kTotal);
+  if (plan.hist16)
+    e = s <= 8 ? fused_set_smem<8, true>() : (s <= 16 ? fused_set_smem<16, true>() : fused_set_smem<32, true>());
   else
-    e = cudaFuncSetAttribute(fused_stream_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedCfg<32>::kTotal);
+    e = s <= 8 ? fused_set_smem<8, false>() : (s <= 16 ? fused_set_smem<16, false>() : fused_set_smem<32, false>());
   return e == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
@@ -358,14 +475,24 @@ inline void fused_plan_destroy(FusedPlan& plan) {
   plan.d_items = nullptr;
 }
 
+template <int SMAX, bool HIST16>
+inline void fused_launch_one(const FusedPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const Hyper* d_hyper,
+                             cudaStream_t stream) {
+  fused_stream_kernel<SMAX, HIST16><<<plan.grid, FusedCfg<SMAX, HIST16>::kThreads, FusedCfg<SMAX, HIST16>::kTotal, stream>>>(
+      d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper);
+}
+
 inline ngalore_status fused_stream_launch(FusedPlan& plan, const MatDesc* d_mats, int /*n_mats*/, Ctrl* d_ctrl,
                                           const Hyper* d_hyper, int s, cudaStream_t stream, int64_t* launches) {
-  if (s <= 8)
-    fused_stream_kernel<8><<<plan.grid, kFusedThreads, FusedCfg<8>::kTotal, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper);
-  else if (s <= 16)
-    fused_stream_kernel<16><<<plan.grid, kFusedThreads, FusedCfg<16>::kTotal, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper);
-  else
-    fused_stream_kernel<32><<<plan.grid, kFusedThreads, FusedCfg<32>::kTotal, stream>>>(d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper);
+  if (plan.hist16) {
+    if (s <= 8) fused_launch_one<8, true>(plan, d_mats, d_ctrl, d_hyper, stream);
+    else if (s <= 16) fused_launch_one<16, true>(plan, d_mats, d_ctrl, d_hyper, stream);
+    else fused_launch_one<32, true>(plan, d_mats, d_ctrl, d_hyper, stream);
+  } else {
+    if (s <= 8) fused_launch_one<8, false>(plan, d_mats, d_ctrl, d_hyper, stream);
+    else if (s <= 16) fused_launch_one<16, false>(plan, d_mats, d_ctrl, d_hyper, stream);
+    else fused_launch_one<32, false>(plan, d_mats, d_ctrl, d_hyper, stream);
+  }
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }

@@ -350,7 +350,8 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
         g.A = G[i]; g.a_rs = hm.N; g.a_cs = 1; g.a_dt = DT_BF16;
         g.B = d.P16; g.b_rs = d.ldp; g.b_cs = 1; g.b_dt = DT_BF16;
       }
-      g.C = d.H + static_cast<long long>(cur) * hm.rn; g.c_rs = hm.lr_cols; g.c_cs = 1; g.c_dt = DT_F32;
+      g.C = d.H16 != nullptr ? d.H : d.H + static_cast<long long>(cur) * hm.rn;
+      g.c_rs = hm.lr_cols; g.c_cs = 1; g.c_dt = DT_F32;
       g.epilogue = EPI_STORE;
       NG_CUDA(launch_simt_gemm<float>(g, stream));
       st->launches += 1;
@@ -440,6 +441,9 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   }
   if (opt != nullptr && opt->struct_size != static_cast<int32_t>(sizeof(ngalore_options))) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && (opt->projection_rule < 0 || opt->projection_rule > 1)) return NGALORE_ERR_INVALID_ARG;
+  if (opt != nullptr && (opt->history_bf16 < 0 || opt->history_bf16 > 1)) return NGALORE_ERR_INVALID_ARG;
+  // the bf16 history lives in the fused stream kernel only
+  if (opt != nullptr && opt->history_bf16 == 1 && (s < 1 || opt->stream_impl == 1)) return NGALORE_ERR_INVALID_ARG;
 
   int dev = 0;
   NG_CUDA(cudaGetDevice(&dev));
@@ -482,7 +486,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     total_rn += hm.rn;
     hash = (hash ^ static_cast<uint64_t>(hm.M)) * 1099511628211ull;
     hash = (hash ^ static_cast<uint64_t>(hm.N)) * 1099511628211ull;
-    hash = (hash ^ static_cast<uint64_t>(hm.right ? 2 : 1)) * 1099511628211ull;
+    hash = (hash ^ static_cast<uint64_t>((hm.right ? 2 : 1) + (st->opt.history_bf16 ? 4 : 0))) * 1099511628211ull;
   }
   st->shape_hash = hash;
   long long te_all = total_rn / (2ll * prop.multiProcessorCount) / 1024 * 1024;
@@ -492,6 +496,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
 
   // ---- arena layout
   const int slots = s > 0 ? s : 1;
+  const bool hist16 = st->opt.history_bf16 == 1;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   struct Offs { size_t H, m, v, P32, P16, Pt16, Kraw, wsol; };
@@ -501,7 +506,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   const size_t o_bad = take(sizeof(int) * n_matrices);
   for (int i = 0; i < n_matrices; ++i) {
     const HostMat& hm = st->mats[i];
-    offs[i].H = take(sizeof(float) * hm.rn * slots);
+    offs[i].H = hist16 ? take(sizeof(uint16_t) * hm.rn * slots) : take(sizeof(float) * hm.rn * slots);
     offs[i].m = take(sizeof(float) * hm.rn);
     offs[i].v = take(sizeof(float) * hm.rn);
     offs[i].P32 = take(sizeof(float) * hm.eM * hm.rp);
@@ -514,7 +519,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
 
   // ---- work layout
   off = 0;
-  struct WOffs { size_t u16, gpart, Ya, Yb, Xa, Xb, C, Gt; };
+  struct WOffs { size_t u16, gpart, Ya, Yb, Xa, Xb, C, Gt, Rcur; };
   std::vector<WOffs> woffs(n_matrices);
   const size_t o_hyper = take(sizeof(Hyper));
   const size_t o_desc = take(sizeof(MatDesc) * n_matrices);
@@ -533,7 +538,8 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     for (int t = 0; t < ntl[i]; ++t) tiles.push_back(StreamTile{i, t});
     n_tiles += ntl[i];
     woffs[i].u16 = take(sizeof(__half) * hm.rn);
-    woffs[i].gpart = take(sizeof(double) * ntl[i] * slots);
+    woffs[i].gpart = take(sizeof(double) * ntl[i] * slots * (hist16 ? 2 : 1));
+    woffs[i].Rcur = hist16 ? take(sizeof(float) * hm.rn) : 0;
     woffs[i].Ya = take(sizeof(float) * hm.eM * hm.rp);
     woffs[i].Yb = take(sizeof(float) * hm.eM * hm.rp);
     woffs[i].Xa = take(sizeof(float) * hm.eN * hm.rp);
@@ -575,7 +581,13 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     d.M = hm.M; d.N = hm.N; d.rp = hm.rp; d.s = s; d.rn = hm.rn;
     d.right = hm.right ? 1 : 0; d.pr = hm.eM; d.lr_rows = hm.lr_rows; d.lr_cols = hm.lr_cols;
     d.ldp = (hm.rp + 7) / 8 * 8; d.ldpt = (hm.eM + 7) / 8 * 8;
-    d.H = reinterpret_cast<float*>(st->arena + offs[i].H);
+    if (hist16) {
+      d.H16 = reinterpret_cast<uint16_t*>(st->arena + offs[i].H);
+      d.H = reinterpret_cast<float*>(st->work + woffs[i].Rcur);
+    } else {
+      d.H16 = nullptr;
+      d.H = reinterpret_cast<float*>(st->arena + offs[i].H);
+    }
     d.m = reinterpret_cast<float*>(st->arena + offs[i].m);
     d.v = reinterpret_cast<float*>(st->arena + offs[i].v);
     d.P32 = reinterpret_cast<float*>(st->arena + offs[i].P32);

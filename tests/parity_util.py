@@ -30,7 +30,7 @@ def rel_err(got: np.ndarray, ref: np.ndarray) -> float:
 
 
 def run_side_by_side(opt, w: wl.Workload, steps: int, mode: str, matrices=None, dev=None, wd=None,
-                     grads=None, W0=None, projection="left"):
+                     grads=None, W0=None, projection="left", oracle_over=None):
     """Run `steps` optimizer steps on both sides; returns the per-step, per-matrix relative errors.
 
     mode "A": the oracle computes each refresh (exact SVD), its bf16-rounded P is injected into the CUDA
@@ -39,7 +39,10 @@ def run_side_by_side(opt, w: wl.Workload, steps: int, mode: str, matrices=None, 
     """
     dev = dev or torch.device("cuda", torch.cuda.current_device())
     idx = list(range(w.n_matrices)) if matrices is None else list(matrices)
-    hp = oracle_hyper(w, projection=projection) if wd is None else oracle_hyper(w, wd=wd, projection=projection)
+    over = dict(oracle_over or {}, projection=projection)
+    if wd is not None:
+        over["wd"] = wd
+    hp = oracle_hyper(w, **over)
     states = {i: orc.MatrixState(w.shapes[i][1], w.shapes[i][2], hp) for i in idx}
     errs = []
     Wdev = [torch.zeros((M, N), dtype=torch.float32, device=dev) for _, M, N in w.shapes]

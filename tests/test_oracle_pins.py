@@ -425,3 +425,30 @@ def test_right_projected_update_lies_in_the_row_space_of_Q():
     assert Q.shape == (12, 3)
     assert np.linalg.norm(dW - dW @ Q @ Q.T) <= 1e-12 * np.linalg.norm(dW)
     assert np.linalg.matrix_rank(dW, tol=1e-10) <= 3
+
+
+# ----------------------------------------------------------------------------- reduced-precision history
+
+def test_bf16_history_keeps_the_current_gradient_exact_and_rounds_the_rest():
+    """With history_bf16 the natural gradient of a step is F~^-1 R for F~ = lambda I + (1/c) sum of outer
+    products of the stored gradients, where the current R enters exactly and the older ones as their bf16
+    roundings: checked by a dense solve, step by step."""
+    rng = np.random.default_rng(61)
+    M, N, r, s, lam = 6, 8, 3, 3, 1e-2
+    st = orc.MatrixState(M, N, orc.Hyper(r=r, s=s, T=0, lam=lam, history_bf16=True, store_P_as_bf16=False))
+    P, _ = np.linalg.qr(rng.standard_normal((M, r)))
+    st.set_subspace(P)
+    stored = []   # what the ring must hold before each step
+    for k in range(6):
+        G = rng.standard_normal((M, N))
+        R = P.T @ G
+        held = stored[-(s - 1):] + [R]
+        F = lam * np.eye(r * N)
+        for H in held:
+            F += np.outer(H.ravel(), H.ravel()) / len(held)
+        want = np.linalg.solve(F, R.ravel()).reshape(r, N)
+        st.step(np.zeros((M, N)), G, auto_refresh=False)
+        assert np.linalg.norm(st.last_natural_gradient - want) <= 1e-9 * np.linalg.norm(want), k
+        stored.append(orc.round_to_bf16(R))
+        ring = [h for h in st.history()]
+        assert all(np.array_equal(h, orc.round_to_bf16(h)) for h in ring)
