@@ -49,7 +49,10 @@ struct StageMeta {
 // bf16 values (the current slot's place stays unused), then the current gradient, m and v as floats.
 template <int SMAX, bool HIST16>
 struct FusedCfg {
-  static constexpr int CE = SMAX <= 16 ? 1024 : 512;  // elements per stage and slot
+  // Elements per stage and slot.  The bf16 history costs more instructions per byte (conversion, two Gram rows),
+  // and the per-stage bookkeeping of a consumer thread weighs as much as its arithmetic on two elements, so its
+  // stages are twice as long (four elements per thread) even though only two or three of them fit.
+  static constexpr int CE = SMAX <= 16 ? (HIST16 ? 2048 : 1024) : 512;
   // consumer threads: the bf16 history costs more instructions per byte (conversion, two Gram rows), so it gets
   // sixteen warps where the registers allow it
   static constexpr int kConsumers = (HIST16 && SMAX <= 16) ? 512 : 256;
@@ -59,7 +62,7 @@ struct FusedCfg {
   static constexpr int kMOff = kHistBytes + (HIST16 ? CE * 4 : 0);
   static constexpr int kVOff = kMOff + CE * 4;
   static constexpr int kStageBytes = kVOff + CE * 4;
-  static constexpr int kStages = HIST16 ? (SMAX <= 8 ? 7 : (SMAX <= 16 ? 4 : 5)) : (SMAX <= 8 ? 5 : 3);
+  static constexpr int kStages = HIST16 ? (SMAX <= 8 ? 3 : (SMAX <= 16 ? 2 : 5)) : (SMAX <= 8 ? 5 : 3);
   static constexpr int kBase = kStages * kStageBytes;
   static constexpr int kFullOff = kBase, kEmptyOff = kBase + 64, kMetaOff = kBase + 128, kFlagOff = kBase + 512;
   static constexpr int kWOff = kBase + 640, kRedOff = kBase + 768;
