@@ -124,7 +124,7 @@ ngalore_status ngalore_step(ngalore_state* st, float* const* W, const uint16_t* 
  * vectors of the gradient).  matrix_index = -1 refreshes all matrices, else one
  * (G is still the full array of n_matrices pointers; only entry matrix_index is read).
  * Uses a randomized subspace iteration; P is orthonormal to fp32 accuracy and is
- * stored both as an fp32 master and as the bf16 working copy the step reads.
+ * stored both as an fp32 master and as the working copies the step reads (the master's values rounded to bf16).
  */
 ngalore_status ngalore_refresh_subspace(ngalore_state* st, const uint16_t* const* G, int matrix_index,
                                         void* stream);
@@ -145,10 +145,10 @@ ngalore_status ngalore_poll_status(ngalore_state* st, int* per_matrix);
 
 /* Copy the fp32 master of the projector of matrix i (ngalore_subspace_rows(i) x r', row-major: P, or Q for a
  * matrix projected on the right) to / from the device buffer P.
- * set also rebuilds the bf16 working copies; the step uses the bf16 values. */
+ * set also rebuilds the working copies; the step uses the values rounded to bf16. */
 ngalore_status ngalore_get_subspace(ngalore_state* st, int i, float* P, void* stream);
 ngalore_status ngalore_set_subspace(ngalore_state* st, int i, const float* P, void* stream);
-/* Copy the bf16 working copy of P, widened to fp32 (rows x r'), to the device buffer P. */
+/* Copy the working copy of the projector (its bf16-rounded values, widened to fp32, same shape) to the device buffer P. */
 ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, void* stream);
 
 /* Checkpoint: with blob == NULL stores the needed size in *bytes; else copies the whole state

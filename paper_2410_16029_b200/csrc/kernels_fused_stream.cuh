@@ -190,7 +190,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
       }
     }
   } else {
-    // ------------------------------------------------------------------ consumers (256 threads)
+    // ------------------------------------------------------------------ consumers (8 or 16 warps)
     const int warp = tid >> 5, lane = tid & 31;
     const Hyper hp = *hyper;
     int stage = 0;

@@ -70,9 +70,6 @@ struct ngalore_state {
   int* d_step_bad = nullptr;
   StreamTile* d_tiles = nullptr;
   int n_tiles = 0;
-  float** d_W = nullptr;
-  const __nv_bfloat16** d_G = nullptr;
-  std::vector<const void*> last_W, last_G;
   std::vector<const uint16_t*> refresh_G;  // the gradients as the refresh reads them (G, or its transposed copy)
   CholProblem* d_chol = nullptr;
   int64_t k = 0;
@@ -127,22 +124,6 @@ void launch_plain_stream(ngalore_state* st, cudaStream_t stream) {
   }
   combine_kernel<SMAX><<<st->n_tiles, kStreamThreads, 0, stream>>>(st->d_desc, st->d_tiles, st->d_ctrl, st->d_hyper);
   st->launches += 1;
-}
-
-ngalore_status upload_pointers(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream,
-                               bool* changed_out) {
-  bool changed = false;
-  for (int i = 0; i < st->n; ++i) {
-    if (W != nullptr && st->last_W[i] != W[i]) { st->last_W[i] = W[i]; changed = true; }
-    if (G != nullptr && st->last_G[i] != G[i]) { st->last_G[i] = G[i]; changed = true; }
-  }
-  if (changed) {
-    // Pageable source: the runtime stages the bytes before returning, so the vectors may change later.
-    NG_CUDA(cudaMemcpyAsync(st->d_W, st->last_W.data(), sizeof(void*) * st->n, cudaMemcpyHostToDevice, stream));
-    NG_CUDA(cudaMemcpyAsync(st->d_G, st->last_G.data(), sizeof(void*) * st->n, cudaMemcpyHostToDevice, stream));
-  }
-  if (changed_out) *changed_out = changed;
-  return NGALORE_OK;
 }
 
 ngalore_status upload_hyper(ngalore_state* st, cudaStream_t stream) {
@@ -328,8 +309,6 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
     if ((rc = refresh_impl(st, G, all, stream))) return rc;
   }
   if (!st->has_subspace) return NGALORE_ERR_NO_SUBSPACE;
-  bool ptr_changed = false;
-  if ((rc = upload_pointers(st, W, G, stream, &ptr_changed))) return rc;
   if ((rc = upload_hyper(st, stream))) return rc;
   if (st->opt.gemm_impl != 1 && (rc = tc_bind_buffers(st->tc, G, W, stream))) return rc;
   const int cur = st->s > 0 ? static_cast<int>(st->n_appended % st->s) : 0;
@@ -462,11 +441,11 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   st->opt.struct_size = sizeof(ngalore_options);
   if (st->opt.seed == 0) st->opt.seed = 0x9E3779B97F4A7C15ull;
 
-  // ---- streaming tile size.  Measured on the 1.1B shapes: the persistent stream kernel pays a fixed latency per
-  // work item (table and descriptor loads, the end-of-tile reduction, the completion counter), so large tiles win
-  // (131072 elements: 5.0 ms, 32768: 5.6 ms, 4096: 9.5 ms per step); tiles shrink only to keep about two
-  // items per SM and pass on small models.  The price: the combination pass finds little of a big matrix's
-  // history still in L2, so the history is read from HBM twice per step.
+  // ---- streaming tile size.  A work item of the persistent stream kernel carries a fixed cost (table and
+  // descriptor loads, the end-of-tile reduction, the completion counter), so tiles are large; measured on the
+  // 1.1B shapes, 65536 to 262144 elements are within 1 % of each other and 16384 costs 4 %.  Tiles shrink only to
+  // keep about two items per pass and SM on small models.  The history is read from HBM twice per step: a big
+  // matrix's history does not survive in L2 between the Gram pass and the combination pass.
   uint64_t hash = 1469598103934665603ull;
   st->mats.resize(n_matrices);
   long long total_rn = 0;
@@ -523,8 +502,6 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   std::vector<WOffs> woffs(n_matrices);
   const size_t o_hyper = take(sizeof(Hyper));
   const size_t o_desc = take(sizeof(MatDesc) * n_matrices);
-  const size_t o_dW = take(sizeof(void*) * n_matrices);
-  const size_t o_dG = take(sizeof(void*) * n_matrices);
   const size_t o_chol = take(sizeof(CholProblem) * n_matrices);
   const size_t o_flags = take(sizeof(int) * 2 * n_matrices);
   int n_tiles = 0;
@@ -565,8 +542,6 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   st->d_step_bad = reinterpret_cast<int*>(st->arena + o_bad);
   st->d_hyper = reinterpret_cast<Hyper*>(st->work + o_hyper);
   st->d_desc = reinterpret_cast<MatDesc*>(st->work + o_desc);
-  st->d_W = reinterpret_cast<float**>(st->work + o_dW);
-  st->d_G = reinterpret_cast<const __nv_bfloat16**>(st->work + o_dG);
   st->d_chol = reinterpret_cast<CholProblem*>(st->work + o_chol);
   st->d_tiles = reinterpret_cast<StreamTile*>(st->work + o_tiles);
   int* flags = reinterpret_cast<int*>(st->work + o_flags);
@@ -618,8 +593,6 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
       cudaMemcpy(st->d_hyper, &st->hyper, sizeof(Hyper), cudaMemcpyHostToDevice) != cudaSuccess)
     return fail(NGALORE_ERR_CUDA);
   st->hyper_dirty = false;
-  st->last_W.assign(n_matrices, nullptr);
-  st->last_G.assign(n_matrices, nullptr);
 
   // kernels with large dynamic shared memory
   int max_rp = 0;
