@@ -28,115 +28,154 @@ __global__ void fill_normal_kernel(float* X, long long n, unsigned long long see
   X[i] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
 }
 
-// ---------------------------------------------------------------- batched Cholesky (fp64, one CTA per matrix)
+// ---------------------------------------------------------------- batched Cholesky (fp64, right-looking, blocked)
 
 struct CholProblem {
-  double* C;  // L x L row-major; lower triangle in, lower Cholesky factor out (C = Lf Lf^T)
+  double* C;    // L x L row-major; lower triangle in, lower Cholesky factor out (C = Lf Lf^T)
   int L;
+  int pad;
+  double tiny;  // pivot floor, written by chol_begin_kernel
 };
 
-// Left-looking blocked Cholesky, block width 32, 512 threads.  A pivot that is not positive
-// (rank-deficient Y) is replaced by a tiny positive number so that the factor stays finite;
-// the caller runs a second orthonormalisation pass at the end of the refresh.
-__global__ void __launch_bounds__(512) chol_batched_kernel(const CholProblem* probs) {
-  constexpr int NB = 32;
-  __shared__ double D[NB][NB + 1];   // diagonal block, or rows j0..j0+31 of the factor for one k-chunk
-  __shared__ double Rs[64][NB + 1];  // 64 panel rows for one k-chunk
-  __shared__ double maxdiag_s;
+constexpr int kCholNB = 32;  // panel width
+
+// Pivot floor of every matrix from its diagonal before the factorisation starts.  A pivot that is not above it
+// (rank-deficient Y) is replaced by it so that the factor stays finite; the caller runs a second
+// orthonormalisation pass at the end of the refresh.  One warp per matrix.
+__global__ void __launch_bounds__(32) chol_begin_kernel(CholProblem* probs) {
+  CholProblem& p = probs[blockIdx.x];
+  double md = 0.0;
+  for (int i = threadIdx.x; i < p.L; i += 32) md = fmax(md, p.C[static_cast<long long>(i) * p.L + i]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) md = fmax(md, __shfl_xor_sync(0xffffffffu, md, o));
+  if (threadIdx.x == 0) p.tiny = fmax(md, 1e-300) * 1e-28;
+}
+
+// Panel step at column j0, one CTA per matrix: factor the diagonal block in shared memory (one warp, lane = row),
+// then solve the rows below it against the block (x D^T = c, forward substitution, one thread per row).
+__global__ void __launch_bounds__(256) chol_panel_kernel(const CholProblem* probs, int j0) {
+  constexpr int NB = kCholNB;
+  __shared__ double D[NB][NB + 1];
   const CholProblem p = probs[blockIdx.x];
   double* C = p.C;
   const int L = p.L;
+  if (j0 >= L) return;
   const int tid = threadIdx.x;
-  if (tid == 0) {
-    double md = 0.0;
-    for (int i = 0; i < L; ++i) md = fmax(md, C[static_cast<long long>(i) * L + i]);
-    maxdiag_s = md;
+  const int nbj = (L - j0 < NB) ? (L - j0) : NB;
+  const double tiny = p.tiny;
+  for (int x = tid; x < NB * NB; x += 256) {
+    const int a = x / NB, b = x % NB;
+    D[a][b] = (a < nbj && b < nbj) ? C[static_cast<long long>(j0 + a) * L + j0 + b] : 0.0;
   }
   __syncthreads();
-  const double tiny = fmax(maxdiag_s, 1e-300) * 1e-28;
-
-  for (int j0 = 0; j0 < L; j0 += NB) {
-    const int nbj = (L - j0 < NB) ? (L - j0) : NB;
-    // (a) panel update: C[i][j0+jj] -= sum_{k<j0} C[i][k] C[j0+jj][k], rows i >= j0.
-    for (int r0 = j0; r0 < L; r0 += 64) {
-      const int row = tid >> 3;      // 0..63
-      const int cg = (tid & 7) * 4;  // 4 consecutive panel columns
-      double acc[4] = {0.0, 0.0, 0.0, 0.0};
-      for (int k0 = 0; k0 < j0; k0 += NB) {
-        for (int x = tid; x < NB * NB; x += 512) {
-          const int a = x / NB, b = x % NB;
-          D[a][b] = (a < nbj) ? C[static_cast<long long>(j0 + a) * L + k0 + b] : 0.0;
-        }
-        for (int x = tid; x < 64 * NB; x += 512) {
-          const int a = x / NB, b = x % NB;
-          Rs[a][b] = (r0 + a < L) ? C[static_cast<long long>(r0 + a) * L + k0 + b] : 0.0;
-        }
-        __syncthreads();
-#pragma unroll 8
-        for (int b = 0; b < NB; ++b) {
-          const double rv = Rs[row][b];
-          acc[0] += rv * D[cg + 0][b];
-          acc[1] += rv * D[cg + 1][b];
-          acc[2] += rv * D[cg + 2][b];
-          acc[3] += rv * D[cg + 3][b];
-        }
-        __syncthreads();
+  if (tid < 32) {
+    const int lane = tid;
+    for (int k = 0; k < nbj; ++k) {
+      double dkk = D[k][k];
+      if (!(dkk > tiny)) dkk = tiny;
+      const double lkk = sqrt(dkk);
+      __syncwarp();
+      if (lane == k) D[k][k] = lkk;
+      if (lane > k && lane < nbj) D[lane][k] /= lkk;
+      __syncwarp();
+      if (lane > k && lane < nbj) {
+        const double lik = D[lane][k];
+        for (int j = k + 1; j <= lane; ++j) D[lane][j] -= lik * D[j][k];
       }
-      if (r0 + row < L) {
-#pragma unroll
-        for (int y = 0; y < 4; ++y)
-          if (cg + y < nbj) C[static_cast<long long>(r0 + row) * L + j0 + cg + y] -= acc[y];
-      }
+      __syncwarp();
     }
-    __syncthreads();
-    // (b) factor the diagonal block in shared memory (warp 0, lane = row).
-    for (int x = tid; x < NB * NB; x += 512) {
-      const int a = x / NB, b = x % NB;
-      D[a][b] = (a < nbj && b < nbj) ? C[static_cast<long long>(j0 + a) * L + j0 + b] : 0.0;
-    }
-    __syncthreads();
-    if (tid < 32) {
-      const int lane = tid;
-      for (int k = 0; k < nbj; ++k) {
-        double dkk = D[k][k];
-        if (!(dkk > tiny)) dkk = tiny;
-        const double lkk = sqrt(dkk);
-        __syncwarp();
-        if (lane == k) D[k][k] = lkk;
-        if (lane > k && lane < nbj) D[lane][k] /= lkk;
-        __syncwarp();
-        if (lane > k && lane < nbj) {
-          const double lik = D[lane][k];
-          for (int j = k + 1; j <= lane; ++j) D[lane][j] -= lik * D[j][k];
-        }
-        __syncwarp();
-      }
-    }
-    __syncthreads();
-    for (int x = tid; x < NB * NB; x += 512) {
-      const int a = x / NB, b = x % NB;
-      if (a < nbj && b <= a) C[static_cast<long long>(j0 + a) * L + j0 + b] = D[a][b];
-    }
-    // (c) rows below the block: x D^T = c, forward substitution, one thread per row.
-    for (int i = j0 + nbj + tid; i < L; i += 512) {
-      double xr[NB];
-      double* crow = C + static_cast<long long>(i) * L + j0;
-#pragma unroll
-      for (int jj = 0; jj < NB; ++jj) {
-        if (jj < nbj) {
-          double a = crow[jj];
-#pragma unroll
-          for (int t = 0; t < NB; ++t)
-            if (t < jj) a -= xr[t] * D[jj][t];
-          xr[jj] = a / D[jj][jj];
-        }
-      }
-#pragma unroll
-      for (int jj = 0; jj < NB; ++jj)
-        if (jj < nbj) crow[jj] = xr[jj];
-    }
-    __syncthreads();
   }
+  __syncthreads();
+  for (int x = tid; x < NB * NB; x += 256) {
+    const int a = x / NB, b = x % NB;
+    if (a < nbj && b <= a) C[static_cast<long long>(j0 + a) * L + j0 + b] = D[a][b];
+  }
+  for (int i = j0 + nbj + tid; i < L; i += 256) {
+    double xr[NB];
+    double* crow = C + static_cast<long long>(i) * L + j0;
+#pragma unroll
+    for (int jj = 0; jj < NB; ++jj) {
+      if (jj < nbj) {
+        double a = crow[jj];
+#pragma unroll
+        for (int t = 0; t < NB; ++t)
+          if (t < jj) a -= xr[t] * D[jj][t];
+        xr[jj] = a / D[jj][jj];
+      }
+    }
+#pragma unroll
+    for (int jj = 0; jj < NB; ++jj)
+      if (jj < nbj) crow[jj] = xr[jj];
+  }
+}
+
+// Trailing update after the panel at column j0: C[i][j] -= sum_k C[i][j0 + k] C[j][j0 + k] on the lower triangle
+// beyond the panel.  blockIdx.y selects the matrix, blockIdx.x a pair (ti >= tj) of 64-row tiles.
+__global__ void __launch_bounds__(256) chol_trailing_kernel(const CholProblem* probs, int j0) {
+  constexpr int NB = kCholNB;
+  __shared__ double As[NB][64 + 1];
+  __shared__ double Bs[NB][64 + 1];
+  const CholProblem p = probs[blockIdx.y];
+  const int L = p.L, base = j0 + NB;
+  if (base >= L) return;
+  const int nt = (L - base + 63) / 64;
+  int ti = static_cast<int>((sqrtf(8.f * blockIdx.x + 1.f) - 1.f) * 0.5f);
+  while ((ti + 1) * (ti + 2) / 2 <= static_cast<int>(blockIdx.x)) ++ti;
+  while (ti * (ti + 1) / 2 > static_cast<int>(blockIdx.x)) --ti;
+  const int tj = blockIdx.x - ti * (ti + 1) / 2;
+  if (ti >= nt) return;
+  const int i0 = base + ti * 64, c0 = base + tj * 64;
+  const int t = threadIdx.x;
+  for (int x = t; x < NB * 64; x += 256) {
+    const int r = x / NB, k = x % NB;  // k contiguous in memory
+    As[k][r] = (i0 + r < L) ? p.C[static_cast<long long>(i0 + r) * L + j0 + k] : 0.0;
+    Bs[k][r] = (c0 + r < L) ? p.C[static_cast<long long>(c0 + r) * L + j0 + k] : 0.0;
+  }
+  __syncthreads();
+  const int tx = t & 15, ty = t >> 4;
+  double acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+#pragma unroll 8
+  for (int k = 0; k < NB; ++k) {
+    double a[4], b[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) { a[x] = As[k][ty * 4 + x]; b[x] = Bs[k][tx * 4 + x]; }
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) acc[x][y] += a[x] * b[y];
+  }
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    const int i = i0 + ty * 4 + x;
+    if (i >= L) continue;
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const int j = c0 + tx * 4 + y;
+      if (j <= i) p.C[static_cast<long long>(i) * L + j] -= acc[x][y];
+    }
+  }
+}
+
+// Factor n matrices (the largest of size Lmax).  Panels of 32 columns: the panel step runs one CTA per matrix, the
+// trailing update spreads over the whole GPU; 2 Lmax / 32 launches.
+inline cudaError_t chol_batched_launch(CholProblem* d_probs, int n, int Lmax, cudaStream_t stream, int64_t* launches) {
+  chol_begin_kernel<<<n, 32, 0, stream>>>(d_probs);
+  *launches += 1;
+  for (int j0 = 0; j0 < Lmax; j0 += kCholNB) {
+    chol_panel_kernel<<<n, 256, 0, stream>>>(d_probs, j0);
+    *launches += 1;
+    const int rows = Lmax - j0 - kCholNB;
+    if (rows > 0) {
+      const int nt = (rows + 63) / 64;
+      chol_trailing_kernel<<<dim3(nt * (nt + 1) / 2, n), 256, 0, stream>>>(d_probs, j0);
+      *launches += 1;
+    }
+  }
+  return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- Q = Y Lf^-T (rows are independent)

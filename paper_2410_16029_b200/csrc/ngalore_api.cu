@@ -162,13 +162,11 @@ ngalore_status orthonormalise(ngalore_state* st, const std::vector<int>& idx, in
   }
   // The problem table holds every matrix; launch over the selected ones.
   if (idx.size() == static_cast<size_t>(st->n)) {
-    chol_batched_kernel<<<st->n, 512, 0, stream>>>(st->d_chol);
-    st->launches += 1;
+    int lmax = 0;
+    for (const HostMat& hm : st->mats) lmax = hm.rp > lmax ? hm.rp : lmax;
+    NG_CUDA(chol_batched_launch(st->d_chol, st->n, lmax, stream, &st->launches));
   } else {
-    for (int i : idx) {
-      chol_batched_kernel<<<1, 512, 0, stream>>>(st->d_chol + i);
-      st->launches += 1;
-    }
+    for (int i : idx) NG_CUDA(chol_batched_launch(st->d_chol + i, 1, st->mats[i].rp, stream, &st->launches));
   }
   NG_CUDA(cudaGetLastError());
   for (int i : idx) {
@@ -583,7 +581,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     hm.Xb = reinterpret_cast<float*>(st->work + woffs[i].Xb);
     hm.C = reinterpret_cast<double*>(st->work + woffs[i].C);
     if (hm.right) hm.Gt = reinterpret_cast<uint16_t*>(st->work + woffs[i].Gt);
-    chol[i].C = hm.C; chol[i].L = hm.rp;
+    chol[i].C = hm.C; chol[i].L = hm.rp; chol[i].pad = 0; chol[i].tiny = 0.0;
     if (s == 0 && cudaMemcpy(d.wsol, w_init.data(), sizeof(float) * kMaxHistory, cudaMemcpyHostToDevice) != cudaSuccess)
       return fail(NGALORE_ERR_CUDA);
   }

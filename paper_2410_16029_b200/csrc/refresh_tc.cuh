@@ -39,11 +39,30 @@ struct SplitJob {
   int cols, ld;
 };
 
-// All matrices in one launch: blockIdx.y selects the matrix, blockIdx.x strides over its elements.
+// All matrices in one launch: blockIdx.y selects the matrix, blockIdx.x strides over its elements, four at a
+// time where the row length allows it (the kernel is a pure stream: 4 bytes in, 4 bytes out per element).
 __global__ void split_hilo_grouped_kernel(const SplitJob* jobs) {
   const SplitJob jb = jobs[blockIdx.y];
-  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < jb.n;
-       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  const long long t0 = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+  if ((jb.cols & 3) == 0 && (jb.ld & 3) == 0) {
+    const int quads_per_row = jb.cols >> 2;
+    for (long long q = t0; q < (jb.n >> 2); q += stride) {
+      const float4 x = reinterpret_cast<const float4*>(jb.src)[q];
+      const long long row = q / quads_per_row;
+      const long long o = row * jb.ld + ((q - row * quads_per_row) << 2);
+      const __nv_bfloat162 h01 = __floats2bfloat162_rn(x.x, x.y), h23 = __floats2bfloat162_rn(x.z, x.w);
+      const __nv_bfloat162 l01 = __floats2bfloat162_rn(x.x - __low2float(h01), x.y - __high2float(h01));
+      const __nv_bfloat162 l23 = __floats2bfloat162_rn(x.z - __low2float(h23), x.w - __high2float(h23));
+      uint2 hv, lv;
+      hv.x = *reinterpret_cast<const uint32_t*>(&h01); hv.y = *reinterpret_cast<const uint32_t*>(&h23);
+      lv.x = *reinterpret_cast<const uint32_t*>(&l01); lv.y = *reinterpret_cast<const uint32_t*>(&l23);
+      *reinterpret_cast<uint2*>(jb.hi + o) = hv;
+      *reinterpret_cast<uint2*>(jb.lo + o) = lv;
+    }
+    return;
+  }
+  for (long long i = t0; i < jb.n; i += stride) {
     const float x = jb.src[i];
     const __nv_bfloat16 h = __float2bfloat16_rn(x);
     const long long o = (i / jb.cols) * jb.ld + (i % jb.cols);
@@ -321,6 +340,7 @@ struct RefreshPlan {
   std::vector<int> atomic_mats[RG_COUNT];  // matrices whose K is split for this GEMM (output must be zeroed)
   GramPrep* d_prep = nullptr;
   CholProblem* d_chol = nullptr;
+  int l_max = 0;  // largest basis width L of the set
   TriInverse* d_tri = nullptr;
   TriLeaf* d_leaves = nullptr;
   int n_leaves = 0;
@@ -461,6 +481,8 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
 
   std::vector<GramPrep> prep(n);
   std::vector<CholProblem> chol(n);
+  plan.l_max = 0;
+  for (const RefreshMat& m : plan.mats) plan.l_max = m.L > plan.l_max ? m.L : plan.l_max;
   std::vector<TriInverse> tri(n);
   std::vector<SplitJob> sy(n), sz(n);
   std::vector<SyrkMat> syrk_m(n);
@@ -481,7 +503,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     m.Rhi = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Rhi);
     m.Rlo = reinterpret_cast<__nv_bfloat16*>(plan.buf + offs[i].Rlo);
     prep[i] = GramPrep{m.C32, m.C64, m.D, m.L};
-    chol[i] = CholProblem{m.C64, m.L};
+    chol[i] = CholProblem{m.C64, m.L, 0, 0.0};
     tri[i] = TriInverse{m.C64, m.D, m.X64, m.Rhi, m.Rlo, m.L, m.ldl};
     syrk_m[i] = SyrkMat{m.Yf, m.X64, m.M, m.L};
     prep64[i] = GramPrep64{m.X64, m.C64, m.D, m.L};
@@ -679,9 +701,8 @@ inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ct
   if ((rc = refresh_tc_split(plan, y_side, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, y_side ? RG_GRAM_Y : RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
   gram_prep_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep, shift_scale);
-  chol_batched_kernel<<<plan.n, 512, 0, stream>>>(plan.d_chol);
-  *launches += 2;
-  if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
+  *launches += 1;
+  if (chol_batched_launch(plan.d_chol, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, y_side ? RG_APPLY_Y : RG_APPLY_Z, d_ctrl, stream, launches))) return rc;
   return refresh_tc_split(plan, y_side, stream, launches);
@@ -698,9 +719,8 @@ inline ngalore_status refresh_tc_final(RefreshPlan& plan, Ctrl* d_ctrl, cudaStre
     if (cudaMemsetAsync(m.X64, 0, sizeof(double) * m.L * m.L, stream) != cudaSuccess) return NGALORE_ERR_CUDA;
   syrk_f64_kernel<<<plan.n_syrk_tiles, 256, 0, stream>>>(plan.d_syrk_mats, plan.d_syrk_tiles);
   gram_prep64_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep64);
-  chol_batched_kernel<<<plan.n, 512, 0, stream>>>(plan.d_chol);
-  *launches += 3;
-  if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
+  *launches += 2;
+  if (chol_batched_launch(plan.d_chol, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
   return refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches);
 }
