@@ -60,6 +60,42 @@ def test_sampled_matrices_of_full_workload(index, steps, svd_shapes):
     print(f"workload {index}: worst relative update error {worst:.2e}")
 
 
+@pytest.mark.parametrize("projection,history_bf16", [("short_side", False), ("left", True), ("short_side", True)])
+def test_options_on_the_full_1p1b_workload(projection, history_bf16):
+    """Workload 4 in the launch configuration bench.py times, under the short-side rule and/or the bf16 history:
+    one matrix of every distinct shape is followed by the oracle with the same options for a few steps."""
+    from paper_2410_16029_b200.ngalore import NGaLore
+
+    w = wl.WORKLOADS[4]
+    dev = torch.device("cuda")
+    shapes = [(M, N) for _, M, N in w.shapes]
+    opt = NGaLore(shapes, w.r, w.s, w.T, lam=w.lam, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, wd=w.wd,
+                  projection=projection, history_bf16=history_bf16)
+    sample = [i for i, _, _ in w.distinct_shapes()]
+    hp = oracle_hyper(w, projection=projection, history_bf16=history_bf16)
+    states = {i: orc.MatrixState(shapes[i][0], shapes[i][1], hp) for i in sample}
+    for i in sample:
+        assert opt.projects_right(i) == states[i].right
+    W = [torch.zeros(s, dtype=torch.float32, device=dev) for s in shapes]
+    for k in range(3):
+        G = [wl.gradient_device(w, i, k, dev) for i in range(len(shapes))]
+        for t in W:
+            t.zero_()
+        opt.step(W, G)
+        torch.cuda.synchronize()
+        for i in sample:
+            st = states[i]
+            g64 = wl.bf16_bits_to_f64(wl.torch_bf16_to_bits(G[i]))
+            if k == 0:
+                st.set_subspace(opt.get_subspace(i, working=True).cpu().numpy().astype(np.float64))
+            dW = st.step(np.zeros(shapes[i]), g64, auto_refresh=False)
+            err = rel_err(W[i].cpu().numpy().astype(np.float64), dW)
+            assert err <= TOL_UPDATE, (projection, history_bf16, k, shapes[i], err)
+        del G
+    code, per = opt.poll_status()
+    assert code == 0, (code, [p for p in per if p])
+
+
 def test_long_run_across_three_refreshes():
     """420 steps of the 60M shapes (T = 200: refreshes at steps 0, 200 and 400, the ring wraps 52 times):
     two matrices are followed by the oracle at every step; nothing drifts, no status is raised."""
