@@ -71,6 +71,10 @@ struct ngalore_state {
   StreamTile* d_tiles = nullptr;
   int n_tiles = 0;
   std::vector<const uint16_t*> refresh_G;  // the gradients as the refresh reads them (G, or its transposed copy)
+  // The tensor-core refresh stores rows of r' floats with 16-byte accesses, so it takes the matrices whose r' is a
+  // multiple of 4; the rest (r' clipped by a tiny dimension) go through the plain fp64 path.
+  std::vector<int> refresh_tc_idx, refresh_plain_idx;
+  std::vector<const uint16_t*> refresh_tc_G;
   CholProblem* d_chol = nullptr;
   int64_t k = 0;
   int64_t n_appended = 0;
@@ -217,7 +221,9 @@ ngalore_status apply_gradient(ngalore_state* st, const std::vector<int>& idx, co
   return NGALORE_OK;
 }
 
-ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bool basis_in_a, cudaStream_t stream) {
+// whole_set: this call completes a refresh of every matrix (even when idx lists only part of them).
+ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bool basis_in_a, cudaStream_t stream,
+                              bool whole_set) {
   ngalore_status rc;
   for (int i : idx) {
     const HostMat& hm = st->mats[i];
@@ -225,11 +231,11 @@ ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bo
                             cudaMemcpyDeviceToDevice, stream));
     if ((rc = make_working_copies(st, i, stream))) return rc;
   }
-  if (st->opt.reset_history_on_refresh && idx.size() == static_cast<size_t>(st->n)) {
+  if (st->opt.reset_history_on_refresh && whole_set) {
     st->n_appended = 0;
     NG_CUDA(cudaMemsetAsync(&st->d_ctrl->n_appended, 0, sizeof(long long), stream));
   }
-  if (idx.size() == static_cast<size_t>(st->n)) st->has_subspace = true;
+  if (whole_set) st->has_subspace = true;
   return NGALORE_OK;
 }
 
@@ -258,7 +264,7 @@ ngalore_status refresh_simt(ngalore_state* st, const uint16_t* const* G, const s
   }
   // Second pass Yb -> Ya so that a clamped pivot of the first pass cannot leave P non-orthonormal.
   if ((rc = orthonormalise(st, idx, 0, false, stream))) return rc;
-  return finish_refresh(st, idx, true, stream);
+  return finish_refresh(st, idx, true, stream, idx.size() == static_cast<size_t>(st->n));
 }
 
 // The subspace a matrix needs is the leading left one of G (left projection) or the leading right one, i.e. the
@@ -281,13 +287,16 @@ ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G_in, cons
   if (st->opt.gemm_impl == 1 || idx.size() != static_cast<size_t>(st->n) || !st->refresh.ready)
     return refresh_simt(st, G, idx, q, stream);
   ngalore_status rc;
-  if ((rc = refresh_tc_run(st->refresh, G, q, st->opt.seed, static_cast<unsigned long long>(st->k) * 65536ull,
-                           st->d_ctrl, stream, &st->launches)))
+  if (!st->refresh_plain_idx.empty() && (rc = refresh_simt(st, G, st->refresh_plain_idx, q, stream))) return rc;
+  st->refresh_tc_G.resize(st->refresh_tc_idx.size());
+  for (size_t p = 0; p < st->refresh_tc_idx.size(); ++p) st->refresh_tc_G[p] = G[st->refresh_tc_idx[p]];
+  if ((rc = refresh_tc_run(st->refresh, st->refresh_tc_G.data(), q, st->opt.seed,
+                           static_cast<unsigned long long>(st->k) * 65536ull, st->d_ctrl, stream, &st->launches)))
     return rc;
   // The basis sits in Ya, orthonormal to about 1e-6 where the matrix has enough rows for the bf16-pair rounding
   // of the last product to average out.  Short matrices get one exact pass (Gram, Cholesky and triangular solve in fp64): Ya -> Yb -> Ya.
   std::vector<int> small;
-  for (int i : idx)
+  for (int i : st->refresh_tc_idx)
     if (st->mats[i].eM < 512) small.push_back(i);
   if (!small.empty()) {
     if ((rc = orthonormalise(st, small, 0, true, stream))) return rc;
@@ -296,7 +305,7 @@ ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G_in, cons
       NG_CUDA(cudaMemcpyAsync(hm.Ya, hm.Yb, sizeof(float) * hm.eM * hm.rp, cudaMemcpyDeviceToDevice, stream));
     }
   }
-  return finish_refresh(st, idx, true, stream);
+  return finish_refresh(st, st->refresh_tc_idx, true, stream, true);
 }
 
 ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream) {
@@ -606,13 +615,20 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   rc = fused_plan_create(st->fused, st->h_desc, s, prop.multiProcessorCount);
   if (rc != NGALORE_OK) return fail(rc);
   if (st->opt.gemm_impl != 1) {
-    std::vector<float*> Yf(n_matrices), Zf(n_matrices);
-    for (int i = 0; i < n_matrices; ++i) { Yf[i] = st->mats[i].Ya; Zf[i] = st->mats[i].Xa; }
-    // the refresh plan sees every matrix in the orientation whose left subspace is wanted
-    std::vector<MatDesc> eff(st->h_desc);
-    for (int i = 0; i < n_matrices; ++i) { eff[i].M = st->mats[i].eM; eff[i].N = st->mats[i].eN; }
-    rc = refresh_plan_create(st->refresh, eff, Yf, Zf, prop.multiProcessorCount);
-    if (rc != NGALORE_OK) return fail(rc);
+    // the refresh plan sees every matrix it takes in the orientation whose left subspace is wanted
+    std::vector<float*> Yf, Zf;
+    std::vector<MatDesc> eff;
+    for (int i = 0; i < n_matrices; ++i) {
+      if (st->mats[i].rp % 4 != 0) { st->refresh_plain_idx.push_back(i); continue; }
+      st->refresh_tc_idx.push_back(i);
+      Yf.push_back(st->mats[i].Ya); Zf.push_back(st->mats[i].Xa);
+      eff.push_back(st->h_desc[i]);
+      eff.back().M = st->mats[i].eM; eff.back().N = st->mats[i].eN;
+    }
+    if (!eff.empty()) {
+      rc = refresh_plan_create(st->refresh, eff, Yf, Zf, prop.multiProcessorCount);
+      if (rc != NGALORE_OK) return fail(rc);
+    }
   }
   for (int e = 0; e < 4; ++e)
     if (cudaEventCreate(&st->ev[e]) != cudaSuccess) return fail(NGALORE_ERR_CUDA);

@@ -184,6 +184,22 @@ def test_long_history_uses_the_32_slot_kernels(impl):
     assert opt.poll_status()[0] == 0
 
 
+EDGE = [(1, 8), (3, 16), (16, 8), (5, 40), (129, 24), (24, 136), (1025, 8), (8, 2056), (257, 264)]
+
+
+@pytest.mark.parametrize("projection", ["left", "short_side"])
+@pytest.mark.parametrize("r,s", [(4, 2), (1, 1), (7, 3), (64, 4)])
+def test_tiny_dimensions_and_odd_ranks(projection, r, s):
+    """One-row and three-row matrices, 8-column matrices, ranks 1 and 7: r' = min(r, M, N) is then no multiple
+    of 4 for some matrices, which the tensor-core refresh cannot take (it stores rows of r' floats with 16-byte
+    accesses); those matrices are refreshed by the plain path inside the same call."""
+    w = wl.tiny_workload(EDGE, r=r, s=s, T=3, inner_rank=2, index=70)
+    opt = _make(w, projection=projection)
+    errs, _, _ = run_side_by_side(opt, w, 7, "B", projection=projection)
+    _assert_errs(errs)
+    assert opt.poll_status()[0] == 0
+
+
 def test_step_replays_from_a_cuda_graph():
     """A step enqueues only kernels once its pointer tables are warm (same W and G buffers, T = 0), so it can
     be captured in a CUDA graph; replays must match eager steps (ring position and counters live on the device)."""
