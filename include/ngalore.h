@@ -92,7 +92,8 @@ typedef struct {
  * hyper-parameters: rank r, history length s, refresh period T, Tikhonov
  * lambda, learning rate, Adam betas and eps, weight decay).
  *   shapes      host array of n_matrices shapes
- *   r >= 1      target rank; per matrix r' = min(r, rows, cols)
+ *   r >= 1      target rank; per matrix r' = min(r, rows, cols); r' may not exceed 875 (the orthonormalisation
+ *               of the refresh keeps 32 rows of r' doubles in shared memory), else NGALORE_ERR_INVALID_ARG
  *   s in [0,32] history length; 0 disables the Fisher term (plain GaLore)
  *   T >= 0      refresh period in steps; 0 = never refresh automatically
  *   lambda > 0 when s > 0

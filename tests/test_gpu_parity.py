@@ -200,6 +200,24 @@ def test_tiny_dimensions_and_odd_ranks(projection, r, s):
     assert opt.poll_status()[0] == 0
 
 
+@pytest.mark.parametrize("projection,history_bf16", [("left", False), ("short_side", True)])
+def test_large_rank_and_longest_history(projection, history_bf16):
+    """r = 768 (not a power of two, near the largest rank the library takes) with s = 32 slots."""
+    w = wl.tiny_workload([(1536, 1024), (1024, 1536)], r=768, s=32, T=40, inner_rank=6, index=71)
+    opt = _make(w, projection=projection, history_bf16=history_bf16)
+    errs, _, _ = run_side_by_side(opt, w, 4, "B", projection=projection,
+                                  oracle_over=dict(history_bf16=history_bf16))
+    _assert_errs(errs)
+    assert opt.poll_status()[0] == 0
+
+
+def test_rank_beyond_the_limit_is_rejected():
+    from paper_2410_16029_b200.ngalore import NGaLore, NGaLoreError
+
+    with pytest.raises(NGaLoreError):
+        NGaLore([(2048, 2048)], 1024, 4, 0)
+
+
 def test_step_replays_from_a_cuda_graph():
     """A step enqueues only kernels once its pointer tables are warm (same W and G buffers, T = 0), so it can
     be captured in a CUDA graph; replays must match eager steps (ring position and counters live on the device)."""
