@@ -138,3 +138,22 @@ def test_checkpoint_roundtrip_under_the_short_side_rule():
     left = _make(w)
     with pytest.raises(Exception):
         left.import_state(_make(w, projection="short_side").export_state())
+
+
+def test_steps_on_a_side_stream_match_the_default_stream():
+    """The stream argument: the same run enqueued on a non-default stream gives the same bits."""
+    w = wl.tiny_workload([(264, 136), (136, 264)], r=16, s=3, T=3, inner_rank=4, index=80)
+    dev = torch.device("cuda")
+    grads = _grads(w, 7, dev)
+    a, b = _make(w), _make(w)
+    Wa = [torch.zeros((M, N), device=dev) for _, M, N in w.shapes]
+    Wb = [torch.zeros((M, N), device=dev) for _, M, N in w.shapes]
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for k in range(7):
+        a.step(Wa, grads[k])
+        b.step(Wb, grads[k], stream=side)
+    side.synchronize()
+    torch.cuda.synchronize()
+    assert all(torch.equal(x, y) for x, y in zip(Wa, Wb))
+    assert a.poll_status()[0] == 0 and b.poll_status()[0] == 0
