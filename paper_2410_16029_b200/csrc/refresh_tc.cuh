@@ -71,6 +71,20 @@ __global__ void split_hilo_grouped_kernel(const SplitJob* jobs) {
   }
 }
 
+// Clear a list of buffers in one launch (a memset per buffer costs more in launch overhead than in work when
+// there are hundreds of small ones): blockIdx.y selects the buffer, blockIdx.x strides over its 16-byte words.
+struct ZeroJob {
+  float4* p;
+  long long n16;
+};
+
+__global__ void zero_jobs_kernel(const ZeroJob* jobs) {
+  const ZeroJob jb = jobs[blockIdx.y];
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < jb.n16;
+       i += static_cast<long long>(gridDim.x) * blockDim.x)
+    jb.p[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
 struct GramPrep {
   const float* C32;  // L x L Gram matrix from the tensor cores
   double* C64;       // L x L, lower triangle written: column-scaled, symmetrised Gram + shift I
@@ -338,6 +352,10 @@ struct RefreshPlan {
   int n_tiles[RG_COUNT] = {};
   int grid[RG_COUNT] = {};
   std::vector<int> atomic_mats[RG_COUNT];  // matrices whose K is split for this GEMM (output must be zeroed)
+  // buffers to clear before GEMM kind g (the outputs of atomic_mats[g]); entry RG_COUNT: every matrix's X64
+  ZeroJob* d_zero[RG_COUNT + 1] = {};
+  int n_zero[RG_COUNT + 1] = {};
+  char* zero_tables = nullptr;
   GramPrep* d_prep = nullptr;
   CholProblem* d_chol = nullptr;
   int l_max = 0;  // largest basis width L of the set
@@ -360,6 +378,8 @@ struct RefreshPlan {
 inline void refresh_plan_destroy(RefreshPlan& plan) {
   if (plan.buf) cudaFree(plan.buf);
   if (plan.tri_tables) cudaFree(plan.tri_tables);
+  if (plan.zero_tables) cudaFree(plan.zero_tables);
+  plan.zero_tables = nullptr;
   plan.buf = nullptr;
   plan.tri_tables = nullptr;
   plan.ready = false;
@@ -616,6 +636,42 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
       cudaMemcpy(plan.d_split_z, sz.data(), sizeof(SplitJob) * n, cudaMemcpyHostToDevice) != cudaSuccess)
     return NGALORE_ERR_CUDA;
 
+  // ---- tables of buffers to clear
+  {
+    std::vector<ZeroJob> jobs;
+    int first[RG_COUNT + 2];
+    for (int g = 0; g <= RG_COUNT; ++g) {
+      first[g] = static_cast<int>(jobs.size());
+      if (g == RG_COUNT) {
+        for (const RefreshMat& m : plan.mats)
+          jobs.push_back(ZeroJob{reinterpret_cast<float4*>(m.X64), static_cast<long long>(m.L) * m.L * 8 / 16});
+        continue;
+      }
+      for (int i : plan.atomic_mats[g]) {
+        const RefreshMat& m = plan.mats[i];
+        float* out; long long bytes;
+        switch (g) {
+          case RG_Y_FROM_Z: case RG_APPLY_Y: out = m.Yf; bytes = 4ll * m.M * m.L; break;
+          case RG_Z_FROM_Y: case RG_APPLY_Z: out = m.Zf; bytes = 4ll * m.N * m.L; break;
+          default: out = m.C32; bytes = 4ll * m.L * m.L; break;
+        }
+        jobs.push_back(ZeroJob{reinterpret_cast<float4*>(out), bytes / 16});  // L is a multiple of 4
+      }
+    }
+    first[RG_COUNT + 1] = static_cast<int>(jobs.size());
+    if (cudaMalloc(&plan.zero_tables, sizeof(ZeroJob) * (jobs.size() + 1)) != cudaSuccess) {
+      plan.zero_tables = nullptr;
+      return NGALORE_ERR_ALLOC;
+    }
+    if (!jobs.empty() && cudaMemcpy(plan.zero_tables, jobs.data(), sizeof(ZeroJob) * jobs.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+      return NGALORE_ERR_CUDA;
+    for (int g = 0; g <= RG_COUNT; ++g) {
+      plan.d_zero[g] = reinterpret_cast<ZeroJob*>(plan.zero_tables) + first[g];
+      plan.n_zero[g] = first[g + 1] - first[g];
+    }
+    plan.device_bytes += sizeof(ZeroJob) * (jobs.size() + 1);
+  }
+
   using L1 = TcSmem<kRefBN, 1, 2, kRefStages1, 4>;
   using L2 = TcSmem<kRefBN, 2, 2, kRefStages2, 4>;
   if (cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, false>,
@@ -634,15 +690,9 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
 
 inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
   // outputs that several K slices accumulate into start from zero
-  for (int i : plan.atomic_mats[g]) {
-    const RefreshMat& m = plan.mats[i];
-    float* out; size_t bytes;
-    switch (g) {
-      case RG_Y_FROM_Z: case RG_APPLY_Y: out = m.Yf; bytes = sizeof(float) * m.M * m.L; break;
-      case RG_Z_FROM_Y: case RG_APPLY_Z: out = m.Zf; bytes = sizeof(float) * m.N * m.L; break;
-      default: out = m.C32; bytes = sizeof(float) * m.L * m.L; break;
-    }
-    if (cudaMemsetAsync(out, 0, bytes, stream) != cudaSuccess) return NGALORE_ERR_CUDA;
+  if (plan.n_zero[g] > 0) {
+    zero_jobs_kernel<<<dim3(32, plan.n_zero[g]), 256, 0, stream>>>(plan.d_zero[g]);
+    *launches += 1;
   }
   using L1 = TcSmem<kRefBN, 1, 2, kRefStages1, 4>;
   using L2 = TcSmem<kRefBN, 2, 2, kRefStages2, 4>;
@@ -672,8 +722,8 @@ inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cu
 
 // X = Lf^-1 for every matrix (blocked), then R^-1 = D^-1 X^T in two bf16 parts.
 inline ngalore_status refresh_tc_tri_inverse(RefreshPlan& plan, cudaStream_t stream, int64_t* launches) {
-  for (const RefreshMat& m : plan.mats)
-    if (cudaMemsetAsync(m.X64, 0, sizeof(double) * m.L * m.L, stream) != cudaSuccess) return NGALORE_ERR_CUDA;
+  zero_jobs_kernel<<<dim3(32, plan.n_zero[RG_COUNT]), 256, 0, stream>>>(plan.d_zero[RG_COUNT]);
+  *launches += 1;
   tri_leaf_kernel<<<(plan.n_leaves + 3) / 4, 128, 0, stream>>>(plan.d_leaves, plan.n_leaves);
   *launches += 1;
   for (int h = 1; h <= plan.tri_levels; ++h) {
@@ -715,8 +765,8 @@ inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ct
 inline ngalore_status refresh_tc_final(RefreshPlan& plan, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
   ngalore_status rc;
   if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;  // bf16 parts of the basis for the apply
-  for (const RefreshMat& m : plan.mats)
-    if (cudaMemsetAsync(m.X64, 0, sizeof(double) * m.L * m.L, stream) != cudaSuccess) return NGALORE_ERR_CUDA;
+  zero_jobs_kernel<<<dim3(32, plan.n_zero[RG_COUNT]), 256, 0, stream>>>(plan.d_zero[RG_COUNT]);
+  *launches += 1;
   syrk_f64_kernel<<<plan.n_syrk_tiles, 256, 0, stream>>>(plan.d_syrk_mats, plan.d_syrk_tiles);
   gram_prep64_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep64);
   *launches += 2;
