@@ -134,7 +134,12 @@ ngalore_status ngalore_refresh_subspace(ngalore_state* st, const uint16_t* const
  * Same step with HOST buffers: copies W and G to internal device staging,
  * steps, copies W back and waits.  W_host / G_host are host arrays of HOST
  * pointers (pinned memory gives asynchronous copies).  Needs staging memory of
- * the size of all W and G, allocated on first use.
+ * the size of all W and G, allocated on first use, together with two internal
+ * copy streams: G goes in first, the projection and the history phase run while
+ * W is still arriving, and W moves in groups of matrices whose copy in,
+ * back-projection and copy out overlap across groups.  The work is ordered
+ * after what `stream` holds at the call, and the call returns when all of it
+ * is complete.
  */
 ngalore_status ngalore_step_host(ngalore_state* st, float* const* W_host, const uint16_t* const* G_host,
                                  void* stream);

@@ -288,7 +288,19 @@ inline ngalore_status tc_backproject_init() {
              : NGALORE_ERR_CUDA;
 }
 
-// W <- (1 - lr wd) W - lr P u for every matrix, through the tensor maps tc_bind_buffers set up.
+// W <- (1 - lr wd) W - lr P u for the matrices [mat0, mat1), through the tensor maps tc_bind_buffers set up.
+inline ngalore_status tc_backproject_range(TcPlan& plan, int mat0, int mat1, const MatDesc* d_mats, Ctrl* d_ctrl,
+                                           const Hyper* d_hyper, cudaStream_t stream, int64_t* launches) {
+  const int t0 = plan.back_tile0[mat0], t1 = plan.back_tile0[mat1];
+  if (t1 <= t0) return NGALORE_OK;
+  const int grid = (t1 - t0) < plan.grid_back ? (t1 - t0) : plan.grid_back;
+  tc_backproject_kernel<<<grid, kBpThreads, BpSmem::kTotal, stream>>>(plan.d_maps, plan.d_tiles_back + t0, t1 - t0,
+                                                                      d_mats, d_ctrl, d_hyper);
+  *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
+}
+
+// W <- (1 - lr wd) W - lr P u for every matrix.
 inline ngalore_status tc_backproject(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const Hyper* d_hyper,
                                      cudaStream_t stream, int64_t* launches) {
   tc_backproject_kernel<<<plan.grid_back, kBpThreads, BpSmem::kTotal, stream>>>(

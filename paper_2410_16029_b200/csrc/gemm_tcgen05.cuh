@@ -423,6 +423,7 @@ struct TcPlan {
   CUtensorMap* d_maps = nullptr;
   TcTile* d_tiles_proj = nullptr;
   TcTile* d_tiles_back = nullptr;
+  std::vector<int> back_tile0;     // first back-projection tile of every matrix, plus the total (n + 1 entries)
   int n_tiles_proj = 0, n_tiles_back = 0;
   int grid_proj = 0, grid_back = 0;
   int* d_split_mats = nullptr;
@@ -515,12 +516,15 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
         }
   }
   std::stable_sort(proj.begin(), proj.end(), [](const TcTile& a, const TcTile& b) { return a.kblocks > b.kblocks; });
+  plan.back_tile0.assign(n + 1, 0);
   for (int i = 0; i < n; ++i) {
     const MatDesc& d = mats[i];
+    plan.back_tile0[i] = static_cast<int>(back.size());
     const int kbn = (d.rp + kTcBK - 1) / kTcBK;
     for (int m0 = 0; m0 < d.M; m0 += kTcBM)
       for (int n0 = 0; n0 < d.N; n0 += kTcBackBN) back.push_back(TcTile{i, m0, n0, 0, kbn, 0, d.M, d.N});
   }
+  plan.back_tile0[n] = static_cast<int>(back.size());
   plan.n_tiles_proj = static_cast<int>(proj.size());
   plan.n_tiles_back = static_cast<int>(back.size());
   plan.grid_proj = std::min(plan.n_tiles_proj, sm_count);

@@ -87,7 +87,12 @@ struct ngalore_state {
   FusedPlan fused;
   // tensor-core refresh plan
   RefreshPlan refresh;
-  // host-buffer staging
+  // host-buffer staging; W travels in groups of matrices so that the copies in, the back-projection and the
+  // copies out of different groups overlap
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t ev_begin = nullptr, ev_G = nullptr, ev_out = nullptr;
+  std::vector<int> group_first;             // first matrix of every group, plus n
+  std::vector<cudaEvent_t> ev_w_in, ev_w_done;
   char* stage = nullptr;
   size_t stage_bytes = 0;
   std::vector<float*> stage_W;
@@ -308,7 +313,10 @@ ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G_in, cons
   return finish_refresh(st, st->refresh_tc_idx, true, stream, true);
 }
 
-ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream) {
+// grouped: the caller delivers W in the groups of ngalore_state::group_first; the back-projection of a group waits
+// for that group's event ev_w_in and records ev_w_done (host-buffer step, tensor-core path only).
+ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* const* G, cudaStream_t stream,
+                         bool grouped = false) {
   ngalore_status rc;
   if (st->T > 0 && st->k % st->T == 0) {
     std::vector<int> all(st->n);
@@ -376,6 +384,14 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       g.skip_flag = d.step_bad;
       NG_CUDA(launch_simt_gemm<float>(g, stream));
       st->launches += 1;
+    }
+  } else if (grouped) {
+    for (size_t g = 0; g + 1 < st->group_first.size(); ++g) {
+      NG_CUDA(cudaStreamWaitEvent(stream, st->ev_w_in[g], 0));
+      if ((rc = tc_backproject_range(st->tc, st->group_first[g], st->group_first[g + 1], st->d_desc, st->d_ctrl,
+                                     st->d_hyper, stream, &st->launches)))
+        return rc;
+      NG_CUDA(cudaEventRecord(st->ev_w_done[g], stream));
     }
   } else {
     if ((rc = tc_backproject(st->tc, st->d_desc, st->d_ctrl, st->d_hyper, stream, &st->launches))) return rc;
@@ -646,6 +662,13 @@ void ngalore_destroy(ngalore_state* st) {
   refresh_plan_destroy(st->refresh);
   for (int e = 0; e < 4; ++e)
     if (st->ev[e]) cudaEventDestroy(st->ev[e]);
+  for (cudaEvent_t e : st->ev_w_in) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : st->ev_w_done) if (e) cudaEventDestroy(e);
+  if (st->ev_begin) cudaEventDestroy(st->ev_begin);
+  if (st->ev_G) cudaEventDestroy(st->ev_G);
+  if (st->ev_out) cudaEventDestroy(st->ev_out);
+  if (st->copy_in) cudaStreamDestroy(st->copy_in);
+  if (st->copy_out) cudaStreamDestroy(st->copy_out);
   if (st->stage) cudaFree(st->stage);
   if (st->work) cudaFree(st->work);
   if (st->arena) cudaFree(st->arena);
@@ -701,17 +724,80 @@ ngalore_status ngalore_step_host(ngalore_state* st, float* const* W_host, const 
       st->stage_G[i] = reinterpret_cast<uint16_t*>(st->stage + og[i]);
     }
   }
+  if (st->opt.gemm_impl == 1) {
+    // debug path: everything in order on the caller's stream
+    for (int i = 0; i < st->n; ++i) {
+      const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+      NG_CUDA(cudaMemcpyAsync(st->stage_G[i], G_host[i], mn * sizeof(uint16_t), cudaMemcpyHostToDevice, s));
+      NG_CUDA(cudaMemcpyAsync(st->stage_W[i], W_host[i], mn * sizeof(float), cudaMemcpyHostToDevice, s));
+    }
+    ngalore_status rc = step_impl(st, st->stage_W.data(), st->stage_G.data(), s);
+    if (rc != NGALORE_OK) return rc;
+    for (int i = 0; i < st->n; ++i) {
+      const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+      NG_CUDA(cudaMemcpyAsync(W_host[i], st->stage_W[i], mn * sizeof(float), cudaMemcpyDeviceToHost, s));
+    }
+    NG_CUDA(cudaStreamSynchronize(s));
+    return NGALORE_OK;
+  }
+  // Pipelined: only the back-projection touches W, so the gradients go in first and the projection and the
+  // history phase run while W is still arriving; W then moves in about eight groups of matrices, each group's
+  // copy in, back-projection and copy out chained by events, so that the two directions of the link overlap.
+  if (st->copy_in == nullptr) {
+    NG_CUDA(cudaStreamCreateWithFlags(&st->copy_in, cudaStreamNonBlocking));
+    NG_CUDA(cudaStreamCreateWithFlags(&st->copy_out, cudaStreamNonBlocking));
+    NG_CUDA(cudaEventCreateWithFlags(&st->ev_begin, cudaEventDisableTiming));
+    NG_CUDA(cudaEventCreateWithFlags(&st->ev_G, cudaEventDisableTiming));
+    NG_CUDA(cudaEventCreateWithFlags(&st->ev_out, cudaEventDisableTiming));
+    size_t total = 0;
+    for (const HostMat& hm : st->mats) total += static_cast<size_t>(hm.M) * hm.N;
+    const int want = st->n < 8 ? st->n : 8;
+    st->group_first.assign(1, 0);
+    size_t acc = 0;
+    for (int i = 0; i < st->n; ++i) {
+      acc += static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+      const size_t done_groups = st->group_first.size();
+      if (i + 1 < st->n && static_cast<int>(done_groups) < want && acc * want >= total * done_groups)
+        st->group_first.push_back(i + 1);
+    }
+    st->group_first.push_back(st->n);
+    const size_t ng = st->group_first.size() - 1;
+    st->ev_w_in.resize(ng); st->ev_w_done.resize(ng);
+    for (size_t g = 0; g < ng; ++g) {
+      NG_CUDA(cudaEventCreateWithFlags(&st->ev_w_in[g], cudaEventDisableTiming));
+      NG_CUDA(cudaEventCreateWithFlags(&st->ev_w_done[g], cudaEventDisableTiming));
+    }
+  }
+  const size_t ng = st->group_first.size() - 1;
+  NG_CUDA(cudaEventRecord(st->ev_begin, s));
+  NG_CUDA(cudaStreamWaitEvent(st->copy_in, st->ev_begin, 0));
   for (int i = 0; i < st->n; ++i) {
     const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
-    NG_CUDA(cudaMemcpyAsync(st->stage_G[i], G_host[i], mn * sizeof(uint16_t), cudaMemcpyHostToDevice, s));
-    NG_CUDA(cudaMemcpyAsync(st->stage_W[i], W_host[i], mn * sizeof(float), cudaMemcpyHostToDevice, s));
+    NG_CUDA(cudaMemcpyAsync(st->stage_G[i], G_host[i], mn * sizeof(uint16_t), cudaMemcpyHostToDevice, st->copy_in));
   }
-  ngalore_status rc = step_impl(st, st->stage_W.data(), st->stage_G.data(), s);
-  if (rc != NGALORE_OK) return rc;
-  for (int i = 0; i < st->n; ++i) {
-    const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
-    NG_CUDA(cudaMemcpyAsync(W_host[i], st->stage_W[i], mn * sizeof(float), cudaMemcpyDeviceToHost, s));
+  NG_CUDA(cudaEventRecord(st->ev_G, st->copy_in));
+  for (size_t g = 0; g < ng; ++g) {
+    for (int i = st->group_first[g]; i < st->group_first[g + 1]; ++i) {
+      const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+      NG_CUDA(cudaMemcpyAsync(st->stage_W[i], W_host[i], mn * sizeof(float), cudaMemcpyHostToDevice, st->copy_in));
+    }
+    NG_CUDA(cudaEventRecord(st->ev_w_in[g], st->copy_in));
   }
+  NG_CUDA(cudaStreamWaitEvent(s, st->ev_G, 0));
+  ngalore_status rc = step_impl(st, st->stage_W.data(), st->stage_G.data(), s, true);
+  if (rc != NGALORE_OK) {
+    cudaStreamSynchronize(st->copy_in);
+    return rc;
+  }
+  for (size_t g = 0; g < ng; ++g) {
+    NG_CUDA(cudaStreamWaitEvent(st->copy_out, st->ev_w_done[g], 0));
+    for (int i = st->group_first[g]; i < st->group_first[g + 1]; ++i) {
+      const size_t mn = static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+      NG_CUDA(cudaMemcpyAsync(W_host[i], st->stage_W[i], mn * sizeof(float), cudaMemcpyDeviceToHost, st->copy_out));
+    }
+  }
+  NG_CUDA(cudaEventRecord(st->ev_out, st->copy_out));
+  NG_CUDA(cudaStreamWaitEvent(s, st->ev_out, 0));
   NG_CUDA(cudaStreamSynchronize(s));
   return NGALORE_OK;
 }
