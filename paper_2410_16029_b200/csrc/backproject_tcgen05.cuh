@@ -3,7 +3,7 @@
 // One persistent warp-specialised CTA per SM walks 128 x 256 tiles of W.  A = P16 (M x r', fp16, K-major),
 // B = u16 (r' x N, fp16), fp32 accumulator in TMEM (two buffers of 256 columns).  W never passes through
 // registers as global traffic: a producer warp streams the tile into shared memory with TMA, 32 columns
-// (one 16 KB slot of a ring) at a time, while the MMAs of the tile run; the epilogue warps update each slot
+// (one 16 KB slot of a short ring) at a time, while the MMAs of the tile run; the epilogue warps update each slot
 // in place, row per lane, against the accumulator they read with tcgen05.ld, and one lane per warp sends
 // its 32 x 32 box back with a TMA store.  The 128-byte swizzle of the W boxes makes the row-per-lane float4
 // accesses free of bank conflicts, so no transposition is needed between the TMEM layout and shared memory.
@@ -20,8 +20,13 @@
 namespace ngalore {
 
 constexpr int kBpBN = kTcBackBN;        // tile columns
-constexpr int kBpStages = 2;            // operand pipeline depth (48 KB per stage)
-constexpr int kBpSlots = 8;             // W ring: slots of 128 rows x 32 columns
+constexpr int kBpStages = 3;            // operand pipeline depth (48 KB per stage)
+// W ring: slots of 128 rows x 32 columns.  Few slots on purpose: measured on the 1.1B shapes, with two operand
+// stages 8 / 7 / 6 / 5 slots ran 2.12 / 2.07 / 1.97 / 1.93 ms, and the memory they free for a third operand stage
+// brings 1.67-1.75 ms (3 stages + 4 slots 2.13 ms, + 3 slots 2.46 ms): a W producer that runs a whole tile ahead
+// takes bandwidth from the operand loads the MMAs are waiting for.  At least four slots are needed: an epilogue
+// warp releases a slot one chunk late (see below), so each of the two chunk parities must fit two slots.
+constexpr int kBpSlots = 5;
 constexpr int kBpWProducerWarp = 10;    // warps 0, 1: operand producer and MMA issuer; 2..9: epilogue; 10: W producer
 constexpr int kBpThreads = 32 * 11;
 
@@ -37,6 +42,7 @@ struct BpSmem {
 };
 static_assert(BpSmem::kTotal <= 232448, "shared memory budget of one CTA");
 static_assert((2 * kBpStages + 4 + 2 * kBpSlots) * 8 + 8 <= 256, "barrier block");
+static_assert(kBpSlots >= 4, "the deferred slot release needs two slots per chunk parity");
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
