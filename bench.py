@@ -29,8 +29,8 @@ if ROOT not in sys.path:
 # and expressed per unit of work so that it scales to the full workload: the stream kernel's traffic grows with
 # the low-rank elements sum(r' N), the GEMMs' with sum(M N).  Valid for r = 512, s = 16 only; set an entry to None
 # when its kernel changes.
-NCU_TRAFFIC_PER_UNIT = {"fused_stream_kernel": ("rn", 145.54), "tc_backproject_kernel": ("mn", 8.383),
-                        "tc_gemm_kernel<project>": ("mn", 3.069)}
+NCU_TRAFFIC_PER_UNIT = {"fused_stream_kernel": ("rn", 145.54), "tc_backproject_kernel": ("mn", 8.361),
+                        "tc_gemm_kernel<project>": ("mn", 3.066)}
 
 METRIC = "optimizer steps/sec over all matrices (device-timed)"
 UNIT = "steps/s"
