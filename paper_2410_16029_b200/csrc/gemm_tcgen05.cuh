@@ -418,6 +418,7 @@ struct TcPlan {
   std::vector<int> rowsN;           // per matrix: M, N for re-encoding the maps of G and W
   std::vector<int> colsN;
   std::vector<int> right;           // per matrix: projected on the right
+  bool tall_proj = false;           // projection tiles are 256 rows high (tc_project2_kernel)
   std::vector<const void*> last_G;
   std::vector<const void*> last_W;
   CUtensorMap* d_maps = nullptr;
@@ -488,6 +489,18 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
 
   // ---- projection tiles: output lr_rows x lr_cols (r' x N with K = M, or M x r' with K = N when the matrix is
   // projected on the right); split K so that no tile dominates the schedule
+  // Tile height: 256 rows (two 128-row halves sharing every staged panel of B, project_tcgen05.cuh) when nearly
+  // all of the work sits in matrices with more than 128 output rows, else 128 rows.
+  {
+    long long work_all = 0, work_tall = 0;
+    for (int i = 0; i < n; ++i) {
+      const long long w = static_cast<long long>(mats[i].M) * mats[i].N;
+      work_all += w;
+      if (mats[i].lr_rows > kTcBM) work_tall += w;
+    }
+    plan.tall_proj = work_tall * 10 >= work_all * 9;
+  }
+  const int proj_bm = plan.tall_proj ? 2 * kTcBM : kTcBM;
   std::vector<TcTile> proj, back;
   long long total_kb = 0;
   for (int i = 0; i < n; ++i) {
@@ -509,7 +522,7 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
     if (splits > 1) split_mats.push_back(i);
     for (int n0 = 0; n0 < d.lr_cols; n0 += kProjBN)
       for (int sp = 0; sp < splits; ++sp)
-        for (int m0 = 0; m0 < d.lr_rows; m0 += kTcBM) {
+        for (int m0 = 0; m0 < d.lr_rows; m0 += proj_bm) {
           const int kb0 = sp * kb_per;
           const int kbn = std::min(kb_per, kb_total - kb0);
           proj.push_back(TcTile{i, m0, n0, kb0 * kTcBK, kbn, splits > 1 ? 1 : 0, d.lr_rows, d.lr_cols});
@@ -546,10 +559,6 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   plan.rowsN.resize(n); plan.colsN.resize(n); plan.right.resize(n);
   for (int i = 0; i < n; ++i) { plan.rowsN[i] = mats[i].M; plan.colsN[i] = mats[i].N; plan.right[i] = mats[i].right; }
 
-  using LP = TcSmem<kProjBN, 1, 1, kProjStages, kProjEpiWarps>;
-  if (cudaFuncSetAttribute(tc_gemm_kernel<kProjBN, 1, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps, false>,
-                           cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess)
-    return NGALORE_ERR_CUDA;
   plan.maps_dirty = true;
   return NGALORE_OK;
 }
@@ -588,20 +597,6 @@ inline ngalore_status tc_bind_buffers(TcPlan& plan, const uint16_t* const* G, fl
     plan.maps_dirty = false;
   }
   return NGALORE_OK;
-}
-
-// R = P^T G for every matrix, into ring slot `cur` (read on the device from Ctrl).
-inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, cudaStream_t stream,
-                                 int64_t* launches) {
-  if (plan.n_split > 0) {
-    zero_split_slots_kernel<<<dim3(64, plan.n_split), 256, 0, stream>>>(d_mats, plan.d_split_mats, d_ctrl);
-    *launches += 1;
-  }
-  using LP = TcSmem<kProjBN, 1, 1, kProjStages, kProjEpiWarps>;
-  tc_gemm_kernel<kProjBN, 1, 1, kProjStages, TC_EPI_PROJECT, kProjEpiWarps, false><<<plan.grid_proj, 64 + 32 * kProjEpiWarps, LP::kTotal, stream>>>(
-      plan.d_maps, plan.d_tiles_proj, plan.n_tiles_proj, d_mats, d_ctrl, nullptr);
-  *launches += 1;
-  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
 }  // namespace ngalore

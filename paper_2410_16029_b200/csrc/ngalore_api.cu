@@ -14,6 +14,7 @@
 #include "kernels_simt_gemm.cuh"
 #include "kernels_stream.cuh"
 #include "gemm_tcgen05.cuh"
+#include "project_tcgen05.cuh"
 #include "backproject_tcgen05.cuh"
 #include "kernels_fused_stream.cuh"
 #include "refresh_tc.cuh"
@@ -627,6 +628,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
 
   ngalore_status rc = tc_plan_create(st->tc, st->h_desc, st->d_desc, s, prop.multiProcessorCount);
   if (rc != NGALORE_OK) return fail(rc);
+  if ((rc = tc_project_init()) != NGALORE_OK) return fail(rc);
   if ((rc = tc_backproject_init()) != NGALORE_OK) return fail(rc);
   rc = fused_plan_create(st->fused, st->h_desc, s, prop.multiProcessorCount);
   if (rc != NGALORE_OK) return fail(rc);
