@@ -20,29 +20,32 @@
 namespace ngalore {
 
 constexpr int kBpBN = kTcBackBN;        // tile columns
-constexpr int kBpStages = 3;            // operand pipeline depth (48 KB per stage)
-// W ring: slots of 128 rows x 32 columns.  Few slots on purpose: measured on the 1.1B shapes, with two operand
-// stages 8 / 7 / 6 / 5 slots ran 2.12 / 2.07 / 1.97 / 1.93 ms, and the memory they free for a third operand stage
-// brings 1.67-1.75 ms (3 stages + 4 slots 2.13 ms, + 3 slots 2.46 ms): a W producer that runs a whole tile ahead
-// takes bandwidth from the operand loads the MMAs are waiting for.  At least four slots are needed: an epilogue
-// warp releases a slot one chunk late (see below), so each of the two chunk parities must fit two slots.
-constexpr int kBpSlots = 5;
+// Two shapes of the shared-memory budget (STAGES operand stages of 48 KB, SLOTS W slots of 128 rows x 32 columns):
+//   3 stages + 5 slots where K = r' is long (six K blocks or more): measured on the 1.1B shapes (r' = 512), with two
+//     stages 8 / 7 / 6 / 5 slots ran 2.12 / 2.07 / 1.97 / 1.93 ms and the memory a short ring frees for a third
+//     stage brings 1.67-1.75 ms (3 stages + 4 slots 2.13 ms, + 3 slots 2.46 ms): a W producer that runs a whole
+//     tile ahead takes bandwidth from the operand loads the MMAs are waiting for;
+//   2 stages + 8 slots where K is short and the kernel is all W traffic (r' = 8 on the same shapes: 1.48 ms
+//     against 1.58 ms with the short ring; r' = 256: 0.525 against 0.545 ms).
+// At least four slots are needed: an epilogue warp releases a slot one chunk late (see below), so each of the two
+// chunk parities must fit two slots.
 constexpr int kBpWProducerWarp = 10;    // warps 0, 1: operand producer and MMA issuer; 2..9: epilogue; 10: W producer
 constexpr int kBpThreads = 32 * 11;
 
+template <int STAGES, int SLOTS>
 struct BpSmem {
+  static_assert(SLOTS >= 4, "the deferred slot release needs two slots per chunk parity");
+  static_assert((2 * STAGES + 4 + 2 * SLOTS) * 8 + 8 <= 256, "barrier block");
   static constexpr int kABytes = kTcBM * kTcBK * 2;                 // 16 KB
   static constexpr int kBChunkBytes = 64 * kTcBK * 2;               // 8 KB: 64 columns x 64 K rows
   static constexpr int kStageBytes = kABytes + (kBpBN / 64) * kBChunkBytes;  // 48 KB
   static constexpr int kWBoxBytes = 32 * 32 * 4;                    // 4 KB: 32 rows x 128 B
   static constexpr int kWSlotBytes = 4 * kWBoxBytes;                // 128 rows x 32 columns
-  static constexpr int kWOffset = kBpStages * kStageBytes;
-  static constexpr int kBarOffset = kWOffset + kBpSlots * kWSlotBytes;
+  static constexpr int kWOffset = STAGES * kStageBytes;
+  static constexpr int kBarOffset = kWOffset + SLOTS * kWSlotBytes;
   static constexpr int kTotal = kBarOffset + 256 + 1024;            // barriers + slack for 1024-byte alignment
 };
-static_assert(BpSmem::kTotal <= 232448, "shared memory budget of one CTA");
-static_assert((2 * kBpStages + 4 + 2 * kBpSlots) * 8 + 8 <= 256, "barrier block");
-static_assert(kBpSlots >= 4, "the deferred slot release needs two slots per chunk parity");
+static_assert(BpSmem<3, 5>::kTotal <= 232448 && BpSmem<2, 8>::kTotal <= 232448, "shared memory budget of one CTA");
 
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
@@ -56,10 +59,11 @@ __device__ __forceinline__ int bp_wchunks(const TcTile& tile) {
   return n_rem >= kBpBN ? kBpBN / 32 : (n_rem + 31) >> 5;
 }
 
+template <int kBpStages, int kBpSlots>
 __global__ void __launch_bounds__(kBpThreads, 1)
 tc_backproject_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__ tiles, int n_tiles,
                       const MatDesc* __restrict__ mats, Ctrl* ctrl, const Hyper* __restrict__ hyper) {
-  using L = BpSmem;
+  using L = BpSmem<kBpStages, kBpSlots>;
   extern __shared__ unsigned char tc_smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
@@ -289,9 +293,12 @@ tc_backproject_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __res
 
 // Launch-time setup of the kernel above (call once per plan).
 inline ngalore_status tc_backproject_init() {
-  return cudaFuncSetAttribute(tc_backproject_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BpSmem::kTotal) == cudaSuccess
-             ? NGALORE_OK
-             : NGALORE_ERR_CUDA;
+  if (cudaFuncSetAttribute(tc_backproject_kernel<3, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           BpSmem<3, 5>::kTotal) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_backproject_kernel<2, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           BpSmem<2, 8>::kTotal) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  return NGALORE_OK;
 }
 
 // W <- (1 - lr wd) W - lr P u for the matrices [mat0, mat1), through the tensor maps tc_bind_buffers set up.
@@ -300,8 +307,12 @@ inline ngalore_status tc_backproject_range(TcPlan& plan, int mat0, int mat1, con
   const int t0 = plan.back_tile0[mat0], t1 = plan.back_tile0[mat1];
   if (t1 <= t0) return NGALORE_OK;
   const int grid = (t1 - t0) < plan.grid_back ? (t1 - t0) : plan.grid_back;
-  tc_backproject_kernel<<<grid, kBpThreads, BpSmem::kTotal, stream>>>(plan.d_maps, plan.d_tiles_back + t0, t1 - t0,
-                                                                      d_mats, d_ctrl, d_hyper);
+  if (plan.long_k_back)
+    tc_backproject_kernel<3, 5><<<grid, kBpThreads, BpSmem<3, 5>::kTotal, stream>>>(plan.d_maps, plan.d_tiles_back + t0,
+                                                                                   t1 - t0, d_mats, d_ctrl, d_hyper);
+  else
+    tc_backproject_kernel<2, 8><<<grid, kBpThreads, BpSmem<2, 8>::kTotal, stream>>>(plan.d_maps, plan.d_tiles_back + t0,
+                                                                                   t1 - t0, d_mats, d_ctrl, d_hyper);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
@@ -309,10 +320,7 @@ inline ngalore_status tc_backproject_range(TcPlan& plan, int mat0, int mat1, con
 // W <- (1 - lr wd) W - lr P u for every matrix.
 inline ngalore_status tc_backproject(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const Hyper* d_hyper,
                                      cudaStream_t stream, int64_t* launches) {
-  tc_backproject_kernel<<<plan.grid_back, kBpThreads, BpSmem::kTotal, stream>>>(
-      plan.d_maps, plan.d_tiles_back, plan.n_tiles_back, d_mats, d_ctrl, d_hyper);
-  *launches += 1;
-  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
+  return tc_backproject_range(plan, 0, plan.n_mats, d_mats, d_ctrl, d_hyper, stream, launches);
 }
 
 }  // namespace ngalore

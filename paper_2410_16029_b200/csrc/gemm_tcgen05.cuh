@@ -419,6 +419,7 @@ struct TcPlan {
   std::vector<int> colsN;
   std::vector<int> right;           // per matrix: projected on the right
   bool tall_proj = false;           // projection tiles are 256 rows high (tc_project2_kernel)
+  bool long_k_back = false;         // back-projection with three operand stages and a short W ring
   std::vector<const void*> last_G;
   std::vector<const void*> last_W;
   CUtensorMap* d_maps = nullptr;
@@ -491,14 +492,19 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   // projected on the right); split K so that no tile dominates the schedule
   // Tile height: 256 rows (two 128-row halves sharing every staged panel of B, project_tcgen05.cuh) when nearly
   // all of the work sits in matrices with more than 128 output rows, else 128 rows.
+  // Measured: on r = 512 shapes (K = 2048) the tall tiles bring 0.99 -> 0.94 ms, on r = 256 shapes (K = 768 or 1024,
+  // one tile covers all output rows) they cost 8 %, because the epilogue no longer overlaps the next tile's MMAs.
+  // The back-projection picks its shared-memory split by the length of K = r' (backproject_tcgen05.cuh).
   {
-    long long work_all = 0, work_tall = 0;
+    long long work_all = 0, work_tall = 0, work_long_k = 0;
     for (int i = 0; i < n; ++i) {
       const long long w = static_cast<long long>(mats[i].M) * mats[i].N;
       work_all += w;
-      if (mats[i].lr_rows > kTcBM) work_tall += w;
+      if (mats[i].lr_rows >= 4 * kTcBM && (mats[i].right ? mats[i].N : mats[i].M) >= 1536) work_tall += w;
+      if (mats[i].rp > 5 * kTcBK) work_long_k += w;
     }
     plan.tall_proj = work_tall * 10 >= work_all * 9;
+    plan.long_k_back = work_long_k * 10 >= work_all * 9;
   }
   const int proj_bm = plan.tall_proj ? 2 * kTcBM : kTcBM;
   std::vector<TcTile> proj, back;

@@ -6,7 +6,7 @@
 // cuts the bytes per output by a third.  The price is that TMEM has no second buffer, so the epilogue of a tile
 // does not overlap the MMAs of the next one (the operand loads of the next tile do run ahead); with K in the
 // thousands the MMAs of a tile take several times longer than its epilogue.  The host picks this kernel when
-// nearly all tiles have more than 128 output rows, else the 128-row kernel of gemm_tcgen05.cuh.
+// nearly all of the work has at least 512 output rows and K >= 1536, else the 128-row kernel of gemm_tcgen05.cuh.
 //
 // A (K-major, bf16): Pt16 (r' x M) or G (M x N); B (N contiguous, bf16): G (M x N) or Q (N x r'); the same tensor
 // maps as the 128-row kernel.  Warp roles: warp 0 TMA producer, warp 1 TMEM owner and MMA issuer, warps 2..9
