@@ -218,6 +218,24 @@ def test_rank_beyond_the_limit_is_rejected():
         NGaLore([(2048, 2048)], 1024, 4, 0)
 
 
+@pytest.mark.parametrize("mix", [0.5, 0.1, 0.01])
+def test_correlated_gradient_sequences(mix):
+    """Consecutive gradients that share 50 %, 90 % and 99 % of their content, as in training: the Gram matrix
+    is then far from diagonal and the s x s system ill conditioned; the update still matches the oracle and no
+    solve fails."""
+    w = wl.tiny_workload([(512, 1376), (1376, 512)], r=128, s=8, T=10, inner_rank=32, index=72)
+
+    def grads(i, k):
+        base = wl.gradient_f32(w, i, 0)
+        fresh = wl.gradient_f32(w, i, k + 1)
+        return wl.f32_to_bf16_bits(((1 - mix) * base + mix * fresh).astype(np.float32))
+
+    opt = _make(w)
+    errs, _, _ = run_side_by_side(opt, w, 14, "B", grads=grads)
+    _assert_errs(errs)
+    assert opt.poll_status()[0] == 0
+
+
 def test_step_replays_from_a_cuda_graph():
     """A step enqueues only kernels once its pointer tables are warm (same W and G buffers, T = 0), so it can
     be captured in a CUDA graph; replays must match eager steps (ring position and counters live on the device)."""
