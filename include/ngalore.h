@@ -91,7 +91,7 @@ typedef struct {
  * Create the state for n_matrices weight matrices (Sec. 2.2-2.4 name the
  * hyper-parameters: rank r, history length s, refresh period T, Tikhonov
  * lambda, learning rate, Adam betas and eps, weight decay).
- *   shapes      host array of n_matrices shapes
+ *   shapes      host array of n_matrices shapes (at most 65535 matrices per state)
  *   r >= 1      target rank; per matrix r' = min(r, rows, cols); r' may not exceed 875 (the orthonormalisation
  *               of the refresh keeps 32 rows of r' doubles in shared memory), else NGALORE_ERR_INVALID_ARG
  *   s in [0,32] history length; 0 disables the Fisher term (plain GaLore)

@@ -436,6 +436,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (out == nullptr) return NGALORE_ERR_INVALID_ARG;
   *out = nullptr;
   if (shapes == nullptr || n_matrices <= 0 || r < 1 || s < 0 || s > kMaxHistory || T < 0) return NGALORE_ERR_INVALID_ARG;
+  if (n_matrices > 65535) return NGALORE_ERR_INVALID_ARG;  // grouped launches index the matrix by blockIdx.y
   if (s > 0 && !(lambda > 0.0)) return NGALORE_ERR_INVALID_ARG;
   if (!(beta1 >= 0.0 && beta1 < 1.0 && beta2 >= 0.0 && beta2 < 1.0) || eps < 0.0) return NGALORE_ERR_INVALID_ARG;
   for (int i = 0; i < n_matrices; ++i) {

@@ -166,12 +166,24 @@ def test_invalid_arguments_are_rejected():
         NGaLore([(64, 64)], 8, 33, 10)           # history too long
     with pytest.raises(NGaLoreError):
         NGaLore([(64, 64)], 8, 4, 10, lam=0.0)   # lambda must be positive with a Fisher term
+    with pytest.raises(NGaLoreError):
+        NGaLore([(8, 8)] * 65536, 8, 1, 0)       # more matrices than one state takes
     opt = NGaLore([(64, 64)], 8, 4, 0)
     W = [torch.zeros((64, 64), device="cuda")]
     G = [torch.zeros((64, 64), device="cuda", dtype=torch.bfloat16)]
     with pytest.raises(NGaLoreError) as e:
         opt.step(W, G)                            # T == 0 and no subspace yet
     assert e.value.code == 5
+
+
+def test_many_small_matrices():
+    """400 matrices in one state (more matrices than SMs, more than two per CTA of every grouped launch)."""
+    shapes = [(24, 16), (16, 40), (40, 40), (8, 24)] * 100
+    w = wl.tiny_workload(shapes, r=8, s=3, T=4, inner_rank=2, index=73)
+    opt = _make(w)
+    errs, _, _ = run_side_by_side(opt, w, 6, "B", matrices=[0, 1, 2, 3, 199, 398, 399])
+    _assert_errs(errs)
+    assert opt.poll_status()[0] == 0
 
 
 @pytest.mark.parametrize("impl", IMPLS[:2])
