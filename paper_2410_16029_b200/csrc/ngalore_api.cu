@@ -497,6 +497,16 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (te_all < 2048) te_all = 2048;
   if (te_all > 131072) te_all = 131072;
   std::vector<int> tile_elems(n_matrices, static_cast<int>(te_all));
+  // The matrices at the end of the item list get tiles a quarter of the size, so that the last wave of the
+  // kernel ends more evenly (the tail of one full-size tile per SM is about 0.1 ms on the 1.1B shapes).
+  if (te_all >= 8192) {
+    const long long tail_budget = static_cast<long long>(prop.multiProcessorCount) * te_all;
+    long long acc = 0;
+    for (int i = n_matrices - 1; i >= 0 && acc < tail_budget; --i) {
+      tile_elems[i] = static_cast<int>(te_all / 4 / 1024 * 1024);
+      acc += st->mats[i].rn;
+    }
+  }
 
   // ---- arena layout
   const int slots = s > 0 ? s : 1;
