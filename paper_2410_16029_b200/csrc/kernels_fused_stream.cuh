@@ -46,8 +46,7 @@ struct StageMeta {
 };
 
 // Stage layout.  fp32 history: SMAX slots of CE floats, then m, then v.  bf16 history (HIST16): SMAX slots of CE
-// bf16 values (the current slot's place stays unused), then the current gradient as floats; m and v do not go
-// through shared memory there (the consumers read them from global memory), which leaves room for a third stage.
+// bf16 values (the current slot's place stays unused), then the current gradient, m and v as floats.
 template <int SMAX, bool HIST16>
 struct FusedCfg {
   // Elements per stage and slot.  The bf16 history costs more instructions per byte (conversion, two Gram rows),
@@ -60,16 +59,16 @@ struct FusedCfg {
   static constexpr int kThreads = kConsumers + 32;
   static constexpr int kHistBytes = SMAX * CE * (HIST16 ? 2 : 4);
   static constexpr int kCurOff = kHistBytes;                          // HIST16: fp32 gradient of this step
-  static constexpr int kMOff = kHistBytes;        // fp32 history only
-  static constexpr int kVOff = kMOff + CE * 4;    // fp32 history only
-  static constexpr int kStageBytes = HIST16 ? kCurOff + CE * 4 : kVOff + CE * 4;
-  static constexpr int kStages = HIST16 ? (SMAX <= 8 ? 5 : (SMAX <= 16 ? 3 : 6)) : (SMAX <= 8 ? 5 : 3);
+  static constexpr int kMOff = kHistBytes + (HIST16 ? CE * 4 : 0);
+  static constexpr int kVOff = kMOff + CE * 4;
+  static constexpr int kStageBytes = kVOff + CE * 4;
+  static constexpr int kStages = HIST16 ? (SMAX <= 8 ? 3 : (SMAX <= 16 ? 2 : 5)) : (SMAX <= 8 ? 5 : 3);
   static constexpr int kBase = kStages * kStageBytes;
   static constexpr int kFullOff = kBase, kEmptyOff = kBase + 64, kMetaOff = kBase + 128, kFlagOff = kBase + 512;
   static constexpr int kWOff = kBase + 640, kRedOff = kBase + 768;
   static constexpr int kRedDoubles = (kConsumers / 32) * SMAX;  // one Gram row per consumer warp
   static constexpr int kAOff = kRedOff + (HIST16 ? 2 : 1) * kRedDoubles * 8;
-  static constexpr int kTotal = kAOff + SMAX * (SMAX + 1) * 8;   // the solve's SMAX x (SMAX + 1) matrix
+  static constexpr int kTotal = kAOff + kMaxHistory * (kMaxHistory + 1) * 8;
   static_assert(kStages * sizeof(StageMeta) <= 384, "stage metadata overflows its slot");
   static_assert(kTotal <= 232448, "shared memory budget of one CTA exceeded");
 };
@@ -152,7 +151,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
         const MatDesc& d = mats[item.mat];
         const int c = ring_count(ctrl, d.s);
         const int cur_slot = ring_cur(ctrl, d.s);
-        const int ncopies = c + ((item.kind == 1 && !HIST16) ? 2 : 0);
+        const int ncopies = c + (item.kind == 1 ? 2 : 0);
         const long long e0 = static_cast<long long>(item.local) * d.te;
         const long long e1 = (e0 + d.te < d.rn) ? e0 + d.te : d.rn;
         for (long long e = e0; e < e1; e += CE) {
@@ -336,7 +335,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
                 }
                 __syncwarp();
               }
-              solve_matrix<SMAX>(d, cur, c, hp.lambda, Amat, red, kConsumerThreads / 32, SMAX);
+              solve_matrix(d, cur, c, hp.lambda, Amat, red, kConsumerThreads / 32, SMAX);
               if (tid == 0) {
                 *d.gram_done = 0;
                 __threadfence();
@@ -386,24 +385,6 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
             }
           } else {
             float n[VEC], mm[VEC], vv[VEC], uu[VEC];
-            float m_old[VEC], v_old[VEC];
-            if (HIST16) {
-              // issued first, so that the loads are in flight while the history is combined
-              if (VEC == 4) {
-                const float4 m4 = __ldcs(reinterpret_cast<const float4*>(it_m + e));
-                const float4 v4 = __ldcs(reinterpret_cast<const float4*>(it_v + e));
-                m_old[0] = m4.x; m_old[1] = m4.y; m_old[2 % VEC] = m4.z; m_old[3 % VEC] = m4.w;
-                v_old[0] = v4.x; v_old[1] = v4.y; v_old[2 % VEC] = v4.z; v_old[3 % VEC] = v4.w;
-              } else {
-                const float2 m2 = __ldcs(reinterpret_cast<const float2*>(it_m + e));
-                const float2 v2 = __ldcs(reinterpret_cast<const float2*>(it_v + e));
-                m_old[0] = m2.x; m_old[1] = m2.y;
-                v_old[0] = v2.x; v_old[1] = v2.y;
-              }
-            } else {
-#pragma unroll
-              for (int q = 0; q < VEC; ++q) { m_old[q] = sm_m[idx + q]; v_old[q] = sm_v[idx + q]; }
-            }
 #pragma unroll
             for (int q = 0; q < VEC; ++q) n[q] = 0.f;
 #pragma unroll
@@ -425,8 +406,8 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
             }
 #pragma unroll
             for (int q = 0; q < VEC; ++q) {
-              mm[q] = hp.beta1 * m_old[q] + (1.f - hp.beta1) * n[q];
-              vv[q] = hp.beta2 * v_old[q] + (1.f - hp.beta2) * n[q] * n[q];
+              mm[q] = hp.beta1 * sm_m[idx + q] + (1.f - hp.beta1) * n[q];
+              vv[q] = hp.beta2 * sm_v[idx + q] + (1.f - hp.beta2) * n[q] * n[q];
               uu[q] = mm[q] / sqrtf(vv[q] + hp.eps);
             }
             if (VEC == 4) {

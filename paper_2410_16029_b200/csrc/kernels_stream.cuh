@@ -61,15 +61,13 @@ __device__ __forceinline__ void gram_tile(const MatDesc& d, int local, int cur, 
 // the weights w of N~ = sum_i w_i H_i, i.e. (lambda I + K) w = e_cur.  This is F^-1 applied to the
 // current gradient by the Woodbury identity, written for the case where the current gradient is a
 // column of the stacked matrix; it avoids the cancellation of the two-term form.
-// A is warp-private shared memory of SDIM x (SDIM + 1) doubles, SDIM >= c (kMaxHistory unless the caller knows a
-// smaller bound on the history length).
+// A is warp-private shared memory of kMaxHistory x (kMaxHistory + 1) doubles.
 // presum (optional, shared memory): groups x stride partial sums of the Gram row, already reduced over
 // disjoint subsets of the tiles by the caller.
-template <int SDIM = kMaxHistory>
 __device__ __forceinline__ void solve_matrix(const MatDesc& d, int cur, int c, double lambda, double* A,
                                              const double* presum = nullptr, int groups = 0, int stride = 0) {
   const int lane = threadIdx.x & 31;
-  constexpr int LD = SDIM + 1;
+  constexpr int LD = kMaxHistory + 1;
   bool finite = true;
   // Gram row: lane j sums tile partials of column j.
   if (d.s > 0) {
