@@ -6,7 +6,8 @@
 One "step" is one optimizer step over every weight matrix of the workload (projection, history
 Gram + solve, natural gradient + Adam moments, back-projection + W update).  Prints ONE JSON line.
 With --gpus N > 1 (launched under torchrun) every rank steps its own replica of the matrix set
-(weak scaling, no data-path collective); the time is the maximum over ranks.
+(weak scaling, no data-path collective); the time is the maximum over ranks.  --shard instead splits one
+matrix set over the ranks and exchanges the updated weights after every step (strong scaling).
 """
 from __future__ import annotations
 
@@ -234,12 +235,27 @@ def run_ours(args, wl):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
+    parts = None
+    if args.shard and world > 1:
+        # one model over all ranks: each rank keeps the optimizer state of its share of the matrices and steps
+        # them; the updated weights of every shard are then broadcast by their owners (inside the timed region)
+        import dataclasses
+
+        from paper_2410_16029_b200 import sharding
+
+        full_shapes = [(M, N) for _, M, N in wl.shapes]
+        parts = sharding.partition(full_shapes, wl.r, wl.s, world, args.projection)
+        wl = dataclasses.replace(wl, shapes=tuple(wl.shapes[i] for i in parts[rank]))
     shapes = [(M, N) for _, M, N in wl.shapes]
     n = len(shapes)
     opt = NGaLore(shapes, wl.r, wl.s, wl.T, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
                   wd=wl.wd, seed=1 + rank, projection=args.projection, history_bf16=args.history == "bf16")
     # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
     wl_rank = rank_workload(wl, rank)
+    if parts is not None:
+        # weights of the matrices other ranks own, received after each step
+        others = {i: torch.empty(full_shapes[i], dtype=torch.float32, device=dev)
+                  for k, p in enumerate(parts) if k != rank for i in p}
     # With fewer than s + 1 distinct sets a gradient would sit twice in the history ring and the Gram matrix
     # would be singular up to lambda; the optimizer never sees that in training.
     pool_sets = args.pool if args.pool > 0 else wl.s + 1
@@ -251,6 +267,13 @@ def run_ours(args, wl):
 
     def step(k):
         opt.step_ptrs(Wp, Gp[k % pool_sets])
+        if parts is not None:
+            Wall = [None] * len(full_shapes)
+            for j, i in enumerate(parts[rank]):
+                Wall[i] = Wt[j]
+            for i, t in others.items():
+                Wall[i] = t
+            sharding.exchange_updated(Wall, parts)
 
     def barrier():
         torch.cuda.synchronize()
@@ -278,7 +301,8 @@ def run_ours(args, wl):
     clocks = sampler.stop() if rank == 0 else None
     ms_total = max_over_ranks(ms_total, dev, world)
     ms_step = ms_total / args.steps
-    value = job_throughput(world, args.steps, ms_total)
+    # sharded: the job made args.steps steps of one model; replicas: every rank made args.steps steps of its own
+    value = job_throughput(1 if parts is not None else world, args.steps, ms_total)
 
     code, per = opt.poll_status()
     if code != 0:
@@ -362,17 +386,19 @@ def run_ours(args, wl):
         cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-           "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+           "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+           "scaling": "strong" if parts is not None else "weak",
            "vs_baseline": None, "dtype": "bf16 (projection) and fp16 (back-projection) GEMM operands, f32 state/accumulation, f64 Gram+solve",
            "data": "synthetic",
            "config": {"workload": wl.name, "matrices": n, "r": wl.r, "s": wl.s, "T": wl.T,
                       "projection": args.projection, "history": args.history,
+                      "sharded": parts is not None,
                       "l2": f"inputs larger than L2: {pool_sets} gradient sets of {grad_bytes / 1e9:.2f} GB cycled",
                       "state_bytes": opt.device_bytes},
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
            "step_roofline": step_roof,
            "refresh": {"ms": refresh_ms, "T": wl.T, "amortised_ms_per_step": ms_step + refresh_ms / max(wl.T, 1),
-                       "amortised_steps_per_s": world * 1e3 / (ms_step + refresh_ms / max(wl.T, 1))},
+                       "amortised_steps_per_s": (1 if parts is not None else world) * 1e3 / (ms_step + refresh_ms / max(wl.T, 1))},
            "cpu_baseline": cpu}
     print(json.dumps(out))
     if world > 1:
@@ -397,6 +423,10 @@ def main():
     ap.add_argument("--history", default="fp32", choices=["fp32", "bf16"],
                     help="fp32: the ring of low-rank gradients in fp32 (the headline configuration); bf16: every "
                          "stored gradient but the current one in bf16 (reduced-precision state option)")
+    ap.add_argument("--shard", action="store_true",
+                    help="with --gpus N > 1: one model's matrices split over the ranks (state memory / N, weights "
+                         "exchanged after every step) instead of N independent replicas; rank 0's phases and "
+                         "roofline then describe its own shard")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -63,3 +63,65 @@ def test_reference_arm_under_two_ranks_prints_one_line():
     rec = json.loads(lines[0])
     assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["value"] > 0
     assert rec["cpu_baseline"]["kind"] == "oracle" and rec["e2e"]["h2d_bytes_per_step"] == 0
+
+
+# ----------------------------------------------------------------------------- sharding one model over ranks
+
+def test_partition_covers_every_matrix_once_and_balances():
+    sys.path.insert(0, ROOT)
+    from paper_2410_16029_b200 import sharding
+    from paper_2410_16029_b200 import workload as wl
+
+    w = wl.WORKLOADS[4]
+    shapes = [(M, N) for _, M, N in w.shapes]
+    for world in (1, 2, 3, 8):
+        parts = sharding.partition(shapes, w.r, w.s, world)
+        flat = sorted(i for p in parts for i in p)
+        assert flat == list(range(len(shapes)))
+        loads = [sum(sharding.matrix_cost(*shapes[i], w.r, w.s) for i in p) for p in parts]
+        assert max(loads) <= 1.05 * sum(loads) / world          # longest-processing-time keeps ranks within 5 %
+        assert sharding.owners(parts, len(shapes)) == [next(k for k, p in enumerate(parts) if i in p)
+                                                       for i in range(len(shapes))]
+    # the byte model is the benchmark's
+    import bench
+    assert sum(sharding.matrix_cost(M, N, w.r, w.s) for M, N in shapes) == bench.byte_model(w)[0]
+    assert sum(sharding.matrix_cost(M, N, w.r, w.s, "short_side") for M, N in shapes) == bench.byte_model(w, "short_side")[0]
+
+
+def _shard_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    from paper_2410_16029_b200 import sharding
+
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    shapes = [(8, 16), (24, 8), (16, 16), (8, 8), (32, 8)]
+    parts = sharding.partition(shapes, 4, 2, world)
+    # every rank starts from the same weights; each "steps" only its own matrices (a stand-in for the CUDA
+    # optimizer: add rank + 1), then the owners' results are exchanged
+    W = [torch.full(s, float(i)) for i, s in enumerate(shapes)]
+    for i in parts[rank]:
+        W[i] += rank + 1
+    sharding.exchange_updated(W, parts)
+    own = sharding.owners(parts, len(shapes))
+    ok = all(torch.equal(W[i], torch.full(shapes[i], float(i + own[i] + 1))) for i in range(len(shapes)))
+    gathered = [None] * world
+    dist.all_gather_object(gathered, (ok, parts))
+    if rank == 0:
+        out.put(gathered)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_exchange_their_shards():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_shard_worker, args=(r, 2, 29747, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (ok0, parts0), (ok1, parts1) = got
+    assert ok0 and ok1
+    assert parts0 == parts1 and sorted(parts0[0] + parts0[1]) == [0, 1, 2, 3, 4]
