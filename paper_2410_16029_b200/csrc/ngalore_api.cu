@@ -493,13 +493,18 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     hash = (hash ^ static_cast<uint64_t>((hm.right ? 2 : 1) + (st->opt.history_bf16 ? 4 : 0))) * 1099511628211ull;
   }
   st->shape_hash = hash;
+  // Stream tiles: two per SM and pass on large workloads.  Where that would make them short, one per SM: every tile
+  // ends with a block-wide reduction and a handful of global round trips, which on small workloads weigh as much
+  // as its traffic (measured, stream phase: RoBERTa-base shapes r = 8 / r = 4 68 -> 44 us / 52 -> 39 us, 60M shapes
+  // 116 -> 106 us; the 130M shapes and larger are 2 % better with two).
   long long te_all = total_rn / (2ll * prop.multiProcessorCount) / 1024 * 1024;
-  if (te_all < 2048) te_all = 2048;
+  if (te_all < 32768) te_all *= 2;
+  if (te_all < 4096) te_all = 4096;
   if (te_all > 131072) te_all = 131072;
   std::vector<int> tile_elems(n_matrices, static_cast<int>(te_all));
   // The matrices at the end of the item list get tiles a quarter of the size, so that the last wave of the
   // kernel ends more evenly (the tail of one full-size tile per SM is about 0.1 ms on the 1.1B shapes).
-  if (te_all >= 8192) {
+  if (te_all >= 32768) {
     const long long tail_budget = static_cast<long long>(prop.multiProcessorCount) * te_all;
     long long acc = 0;
     for (int i = n_matrices - 1; i >= 0 && acc < tail_budget; --i) {
