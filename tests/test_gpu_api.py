@@ -157,3 +157,40 @@ def test_steps_on_a_side_stream_match_the_default_stream():
     torch.cuda.synchronize()
     assert all(torch.equal(x, y) for x, y in zip(Wa, Wb))
     assert a.poll_status()[0] == 0 and b.poll_status()[0] == 0
+
+
+def test_sharded_wrapper_with_one_rank_equals_the_plain_optimizer():
+    """One rank owns every matrix: the sharded wrapper (partition, subset stepping, weight exchange over the
+    process group) must then give the bits of the plain optimizer.  The refresh draws its random test matrix from
+    the seed and the matrix's position, so both sides get the subspaces injected."""
+    import os
+
+    import torch.distributed as dist
+
+    from paper_2410_16029_b200.sharding import ShardedNGaLore
+
+    w = wl.tiny_workload([(136, 264), (264, 136), (72, 40), (200, 96)], r=16, s=3, T=0, inner_rank=4, index=83)
+    dev = torch.device("cuda")
+    shapes = [(M, N) for _, M, N in w.shapes]
+    grads = _grads(w, 5, dev)
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29761")
+    dist.init_process_group("gloo", rank=0, world_size=1)
+    try:
+        kw = dict(lam=w.lam, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, wd=w.wd)
+        sharded = ShardedNGaLore(shapes, w.r, w.s, 0, **kw)
+        assert sharded.mine == [0, 1, 2, 3] and sharded.parts == [[0, 1, 2, 3]]
+        plain = _make(w, T=0)
+        plain.refresh_subspace(grads[0])
+        for i in range(len(shapes)):
+            sharded.opt.set_subspace(i, plain.get_subspace(i))
+        Wa = [wl.initial_weight_device(w, i, dev) for i in range(w.n_matrices)]
+        Wb = [t.clone() for t in Wa]
+        for k in range(5):
+            plain.step(Wa, grads[k])
+            sharded.step(Wb, grads[k])
+        torch.cuda.synchronize()
+        for x, y in zip(Wa, Wb):
+            assert torch.equal(x, y)
+    finally:
+        dist.destroy_process_group()
