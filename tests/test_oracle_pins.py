@@ -219,6 +219,43 @@ def test_full_rank_identity_reduces_to_elementwise_adam():
         np.testing.assert_allclose(W, Wref, rtol=1e-12)
 
 
+@pytest.mark.parametrize("projection,s", [("left", 0), ("left", 3), ("short_side", 0), ("short_side", 3)])
+def test_cyclic_shift_projector_gives_the_update_of_the_identity_projector(projection, s):
+    """A square projector that is a cyclic shift (a permutation, so not symmetric) only relabels the rows of
+    the low-rank gradient (the columns, on the right); Adam is elementwise and the Fisher solve sees the same
+    inner products, so projecting and projecting back must give exactly the update of P = I.  A transposed
+    P in either product shifts twice instead of shifting there and back."""
+    rng = np.random.default_rng(61)
+    n = 6
+    shift = np.roll(np.eye(n), 1, axis=0)          # row i of shift^T G is row i + 1 of G
+    assert not np.array_equal(shift, shift.T)
+    hp = orc.Hyper(r=n, s=s, T=0, lr=1e-2, projection=projection)
+    a, b = orc.MatrixState(n, n, hp), orc.MatrixState(n, n, hp)
+    a.set_subspace(shift)
+    b.set_subspace(np.eye(n))
+    for _ in range(5):
+        G = rng.standard_normal((n, n))
+        da = a.step(np.zeros((n, n)), G)
+        db = b.step(np.zeros((n, n)), G)
+        np.testing.assert_allclose(da, db, rtol=1e-9, atol=1e-15)
+    R = orc.project(shift, G)
+    for i in range(n):
+        np.testing.assert_array_equal(R[i], G[(i + 1) % n])
+
+
+def test_stored_projector_holds_bf16_values():
+    """The projector is kept in the storage format of the step's GEMM operand (bf16): every stored value has
+    an 8-bit significand and lies within half a bf16 spacing of what was set."""
+    rng = np.random.default_rng(62)
+    P, _ = np.linalg.qr(rng.standard_normal((12, 5)))
+    st = orc.MatrixState(12, 9, orc.Hyper(r=5, s=0, T=0))
+    st.set_subspace(P)
+    mant, _ = np.frexp(st.P)
+    assert np.array_equal(mant * 256.0, np.round(mant * 256.0))      # 8 significant bits
+    assert np.all(np.abs(st.P - P) <= np.abs(P) * 2.0 ** -8)      # half of the spacing 2^(e-7)
+    assert np.any(st.P != P)
+
+
 def test_large_lambda_limit_returns_scaled_gradient():
     rng = np.random.default_rng(8)
     hist = _rand_history(rng, 6, 4, 9)
