@@ -37,7 +37,7 @@ MUTANTS = [
     ("right basis taken from the left singular vectors",
      "return np.ascontiguousarray(Vt[:rp, :].T)", "return np.ascontiguousarray(np.linalg.svd(G.T, full_matrices=False)[2][:rp, :].T)"),
     ("projection without the transpose of P (square P)", "return P.T @ G", "return (P @ G) if P.shape[0] == P.shape[1] else P.T @ G"),
-    ("history always divided by s", "self.count = min(self.count + 1, hp.s)", "self.count = hp.s if self.slots[hp.s - 1] is not None or True else 0"),
+    ("count of gradients held grows past the ring", "self.count = min(self.count + 1, hp.s)", "self.count = self.count + 1"),
     ("ring never wraps onto the oldest slot", "self.head = (self.head + 1) % hp.s", "self.head = min(self.head + 1, hp.s - 1)"),
     ("refresh one step late", "if auto_refresh and hp.T > 0 and self.k % hp.T == 0:", "if auto_refresh and hp.T > 0 and self.k % hp.T == 1 % hp.T:"),
     ("update not scaled by the learning rate", "dW = -hp.lr * back - hp.lr * hp.wd * W", "dW = -back - hp.lr * hp.wd * W"),
