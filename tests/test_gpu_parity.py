@@ -174,6 +174,17 @@ def test_invalid_arguments_are_rejected():
     with pytest.raises(NGaLoreError) as e:
         opt.step(W, G)                            # T == 0 and no subspace yet
     assert e.value.code == 5
+    # pointers that are not 16-byte aligned are turned away on the host, before any kernel sees them
+    opt.set_subspace(0, torch.eye(64)[:, :8].contiguous())
+    flat = torch.zeros(64 * 64 + 4, device="cuda")
+    W_off = [flat[1:1 + 64 * 64].view(64, 64)]
+    assert W_off[0].data_ptr() % 16 == 4 and W_off[0].is_contiguous()
+    with pytest.raises(NGaLoreError) as e:
+        opt.step(W_off, G, check=False)
+    assert e.value.code == 1
+    assert opt.step_count == 0                    # a rejected call leaves the state where it was
+    opt.step(W, G)
+    assert opt.step_count == 1 and opt.poll_status()[0] == 0
 
 
 def test_many_small_matrices():
