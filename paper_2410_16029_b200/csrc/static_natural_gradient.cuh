@@ -6,6 +6,8 @@
 // the same translation unit.
 #pragma once
 
+#include <atomic>
+
 #include "../../include/ngalore.h"
 #include "common.cuh"
 #include "kernels_stream.cuh"
@@ -89,18 +91,20 @@ __global__ void __launch_bounds__(kStreamThreads) static_combine_kernel(StaticAr
 // host-side handle in host code; kernels must be given the address the runtime reports).
 inline cudaError_t static_scratch_address(unsigned char** out) {
   constexpr int kMaxDevices = 64;
-  static unsigned char* cached[kMaxDevices] = {nullptr};
-  int dev = 0;
+  static std::atomic<unsigned char*> cached[kMaxDevices];  // zero-initialised; threads may race to fill an entry
+  int dev = 0;                                             // with the same value
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  if (cached[dev] == nullptr) {
+  unsigned char* addr = cached[dev].load(std::memory_order_acquire);
+  if (addr == nullptr) {
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_static_scratch);
     if (e != cudaSuccess) return e;
-    cached[dev] = static_cast<unsigned char*>(p);
+    addr = static_cast<unsigned char*>(p);
+    cached[dev].store(addr, std::memory_order_release);
   }
-  *out = cached[dev];
+  *out = addr;
   return cudaSuccess;
 }
 
