@@ -294,7 +294,8 @@ def run_ours(args, wl):
     shapes = [(M, N) for _, M, N in wl.shapes]
     n = len(shapes)
     opt = NGaLore(shapes, wl.r, wl.s, wl.T, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
-                  wd=wl.wd, seed=1 + rank, projection=args.projection, history_bf16=args.history == "bf16")
+                  wd=wl.wd, seed=1 + rank, projection=args.projection, history_bf16=args.history == "bf16",
+                  gram_fusion=args.gram_fusion == "on")
     # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
     wl_rank = rank_workload(wl, rank)
     if parts is not None:
@@ -440,7 +441,7 @@ def run_ours(args, wl):
                            "f64 Gram reduction and solve",
            "data": "synthetic",
            "config": {"workload": wl.name, "matrices": n, "r": wl.r, "s": wl.s, "T": wl.T,
-                      "projection": args.projection, "history": args.history,
+                      "projection": args.projection, "history": args.history, "gram_fusion": args.gram_fusion,
                       "sharded": parts is not None,
                       "l2": f"inputs larger than L2: {pool_sets} gradient sets of {grad_bytes / 1e9:.2f} GB cycled",
                       "state_bytes": opt.device_bytes},
@@ -472,6 +473,9 @@ def main():
     ap.add_argument("--history", default="fp32", choices=["fp32", "bf16"],
                     help="fp32: the ring of low-rank gradients in fp32 (the headline configuration); bf16: every "
                          "stored gradient but the current one in bf16 (reduced-precision state option)")
+    ap.add_argument("--gram-fusion", default="off", choices=["on", "off"],
+                    help="off (the library's default): the Gram tiles run in the stream kernel; on: where the workload "
+                         "allows it the new Gram row is formed in the projection's epilogue")
     ap.add_argument("--shard", action="store_true",
                     help="with --gpus N > 1: one model's matrices split over the ranks (state memory / N, weights "
                          "exchanged after every step) instead of N independent replicas; rank 0's phases and "

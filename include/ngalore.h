@@ -84,7 +84,14 @@ typedef struct {
                                        step takes part in fp32, which the Woodbury form needs, and is stored as bf16
                                        afterwards; the Gram matrix is kept that of the stored values.  Halves the
                                        history traffic and memory.  Needs s >= 1 and the fused stream kernel. */
-  int32_t reserved;
+  int32_t gram_fusion;              /* 0 (default): the new Gram row comes from the Gram tiles of the stream kernel.
+                                       1: where the workload allows it (rank-512 class shapes, left projection, K of
+                                       at most 8192, fp32 history of at most 16 slots, rows and columns multiples of
+                                       32) it is formed in the epilogue of the projection GEMM instead, so that the
+                                       first read of the history runs under the tensor-core work; same results to
+                                       rounding.  Measured slower than the default on the 1.1B shapes as built (the
+                                       history arrives in boxes of 128 scattered row pieces, which keeps too few bytes
+                                       in flight), hence off unless asked for. */
 } ngalore_options;
 
 /*

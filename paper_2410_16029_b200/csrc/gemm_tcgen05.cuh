@@ -57,7 +57,8 @@ enum {
   TC_MAP_B_BACK = 3,   // u16: r' (K) rows x N, box 64 x 64        Pt16 = Q^T (fp16): r' (K) rows x N
   TC_MAP_W_LOAD = 4,   // W (fp32): M rows x N, box 32 columns x 128 rows
   TC_MAP_W_STORE = 5,  // W (fp32): box 32 x 32
-  kTcMapsPerMat = 6
+  TC_MAP_H_LOAD = 6,   // history ring (fp32) as one matrix of s * lr_rows rows x lr_cols, box 32 columns x 128 rows
+  kTcMapsPerMat = 7
 };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
@@ -410,6 +411,20 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 constexpr int kProjBN = 256, kProjStages = 4, kProjEpiWarps = 4;
 constexpr int kTcBackBN = 256;  // tile width of the back-projection kernel
 
+// Projection with the Gram row in its epilogue (project_gram_tcgen05.cuh): tile width, the longest history that
+// takes part, partial rows per tile (one per epilogue warp).
+constexpr int kPgBN = 256;
+constexpr int kPgSMax = 16;
+constexpr int kPgWarpRows = 8;
+
+// Per matrix: where its partial rows start in the partial buffer (in doubles; -1: the matrix does not take part)
+// and its tile grid.  Partial row of (tile, epilogue warp e): part_off + (tile * 8 + e) * kPgSMax.
+struct PgMat {
+  long long part_off;
+  int ntiles;
+  int tiles_n;   // tiles per 128-row band (columns / 256, rounded up)
+};
+
 struct TcPlan {
   size_t device_bytes = 0;
   EncodeTiledFn encode = nullptr;
@@ -431,6 +446,14 @@ struct TcPlan {
   int* d_split_mats = nullptr;
   int n_split = 0;
   bool maps_dirty = true;
+  // projection with the Gram row in its epilogue: the matrices that take part, their tiles and partial rows
+  std::vector<int> gram_fused;     // per matrix: 1 when its Gram row comes from the projection's epilogue
+  TcTile* d_tiles_pg = nullptr;
+  int n_tiles_pg = 0, grid_pg = 0;
+  PgMat* d_pgm = nullptr;
+  double* d_pg_part = nullptr;
+  int* d_pg_list = nullptr;
+  int n_pg = 0;
 };
 
 // 16-bit elements unless fp32 is asked for (TMA moves fp16 and bf16 alike).
@@ -450,11 +473,16 @@ inline void tc_plan_destroy(TcPlan& plan) {
   if (plan.d_tiles_proj) cudaFree(plan.d_tiles_proj);
   if (plan.d_tiles_back) cudaFree(plan.d_tiles_back);
   if (plan.d_split_mats) cudaFree(plan.d_split_mats);
+  if (plan.d_tiles_pg) cudaFree(plan.d_tiles_pg);
+  if (plan.d_pgm) cudaFree(plan.d_pgm);
+  if (plan.d_pg_part) cudaFree(plan.d_pg_part);
+  if (plan.d_pg_list) cudaFree(plan.d_pg_list);
   plan.d_maps = nullptr; plan.d_tiles_proj = nullptr; plan.d_tiles_back = nullptr; plan.d_split_mats = nullptr;
+  plan.d_tiles_pg = nullptr; plan.d_pgm = nullptr; plan.d_pg_part = nullptr; plan.d_pg_list = nullptr;
 }
 
-inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& mats, const MatDesc* /*d_mats*/, int /*s*/,
-                                     int sm_count) {
+inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& mats, const MatDesc* /*d_mats*/, int s,
+                                     int sm_count, bool allow_gram_fusion) {
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr)
@@ -518,6 +546,16 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   long long target_kb = per_cta / 4;
   if (target_kb < 16) target_kb = 16;
   std::vector<int> split_mats;
+  // Matrices whose Gram row is formed in the projection's epilogue (project_gram_tcgen05.cuh): the workload class
+  // of the tall projection tiles (long K, rank 512: there the history read is long enough to hide the MMAs),
+  // left projection, K short enough to stay unsplit, fp32 history of at most kPgSMax slots, rows and columns
+  // multiples of 32.
+  plan.gram_fused.assign(n, 0);
+  std::vector<TcTile> pg;
+  std::vector<PgMat> pgm(n, PgMat{-1, 0, 0});
+  std::vector<int> pg_list;
+  long long pg_rows = 0;
+  const bool fuse_class = allow_gram_fusion && plan.tall_proj && s >= 1 && s <= kPgSMax;
   for (int i = 0; i < n; ++i) {
     const MatDesc& d = mats[i];
     const int kb_total = ((d.right ? d.N : d.M) + kTcBK - 1) / kTcBK;
@@ -525,6 +563,18 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
     if (splits < 1) splits = 1;
     const int kb_per = (kb_total + splits - 1) / splits;
     splits = (kb_total + kb_per - 1) / kb_per;
+    // (a K of up to 128 blocks stays in one piece for it even where the schedule would rather split it)
+    if (fuse_class && kb_total <= 128 && !d.right && d.H16 == nullptr && d.s == s && d.lr_rows % 32 == 0 && d.lr_cols % 32 == 0) {
+      plan.gram_fused[i] = 1;
+      pg_list.push_back(i);
+      const int tiles_m = (d.lr_rows + kTcBM - 1) / kTcBM, tiles_n = (d.lr_cols + kPgBN - 1) / kPgBN;
+      pgm[i] = PgMat{pg_rows * kPgSMax, tiles_m * tiles_n, tiles_n};
+      pg_rows += static_cast<long long>(tiles_m) * tiles_n * kPgWarpRows;
+      for (int n0 = 0; n0 < d.lr_cols; n0 += kPgBN)
+        for (int m0 = 0; m0 < d.lr_rows; m0 += kTcBM)
+          pg.push_back(TcTile{i, m0, n0, 0, kb_total, 0, d.lr_rows, d.lr_cols});
+      continue;
+    }
     if (splits > 1) split_mats.push_back(i);
     for (int n0 = 0; n0 < d.lr_cols; n0 += kProjBN)
       for (int sp = 0; sp < splits; ++sp)
@@ -535,6 +585,7 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
         }
   }
   std::stable_sort(proj.begin(), proj.end(), [](const TcTile& a, const TcTile& b) { return a.kblocks > b.kblocks; });
+  std::stable_sort(pg.begin(), pg.end(), [](const TcTile& a, const TcTile& b) { return a.kblocks > b.kblocks; });
   plan.back_tile0.assign(n + 1, 0);
   for (int i = 0; i < n; ++i) {
     const MatDesc& d = mats[i];
@@ -549,13 +600,35 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   plan.grid_proj = std::min(plan.n_tiles_proj, sm_count);
   plan.grid_back = std::min(plan.n_tiles_back, sm_count);
   plan.n_split = static_cast<int>(split_mats.size());
+  plan.n_tiles_pg = static_cast<int>(pg.size());
+  plan.grid_pg = std::min(plan.n_tiles_pg, sm_count);
+  plan.n_pg = static_cast<int>(pg_list.size());
+  for (int i : pg_list) {
+    // the whole ring of the matrix as one tall fp32 matrix: slot j starts at row j * lr_rows
+    const MatDesc& d = mats[i];
+    if (!tc_encode_2d(plan.encode, &plan.h_maps[static_cast<size_t>(i) * kTcMapsPerMat + TC_MAP_H_LOAD], d.H, d.lr_cols,
+                      static_cast<uint64_t>(s) * d.lr_rows, static_cast<uint64_t>(d.lr_cols) * 4, 32, kTcBM, true))
+      return NGALORE_ERR_CUDA;
+  }
+  if (plan.n_pg > 0) {
+    if (cudaMalloc(&plan.d_tiles_pg, sizeof(TcTile) * pg.size()) != cudaSuccess) { plan.d_tiles_pg = nullptr; return NGALORE_ERR_ALLOC; }
+    if (cudaMalloc(&plan.d_pgm, sizeof(PgMat) * n) != cudaSuccess) { plan.d_pgm = nullptr; return NGALORE_ERR_ALLOC; }
+    if (cudaMalloc(&plan.d_pg_part, sizeof(double) * pg_rows * kPgSMax) != cudaSuccess) { plan.d_pg_part = nullptr; return NGALORE_ERR_ALLOC; }
+    if (cudaMalloc(&plan.d_pg_list, sizeof(int) * pg_list.size()) != cudaSuccess) { plan.d_pg_list = nullptr; return NGALORE_ERR_ALLOC; }
+    if (cudaMemcpy(plan.d_tiles_pg, pg.data(), sizeof(TcTile) * pg.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(plan.d_pgm, pgm.data(), sizeof(PgMat) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(plan.d_pg_list, pg_list.data(), sizeof(int) * pg_list.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(plan.d_pg_part, 0, sizeof(double) * pg_rows * kPgSMax) != cudaSuccess)
+      return NGALORE_ERR_CUDA;
+    plan.device_bytes += sizeof(TcTile) * pg.size() + sizeof(PgMat) * n + sizeof(double) * pg_rows * kPgSMax + sizeof(int) * pg_list.size();
+  }
 
   const size_t maps_bytes = sizeof(CUtensorMap) * plan.h_maps.size();
   if (cudaMalloc(&plan.d_maps, maps_bytes) != cudaSuccess) { plan.d_maps = nullptr; return NGALORE_ERR_ALLOC; }
   if (cudaMalloc(&plan.d_tiles_proj, sizeof(TcTile) * proj.size()) != cudaSuccess) { plan.d_tiles_proj = nullptr; return NGALORE_ERR_ALLOC; }
   if (cudaMalloc(&plan.d_tiles_back, sizeof(TcTile) * back.size()) != cudaSuccess) { plan.d_tiles_back = nullptr; return NGALORE_ERR_ALLOC; }
   if (cudaMalloc(&plan.d_split_mats, sizeof(int) * (split_mats.size() + 1)) != cudaSuccess) { plan.d_split_mats = nullptr; return NGALORE_ERR_ALLOC; }
-  plan.device_bytes = maps_bytes + sizeof(TcTile) * (proj.size() + back.size()) + sizeof(int) * (split_mats.size() + 1);
+  plan.device_bytes += maps_bytes + sizeof(TcTile) * (proj.size() + back.size()) + sizeof(int) * (split_mats.size() + 1);
   if (cudaMemcpy(plan.d_tiles_proj, proj.data(), sizeof(TcTile) * proj.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_tiles_back, back.data(), sizeof(TcTile) * back.size(), cudaMemcpyHostToDevice) != cudaSuccess)
     return NGALORE_ERR_CUDA;

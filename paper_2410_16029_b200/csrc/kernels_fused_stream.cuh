@@ -441,7 +441,10 @@ inline cudaError_t fused_set_smem() {
                               FusedCfg<SMAX, HIST16>::kTotal);
 }
 
-inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDesc>& mats, int s, int sm_count) {
+// skip_gram (optional, one entry per matrix): 1 where the Gram row and the solve of a matrix are done before this
+// kernel runs (projection with the Gram row in its epilogue); such a matrix gets combination tiles only.
+inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDesc>& mats, int s, int sm_count,
+                                        const std::vector<int>* skip_gram = nullptr) {
   plan.grid = sm_count;
   // Item order: every Gram tile (matrix order), then every combination tile (same order).  A CTA that picks
   // up a combination tile then never waits for a Gram tile that is still running, except for the last few
@@ -452,6 +455,7 @@ inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDe
   const int n = static_cast<int>(mats.size());
   for (int i = 0; i < n; ++i) {
     if (mats[i].s == 0) continue;
+    if (skip_gram != nullptr && (*skip_gram)[i]) continue;
     for (int t = 0; t < mats[i].ntiles; ++t) items.push_back(FusedItem{i, t, 0, 0});
   }
   for (int i = 0; i < n; ++i)

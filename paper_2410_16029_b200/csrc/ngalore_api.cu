@@ -352,7 +352,7 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       st->launches += 1;
     }
   } else {
-    if ((rc = tc_project(st->tc, st->d_desc, st->d_ctrl, stream, &st->launches))) return rc;
+    if ((rc = tc_project(st->tc, st->d_desc, st->d_ctrl, st->d_hyper, stream, &st->launches))) return rc;
   }
   if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[1], stream));
   // ---- phase 1: Gram row, solve, natural gradient + moments
@@ -446,6 +446,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (opt != nullptr && opt->struct_size != static_cast<int32_t>(sizeof(ngalore_options))) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && (opt->projection_rule < 0 || opt->projection_rule > 1)) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && (opt->history_bf16 < 0 || opt->history_bf16 > 1)) return NGALORE_ERR_INVALID_ARG;
+  if (opt != nullptr && (opt->gram_fusion < 0 || opt->gram_fusion > 1)) return NGALORE_ERR_INVALID_ARG;
   // the bf16 history lives in the fused stream kernel only
   if (opt != nullptr && opt->history_bf16 == 1 && (s < 1 || opt->stream_impl == 1)) return NGALORE_ERR_INVALID_ARG;
 
@@ -642,11 +643,12 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
                            static_cast<int>(orth_apply_smem_bytes(max_rp))) != cudaSuccess)
     return fail(NGALORE_ERR_CUDA);
 
-  ngalore_status rc = tc_plan_create(st->tc, st->h_desc, st->d_desc, s, prop.multiProcessorCount);
+  const bool allow_gram_fusion = st->opt.gemm_impl != 1 && st->opt.stream_impl != 1 && !hist16 && st->opt.gram_fusion == 1;
+  ngalore_status rc = tc_plan_create(st->tc, st->h_desc, st->d_desc, s, prop.multiProcessorCount, allow_gram_fusion);
   if (rc != NGALORE_OK) return fail(rc);
   if ((rc = tc_project_init()) != NGALORE_OK) return fail(rc);
   if ((rc = tc_backproject_init()) != NGALORE_OK) return fail(rc);
-  rc = fused_plan_create(st->fused, st->h_desc, s, prop.multiProcessorCount);
+  rc = fused_plan_create(st->fused, st->h_desc, s, prop.multiProcessorCount, &st->tc.gram_fused);
   if (rc != NGALORE_OK) return fail(rc);
   if (st->opt.gemm_impl != 1) {
     // the refresh plan sees every matrix it takes in the orientation whose left subspace is wanted

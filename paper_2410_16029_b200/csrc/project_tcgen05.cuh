@@ -16,6 +16,7 @@
 #pragma once
 
 #include "gemm_tcgen05.cuh"
+#include "project_gram_tcgen05.cuh"
 
 namespace ngalore {
 
@@ -213,16 +214,24 @@ inline ngalore_status tc_project_init() {
                            cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess ||
       cudaFuncSetAttribute(tc_project2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, P2Smem::kTotal) != cudaSuccess)
     return NGALORE_ERR_CUDA;
-  return NGALORE_OK;
+  return tc_project_gram_init();
 }
 
 // R = P^T G (or G Q) for every matrix, into the buffer of the current step (ring slot `cur`, read on the device
 // from Ctrl), through the tensor maps tc_bind_buffers set up.
-inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, cudaStream_t stream,
-                                 int64_t* launches) {
+inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const Hyper* d_hyper,
+                                 cudaStream_t stream, int64_t* launches) {
   if (plan.n_split > 0) {
     zero_split_slots_kernel<<<dim3(64, plan.n_split), 256, 0, stream>>>(d_mats, plan.d_split_mats, d_ctrl);
     *launches += 1;
+  }
+  if (plan.n_tiles_pg > 0) {
+    // the matrices whose Gram row comes out of the projection's epilogue, then their s x s solves
+    tc_project_gram_kernel<kPgStages, kPgSlots><<<plan.grid_pg, kPgThreads, BpSmem<kPgStages, kPgSlots>::kTotal, stream>>>(
+        plan.d_maps, plan.d_tiles_pg, plan.n_tiles_pg, d_mats, plan.d_pgm, plan.d_pg_part, d_ctrl);
+    pg_solve_kernel<<<plan.n_pg, 256, 0, stream>>>(d_mats, plan.d_pgm, plan.d_pg_part, plan.d_pg_list, d_ctrl, d_hyper);
+    *launches += 2;
+    if (plan.n_tiles_proj == 0) return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
   }
   if (plan.tall_proj) {
     tc_project2_kernel<<<plan.grid_proj, kP2Threads, P2Smem::kTotal, stream>>>(plan.d_maps, plan.d_tiles_proj,
