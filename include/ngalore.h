@@ -89,9 +89,9 @@ typedef struct {
                                        at most 8192, fp32 history of at most 16 slots, rows and columns multiples of
                                        32) it is formed in the epilogue of the projection GEMM instead, so that the
                                        first read of the history runs under the tensor-core work; same results to
-                                       rounding.  Measured slower than the default on the 1.1B shapes as built (the
-                                       history arrives in boxes of 128 scattered row pieces, which keeps too few bytes
-                                       in flight), hence off unless asked for. */
+                                       rounding.  Measured slower than the default on the 1.1B shapes as built (about
+                                       7.0 against 6.7 ms per step: with the memory system saturated by the history the
+                                       MMAs wait for their operands), hence off unless asked for. */
 } ngalore_options;
 
 /*

@@ -57,7 +57,7 @@ enum {
   TC_MAP_B_BACK = 3,   // u16: r' (K) rows x N, box 64 x 64        Pt16 = Q^T (fp16): r' (K) rows x N
   TC_MAP_W_LOAD = 4,   // W (fp32): M rows x N, box 32 columns x 128 rows
   TC_MAP_W_STORE = 5,  // W (fp32): box 32 x 32
-  TC_MAP_H_LOAD = 6,   // history ring (fp32) as one matrix of s * lr_rows rows x lr_cols, box 32 columns x 128 rows
+  TC_MAP_H_LOAD = 6,   // history ring (fp32) as one matrix of s * lr_rows rows x lr_cols, box 32 columns x 32 rows
   kTcMapsPerMat = 7
 };
 
@@ -607,7 +607,7 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
     // the whole ring of the matrix as one tall fp32 matrix: slot j starts at row j * lr_rows
     const MatDesc& d = mats[i];
     if (!tc_encode_2d(plan.encode, &plan.h_maps[static_cast<size_t>(i) * kTcMapsPerMat + TC_MAP_H_LOAD], d.H, d.lr_cols,
-                      static_cast<uint64_t>(s) * d.lr_rows, static_cast<uint64_t>(d.lr_cols) * 4, 32, kTcBM, true))
+                      static_cast<uint64_t>(s) * d.lr_rows, static_cast<uint64_t>(d.lr_cols) * 4, 32, 32, true))
       return NGALORE_ERR_CUDA;
   }
   if (plan.n_pg > 0) {

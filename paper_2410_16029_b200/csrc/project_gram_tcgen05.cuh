@@ -1,24 +1,26 @@
 // Projection R = P^T G with the new row of the history's Gram matrix formed in its epilogue (Sec. 1; Sec. 2.4:
-// y = G^T g, the inner products of the current low-rank gradient with the stacked past ones).
+// y = G^T g, the inner products of the current low-rank gradient with the stacked past ones).  Option
+// gram_fusion; off by default because it measured slower than the separate kernels as built.
 //
 // The Gram row needs one read of the whole history ring, which is HBM traffic with no arithmetic to speak of,
 // and the projection is tensor-core time with little traffic.  Run one after the other neither hides the other;
-// here the old ring slots of the tile an epilogue warp is draining stream through a short shared-memory ring
-// (TMA, 128 rows x 32 columns per slot, 128-byte swizzle: the row-per-lane float4 reads are conflict-free) while
-// the MMAs of the next tile run into the second accumulator buffer.  Each epilogue thread holds its row of the
-// 32-column chunk of R from tcgen05.ld, writes it to the ring slot of the current step and multiplies it into the
-// same rows of every older slot.  Products and the per-thread sums over a tile are fp32, everything across
-// threads is fp64, as in the stream kernel's Gram pass.  Every epilogue warp writes its partial row per tile
-// (no synchronisation between warps); pg_solve_kernel, launched behind this kernel, adds the partial rows of
-// a matrix in a fixed order, solves the s x s system and publishes the weights for the combination pass.
+// here every epilogue warp streams the older ring slots of the rows it is draining through a small ring of its
+// own in shared memory (TMA boxes of 32 rows x 32 columns, 128-byte swizzle: the row-per-lane float4 reads are
+// conflict-free), a few boxes ahead and across tile boundaries, while the MMAs of the next tile run into the
+// second accumulator buffer.  Each epilogue thread holds its row of a 32-column chunk of R from tcgen05.ld,
+// writes it to the ring slot of the current step and multiplies it into the same piece of every older slot.
+// Products and the per-thread sums over a tile are fp32, everything across threads is fp64, as in the stream
+// kernel's Gram pass.  Every epilogue warp writes its partial row per tile (no synchronisation between warps);
+// pg_solve_kernel, launched behind this kernel, adds the partial rows of a matrix in a fixed order, solves the
+// s x s system and publishes the weights for the combination pass.
 //
-// Only matrices whose R comes out of a single CTA per tile take part (left projection, K not split, row and
-// column counts multiples of 32, 1 <= s <= 16, fp32 history); the others keep the plain projection and the Gram
-// tiles of the stream kernel.
+// Only matrices whose R comes out of a single CTA per tile take part (left projection, K of at most 128 blocks so
+// that it stays unsplit, row and column counts multiples of 32, 1 <= s <= 16, fp32 history); the others keep the
+// plain projection and the Gram tiles of the stream kernel.
 //
-// Warp roles as in the back-projection: warp 0 TMA producer of the operands, warp 1 TMEM owner and MMA issuer,
-// warps 2..9 epilogue (quarter = warp % 4 owns 32 rows; the two warps of a quarter share the history boxes of
-// every chunk), warp 10 TMA producer of the history boxes.  Every mbarrier wait is bounded (see mbar_wait).
+// Warp roles: warp 0 TMA producer of the operands, warp 1 TMEM owner and MMA issuer, warps 2..9 epilogue
+// (quarter = warp % 4 owns 32 rows; the two warps of a quarter take the even and the odd 32-column chunks).
+// Every mbarrier wait is bounded (see mbar_wait).
 #pragma once
 
 #include "backproject_tcgen05.cuh"
@@ -26,11 +28,7 @@
 
 namespace ngalore {
 
-constexpr int kPgHProducerWarp = 10;
-constexpr int kPgThreads = 32 * 11;
-// Two operand stages of 48 KB and eight history slots of 16 KB: the kernel is bound by the history stream, which
-// wants bytes in flight; the MMAs of a tile take a third of the time its history takes to arrive.
-constexpr int kPgStages = 2, kPgSlots = 8;
+constexpr int kPgThreads = 32 * 10;
 
 // Inner product of a thread's 32 accumulator columns with 32 values of the same row of another matrix, in one
 // fixed order of operations (see the epilogue).
@@ -43,14 +41,76 @@ __device__ __forceinline__ float pg_dot32(const uint32_t (&r)[32], const float4 
   return t;
 }
 
-template <int STAGES, int SLOTS>
+// Three operand stages of 48 KB and two history boxes of 4 KB in flight per epilogue warp.  Measured on the 1.1B
+// shapes (kernel + solves + the embeddings' plain projection): 2 stages with 4 boxes per warp 2.93 ms, 3 stages
+// with 2 boxes 2.78 ms: under a saturated memory system the operand loads of the MMAs are what the kernel waits
+// for.  An earlier arrangement with a producer warp and 16 KB boxes shared by four warps (128 rows) ran 2.96 ms.
+constexpr int kPgStages = 3;      // operand stages of 48 KB
+constexpr int kPgBoxes = 2;       // boxes in flight per epilogue warp
+struct PgSmem {
+  static constexpr int kABytes = kTcBM * kTcBK * 2;
+  static constexpr int kBChunkBytes = 64 * kTcBK * 2;
+  static constexpr int kStageBytes = kABytes + (kPgBN / 64) * kBChunkBytes;   // 48 KB
+  static constexpr int kBoxBytes = 32 * 32 * 4;                               // 4 KB
+  static constexpr int kRingOffset = kPgStages * kStageBytes;
+  static constexpr int kBarOffset = kRingOffset + 8 * kPgBoxes * kBoxBytes;
+  static constexpr int kBarBytes = 512;
+  static constexpr int kTotal = kBarOffset + kBarBytes + 1024;
+};
+static_assert((2 * kPgStages + 4 + 8 * kPgBoxes) * 8 + 8 <= PgSmem::kBarBytes, "barrier block");
+static_assert(PgSmem::kTotal <= 232448, "shared memory budget of one CTA");
+
+// Walks the boxes of one epilogue warp in the order it uses them: tile (this CTA's), older slot, own chunk
+// (slot-major, so that DRAM sees 1 KB of a row within a few boxes: measured 2.78 ms against 3.03 ms chunk-major).
+struct PgBoxIter {
+  int t, j, c, wchunks;
+  int n0, m0, rows, mat;
+  bool valid;
+};
+__device__ __forceinline__ int pg_next_slot(int j, int cur, int count) {
+  ++j;
+  if (j == cur) ++j;
+  return j < count ? j : -1;
+}
+__device__ __forceinline__ void pg_iter_load_tile(PgBoxIter& it, const TcTile* tiles) {
+  const TcTile tile = tiles[it.t];
+  const int n_rem = tile.cols - tile.n0;
+  it.wchunks = (n_rem >= kPgBN ? kPgBN : n_rem) >> 5;
+  it.n0 = tile.n0; it.m0 = tile.m0; it.rows = tile.rows; it.mat = tile.mat;
+}
+// First box at or after tile it.t (tiles that have no chunk of this warp's parity are skipped).
+__device__ __forceinline__ void pg_iter_seek(PgBoxIter& it, const TcTile* tiles, int n_tiles, int stride, int parity,
+                                             int cur, int count) {
+  it.valid = false;
+  if (count < 2) return;
+  while (it.t < n_tiles) {
+    pg_iter_load_tile(it, tiles);
+    if (parity < it.wchunks) {
+      it.j = pg_next_slot(-1, cur, count);
+      it.c = parity;
+      it.valid = true;
+      return;
+    }
+    it.t += stride;
+  }
+}
+__device__ __forceinline__ void pg_iter_advance(PgBoxIter& it, const TcTile* tiles, int n_tiles, int stride, int parity,
+                                                int cur, int count) {
+  it.c += 2;
+  if (it.c < it.wchunks) return;
+  it.c = parity;
+  it.j = pg_next_slot(it.j, cur, count);
+  if (it.j >= 0) return;
+  it.t += stride;
+  pg_iter_seek(it, tiles, n_tiles, stride, parity, cur, count);
+}
+
 __global__ void __launch_bounds__(kPgThreads, 1)
 tc_project_gram_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__ tiles, int n_tiles,
-                       const MatDesc* __restrict__ mats, const PgMat* __restrict__ pgm, double* __restrict__ part,
-                       Ctrl* ctrl) {
-  using L = BpSmem<STAGES, SLOTS>;
-  static_assert(SLOTS % 2 == 0, "the ring is split into two halves");
-  constexpr int kHalf = SLOTS / 2;
+                        const MatDesc* __restrict__ mats, const PgMat* __restrict__ pgm, double* __restrict__ part,
+                        Ctrl* ctrl) {
+  using L = PgSmem;
+  constexpr int STAGES = kPgStages;
   extern __shared__ unsigned char tc_smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(tc_smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
@@ -58,16 +118,15 @@ tc_project_gram_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __re
   uint64_t* empty_bar = bars + STAGES;           // [STAGES] operands consumed
   uint64_t* tfull_bar = bars + 2 * STAGES;       // [2] accumulator complete
   uint64_t* tempty_bar = bars + 2 * STAGES + 2;  // [2] accumulator drained
-  uint64_t* hfull_bar = bars + 2 * STAGES + 4;   // [SLOTS] history box landed
-  uint64_t* hempty_bar = hfull_bar + SLOTS;      // [SLOTS] history box read by its four warps
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(hempty_bar + SLOTS);
+  uint64_t* hfull_bar = bars + 2 * STAGES + 4;   // [8 warps][kPgBoxes] history box landed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(hfull_bar + 8 * kPgBoxes);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + s, 1); mbar_init(empty_bar + s, 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + b, 1); mbar_init(tempty_bar + b, 8); }
-    for (int s = 0; s < SLOTS; ++s) { mbar_init(hfull_bar + s, 1); mbar_init(hempty_bar + s, 4); }
+    for (int s = 0; s < 8 * kPgBoxes; ++s) mbar_init(hfull_bar + s, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -82,10 +141,8 @@ tc_project_gram_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __re
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int stride = gridDim.x;
-  // ring position and number of gradients held, the same for every matrix of the state
   const int s_len = mats[0].s;
   const int cur = ring_cur(ctrl, s_len), count = ring_count(ctrl, s_len);
-  const int n_old = count - 1;  // history boxes per 32-column chunk
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer of the operands
@@ -109,34 +166,6 @@ tc_project_gram_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __re
           for (int c = 0; c < nchunks; ++c)
             tma_load_2d(sA + L::kABytes + c * L::kBChunkBytes, maps + TC_MAP_B_PROJ, tile.n0 + c * 64, k, full_bar + stage);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-        }
-      }
-    }
-  } else if (warp == kPgHProducerWarp) {
-    // ------------------------------------------------------------------ TMA producer of the history boxes
-    // Order: tile, history slot (ascending, the current one left out), 32-column chunk: the boxes of one slot
-    // follow each other along the rows, so that DRAM sees 1 KB of a row within a few boxes rather than 128 bytes.
-    // The history is one tall matrix of s * lr_rows rows to the tensor map: slot j starts at row j * lr_rows.
-    if (lane == 0 && n_old > 0) {
-      int pos[2] = {0, 0};           // position inside each half of the ring
-      uint32_t phase[2] = {0u, 0u};
-      bool ok = true;
-      for (int t = blockIdx.x; t < n_tiles && ok; t += stride) {
-        const TcTile tile = tiles[t];
-        const CUtensorMap* mapH = tmaps + tile.mat * kTcMapsPerMat + TC_MAP_H_LOAD;
-        const int n_rem = tile.cols - tile.n0;
-        const int wchunks = (n_rem >= kPgBN ? kPgBN : n_rem) >> 5;
-        for (int j = 0; j < count && ok; ++j) {
-          if (j == cur) continue;
-          for (int c = 0; c < wchunks; ++c) {
-            const int h = c & 1;     // even chunks go through the first half of the ring, odd ones through the second
-            const int slot = h * kHalf + pos[h];
-            if (!mbar_wait(hempty_bar + slot, phase[h] ^ 1u, abort_flag)) { ok = false; break; }
-            mbar_expect_tx(hfull_bar + slot, L::kWSlotBytes);
-            tma_load_2d(smem + L::kWOffset + slot * L::kWSlotBytes, mapH, tile.n0 + c * 32, j * tile.rows + tile.m0,
-                        hfull_bar + slot);
-            if (++pos[h] == kHalf) { pos[h] = 0; phase[h] ^= 1u; }
-          }
         }
       }
     }
@@ -178,15 +207,31 @@ tc_project_gram_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __re
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2 .. 9)
     // The two warps of a quarter take the even and the odd 32-column chunks, for R itself and for every older
-    // slot alike, and each has its own half of the ring (the producer sends a chunk's box to the half of the
-    // chunk's parity), so every warp waits for every use of its slots in order, which is what the one phase bit
-    // of an mbarrier can tell apart.  The inner products of R with itself and with an older slot go through the
-    // same function, chunk by chunk in the same order on the same thread: where a gradient repeats bit for bit,
-    // <R, H_j> equals the <H_j, H_j> computed when H_j was new, and the Gram matrix stays exactly singular
-    // rather than indefinite by a rounding (lambda then keeps it positive definite).
+    // slot alike.  <R, R> and <R, H_j> go through the same function, chunk by chunk in the same order on the same
+    // thread (see pg_dot32), so a gradient that repeats bit for bit gives an exactly singular Gram matrix.
     const int quarter = warp & 3;        // TMEM lanes 32 * quarter .. + 31 belong to this warp
     const int parity = (warp - 2) >> 2;
-    int pos = 0;                         // position inside this warp's half of the ring
+    const int e = warp - 2;
+    unsigned char* my_ring = smem + L::kRingOffset + e * kPgBoxes * L::kBoxBytes;
+    uint64_t* my_full = hfull_bar + e * kPgBoxes;
+    // the box this warp uses next sits in ring position `pos`; `ahead` walks kPgBoxes boxes in front of it
+    PgBoxIter ahead;
+    ahead.t = blockIdx.x;
+    pg_iter_seek(ahead, tiles, n_tiles, stride, parity, cur, count);
+    auto issue = [&](int k) {
+      // all lanes know the box; lane 0 sends the copy
+      if (lane == 0) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the place was just read with plain loads
+        mbar_expect_tx(my_full + k, L::kBoxBytes);
+        tma_load_2d(my_ring + k * L::kBoxBytes, tmaps + ahead.mat * kTcMapsPerMat + TC_MAP_H_LOAD, ahead.n0 + ahead.c * 32,
+                    ahead.j * ahead.rows + ahead.m0 + quarter * 32, my_full + k);
+      }
+    };
+    for (int k = 0; k < kPgBoxes && ahead.valid; ++k) {
+      issue(k);
+      pg_iter_advance(ahead, tiles, n_tiles, stride, parity, cur, count);
+    }
+    int pos = 0;
     uint32_t phase = 0;
     int local = 0;
     bool ok = true;
@@ -237,21 +282,23 @@ tc_project_gram_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __re
             uint32_t r[32];
             tc_ld32(tmem_row + static_cast<uint32_t>(c * 32), r);
             tc_wait_ld();
-            const int slot = parity * kHalf + pos;
-            if (!__all_sync(0xffffffffu, mbar_wait(hfull_bar + slot, phase, abort_flag))) {
+            if (!__all_sync(0xffffffffu, mbar_wait(my_full + pos, phase, abort_flag))) {
               ok = false;
             } else {
               // this lane's row of the box: 16-byte piece q sits at piece (q ^ (row & 7)) of the 128-byte row
-              const unsigned char* rowp =
-                  smem + L::kWOffset + slot * L::kWSlotBytes + quarter * L::kWBoxBytes + lane * 128;
+              const unsigned char* rowp = my_ring + pos * L::kBoxBytes + lane * 128;
               float4 h[8];
 #pragma unroll
               for (int q = 0; q < 8; ++q) h[q] = *reinterpret_cast<const float4*>(rowp + ((q ^ (lane & 7)) << 4));
               const float tsum = pg_dot32(r, h);
               if (row_ok) acc[j] += tsum;
+              // every lane has read the box: refill its place with the box kPgBoxes further on
               __syncwarp();
-              if (lane == 0) mbar_arrive(hempty_bar + slot);
-              if (++pos == kHalf) { pos = 0; phase ^= 1u; }
+              if (ahead.valid) {
+                issue(pos);
+                pg_iter_advance(ahead, tiles, n_tiles, stride, parity, cur, count);
+              }
+              if (++pos == kPgBoxes) { pos = 0; phase ^= 1u; }
             }
           }
         }
@@ -263,7 +310,7 @@ tc_project_gram_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __re
       if (!ok) break;
       // this warp's partial row of the tile (zeros for the slots it took no box of)
       const int tile_local = (tile.m0 / kTcBM) * pm.tiles_n + tile.n0 / kPgBN;
-      double* prow = part + pm.part_off + (static_cast<long long>(tile_local) * kPgWarpRows + (warp - 2)) * kPgSMax;
+      double* prow = part + pm.part_off + (static_cast<long long>(tile_local) * kPgWarpRows + e) * kPgSMax;
 #pragma unroll
       for (int j = 0; j < kPgSMax; ++j) {
         const double tj = warp_sum(static_cast<double>(acc[j]));
@@ -320,8 +367,7 @@ __global__ void __launch_bounds__(256) pg_solve_kernel(const MatDesc* __restrict
 }
 
 inline ngalore_status tc_project_gram_init() {
-  if (cudaFuncSetAttribute(tc_project_gram_kernel<kPgStages, kPgSlots>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           BpSmem<kPgStages, kPgSlots>::kTotal) != cudaSuccess)
+  if (cudaFuncSetAttribute(tc_project_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PgSmem::kTotal) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   return NGALORE_OK;
 }

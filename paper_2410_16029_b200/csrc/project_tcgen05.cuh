@@ -227,7 +227,7 @@ inline ngalore_status tc_project(TcPlan& plan, const MatDesc* d_mats, Ctrl* d_ct
   }
   if (plan.n_tiles_pg > 0) {
     // the matrices whose Gram row comes out of the projection's epilogue, then their s x s solves
-    tc_project_gram_kernel<kPgStages, kPgSlots><<<plan.grid_pg, kPgThreads, BpSmem<kPgStages, kPgSlots>::kTotal, stream>>>(
+    tc_project_gram_kernel<<<plan.grid_pg, kPgThreads, PgSmem::kTotal, stream>>>(
         plan.d_maps, plan.d_tiles_pg, plan.n_tiles_pg, d_mats, plan.d_pgm, plan.d_pg_part, d_ctrl);
     pg_solve_kernel<<<plan.n_pg, 256, 0, stream>>>(d_mats, plan.d_pgm, plan.d_pg_part, plan.d_pg_list, d_ctrl, d_hyper);
     *launches += 2;
