@@ -406,6 +406,11 @@ def run_ours(args, wl):
     # least 512 output rows and a long K, which of the workloads here are those of rank 512; elsewhere the
     # 128-row tc_gemm_kernel does the same work
     names = ["tc_project2_kernel" if wl.r >= 512 else "tc_gemm_kernel", "fused_stream_kernel", "tc_backproject_kernel"]
+    fused_gram = args.gram_fusion == "on" and wl.r >= 512 and args.projection == "left" and args.history == "fp32"
+    if fused_gram:
+        # phase 0 is then the projection with the Gram row in its epilogue (plus the solves and the plain projection
+        # of the matrices that do not take part); the byte split between the phases below is that of the default path
+        names[0] = "tc_project_gram_kernel"
     proj_bytes = sum(2 * M * N + 2 * dims[i][1] * dims[i][0] + 4 * dims[i][2] for i, (M, N) in enumerate(shapes))
     back_bytes = sum(8 * M * N + 2 * dims[i][1] * dims[i][0] for i, (M, N) in enumerate(shapes))
     alg = [proj_bytes, stream_bytes, back_bytes]
@@ -413,7 +418,8 @@ def run_ours(args, wl):
     achieved = alg[dom] / (phase[dom] * 1e-3) / 1e9
     traffic = None
     per_unit = NCU_TRAFFIC_PER_UNIT.get(names[dom])
-    if per_unit is not None and wl.r == 512 and wl.s == 16 and args.projection == "left" and args.history == "fp32":
+    if (per_unit is not None and wl.r == 512 and wl.s == 16 and args.projection == "left" and args.history == "fp32"
+            and not fused_gram):
         units = sum(d[2] for d in dims) if per_unit[0] == "rn" else sum(M * N for M, N in shapes)
         traffic = per_unit[1] * units
     roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s",
