@@ -37,6 +37,21 @@ METRIC = "optimizer steps/sec over all matrices (device-timed)"
 UNIT = "steps/s"
 
 
+def pool_size(args, wl):
+    """Gradient sets kept resident and cycled.  With fewer than s + 1 distinct sets a gradient would sit twice in
+    the history ring and the Gram matrix would be singular up to lambda; the optimizer never sees that in training."""
+    return args.pool if args.pool > 0 else wl.s + 1
+
+
+def config_dict(args, wl, n_matrices, sharded):
+    """The workload and protocol of a run; both arms (CUDA path and oracle) describe the same one."""
+    grad_bytes = sum(M * N * 2 for _, M, N in wl.shapes)
+    return {"workload": wl.name, "matrices": n_matrices, "r": wl.r, "s": wl.s, "T": wl.T,
+            "projection": args.projection, "history": args.history, "gram_fusion": args.gram_fusion,
+            "sharded": sharded, "history_filled": True, "refresh_in_timed_region": False,
+            "l2": f"inputs larger than L2: {pool_size(args, wl)} gradient sets of {grad_bytes / 1e9:.2f} GB cycled"}
+
+
 def measured_peaks():
     """(HBM copy GB/s, sustained bf16 TFLOP/s, "measured" | "fallback"): the machine's own measured peaks when
     the file with them is present, else the documented earlier measurement.  The step is timed inside a long
@@ -230,8 +245,7 @@ def run_reference(args, wl):
     out = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": wl.name, "matrices": wl.n_matrices, "r": wl.r, "s": wl.s, "projection": args.projection,
-                      "history": args.history},
+           "config": config_dict(args, wl, wl.n_matrices, False),
            "cpu_baseline": {"value": val, "unit": UNIT, "cores": smp.threads(), "kind": "oracle", "sample": desc},
            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out))
@@ -293,7 +307,9 @@ def run_ours(args, wl):
         wl = dataclasses.replace(wl, shapes=tuple(wl.shapes[i] for i in parts[rank]))
     shapes = [(M, N) for _, M, N in wl.shapes]
     n = len(shapes)
-    opt = NGaLore(shapes, wl.r, wl.s, wl.T, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
+    # The state is created without automatic refreshes: the timed steps are steady-state steps (history ring full,
+    # no refresh among them, whatever T is); the refresh is run once before them and timed alone further down.
+    opt = NGaLore(shapes, wl.r, wl.s, 0, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
                   wd=wl.wd, seed=1 + rank, projection=args.projection, history_bf16=args.history == "bf16",
                   gram_fusion=args.gram_fusion == "on")
     # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
@@ -302,24 +318,26 @@ def run_ours(args, wl):
         # weights of the matrices other ranks own, received after each step
         others = {i: torch.empty(full_shapes[i], dtype=torch.float32, device=dev)
                   for k, p in enumerate(parts) if k != rank for i in p}
-    # With fewer than s + 1 distinct sets a gradient would sit twice in the history ring and the Gram matrix
-    # would be singular up to lambda; the optimizer never sees that in training.
-    pool_sets = args.pool if args.pool > 0 else wl.s + 1
+    pool_sets = pool_size(args, wl)
     pool = [[W.gradient_device(wl_rank, i, k, dev) for i in range(n)] for k in range(pool_sets)]
     Wt = [W.initial_weight_device(wl_rank, i, dev) for i in range(n)]
     Wp = NGaLore.pointer_array(Wt)
     Gp = [NGaLore.pointer_array(g) for g in pool]
     grad_bytes = sum(M * N * 2 for M, N in shapes)
+    opt.refresh_subspace(pool[0])
+
+    def exchange():
+        Wall = [None] * len(full_shapes)
+        for j, i in enumerate(parts[rank]):
+            Wall[i] = Wt[j]
+        for i, t in others.items():
+            Wall[i] = t
+        sharding.exchange_updated(Wall, parts)
 
     def step(k):
         opt.step_ptrs(Wp, Gp[k % pool_sets])
         if parts is not None:
-            Wall = [None] * len(full_shapes)
-            for j, i in enumerate(parts[rank]):
-                Wall[i] = Wt[j]
-            for i, t in others.items():
-                Wall[i] = t
-            sharding.exchange_updated(Wall, parts)
+            exchange()
 
     def barrier():
         torch.cuda.synchronize()
@@ -327,28 +345,68 @@ def run_ours(args, wl):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for k in range(args.warmup):
+    # ---- untimed: fill the history ring (a step with c < s slots held moves fewer bytes than a steady-state one)
+    # and show the library every gradient set once, so that no timed step encodes or uploads TMA descriptors
+    fill = max(args.warmup, wl.s, pool_sets)
+    for k in range(fill):
         step(k)
+    barrier()
+    assert opt.step_count >= wl.s, "the history ring must be full before the timed region"
+    uploads_before = opt.descriptor_uploads
+
+    # ---- launch: one CUDA graph per gradient set (the step's kernel arguments do not change from step to step;
+    # only the descriptors of the gradient buffers differ between sets), or plain stream launches
+    use_graph = args.launch == "graph" and parts is None
+    graphs = None
+    if use_graph:
+        graphs = []
+        for j in range(pool_sets):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                opt.step_ptrs(Wp, Gp[j])
+            graphs.append(g)
+        barrier()
+
+    launches_per_step = [0]
+
+    def timed_step(k):
+        if graphs is not None:
+            graphs[k % pool_sets].replay()
+        else:
+            l0 = opt.launch_count
+            step(k)
+            launches_per_step[0] = opt.launch_count - l0
+
+    if graphs is not None:
+        l0 = opt.launch_count
+        opt.step_ptrs(Wp, Gp[fill % pool_sets])      # counts the kernels of one step; also one more warm step
+        launches_per_step[0] = opt.launch_count - l0
+        fill += 1
+    for k in range(args.warmup):
+        timed_step(fill + k)
     barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    l0 = opt.launch_count
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
-    e0.record()
+    ev[0].record()
     for k in range(args.steps):
-        step(args.warmup + k)
-    e1.record()
+        timed_step(fill + args.warmup + k)
+        ev[k + 1].record()
     barrier()
-    ms_total = e0.elapsed_time(e1)
-    launches = opt.launch_count - l0
+    ms_total = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    launches = launches_per_step[0] * args.steps
     clocks = sampler.stop() if rank == 0 else None
     ms_total = max_over_ranks(ms_total, dev, world)
+    ms_median = max_over_ranks(float(np.median(per_step)), dev, world)
     ms_step = ms_total / args.steps
     # sharded: the job made args.steps steps of one model; replicas: every rank made args.steps steps of its own
     value = job_throughput(1 if parts is not None else world, args.steps, ms_total)
+    assert opt.descriptor_uploads == uploads_before, "a timed step uploaded TMA descriptors"
+    done_steps = fill + args.warmup + args.steps
 
     code, per = opt.poll_status()
     if code != 0:
@@ -359,7 +417,7 @@ def run_ours(args, wl):
     phase = np.zeros(3)
     reps = 10
     for k in range(reps):
-        step(args.warmup + args.steps + k)
+        step(done_steps + k)
         phase += np.array([opt.last_phase_ms(p) for p in range(3)])
     phase /= reps
     opt.set_profiling(False)
@@ -446,11 +504,9 @@ def run_ours(args, wl):
            "dtype_detail": "bf16 (projection) and fp16 (back-projection) GEMM operands, f32 state and accumulation, "
                            "f64 Gram reduction and solve",
            "data": "synthetic",
-           "config": {"workload": wl.name, "matrices": n, "r": wl.r, "s": wl.s, "T": wl.T,
-                      "projection": args.projection, "history": args.history, "gram_fusion": args.gram_fusion,
-                      "sharded": parts is not None,
-                      "l2": f"inputs larger than L2: {pool_sets} gradient sets of {grad_bytes / 1e9:.2f} GB cycled",
-                      "state_bytes": opt.device_bytes},
+           "config": config_dict(args, wl, n, parts is not None),
+           "launch": "cuda_graph" if use_graph else "stream", "ms_per_step_median": ms_median,
+           "untimed_steps_before": fill + args.warmup, "state_bytes": opt.device_bytes,
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
            "step_roofline": step_roof,
            "refresh": {"ms": refresh_ms, "T": wl.T, "amortised_ms_per_step": ms_step + refresh_ms / max(wl.T, 1),
@@ -486,6 +542,9 @@ def main():
                     help="with --gpus N > 1: one model's matrices split over the ranks (state memory / N, weights "
                          "exchanged after every step) instead of N independent replicas; rank 0's phases and "
                          "roofline then describe its own shard")
+    ap.add_argument("--launch", default="graph", choices=["graph", "stream"],
+                    help="graph (default): every timed step is one replay of a CUDA graph captured from ngalore_step, one "
+                         "graph per gradient set; stream: plain calls of ngalore_step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -30,10 +30,16 @@
  *    ngalore_step and ngalore_refresh_subspace enqueue work and return; they do
  *    not synchronise and do not allocate.
  *  - Host-detectable errors are returned at once and leave the state untouched.
- *    Errors found on the device (a non-finite gradient, a non-positive Cholesky
- *    pivot, a wait that ran out) set a per-matrix status word; that matrix's W,
- *    m and v are left unchanged for the step and ngalore_poll_status reports it.
- *    No call traps or aborts.
+ *    Errors found on the device set a per-matrix status word that
+ *    ngalore_poll_status reports.  A non-finite gradient or a non-positive
+ *    Cholesky pivot leaves that matrix's W, m and v unchanged for the step (its
+ *    gradient enters the history as zero).  Every wait inside a kernel is
+ *    bounded; when the wait for a matrix's solved weights runs out, that
+ *    matrix's W is left unchanged for the step and its status is
+ *    NGALORE_ERR_TIMEOUT (parts of its m and v may already have advanced); when
+ *    a wait inside a GEMM pipeline runs out, the kernel stops issuing work and
+ *    ngalore_poll_status returns NGALORE_ERR_TIMEOUT for the state as a whole:
+ *    restore it from a checkpoint.  No call traps, aborts or spins for ever.
  *  - A state is bound to the device that was current in ngalore_create and is
  *    not safe for concurrent calls from several threads.
  */
@@ -89,9 +95,7 @@ typedef struct {
                                        at most 8192, fp32 history of at most 16 slots, rows and columns multiples of
                                        32) it is formed in the epilogue of the projection GEMM instead, so that the
                                        first read of the history runs under the tensor-core work; same results to
-                                       rounding.  Measured slower than the default on the 1.1B shapes as built (about
-                                       7.0 against 6.7 ms per step: with the memory system saturated by the history the
-                                       MMAs wait for their operands), hence off unless asked for. */
+                                       rounding.  Not faster than the default as built, hence off unless asked for. */
 } ngalore_options;
 
 /*
@@ -121,9 +125,13 @@ void ngalore_destroy(ngalore_state* st);
  *   G  host array of n_matrices device pointers, bf16 bit patterns M x N, read only
  * If T > 0 and the step index k satisfies k mod T == 0, the subspace of every
  * matrix is refreshed from G first.  Increments k.
- * After one call with the same W and G pointers a further call enqueues kernels only (no copies), so it can
- * be captured in a CUDA graph.  A replay advances the device-side ring position but not the host-side k:
- * create the state with T = 0 when replaying from a graph and call ngalore_refresh_subspace yourself.
+ * The TMA descriptors of W and G are cached per array of pointers (at most 32 arrays, fewer for very many
+ * matrices; the least recently used is overwritten): the first call with a given pair of arrays encodes and
+ * uploads them, a later call with the same pointers enqueues kernels only (no copies), so it can be captured in a
+ * CUDA graph.  Such a graph stays valid until its array of pointers has been pushed out of that cache.  A call
+ * under stream capture leaves the host-side step counter alone and a replay advances the device-side ring
+ * position and step index only, so the automatic refresh (which the host decides) cannot follow replays: create
+ * the state with T = 0 when replaying from a graph and call ngalore_refresh_subspace yourself.
  */
 ngalore_status ngalore_step(ngalore_state* st, float* const* W, const uint16_t* const* G, void* stream);
 
@@ -170,6 +178,16 @@ ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, 
 ngalore_status ngalore_state_export(ngalore_state* st, void* blob, size_t* bytes);
 ngalore_status ngalore_state_import(ngalore_state* st, const void* blob, size_t bytes);
 
+/*
+ * Testing aid (no counterpart in the paper): in the next ngalore_step only, the solved weights of matrix
+ * `matrix_index` are computed but not announced, and the tiles that wait for them give up after `polls` polls
+ * (1 .. 1000000, about 100 ns each) instead of the default limit.  The step then ends normally with
+ * NGALORE_ERR_TIMEOUT in that matrix's status word and its W unchanged; the following step is a regular one.
+ * This is how the tests exercise a bounded wait that runs out; nothing hangs or traps.  Synchronises the device.
+ * Not available with s = 0, stream_impl = 1, or for a matrix whose Gram row is formed by gram_fusion.
+ */
+ngalore_status ngalore_debug_withhold_solution(ngalore_state* st, int matrix_index, int polls);
+
 /* Change the learning rate used from the next step on. */
 ngalore_status ngalore_set_lr(ngalore_state* st, double lr);
 
@@ -178,10 +196,15 @@ int ngalore_num_matrices(const ngalore_state* st);
 int ngalore_rank(const ngalore_state* st, int i);          /* r' of matrix i, -1 if i is out of range */
 int ngalore_projects_right(const ngalore_state* st, int i); /* 1 if matrix i is projected on the right, 0 if on the left, -1 if out of range */
 int ngalore_subspace_rows(const ngalore_state* st, int i);  /* rows of its projector: M (left) or N (right), -1 if out of range */
-int64_t ngalore_step_count(const ngalore_state* st);        /* k */
+int64_t ngalore_step_count(const ngalore_state* st);        /* k as the host last knew it: steps replayed from a CUDA
+                                                               graph are counted on the device and taken over by
+                                                               ngalore_poll_status and ngalore_state_export */
 size_t ngalore_device_bytes(const ngalore_state* st);       /* device memory held by the state */
 /* Kernels launched by the library on behalf of this state since creation. */
 int64_t ngalore_launch_count(const ngalore_state* st);
+/* How many times ngalore_step had to encode and upload the TMA descriptors of a (W, G) pair of pointer arrays
+ * (see ngalore_step: once per distinct pair while it stays cached). */
+int64_t ngalore_descriptor_uploads(const ngalore_state* st);
 
 /* Per-phase timing of ngalore_step with CUDA events recorded on the launching stream.
  * phase: 0 projection GEMM (R = P^T G), 1 Gram / solve / moment kernels, 2 back-projection + W update.

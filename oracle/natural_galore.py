@@ -20,8 +20,7 @@ paper gives:
 
 with U = [vec(H_1) ... vec(H_c)] / sqrt(c) and c the number of gradients held.
 
-Readings taken where the paper is silent or inconsistent (each is listed in the
-design notes): left projection only (the default; ``Hyper.projection =
+Readings taken where the paper is silent or inconsistent: left projection only (the default; ``Hyper.projection =
 "short_side"`` selects the GaLore convention the paper inherits when it says, at
 the start of Sec. 2.4, that most steps are those of GaLore: project on the
 right, R = G Q with Q the first r' right singular vectors, when M >= N);
@@ -55,8 +54,11 @@ import numpy as np
 def round_to_bf16(x: np.ndarray) -> np.ndarray:
     """Values of x rounded to the nearest bf16 (ties to even), returned as float64.
 
-    Used only to hold the projection matrix in the storage format the update is
-    defined on (P is kept as bf16 by contract; see the design notes)."""
+    Used to hold the projection matrix in the storage format the update is defined
+    on: the optimizer keeps the working copy of P in bf16, so the step (both here
+    and in the CUDA path) is the paper's update with P replaced by its bf16 rounding,
+    and the rounding of P is then not an error term of the comparison.  Also used by
+    the bf16-history option."""
     f = np.ascontiguousarray(x, dtype=np.float32)
     u = f.view(np.uint32).astype(np.uint64)
     u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000

@@ -51,6 +51,11 @@ struct Ctrl {
   unsigned int work_counter;  // dynamic tile counter of the fused streaming kernel
   unsigned int gemm_counter0; // dynamic tile counter of the projection GEMM
   unsigned int gemm_counter1; // dynamic tile counter of the back-projection GEMM
+  // Testing aids, both cleared at the end of every step.  They exist so that a test can make a bounded wait run
+  // out without hanging or trapping anything: the solution of one matrix is computed but not published, and the
+  // tiles that wait for it give up after a few polls.
+  int spin_limit;             // > 0: polls before a flag wait of the stream kernel is abandoned (0: the default)
+  int debug_withhold;         // > 0: the weights of matrix (debug_withhold - 1) are not published in this step
 };
 
 struct Hyper {

@@ -19,6 +19,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstring>
 #include <vector>
 
 #include "../../include/ngalore.h"
@@ -435,9 +436,26 @@ struct TcPlan {
   std::vector<int> right;           // per matrix: projected on the right
   bool tall_proj = false;           // projection tiles are 256 rows high (tc_project2_kernel)
   bool long_k_back = false;         // back-projection with three operand stages and a short W ring
-  std::vector<const void*> last_G;
-  std::vector<const void*> last_W;
-  CUtensorMap* d_maps = nullptr;
+  // Binding sets: the tensor maps of one particular array of G and W pointers, encoded once, kept in pinned host
+  // memory and uploaded once.  A training loop that cycles through a few gradient buffers (or always passes the
+  // same ones) pays for encoding and upload only the first time it shows a set; afterwards a step does no host
+  // work beyond comparing the pointers.  All sets are allocated with the plan; the least recently used one is
+  // overwritten when a new array of pointers arrives and every set is taken.
+  struct Binding {
+    std::vector<const void*> G, W;
+    uint64_t hash = 0;
+    bool valid = false;
+    int64_t last_use = 0;
+    cudaEvent_t uploaded = nullptr;  // recorded after the upload from h_pinned: the pinned copy may be rewritten after it
+    CUtensorMap* d_maps = nullptr;
+    CUtensorMap* h_pinned = nullptr;
+  };
+  std::vector<Binding> bindings;
+  int64_t bind_clock = 0;
+  int64_t bind_uploads = 0;         // how many times a set had to be encoded and uploaded
+  CUtensorMap* d_maps_all = nullptr;
+  CUtensorMap* h_pinned_all = nullptr;
+  CUtensorMap* d_maps = nullptr;    // the set of the current call (one of bindings[*].d_maps)
   TcTile* d_tiles_proj = nullptr;
   TcTile* d_tiles_back = nullptr;
   std::vector<int> back_tile0;     // first back-projection tile of every matrix, plus the total (n + 1 entries)
@@ -445,7 +463,6 @@ struct TcPlan {
   int grid_proj = 0, grid_back = 0;
   int* d_split_mats = nullptr;
   int n_split = 0;
-  bool maps_dirty = true;
   // projection with the Gram row in its epilogue: the matrices that take part, their tiles and partial rows
   std::vector<int> gram_fused;     // per matrix: 1 when its Gram row comes from the projection's epilogue
   TcTile* d_tiles_pg = nullptr;
@@ -469,7 +486,12 @@ inline bool tc_encode_2d(EncodeTiledFn fn, CUtensorMap* map, const void* base, u
 }
 
 inline void tc_plan_destroy(TcPlan& plan) {
-  if (plan.d_maps) cudaFree(plan.d_maps);
+  for (TcPlan::Binding& b : plan.bindings)
+    if (b.uploaded) cudaEventDestroy(b.uploaded);
+  plan.bindings.clear();
+  if (plan.d_maps_all) cudaFree(plan.d_maps_all);
+  if (plan.h_pinned_all) cudaFreeHost(plan.h_pinned_all);
+  plan.d_maps_all = nullptr; plan.h_pinned_all = nullptr;
   if (plan.d_tiles_proj) cudaFree(plan.d_tiles_proj);
   if (plan.d_tiles_back) cudaFree(plan.d_tiles_back);
   if (plan.d_split_mats) cudaFree(plan.d_split_mats);
@@ -491,8 +513,6 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   const int n = static_cast<int>(mats.size());
   plan.n_mats = n;
   plan.h_maps.resize(static_cast<size_t>(n) * kTcMapsPerMat);
-  plan.last_G.assign(n, nullptr);
-  plan.last_W.assign(n, nullptr);
   std::memset(plan.h_maps.data(), 0, sizeof(CUtensorMap) * plan.h_maps.size());
   for (int i = 0; i < n; ++i) {
     const MatDesc& d = mats[i];
@@ -623,8 +643,23 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
     plan.device_bytes += sizeof(TcTile) * pg.size() + sizeof(PgMat) * n + sizeof(double) * pg_rows * kPgSMax + sizeof(int) * pg_list.size();
   }
 
-  const size_t maps_bytes = sizeof(CUtensorMap) * plan.h_maps.size();
-  if (cudaMalloc(&plan.d_maps, maps_bytes) != cudaSuccess) { plan.d_maps = nullptr; return NGALORE_ERR_ALLOC; }
+  // binding sets: as many as fit in 64 MB, between 2 and 32
+  const size_t set_bytes = sizeof(CUtensorMap) * plan.h_maps.size();
+  int n_sets = static_cast<int>((64u << 20) / set_bytes);
+  n_sets = n_sets < 2 ? 2 : (n_sets > 32 ? 32 : n_sets);
+  const size_t maps_bytes = set_bytes * n_sets;
+  if (cudaMalloc(&plan.d_maps_all, maps_bytes) != cudaSuccess) { plan.d_maps_all = nullptr; return NGALORE_ERR_ALLOC; }
+  if (cudaMallocHost(&plan.h_pinned_all, maps_bytes) != cudaSuccess) { plan.h_pinned_all = nullptr; return NGALORE_ERR_ALLOC; }
+  plan.bindings.resize(n_sets);
+  for (int b = 0; b < n_sets; ++b) {
+    plan.bindings[b].d_maps = plan.d_maps_all + static_cast<size_t>(b) * plan.h_maps.size();
+    plan.bindings[b].h_pinned = plan.h_pinned_all + static_cast<size_t>(b) * plan.h_maps.size();
+    if (cudaEventCreateWithFlags(&plan.bindings[b].uploaded, cudaEventDisableTiming) != cudaSuccess) {
+      plan.bindings[b].uploaded = nullptr;
+      return NGALORE_ERR_CUDA;
+    }
+  }
+  plan.d_maps = plan.bindings[0].d_maps;
   if (cudaMalloc(&plan.d_tiles_proj, sizeof(TcTile) * proj.size()) != cudaSuccess) { plan.d_tiles_proj = nullptr; return NGALORE_ERR_ALLOC; }
   if (cudaMalloc(&plan.d_tiles_back, sizeof(TcTile) * back.size()) != cudaSuccess) { plan.d_tiles_back = nullptr; return NGALORE_ERR_ALLOC; }
   if (cudaMalloc(&plan.d_split_mats, sizeof(int) * (split_mats.size() + 1)) != cudaSuccess) { plan.d_split_mats = nullptr; return NGALORE_ERR_ALLOC; }
@@ -638,43 +673,61 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   plan.rowsN.resize(n); plan.colsN.resize(n); plan.right.resize(n);
   for (int i = 0; i < n; ++i) { plan.rowsN[i] = mats[i].M; plan.colsN[i] = mats[i].N; plan.right[i] = mats[i].right; }
 
-  plan.maps_dirty = true;
   return NGALORE_OK;
 }
 
 // Point the tensor maps of the step at this call's gradients and weights (host arrays of device pointers,
-// 16-byte aligned, row-major M x N).  Maps are rebuilt and uploaded only when a pointer differs from the
-// last call's, so a step with unchanged buffers enqueues kernels only.
+// 16-byte aligned, row-major M x N).  An array of pointers that was seen before (and whose binding set has not
+// been overwritten since) costs a comparison of the pointers; a new one is encoded into its set's pinned host
+// copy and uploaded from there, asynchronously on `stream`.
 inline ngalore_status tc_bind_buffers(TcPlan& plan, const uint16_t* const* G, float* const* W, cudaStream_t stream) {
-  bool changed = plan.maps_dirty;
-  for (int i = 0; i < plan.n_mats; ++i) {
-    CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * kTcMapsPerMat];
-    if (plan.last_G[i] != G[i]) {
-      plan.last_G[i] = G[i];
-      // G is the B operand of a left projection (K = M rows) and the A operand of a right one (K = N columns)
-      const bool enc = plan.right[i]
-                           ? tc_encode_2d(plan.encode, mp + TC_MAP_A_PROJ, G[i], plan.colsN[i], plan.rowsN[i],
-                                          static_cast<uint64_t>(plan.colsN[i]) * 2, kTcBK, kTcBM)
-                           : tc_encode_2d(plan.encode, mp + TC_MAP_B_PROJ, G[i], plan.colsN[i], plan.rowsN[i],
-                                          static_cast<uint64_t>(plan.colsN[i]) * 2, 64, kTcBK);
-      if (!enc) return NGALORE_ERR_CUDA;
-      changed = true;
-    }
-    if (plan.last_W[i] != W[i]) {
-      plan.last_W[i] = W[i];
-      const uint64_t row_bytes = static_cast<uint64_t>(plan.colsN[i]) * 4;
-      if (!tc_encode_2d(plan.encode, mp + TC_MAP_W_LOAD, W[i], plan.colsN[i], plan.rowsN[i], row_bytes, 32, kTcBM, true) ||
-          !tc_encode_2d(plan.encode, mp + TC_MAP_W_STORE, W[i], plan.colsN[i], plan.rowsN[i], row_bytes, 32, 32, true))
-        return NGALORE_ERR_CUDA;
-      changed = true;
-    }
+  const int n = plan.n_mats;
+  uint64_t hash = 1469598103934665603ull;
+  for (int i = 0; i < n; ++i) {
+    hash = (hash ^ reinterpret_cast<uintptr_t>(G[i])) * 1099511628211ull;
+    hash = (hash ^ reinterpret_cast<uintptr_t>(W[i])) * 1099511628211ull;
   }
-  if (changed) {
-    if (cudaMemcpyAsync(plan.d_maps, plan.h_maps.data(), sizeof(CUtensorMap) * plan.h_maps.size(),
-                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
+  plan.bind_clock += 1;
+  TcPlan::Binding* victim = nullptr;  // a free set if there is one, else the least recently used
+  for (TcPlan::Binding& b : plan.bindings) {
+    if (b.valid && b.hash == hash && std::equal(b.G.begin(), b.G.end(), reinterpret_cast<const void* const*>(G)) &&
+        std::equal(b.W.begin(), b.W.end(), reinterpret_cast<const void* const*>(W))) {
+      b.last_use = plan.bind_clock;
+      plan.d_maps = b.d_maps;
+      return NGALORE_OK;
+    }
+    if (victim == nullptr || (victim->valid && (!b.valid || b.last_use < victim->last_use))) victim = &b;
+  }
+  TcPlan::Binding& b = *victim;
+  // the previous upload from this pinned copy must have been read before it is rewritten
+  if (b.valid && cudaEventSynchronize(b.uploaded) != cudaSuccess) return NGALORE_ERR_CUDA;
+  b.valid = false;
+  std::memcpy(b.h_pinned, plan.h_maps.data(), sizeof(CUtensorMap) * plan.h_maps.size());
+  for (int i = 0; i < n; ++i) {
+    CUtensorMap* mp = b.h_pinned + static_cast<size_t>(i) * kTcMapsPerMat;
+    // G is the B operand of a left projection (K = M rows) and the A operand of a right one (K = N columns)
+    const bool enc = plan.right[i]
+                         ? tc_encode_2d(plan.encode, mp + TC_MAP_A_PROJ, G[i], plan.colsN[i], plan.rowsN[i],
+                                        static_cast<uint64_t>(plan.colsN[i]) * 2, kTcBK, kTcBM)
+                         : tc_encode_2d(plan.encode, mp + TC_MAP_B_PROJ, G[i], plan.colsN[i], plan.rowsN[i],
+                                        static_cast<uint64_t>(plan.colsN[i]) * 2, 64, kTcBK);
+    if (!enc) return NGALORE_ERR_CUDA;
+    const uint64_t row_bytes = static_cast<uint64_t>(plan.colsN[i]) * 4;
+    if (!tc_encode_2d(plan.encode, mp + TC_MAP_W_LOAD, W[i], plan.colsN[i], plan.rowsN[i], row_bytes, 32, kTcBM, true) ||
+        !tc_encode_2d(plan.encode, mp + TC_MAP_W_STORE, W[i], plan.colsN[i], plan.rowsN[i], row_bytes, 32, 32, true))
       return NGALORE_ERR_CUDA;
-    plan.maps_dirty = false;
   }
+  if (cudaMemcpyAsync(b.d_maps, b.h_pinned, sizeof(CUtensorMap) * plan.h_maps.size(), cudaMemcpyHostToDevice, stream) !=
+          cudaSuccess ||
+      cudaEventRecord(b.uploaded, stream) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  b.G.assign(reinterpret_cast<const void* const*>(G), reinterpret_cast<const void* const*>(G) + n);
+  b.W.assign(reinterpret_cast<const void* const*>(W), reinterpret_cast<const void* const*>(W) + n);
+  b.hash = hash;
+  b.valid = true;
+  b.last_use = plan.bind_clock;
+  plan.bind_uploads += 1;
+  plan.d_maps = b.d_maps;
   return NGALORE_OK;
 }
 

@@ -339,7 +339,7 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
               if (tid == 0) {
                 *d.gram_done = 0;
                 __threadfence();
-                atomicExch(d.w_ready, tag);
+                if (ctrl->debug_withhold != mt.mat + 1) atomicExch(d.w_ready, tag);
               }
             }
           }
@@ -351,13 +351,20 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
           if (d.s > 0) {
             if (tid == 0) {
               const volatile int* flag = d.w_ready;
+              const long long limit = ctrl->spin_limit > 0 ? ctrl->spin_limit : kSpinLimit;
               long long spins = 0;
               int ok = 1;
               while (*flag != tag) {
-                if (++spins > kSpinLimit) { ok = 0; break; }
+                if (++spins > limit) { ok = 0; break; }
                 __nanosleep(100);
               }
-              if (!ok) atomicExch(&ctrl->timeout_flag, 1);
+              if (!ok) {
+                // The weights never came: this matrix takes no update in this step (the back-projection skips it)
+                // and says why.  Tiles of it that other CTAs did combine have advanced their part of m and v.
+                atomicExch(&ctrl->timeout_flag, 1);
+                atomicExch(d.step_bad, 1);
+                atomicCAS(d.status, 0, 8 /* NGALORE_ERR_TIMEOUT */);
+              }
               *s_flag = ok;
             }
             consumer_sync<kConsumerThreads>();

@@ -236,6 +236,8 @@ __global__ void advance_kernel(Ctrl* ctrl) {
   ctrl->work_counter = 0u;
   ctrl->gemm_counter0 = 0u;
   ctrl->gemm_counter1 = 0u;
+  ctrl->spin_limit = 0;
+  ctrl->debug_withhold = 0;
 }
 
 }  // namespace ngalore

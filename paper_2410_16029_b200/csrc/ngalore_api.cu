@@ -69,6 +69,7 @@ struct ngalore_state {
   Hyper* d_hyper = nullptr;
   int* d_status = nullptr;
   int* d_step_bad = nullptr;
+  int* d_flags = nullptr;            // gram_done / w_ready of every matrix (scratch, not part of a checkpoint)
   StreamTile* d_tiles = nullptr;
   int n_tiles = 0;
   std::vector<const uint16_t*> refresh_G;  // the gradients as the refresh reads them (G, or its transposed copy)
@@ -79,7 +80,8 @@ struct ngalore_state {
   CholProblem* d_chol = nullptr;
   int64_t k = 0;
   int64_t n_appended = 0;
-  bool has_subspace = false;
+  bool has_subspace = false;         // every matrix has a projector
+  std::vector<char> subspace_set;    // per matrix: refreshed or set at least once
   int64_t launches = 0;
   uint64_t shape_hash = 0;
   // tensor-core GEMM plan (tile tables, tensor maps)
@@ -241,7 +243,9 @@ ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bo
     st->n_appended = 0;
     NG_CUDA(cudaMemsetAsync(&st->d_ctrl->n_appended, 0, sizeof(long long), stream));
   }
-  if (whole_set) st->has_subspace = true;
+  for (int i : idx) st->subspace_set[i] = 1;
+  st->has_subspace = true;
+  for (char c : st->subspace_set) st->has_subspace = st->has_subspace && c != 0;
   return NGALORE_OK;
 }
 
@@ -404,8 +408,15 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
     NG_CUDA(cudaEventRecord(st->ev[3], stream));
     st->ev_valid = true;
   }
-  st->k += 1;
-  st->n_appended += 1;
+  // A call that is being captured into a CUDA graph enqueues nothing yet: the host-side counters then stay where
+  // they are (replays advance the device-side counters only; ngalore_poll_status and ngalore_state_export read
+  // those back).
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) cap = cudaStreamCaptureStatusNone;
+  if (cap == cudaStreamCaptureStatusNone) {
+    st->k += 1;
+    st->n_appended += 1;
+  }
   return NGALORE_OK;
 }
 
@@ -586,6 +597,8 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   st->d_chol = reinterpret_cast<CholProblem*>(st->work + o_chol);
   st->d_tiles = reinterpret_cast<StreamTile*>(st->work + o_tiles);
   int* flags = reinterpret_cast<int*>(st->work + o_flags);
+  st->d_flags = flags;
+  st->subspace_set.assign(n_matrices, 0);
 
   st->h_desc.resize(n_matrices);
   std::vector<CholProblem> chol(n_matrices);
@@ -832,6 +845,9 @@ ngalore_status ngalore_poll_status(ngalore_state* st, int* per_matrix) {
   Ctrl c{};
   NG_CUDA(cudaMemcpy(&c, st->d_ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost));
   NG_CUDA(cudaMemset(st->d_status, 0, sizeof(int) * st->n));
+  // steps replayed from a CUDA graph advance only the device-side counters: take those over
+  st->k = c.k;
+  st->n_appended = c.n_appended;
   if (c.timeout_flag != 0) NG_CUDA(cudaMemset(&st->d_ctrl->timeout_flag, 0, sizeof(int)));
   ngalore_status first = NGALORE_OK;
   for (int i = 0; i < st->n; ++i) {
@@ -845,6 +861,7 @@ ngalore_status ngalore_poll_status(ngalore_state* st, int* per_matrix) {
 ngalore_status ngalore_get_subspace(ngalore_state* st, int i, float* P, void* stream) {
   if (st == nullptr || i < 0 || i >= st->n || P == nullptr) return NGALORE_ERR_INVALID_ARG;
   DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
   const HostMat& hm = st->mats[i];
   NG_CUDA(cudaMemcpyAsync(P, st->h_desc[i].P32, sizeof(float) * hm.eM * hm.rp, cudaMemcpyDeviceToDevice,
                           static_cast<cudaStream_t>(stream)));
@@ -854,6 +871,7 @@ ngalore_status ngalore_get_subspace(ngalore_state* st, int i, float* P, void* st
 ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, void* stream) {
   if (st == nullptr || i < 0 || i >= st->n || P == nullptr) return NGALORE_ERR_INVALID_ARG;
   DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
   const HostMat& hm = st->mats[i];
   const long long cnt = static_cast<long long>(hm.eM) * hm.rp;
   widen_16_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
@@ -866,12 +884,15 @@ ngalore_status ngalore_get_working_subspace(ngalore_state* st, int i, float* P, 
 ngalore_status ngalore_set_subspace(ngalore_state* st, int i, const float* P, void* stream) {
   if (st == nullptr || i < 0 || i >= st->n || P == nullptr) return NGALORE_ERR_INVALID_ARG;
   DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
   const HostMat& hm = st->mats[i];
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, P, sizeof(float) * hm.eM * hm.rp, cudaMemcpyDeviceToDevice, s));
   ngalore_status rc = make_working_copies(st, i, s);
   if (rc != NGALORE_OK) return rc;
-  st->has_subspace = true;  // the caller is responsible for setting every matrix before stepping
+  st->subspace_set[i] = 1;
+  st->has_subspace = true;  // stepping needs a projector for every matrix
+  for (char c : st->subspace_set) st->has_subspace = st->has_subspace && c != 0;
   return NGALORE_OK;
 }
 
@@ -881,7 +902,12 @@ ngalore_status ngalore_state_export(ngalore_state* st, void* blob, size_t* bytes
   if (blob == nullptr) { *bytes = need; return NGALORE_OK; }
   if (*bytes < need) return NGALORE_ERR_INVALID_ARG;
   DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
   NG_CUDA(cudaDeviceSynchronize());
+  Ctrl c{};
+  NG_CUDA(cudaMemcpy(&c, st->d_ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost));
+  st->k = c.k;                      // the device-side counters are the authority (graph replays advance only them)
+  st->n_appended = c.n_appended;
   BlobHeader h{};
   h.magic = kBlobMagic; h.arena_bytes = st->arena_bytes; h.k = st->k; h.n_appended = st->n_appended;
   h.n = st->n; h.r = st->r; h.s = st->s; h.has_subspace = st->has_subspace ? 1 : 0; h.shape_hash = st->shape_hash;
@@ -899,9 +925,32 @@ ngalore_status ngalore_state_import(ngalore_state* st, const void* blob, size_t 
       h.shape_hash != st->shape_hash || bytes < sizeof(h) + h.arena_bytes)
     return NGALORE_ERR_INVALID_ARG;
   DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
   NG_CUDA(cudaDeviceSynchronize());
   NG_CUDA(cudaMemcpy(st->arena, static_cast<const char*>(blob) + sizeof(h), st->arena_bytes, cudaMemcpyHostToDevice));
+  // The blob brings back the step epoch of the exporting state.  The per-matrix flags of the stream kernel hold
+  // epochs of steps this state ran before the import and could equal the next step's tag by accident (export, step,
+  // import, step): clear them, together with the scheduling counters and anything a testing aid left behind.
+  NG_CUDA(cudaMemset(st->d_flags, 0, sizeof(int) * 2 * st->n));
+  Ctrl c{};
+  NG_CUDA(cudaMemcpy(&c, st->d_ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost));
+  c.timeout_flag = 0; c.work_counter = 0u; c.gemm_counter0 = 0u; c.gemm_counter1 = 0u;
+  c.spin_limit = 0; c.debug_withhold = 0;
+  NG_CUDA(cudaMemcpy(st->d_ctrl, &c, sizeof(Ctrl), cudaMemcpyHostToDevice));
   st->k = h.k; st->n_appended = h.n_appended; st->has_subspace = h.has_subspace != 0;
+  st->subspace_set.assign(st->n, st->has_subspace ? 1 : 0);
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_debug_withhold_solution(ngalore_state* st, int matrix_index, int polls) {
+  if (st == nullptr || matrix_index < 0 || matrix_index >= st->n || polls < 1 || polls > 1000000) return NGALORE_ERR_INVALID_ARG;
+  if (st->s < 1 || st->opt.stream_impl == 1) return NGALORE_ERR_INVALID_ARG;
+  if (!st->tc.gram_fused.empty() && st->tc.gram_fused[matrix_index]) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
+  NG_CUDA(cudaDeviceSynchronize());
+  const int v[2] = {polls, matrix_index + 1};
+  NG_CUDA(cudaMemcpy(&st->d_ctrl->spin_limit, v, sizeof(v), cudaMemcpyHostToDevice));
   return NGALORE_OK;
 }
 
@@ -919,6 +968,7 @@ int ngalore_subspace_rows(const ngalore_state* st, int i) { return (st && i >= 0
 int64_t ngalore_step_count(const ngalore_state* st) { return st ? st->k : -1; }
 size_t ngalore_device_bytes(const ngalore_state* st) { return st ? st->arena_bytes + st->work_bytes + st->stage_bytes + st->tc.device_bytes + st->refresh.device_bytes : 0; }
 int64_t ngalore_launch_count(const ngalore_state* st) { return st ? st->launches : 0; }
+int64_t ngalore_descriptor_uploads(const ngalore_state* st) { return st ? st->tc.bind_uploads : 0; }
 
 ngalore_status ngalore_set_profiling(ngalore_state* st, int on) {
   if (st == nullptr) return NGALORE_ERR_INVALID_ARG;

@@ -60,6 +60,8 @@ _lib.ngalore_state_export.restype = ctypes.c_int
 _lib.ngalore_state_export.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_size_t)]
 _lib.ngalore_state_import.restype = ctypes.c_int
 _lib.ngalore_state_import.argtypes = [_vp, _vp, ctypes.c_size_t]
+_lib.ngalore_debug_withhold_solution.restype = ctypes.c_int
+_lib.ngalore_debug_withhold_solution.argtypes = [_vp, ctypes.c_int, ctypes.c_int]
 _lib.ngalore_set_lr.restype = ctypes.c_int
 _lib.ngalore_set_lr.argtypes = [_vp, ctypes.c_double]
 _lib.ngalore_num_matrices.restype = ctypes.c_int
@@ -73,6 +75,8 @@ _lib.ngalore_device_bytes.restype = ctypes.c_size_t
 _lib.ngalore_device_bytes.argtypes = [_vp]
 _lib.ngalore_launch_count.restype = ctypes.c_int64
 _lib.ngalore_launch_count.argtypes = [_vp]
+_lib.ngalore_descriptor_uploads.restype = ctypes.c_int64
+_lib.ngalore_descriptor_uploads.argtypes = [_vp]
 _lib.ngalore_set_profiling.restype = ctypes.c_int
 _lib.ngalore_set_profiling.argtypes = [_vp, ctypes.c_int]
 _lib.ngalore_last_phase_ms.restype = ctypes.c_double
@@ -206,6 +210,10 @@ class NGaLore:
     def import_state(self, blob: bytes):
         _check(_lib.ngalore_state_import(self._h, blob, len(blob)), "ngalore_state_import")
 
+    def debug_withhold_solution(self, matrix_index: int, polls: int):
+        """Testing aid: the next step does not announce matrix_index's solved weights (see include/ngalore.h)."""
+        _check(_lib.ngalore_debug_withhold_solution(self._h, matrix_index, polls), "ngalore_debug_withhold_solution")
+
     def set_lr(self, lr: float):
         _check(_lib.ngalore_set_lr(self._h, lr), "ngalore_set_lr")
 
@@ -220,6 +228,10 @@ class NGaLore:
     @property
     def launch_count(self) -> int:
         return _lib.ngalore_launch_count(self._h)
+
+    @property
+    def descriptor_uploads(self) -> int:
+        return _lib.ngalore_descriptor_uploads(self._h)
 
     def set_profiling(self, on: bool):
         _check(_lib.ngalore_set_profiling(self._h, int(on)), "ngalore_set_profiling")

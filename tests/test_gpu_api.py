@@ -194,3 +194,120 @@ def test_sharded_wrapper_with_one_rank_equals_the_plain_optimizer():
             assert torch.equal(x, y)
     finally:
         dist.destroy_process_group()
+
+
+def test_import_into_a_state_that_has_stepped_since_the_export():
+    """Export, step once more, import the blob back into the SAME state, step again: the bits of a straight run.
+    The import brings back the exporting step's epoch; whatever the step in between left in the stream kernel's
+    readiness flags must not be taken for the next step's."""
+    w = wl.tiny_workload([(136, 264)], r=16, s=3, T=0, inner_rank=4, index=86)
+    dev = torch.device("cuda")
+    grads = _grads(w, 8, dev)
+    P = None
+
+    def run(detour):
+        nonlocal P
+        opt = _make(w)
+        if P is None:
+            opt.refresh_subspace(grads[0])
+            P = opt.get_subspace(0).clone()
+        else:
+            opt.set_subspace(0, P)
+        W = [torch.zeros((136, 264), device=dev)]
+        for k in range(8):
+            if detour and k == 5:
+                blob = opt.export_state()
+                scratch = [W[0].clone()]
+                opt.step(scratch, grads[7])      # a step the straight run never makes
+                torch.cuda.synchronize()
+                opt.import_state(blob)
+            opt.step(W, grads[k])
+        torch.cuda.synchronize()
+        assert opt.poll_status()[0] == 0
+        return W[0].clone()
+
+    a, b = run(False), run(True)
+    assert torch.equal(a, b)
+
+
+def test_a_wait_that_runs_out_is_reported_and_skips_only_that_matrix():
+    """The bounded wait of the stream kernel's combination tiles: with the testing aid the weights of matrix 1 are
+    computed but never announced, its tiles give up after a bounded number of polls, and the step ends by itself: status
+    TIMEOUT for matrix 1, its W bitwise untouched, the other matrices updated as usual, and the next step clean."""
+    from paper_2410_16029_b200.ngalore import NGaLoreError
+
+    w = wl.tiny_workload([(136, 264), (264, 136), (72, 200)], r=16, s=3, T=0, inner_rank=4, index=87, wd=0.1)
+    dev = torch.device("cuda")
+    grads = _grads(w, 4, dev)
+    a, b = _make(w), _make(w)
+    a.refresh_subspace(grads[0])
+    for i in range(3):
+        b.set_subspace(i, a.get_subspace(i))
+    Wa = [wl.initial_weight_device(w, i, dev) for i in range(3)]
+    Wb = [t.clone() for t in Wa]
+    for k in range(2):
+        a.step(Wa, grads[k])
+        b.step(Wb, grads[k])
+    torch.cuda.synchronize()
+    before = Wb[1].clone()
+    b.debug_withhold_solution(1, 20000)
+    a.step(Wa, grads[2])
+    b.step(Wb, grads[2])
+    torch.cuda.synchronize()
+    code, per = b.poll_status()
+    assert code == 8 and per == [0, 8, 0], (code, per)
+    assert torch.equal(Wb[1], before)                       # neither decay nor update reached it
+    assert torch.equal(Wb[0], Wa[0]) and torch.equal(Wb[2], Wa[2])
+    # the aid lasts one step: the next one is regular again for every matrix
+    before = [t.clone() for t in Wb]
+    b.step(Wb, grads[3])
+    torch.cuda.synchronize()
+    assert b.poll_status() == (0, [0, 0, 0])
+    assert all(not torch.equal(x, y) for x, y in zip(before, Wb))
+    with pytest.raises(NGaLoreError):
+        b.debug_withhold_solution(7, 20000)
+
+
+def test_stepping_needs_a_projector_for_every_matrix():
+    from paper_2410_16029_b200.ngalore import NGaLoreError
+
+    w = wl.tiny_workload([(72, 40), (40, 72)], r=8, s=2, T=0, inner_rank=4, index=88)
+    dev = torch.device("cuda")
+    grads = _grads(w, 1, dev)
+    opt = _make(w)
+    W = [torch.zeros((M, N), device=dev) for _, M, N in w.shapes]
+    ref = _make(w)
+    ref.refresh_subspace(grads[0])
+    opt.set_subspace(0, ref.get_subspace(0))
+    with pytest.raises(NGaLoreError) as e:
+        opt.step(W, grads[0])
+    assert e.value.code == 5                                 # NO_SUBSPACE: matrix 1 has none yet
+    opt.refresh_subspace(grads[0], matrix_index=1)
+    opt.step(W, grads[0])
+    torch.cuda.synchronize()
+    assert opt.poll_status()[0] == 0
+
+
+def test_more_buffer_sets_than_cached_descriptor_sets():
+    """The TMA descriptors of (W, G) pointer arrays are cached; a run that shows more distinct gradient buffers
+    than the cache holds (sets get overwritten and come back) gives the bits of a run that always passes the same
+    buffer."""
+    w = wl.tiny_workload([(136, 264), (264, 136)], r=16, s=3, T=0, inner_rank=4, index=89)
+    dev = torch.device("cuda")
+    steps = 80
+    grads = _grads(w, 40, dev)                               # 40 distinct buffer sets, cycled twice
+    a, b = _make(w), _make(w)
+    a.refresh_subspace(grads[0])
+    for i in range(2):
+        b.set_subspace(i, a.get_subspace(i))
+    Wa = [torch.zeros((M, N), device=dev) for _, M, N in w.shapes]
+    Wb = [torch.zeros((M, N), device=dev) for _, M, N in w.shapes]
+    fixed = [torch.empty_like(g) for g in grads[0]]
+    for k in range(steps):
+        a.step(Wa, grads[k % 40])
+        for f, g in zip(fixed, grads[k % 40]):
+            f.copy_(g)
+        b.step(Wb, fixed)
+    torch.cuda.synchronize()
+    assert all(torch.equal(x, y) for x, y in zip(Wa, Wb))
+    assert a.poll_status()[0] == 0 and b.poll_status()[0] == 0

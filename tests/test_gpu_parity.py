@@ -290,3 +290,19 @@ def test_step_replays_from_a_cuda_graph():
         for a, b in zip(Wa, Wb):
             assert rel_err(b.cpu().numpy(), a.cpu().numpy()) <= 1e-6
     assert eager.poll_status()[0] == 0 and graphed.poll_status()[0] == 0
+
+
+def test_full_wrapping_ring_of_sixteen_on_the_default_path():
+    """s = 16 with more steps than slots on the default path (tensor-core GEMMs, fused stream kernel, default
+    options): the Gram tiles of the 16-slot instantiation of the stream kernel run with every slot held and the
+    ring position wrapping, on shapes with several stream tiles and ragged tails, r = 128.  T = 30 puts the only
+    refresh at step 0."""
+    shapes = [(512, 768), (640, 1000), (1376, 512), (200, 264), (512, 4096)]
+    w = wl.tiny_workload(shapes, r=128, s=16, T=30, inner_rank=8, index=95)
+    for mode in ("B", "A"):
+        opt = _make(w, T=w.T if mode == "B" else 0)
+        errs, _, _ = run_side_by_side(opt, w, 22, mode)
+        _assert_errs(errs)
+        worst_full = max(max(row.values()) for row in errs[16:])
+        print(f"16-slot ring, mode {mode}, steps 16..21 (full, wrapping): worst relative update error {worst_full:.2e}")
+        assert opt.poll_status()[0] == 0

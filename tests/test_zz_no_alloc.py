@@ -9,13 +9,15 @@ that both produce the same natural gradient, on several calls in a row (the call
 How the comparison works: with M = r (so P can be the identity), beta1 = beta2 = 0 and lr = 1 the step
 writes W = -N~ / sqrt(N~^2 + eps) into a zeroed W, where N~ is the natural gradient of the current
 low-rank gradient R = G; the static entry point returns N~ itself from a caller-kept history ring.
+The same N~ is also computed by the fp64 oracle from a host copy of that ring and compared directly.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import natural_galore as orc
 from paper_2410_16029_b200 import workload as wl
-from tests.parity_util import TOL_UPDATE, to_device_bf16
+from tests.parity_util import TOL_UPDATE, rel_err, to_device_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -46,6 +48,10 @@ def test_static_natural_gradient_matches_step_on_consecutive_calls():
         err = (torch.linalg.norm(W.double() - expect) / torch.linalg.norm(expect)).item()
         assert err <= TOL_UPDATE, (k, err)
         assert status.item() == 0
+        # directly against the oracle: F^-1 applied to the newest gradient over the gradients the ring holds
+        ring = H.double().cpu().numpy()
+        want = orc.natural_gradient(ring[cur], [ring[j] for j in range(count)], lam)
+        assert rel_err(out.double().cpu().numpy(), want) <= TOL_UPDATE, (k, rel_err(out.double().cpu().numpy(), want))
     assert opt.poll_status()[0] == 0
 
 
