@@ -96,6 +96,17 @@ typedef struct {
                                        32) it is formed in the epilogue of the projection GEMM instead, so that the
                                        first read of the history runs under the tensor-core work; same results to
                                        rounding.  Not faster than the default as built, hence off unless asked for. */
+  int32_t ritz_columns;             /* the eigensolve at the end of a refresh rotates the leading ritz_columns
+                                       columns of the refreshed basis into Ritz vectors (approximate singular
+                                       vectors, in falling order of their singular value) within their own span; the
+                                       remaining columns complete an orthonormal basis of the subspace as the
+                                       subspace iteration left them.  0 (default): 256 (at most about a hundred
+                                       singular values can be separated from both neighbours by 1e-2 sigma_1, and the
+                                       iteration orders its basis by strength, so the determined singular vectors sit
+                                       at the front; a weak one close to the noise level is still spread over a few
+                                       hundred columns of an unconverged basis, which is why the default is not
+                                       smaller); -1: all r' columns (the full Rayleigh-Ritz step, about 2.5 times the
+                                       refresh time at r' = 512). */
 } ngalore_options;
 
 /*

@@ -78,6 +78,11 @@ struct ngalore_state {
   std::vector<int> refresh_tc_idx, refresh_plain_idx;
   std::vector<const uint16_t*> refresh_tc_G;
   CholProblem* d_chol = nullptr;
+  // Rayleigh-Ritz rotation of the plain refresh path: X of the Jacobi kernels lives in Xa, V (fp64) in C
+  JacobiMat* d_jac = nullptr;
+  JacobiInit* d_jac_init = nullptr;
+  JacobiOut* d_jac_out = nullptr;
+  JacobiSlot* d_jac_slots = nullptr;   // one matrix's worth (the plain path diagonalises the matrices one by one)
   int64_t k = 0;
   int64_t n_appended = 0;
   bool has_subspace = false;         // every matrix has a projector
@@ -249,6 +254,11 @@ ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bo
   return NGALORE_OK;
 }
 
+// Leading columns of the basis that the Rayleigh-Ritz rotation turns into Ritz vectors (see ritz_jacobi.cuh).
+inline int ritz_columns(const ngalore_state* st) {
+  return st->opt.ritz_columns == 0 ? 256 : (st->opt.ritz_columns < 0 ? (1 << 20) : st->opt.ritz_columns);
+}
+
 // Plain SIMT refresh (debug path, and single-matrix refreshes).
 ngalore_status refresh_simt(ngalore_state* st, const uint16_t* const* G, const std::vector<int>& idx, int q,
                             cudaStream_t stream) {
@@ -273,6 +283,39 @@ ngalore_status refresh_simt(ngalore_state* st, const uint16_t* const* G, const s
     if ((rc = orthonormalise(st, idx, 0, true, stream))) return rc;
   }
   // Second pass Yb -> Ya so that a clamped pivot of the first pass cannot leave P non-orthonormal.
+  if ((rc = orthonormalise(st, idx, 0, false, stream))) return rc;
+  // Rayleigh-Ritz rotation (Sec. 1: P holds the singular vectors): Z = G^T Q into Xa, C = Z^T Z (fp64) into C,
+  // eigenvectors V of C by Jacobi rotations (X in Xa; V, fp64, takes over the memory of C once C has been read),
+  // V with its columns in falling order of the eigenvalue into Xb (as fp32), Yb = Ya V, and a last
+  // orthonormalisation Yb -> Ya (its triangular factor is the identity to about 1e-6, so the columns keep their
+  // directions).
+  if ((rc = apply_gradient(st, idx, G, 1, BUF_YA, BUF_XA, stream))) return rc;
+  for (int i : idx) {
+    const HostMat& hm = st->mats[i];
+    SimtGemm g{};
+    g.m = hm.rp; g.n = hm.rp; g.k = hm.eN;
+    g.A = hm.Xa; g.a_rs = 1; g.a_cs = hm.rp; g.a_dt = DT_F32;
+    g.B = hm.Xa; g.b_rs = hm.rp; g.b_cs = 1; g.b_dt = DT_F32;
+    g.C = hm.C; g.c_rs = hm.rp; g.c_cs = 1; g.c_dt = DT_F64;
+    g.epilogue = EPI_STORE;
+    NG_CUDA(launch_simt_gemm<double>(g, stream));
+    st->launches += 1;
+    jacobi_init_kernel<<<1, 256, 0, stream>>>(st->d_jac + i, st->d_jac_init + i);
+    st->launches += 1;
+    const int Lj = std::min(hm.rp, ritz_columns(st));
+    NG_CUDA(jacobi_batched_launch(st->d_jac + i, 1, jacobi_blocks(Lj), (Lj + 3) & ~3, st->d_jac_slots, stream, &st->launches));
+    jacobi_finish_kernel<<<dim3(1, kJacFinishSplit), 256, 0, stream>>>(st->d_jac + i, st->d_jac_out + i);
+    st->launches += 1;
+    SimtGemm a{};
+    a.m = hm.eM; a.n = hm.rp; a.k = hm.rp;
+    a.A = hm.Ya; a.a_rs = hm.rp; a.a_cs = 1; a.a_dt = DT_F32;
+    a.B = hm.Xb; a.b_rs = hm.rp; a.b_cs = 1; a.b_dt = DT_F32;  // the sorted eigenvectors
+    a.C = hm.Yb; a.c_rs = hm.rp; a.c_cs = 1; a.c_dt = DT_F32;
+    a.epilogue = EPI_STORE;
+    NG_CUDA(launch_simt_gemm<float>(a, stream));
+    st->launches += 1;
+  }
+  NG_CUDA(cudaGetLastError());
   if ((rc = orthonormalise(st, idx, 0, false, stream))) return rc;
   return finish_refresh(st, idx, true, stream, idx.size() == static_cast<size_t>(st->n));
 }
@@ -458,6 +501,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (opt != nullptr && (opt->projection_rule < 0 || opt->projection_rule > 1)) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && (opt->history_bf16 < 0 || opt->history_bf16 > 1)) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && (opt->gram_fusion < 0 || opt->gram_fusion > 1)) return NGALORE_ERR_INVALID_ARG;
+  if (opt != nullptr && opt->ritz_columns < -1) return NGALORE_ERR_INVALID_ARG;
   // the bf16 history lives in the fused stream kernel only
   if (opt != nullptr && opt->history_bf16 == 1 && (s < 1 || opt->stream_impl == 1)) return NGALORE_ERR_INVALID_ARG;
 
@@ -556,6 +600,13 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   const size_t o_desc = take(sizeof(MatDesc) * n_matrices);
   const size_t o_chol = take(sizeof(CholProblem) * n_matrices);
   const size_t o_flags = take(sizeof(int) * 2 * n_matrices);
+  const size_t o_jac = take(sizeof(JacobiMat) * n_matrices);
+  const size_t o_jac_init = take(sizeof(JacobiInit) * n_matrices);
+  const size_t o_jac_out = take(sizeof(JacobiOut) * n_matrices);
+  const size_t o_jac_flags = take(sizeof(int) * 2 * n_matrices);
+  int jac_tables = 1;
+  for (const HostMat& hm : st->mats) jac_tables = std::max(jac_tables, jacobi_blocks(std::min(hm.rp, ritz_columns(st))) / 2);
+  const size_t o_jac_slots = take(sizeof(JacobiSlot) * jac_tables);
   int n_tiles = 0;
   std::vector<StreamTile> tiles;
   std::vector<int> tile0(n_matrices), ntl(n_matrices);
@@ -573,7 +624,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     woffs[i].Yb = take(sizeof(float) * hm.eM * hm.rp);
     woffs[i].Xa = take(sizeof(float) * hm.eN * hm.rp);
     woffs[i].Xb = take(sizeof(float) * hm.eN * hm.rp);
-    woffs[i].C = take(sizeof(double) * hm.rp * hm.rp);
+    woffs[i].C = take(sizeof(double) * hm.rp * ((hm.rp + 3) / 4 * 4));
     woffs[i].Gt = hm.right ? take(sizeof(uint16_t) * hm.N * hm.eN) : 0;
   }
   st->n_tiles = n_tiles;
@@ -598,6 +649,13 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   st->d_tiles = reinterpret_cast<StreamTile*>(st->work + o_tiles);
   int* flags = reinterpret_cast<int*>(st->work + o_flags);
   st->d_flags = flags;
+  st->d_jac = reinterpret_cast<JacobiMat*>(st->work + o_jac);
+  st->d_jac_init = reinterpret_cast<JacobiInit*>(st->work + o_jac_init);
+  st->d_jac_out = reinterpret_cast<JacobiOut*>(st->work + o_jac_out);
+  st->d_jac_slots = reinterpret_cast<JacobiSlot*>(st->work + o_jac_slots);
+  std::vector<JacobiMat> jac(n_matrices);
+  std::vector<JacobiInit> jac_init(n_matrices);
+  std::vector<JacobiOut> jac_out(n_matrices);
   st->subspace_set.assign(n_matrices, 0);
 
   st->h_desc.resize(n_matrices);
@@ -638,13 +696,23 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     hm.C = reinterpret_cast<double*>(st->work + woffs[i].C);
     if (hm.right) hm.Gt = reinterpret_cast<uint16_t*>(st->work + woffs[i].Gt);
     chol[i].C = hm.C; chol[i].L = hm.rp; chol[i].pad = 0; chol[i].tiny = 0.0;
+    // eN >= r' and a multiple of 8, so r' rows of ld <= eN floats fit in the eN x r' floats of Xa; V (r' x ld
+    // doubles) takes over C, which is allocated with that leading dimension
+    const int Lj = std::min(hm.rp, ritz_columns(st));
+    jac[i] = JacobiMat{hm.Xa, hm.C, Lj, (Lj + 3) & ~3, jacobi_blocks(Lj),
+                       reinterpret_cast<int*>(st->work + o_jac_flags) + 2 * i};
+    jac_init[i] = JacobiInit{nullptr, hm.C, hm.rp};
+    jac_out[i] = JacobiOut{hm.Xb, hm.rp, nullptr, nullptr, 0, hm.rp};
     if (s == 0 && cudaMemcpy(d.wsol, w_init.data(), sizeof(float) * kMaxHistory, cudaMemcpyHostToDevice) != cudaSuccess)
       return fail(NGALORE_ERR_CUDA);
   }
   if (cudaMemcpy(st->d_desc, st->h_desc.data(), sizeof(MatDesc) * n_matrices, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(st->d_chol, chol.data(), sizeof(CholProblem) * n_matrices, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(st->d_tiles, tiles.data(), sizeof(StreamTile) * n_tiles, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemcpy(st->d_hyper, &st->hyper, sizeof(Hyper), cudaMemcpyHostToDevice) != cudaSuccess)
+      cudaMemcpy(st->d_hyper, &st->hyper, sizeof(Hyper), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(st->d_jac, jac.data(), sizeof(JacobiMat) * n_matrices, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(st->d_jac_init, jac_init.data(), sizeof(JacobiInit) * n_matrices, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(st->d_jac_out, jac_out.data(), sizeof(JacobiOut) * n_matrices, cudaMemcpyHostToDevice) != cudaSuccess)
     return fail(NGALORE_ERR_CUDA);
   st->hyper_dirty = false;
 
@@ -653,7 +721,9 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   for (const HostMat& hm : st->mats) max_rp = hm.rp > max_rp ? hm.rp : max_rp;
   if (orth_apply_smem_bytes(max_rp) > static_cast<size_t>(prop.sharedMemPerBlockOptin)) return fail(NGALORE_ERR_INVALID_ARG);
   if (cudaFuncSetAttribute(orth_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(orth_apply_smem_bytes(max_rp))) != cudaSuccess)
+                           static_cast<int>(orth_apply_smem_bytes(max_rp))) != cudaSuccess ||
+      cudaFuncSetAttribute(jacobi_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(jacobi_smem_bytes(kJacMaxL))) != cudaSuccess)
     return fail(NGALORE_ERR_CUDA);
 
   const bool allow_gram_fusion = st->opt.gemm_impl != 1 && st->opt.stream_impl != 1 && !hist16 && st->opt.gram_fusion == 1;
@@ -675,7 +745,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
       eff.back().M = st->mats[i].eM; eff.back().N = st->mats[i].eN;
     }
     if (!eff.empty()) {
-      rc = refresh_plan_create(st->refresh, eff, Yf, Zf, prop.multiProcessorCount);
+      rc = refresh_plan_create(st->refresh, eff, Yf, Zf, prop.multiProcessorCount, ritz_columns(st));
       if (rc != NGALORE_OK) return fail(rc);
     }
   }

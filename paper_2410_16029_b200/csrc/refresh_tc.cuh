@@ -9,7 +9,9 @@
 // is added before the fp64 Cholesky factorisation so that the fp32 accumulation error cannot make it
 // indefinite, and
 // Q = Y R^-1 is again a tensor-core GEMM with R^-1 split in two bf16 parts.  The last basis is then
-// orthonormalised exactly (Gram, Cholesky and triangular solve in fp64) by the caller.
+// orthonormalised exactly (Gram, Cholesky and triangular solve in fp64), rotated to the Ritz vectors of G inside
+// the subspace (Z = G^T Q, eigenvectors V of Z^T Z by the Jacobi kernels of ritz_jacobi.cuh, P = Q V on the tensor
+// cores, columns in falling order of their singular value) and orthonormalised once more.
 #pragma once
 
 #include <cstring>
@@ -17,6 +19,7 @@
 
 #include "gemm_tcgen05.cuh"
 #include "kernels_refresh.cuh"
+#include "ritz_jacobi.cuh"
 
 namespace ngalore {
 
@@ -102,19 +105,22 @@ __host__ __device__ inline double gram_shift(int L) { return static_cast<double>
 // One CTA per matrix: C64 = D^-1 ((C32 + C32^T) / 2) D^-1 + shift I with D = diag(sqrt(C_ii)).
 // Scaling the columns to unit norm first makes the shift act on every column alike, whatever its
 // norm, so weak directions are still orthogonalised against each other and re-normalised.
+// (blockIdx.y shares the entries of a matrix among several CTAs; each of them forms the column norms for itself)
 __global__ void __launch_bounds__(256) gram_prep_kernel(const GramPrep* probs, double shift_scale) {
+  __shared__ double Ds[880];
   const GramPrep p = probs[blockIdx.x];
   for (int i = threadIdx.x; i < p.L; i += 256) {
     const double c = static_cast<double>(p.C32[static_cast<long long>(i) * p.L + i]);
-    p.D[i] = sqrt(fmax(c, 1e-60));
+    Ds[i] = sqrt(fmax(c, 1e-60));
+    if (blockIdx.y == 0) p.D[i] = Ds[i];
   }
   __syncthreads();
   const long long total = static_cast<long long>(p.L) * p.L;
-  for (long long x = threadIdx.x; x < total; x += 256) {
+  for (long long x = blockIdx.y * 256 + threadIdx.x; x < total; x += 256ll * gridDim.y) {
     const int i = static_cast<int>(x / p.L), j = static_cast<int>(x % p.L);
     if (j > i) continue;
     double v = 0.5 * (static_cast<double>(p.C32[x]) + static_cast<double>(p.C32[static_cast<long long>(j) * p.L + i]));
-    v /= p.D[i] * p.D[j];
+    v /= Ds[i] * Ds[j];
     if (i == j) v = 1.0 + shift_scale * gram_shift(p.L);
     p.C64[x] = v;
   }
@@ -300,17 +306,53 @@ __global__ void __launch_bounds__(256) tri_gemm_kernel(const TriGemm* probs) {
   }
 }
 
-// R^-1 = D^-1 X^T (upper triangular) split into two bf16 parts; one CTA per matrix.
+// R^-1 = D^-1 X^T (upper triangular) split into two bf16 parts; blockIdx.x = matrix, blockIdx.y = share of its entries.
 __global__ void __launch_bounds__(256) tri_convert_kernel(const TriInverse* probs) {
   const TriInverse p = probs[blockIdx.x];
   const long long total = static_cast<long long>(p.L) * p.L;
-  for (long long x = threadIdx.x; x < total; x += 256) {
+  for (long long x = blockIdx.y * 256 + threadIdx.x; x < total; x += 256ll * gridDim.y) {
     const int j = static_cast<int>(x / p.L), i = static_cast<int>(x % p.L);  // entry (j, i) of R^-1
     const double v = (i >= j) ? p.X[static_cast<long long>(i) * p.L + j] / p.D[j] : 0.0;
     const float f = static_cast<float>(fmin(fmax(v, -1e30), 1e30));
     const __nv_bfloat16 h = __float2bfloat16_rn(f);
     p.Rhi[static_cast<long long>(j) * p.ld + i] = h;
     p.Rlo[static_cast<long long>(j) * p.ld + i] = __float2bfloat16_rn(f - __bfloat162float(h));
+  }
+}
+
+// Scale every column of Y (rows x L, fp32) to unit norm, the norm summed in fp64.  The products of the refresh go
+// through operands split in two bf16 parts; the rounding of the diagonal of a triangular factor or of a rotation
+// (a relative 2^-17) scales a whole column, which is the largest part of what the last product leaves of
+// non-orthonormality.  Block (32, 8): blockIdx.x = strip of 32 columns, blockIdx.y = matrix.
+struct NormJob {
+  float* Y;
+  int rows, L;
+};
+
+__global__ void __launch_bounds__(256) normalize_columns_kernel(const NormJob* jobs) {
+  __shared__ double part[8][33];
+  __shared__ float scale[32];
+  const NormJob jb = jobs[blockIdx.y];
+  const int col = blockIdx.x * 32 + threadIdx.x;
+  if (blockIdx.x * 32 >= jb.L) return;
+  double s = 0.0;
+  if (col < jb.L)
+    for (int r = threadIdx.y; r < jb.rows; r += 8) {
+      const double v = static_cast<double>(jb.Y[static_cast<long long>(r) * jb.L + col]);
+      s += v * v;
+    }
+  part[threadIdx.y][threadIdx.x] = s;
+  __syncthreads();
+  if (threadIdx.y == 0) {
+    double t = 0.0;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) t += part[g][threadIdx.x];
+    scale[threadIdx.x] = t > 0.0 ? static_cast<float>(1.0 / sqrt(t)) : 0.f;
+  }
+  __syncthreads();
+  if (col < jb.L) {
+    const float f = scale[threadIdx.x];
+    for (int r = threadIdx.y; r < jb.rows; r += 8) jb.Y[static_cast<long long>(r) * jb.L + col] *= f;
   }
 }
 
@@ -373,6 +415,13 @@ struct RefreshPlan {
   int n_syrk_tiles = 0;
   GramPrep64* d_prep64 = nullptr;
   SplitJob* d_split_z = nullptr;
+  // Rayleigh-Ritz rotation: the Jacobi kernels work in the T64 (X, fp32) and X64 (V, fp64) buffers
+  JacobiMat* d_jac = nullptr;
+  JacobiInit* d_jac_init = nullptr;
+  JacobiOut* d_jac_out = nullptr;
+  JacobiSlot* d_jac_slots = nullptr;
+  int jac_nblk_max = 0, jac_ld_max = 0;
+  NormJob* d_norm = nullptr;
 };
 
 inline void refresh_plan_destroy(RefreshPlan& plan) {
@@ -386,7 +435,8 @@ inline void refresh_plan_destroy(RefreshPlan& plan) {
 }
 
 inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<MatDesc>& mats,
-                                          const std::vector<float*>& Yf, const std::vector<float*>& Zf, int sm_count) {
+                                          const std::vector<float*>& Yf, const std::vector<float*>& Zf, int sm_count,
+                                          int ritz_columns) {
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || fn == nullptr)
@@ -495,6 +545,14 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   const size_t o_prep64 = take(sizeof(GramPrep64) * n);
   const size_t o_sy = take(sizeof(SplitJob) * n);
   const size_t o_sz = take(sizeof(SplitJob) * n);
+  const size_t o_jac = take(sizeof(JacobiMat) * n);
+  const size_t o_jac_init = take(sizeof(JacobiInit) * n);
+  const size_t o_jac_out = take(sizeof(JacobiOut) * n);
+  const size_t o_norm = take(sizeof(NormJob) * n);
+  const size_t o_jac_flags = take(sizeof(int) * 2 * n);
+  int nblk_max_all = 2;
+  for (int i = 0; i < n; ++i) nblk_max_all = std::max(nblk_max_all, jacobi_blocks(std::min(mats[i].rp, (ritz_columns + 3) & ~3)));
+  const size_t o_jac_slots = take(sizeof(JacobiSlot) * n * (nblk_max_all / 2));
   if (cudaMalloc(&plan.buf, off) != cudaSuccess) { plan.buf = nullptr; return NGALORE_ERR_ALLOC; }
   if (cudaMemset(plan.buf, 0, off) != cudaSuccess) return NGALORE_ERR_CUDA;
   plan.device_bytes = off;
@@ -507,6 +565,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   std::vector<SplitJob> sy(n), sz(n);
   std::vector<SyrkMat> syrk_m(n);
   std::vector<GramPrep64> prep64(n);
+  std::vector<JacobiMat> jac(n);
+  std::vector<JacobiInit> jac_init(n);
+  std::vector<JacobiOut> jac_out(n);
+  std::vector<NormJob> norm(n);
   plan.h_maps.resize(static_cast<size_t>(RM_COUNT) * n);
   std::memset(plan.h_maps.data(), 0, sizeof(CUtensorMap) * plan.h_maps.size());
   for (int i = 0; i < n; ++i) {
@@ -529,6 +591,16 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     prep64[i] = GramPrep64{m.X64, m.C64, m.D, m.L};
     sy[i] = SplitJob{m.Yf, m.Yhi, m.Ylo, static_cast<long long>(m.M) * m.L, m.L, m.ldl};
     sz[i] = SplitJob{m.Zf, m.Zhi, m.Zlo, static_cast<long long>(m.N) * m.L, m.L, m.ldl};
+    // the Jacobi rotation keeps X (fp32) in the memory of T64 and V (fp64) in X64 (L is a multiple of 4 on this path)
+    // (width of the rotated part: all of the basis, or its leading ritz_columns, kept a multiple of 4)
+    const int Lj = std::min(m.L, (ritz_columns + 3) & ~3);
+    jac[i] = JacobiMat{reinterpret_cast<float*>(m.T64), m.X64, Lj, Lj, jacobi_blocks(Lj),
+                       reinterpret_cast<int*>(plan.buf + o_jac_flags) + 2 * i};
+    norm[i] = NormJob{m.Yf, m.M, m.L};
+    jac_init[i] = JacobiInit{m.C32, nullptr, m.L};
+    jac_out[i] = JacobiOut{nullptr, 0, m.Rhi, m.Rlo, m.ldl, m.L};
+    plan.jac_nblk_max = std::max(plan.jac_nblk_max, jac[i].nblk);
+    plan.jac_ld_max = std::max(plan.jac_ld_max, Lj);
     CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * RM_COUNT];
     const uint64_t sl = static_cast<uint64_t>(m.ldl) * 2;
     bool ok = true;
@@ -626,6 +698,11 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   plan.d_syrk_tiles = reinterpret_cast<SyrkTile*>(plan.buf + o_syrk_t);
   plan.d_prep64 = reinterpret_cast<GramPrep64*>(plan.buf + o_prep64);
   plan.d_split_z = reinterpret_cast<SplitJob*>(plan.buf + o_sz);
+  plan.d_jac = reinterpret_cast<JacobiMat*>(plan.buf + o_jac);
+  plan.d_jac_init = reinterpret_cast<JacobiInit*>(plan.buf + o_jac_init);
+  plan.d_jac_out = reinterpret_cast<JacobiOut*>(plan.buf + o_jac_out);
+  plan.d_norm = reinterpret_cast<NormJob*>(plan.buf + o_norm);
+  plan.d_jac_slots = reinterpret_cast<JacobiSlot*>(plan.buf + o_jac_slots);
   if (cudaMemcpy(plan.d_prep, prep.data(), sizeof(GramPrep) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_chol, chol.data(), sizeof(CholProblem) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_tri, tri.data(), sizeof(TriInverse) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -633,7 +710,11 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
       cudaMemcpy(plan.d_syrk_tiles, syrk_tiles.data(), sizeof(SyrkTile) * syrk_tiles.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_prep64, prep64.data(), sizeof(GramPrep64) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_split_y, sy.data(), sizeof(SplitJob) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
-      cudaMemcpy(plan.d_split_z, sz.data(), sizeof(SplitJob) * n, cudaMemcpyHostToDevice) != cudaSuccess)
+      cudaMemcpy(plan.d_split_z, sz.data(), sizeof(SplitJob) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_jac, jac.data(), sizeof(JacobiMat) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_jac_init, jac_init.data(), sizeof(JacobiInit) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_jac_out, jac_out.data(), sizeof(JacobiOut) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_norm, norm.data(), sizeof(NormJob) * n, cudaMemcpyHostToDevice) != cudaSuccess)
     return NGALORE_ERR_CUDA;
 
   // ---- tables of buffers to clear
@@ -682,6 +763,9 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
                            cudaFuncAttributeMaxDynamicSharedMemorySize, L2::kTotal) != cudaSuccess ||
       cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 2, 2, kRefStages2, TC_EPI_STORE, 4, true>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, L2::kTotal) != cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  if (cudaFuncSetAttribute(jacobi_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(jacobi_smem_bytes(kJacMaxL))) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   plan.ready = true;
   return NGALORE_OK;
@@ -733,7 +817,7 @@ inline ngalore_status refresh_tc_tri_inverse(RefreshPlan& plan, cudaStream_t str
     tri_gemm_kernel<<<dim3(tiles, tiles, plan.n_tg[h]), 256, 0, stream>>>(plan.d_tg2[h]);
     *launches += 2;
   }
-  tri_convert_kernel<<<plan.n, 256, 0, stream>>>(plan.d_tri);
+  tri_convert_kernel<<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_tri);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
@@ -750,7 +834,7 @@ inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ct
   ngalore_status rc;
   if ((rc = refresh_tc_split(plan, y_side, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, y_side ? RG_GRAM_Y : RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
-  gram_prep_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep, shift_scale);
+  gram_prep_kernel<<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_prep, shift_scale);
   *launches += 1;
   if (chol_batched_launch(plan.d_chol, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
@@ -812,11 +896,31 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
     if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches))) return rc;
     if ((rc = refresh_tc_orth(plan, true, d_ctrl, stream, launches))) return rc;
   }
-  // twice: the basis that leaves the sweeps can be ill conditioned in its weak directions, and the bf16-pair
-  // product then carries its rounding amplified by that condition number; the second pass starts from a
-  // nearly orthonormal basis
+  // Exact orthonormalisation of the basis that leaves the sweeps, twice: the basis can be ill conditioned in its
+  // weak directions, so the product with the first triangular factor leaves it orthonormal to about 1e-5 only; the
+  // second pass starts from that and ends at about 1e-6.  The Rayleigh-Ritz step below relies on it (it solves
+  // C v = lambda v, not C v = lambda (Q^T Q) v, and what Q lacks in orthonormality goes into the Ritz vectors).
   if ((rc = refresh_tc_final(plan, d_ctrl, stream, launches))) return rc;
-  return refresh_tc_final(plan, d_ctrl, stream, launches);
+  if ((rc = refresh_tc_final(plan, d_ctrl, stream, launches))) return rc;
+  if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;
+  // Rayleigh-Ritz: Z = G^T Q, C = Z^T Z (tensor cores: its entries are good to about 2^-17 of the diagonal, far
+  // finer than the gaps that decide a Ritz vector), V = eigenvectors of C (or of its leading block, see
+  // ritz_jacobi.cuh), P = Q V.
+  if ((rc = refresh_tc_gemm(plan, RG_Z_FROM_Y, d_ctrl, stream, launches))) return rc;
+  if ((rc = refresh_tc_split(plan, false, stream, launches))) return rc;
+  if ((rc = refresh_tc_gemm(plan, RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
+  jacobi_init_kernel<<<plan.n, 256, 0, stream>>>(plan.d_jac, plan.d_jac_init);
+  *launches += 1;
+  if (jacobi_batched_launch(plan.d_jac, plan.n, plan.jac_nblk_max, plan.jac_ld_max, plan.d_jac_slots, stream, launches) !=
+      cudaSuccess)
+    return NGALORE_ERR_CUDA;
+  jacobi_finish_kernel<<<dim3(plan.n, kJacFinishSplit), 256, 0, stream>>>(plan.d_jac, plan.d_jac_out);
+  *launches += 1;
+  // Q orthonormal to about 1e-6 and V orthogonal: so is their product, once its columns are scaled back to unit norm
+  if ((rc = refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches))) return rc;
+  normalize_columns_kernel<<<dim3((plan.l_max + 31) / 32, plan.n), dim3(32, 8), 0, stream>>>(plan.d_norm);
+  *launches += 1;
+  return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
 }  // namespace ngalore
