@@ -326,18 +326,36 @@ def run_ours(args, wl):
     grad_bytes = sum(M * N * 2 for M, N in shapes)
     opt.refresh_subspace(pool[0])
 
-    def exchange():
+    groups_by_owner, comm = None, None
+    if parts is not None:
         Wall = [None] * len(full_shapes)
         for j, i in enumerate(parts[rank]):
             Wall[i] = Wt[j]
         for i, t in others.items():
             Wall[i] = t
-        sharding.exchange_updated(Wall, parts)
+        if args.exchange == "overlapped":
+            # the weight update in groups, each group on the wire as soon as it is done (sharding.exchange_overlapped)
+            opt.set_update_groups(args.update_groups)
+            mine_groups = [[parts[rank][j] for j in range(a, b)] for a, b in opt.update_groups()]
+            groups_by_owner = [None] * world
+            dist.all_gather_object(groups_by_owner, mine_groups)
+            comm = torch.cuda.Stream()
 
     def step(k):
+        if groups_by_owner is not None:
+            main = torch.cuda.current_stream()
+            before = torch.cuda.Event()
+            before.record(main)
+            comm.wait_event(before)
         opt.step_ptrs(Wp, Gp[k % pool_sets])
-        if parts is not None:
-            exchange()
+        if parts is None:
+            return
+        if groups_by_owner is None:
+            sharding.exchange_updated(Wall, parts)
+        else:
+            sharding.exchange_overlapped(Wall, groups_by_owner, wait_update=lambda g: opt.stream_wait_update(g, comm),
+                                         comm_stream=comm, wire=args.wire)
+            torch.cuda.current_stream().wait_stream(comm)
 
     def barrier():
         torch.cuda.synchronize()
@@ -506,6 +524,8 @@ def run_ours(args, wl):
            "data": "synthetic",
            "config": config_dict(args, wl, n, parts is not None),
            "launch": "cuda_graph" if use_graph else "stream", "ms_per_step_median": ms_median,
+           "exchange": None if parts is None else {"mode": args.exchange, "wire": args.wire,
+                                                   "update_groups": args.update_groups},
            "untimed_steps_before": fill + args.warmup, "state_bytes": opt.device_bytes,
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
            "step_roofline": step_roof,
@@ -545,6 +565,13 @@ def main():
     ap.add_argument("--launch", default="graph", choices=["graph", "stream"],
                     help="graph (default): every timed step is one replay of a CUDA graph captured from ngalore_step, one "
                          "graph per gradient set; stream: plain calls of ngalore_step")
+    ap.add_argument("--exchange", default="overlapped", choices=["overlapped", "after"],
+                    help="with --shard: overlapped (default): the weights are updated in groups and every group is "
+                         "broadcast by its owner while the next one is being updated; after: one broadcast per owner "
+                         "after the step")
+    ap.add_argument("--update-groups", type=int, default=4, help="with --shard --exchange overlapped: groups per rank")
+    ap.add_argument("--wire", default="fp32", choices=["fp32", "bf16"],
+                    help="with --shard --exchange overlapped: format of the weights on the wire")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -190,6 +190,21 @@ ngalore_status ngalore_state_export(ngalore_state* st, void* blob, size_t* bytes
 ngalore_status ngalore_state_import(ngalore_state* st, const void* blob, size_t bytes);
 
 /*
+ * Update groups (the paper's related work: optimizer-state sharding, where ranks exchange updated weights; also any
+ * consumer that wants the weights of the first layers before the last ones are done).  With n_groups >= 2 the
+ * back-projection + weight update of ngalore_step runs as n_groups launches over contiguous ranges of matrices of
+ * about equal size, and an event is recorded on the stepping stream after each.  ngalore_update_group_range gives
+ * the matrices [first, last) of group g; ngalore_stream_wait_update makes `stream` wait until the latest enqueued
+ * step has updated group g, so work on that stream (a copy, a collective, a forward pass) overlaps the update of
+ * the later groups.  n_groups <= 1 restores the single launch.  Synchronises the device; not meant for steps
+ * replayed from a CUDA graph (the events belong to the live stream).
+ */
+ngalore_status ngalore_set_update_groups(ngalore_state* st, int n_groups);
+int ngalore_num_update_groups(const ngalore_state* st);
+ngalore_status ngalore_update_group_range(const ngalore_state* st, int g, int* first, int* last);
+ngalore_status ngalore_stream_wait_update(ngalore_state* st, int g, void* stream);
+
+/*
  * Testing aid (no counterpart in the paper): in the next ngalore_step only, the solved weights of matrix
  * `matrix_index` are computed but not announced, and the tiles that wait for them give up after `polls` polls
  * (1 .. 1000000, about 100 ns each) instead of the default limit.  The step then ends normally with

@@ -105,6 +105,11 @@ struct ngalore_state {
   size_t stage_bytes = 0;
   std::vector<float*> stage_W;
   std::vector<uint16_t*> stage_G;
+  // update groups: the back-projection runs group by group and records an event after each, so that a consumer of
+  // the updated weights (an exchange between ranks, the next forward pass) can start on a group while the next
+  // one is still being updated
+  std::vector<int> upd_first;               // first matrix of every group, plus n (empty: one launch, no events)
+  std::vector<cudaEvent_t> ev_upd;
   // profiling
   bool profiling = false;
   cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -432,6 +437,8 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
       g.skip_flag = d.step_bad;
       NG_CUDA(launch_simt_gemm<float>(g, stream));
       st->launches += 1;
+      for (size_t ug = 0; ug + 1 < st->upd_first.size(); ++ug)
+        if (st->upd_first[ug + 1] == i + 1) NG_CUDA(cudaEventRecord(st->ev_upd[ug], stream));
     }
   } else if (grouped) {
     for (size_t g = 0; g + 1 < st->group_first.size(); ++g) {
@@ -440,6 +447,13 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
                                      st->d_hyper, stream, &st->launches)))
         return rc;
       NG_CUDA(cudaEventRecord(st->ev_w_done[g], stream));
+    }
+  } else if (st->upd_first.size() > 1) {
+    for (size_t ug = 0; ug + 1 < st->upd_first.size(); ++ug) {
+      if ((rc = tc_backproject_range(st->tc, st->upd_first[ug], st->upd_first[ug + 1], st->d_desc, st->d_ctrl,
+                                     st->d_hyper, stream, &st->launches)))
+        return rc;
+      NG_CUDA(cudaEventRecord(st->ev_upd[ug], stream));
     }
   } else {
     if ((rc = tc_backproject(st->tc, st->d_desc, st->d_ctrl, st->d_hyper, stream, &st->launches))) return rc;
@@ -765,6 +779,7 @@ void ngalore_destroy(ngalore_state* st) {
   refresh_plan_destroy(st->refresh);
   for (int e = 0; e < 4; ++e)
     if (st->ev[e]) cudaEventDestroy(st->ev[e]);
+  for (cudaEvent_t e : st->ev_upd) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : st->ev_w_in) if (e) cudaEventDestroy(e);
   for (cudaEvent_t e : st->ev_w_done) if (e) cudaEventDestroy(e);
   if (st->ev_begin) cudaEventDestroy(st->ev_begin);
@@ -1009,6 +1024,53 @@ ngalore_status ngalore_state_import(ngalore_state* st, const void* blob, size_t 
   NG_CUDA(cudaMemcpy(st->d_ctrl, &c, sizeof(Ctrl), cudaMemcpyHostToDevice));
   st->k = h.k; st->n_appended = h.n_appended; st->has_subspace = h.has_subspace != 0;
   st->subspace_set.assign(st->n, st->has_subspace ? 1 : 0);
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_set_update_groups(ngalore_state* st, int n_groups) {
+  if (st == nullptr || n_groups < 0 || n_groups > 4096) return NGALORE_ERR_INVALID_ARG;
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
+  NG_CUDA(cudaDeviceSynchronize());
+  for (cudaEvent_t e : st->ev_upd) if (e) cudaEventDestroy(e);
+  st->ev_upd.clear();
+  st->upd_first.clear();
+  if (n_groups <= 1) return NGALORE_OK;
+  // contiguous groups of about equal weight traffic
+  size_t total = 0;
+  for (const HostMat& hm : st->mats) total += static_cast<size_t>(hm.M) * hm.N;
+  const int want = n_groups < st->n ? n_groups : st->n;
+  st->upd_first.assign(1, 0);
+  size_t acc = 0;
+  for (int i = 0; i < st->n; ++i) {
+    acc += static_cast<size_t>(st->mats[i].M) * st->mats[i].N;
+    const size_t done = st->upd_first.size();
+    if (i + 1 < st->n && static_cast<int>(done) < want && acc * want >= total * done) st->upd_first.push_back(i + 1);
+  }
+  st->upd_first.push_back(st->n);
+  st->ev_upd.assign(st->upd_first.size() - 1, nullptr);
+  for (cudaEvent_t& e : st->ev_upd)
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { e = nullptr; return NGALORE_ERR_CUDA; }
+  return NGALORE_OK;
+}
+
+int ngalore_num_update_groups(const ngalore_state* st) {
+  return st == nullptr ? 0 : (st->upd_first.size() > 1 ? static_cast<int>(st->upd_first.size()) - 1 : 1);
+}
+
+ngalore_status ngalore_update_group_range(const ngalore_state* st, int g, int* first, int* last) {
+  if (st == nullptr || first == nullptr || last == nullptr || g < 0 || g >= ngalore_num_update_groups(st)) return NGALORE_ERR_INVALID_ARG;
+  if (st->upd_first.size() > 1) { *first = st->upd_first[g]; *last = st->upd_first[g + 1]; }
+  else { *first = 0; *last = st->n; }
+  return NGALORE_OK;
+}
+
+ngalore_status ngalore_stream_wait_update(ngalore_state* st, int g, void* stream) {
+  if (st == nullptr || g < 0 || g >= ngalore_num_update_groups(st)) return NGALORE_ERR_INVALID_ARG;
+  if (st->upd_first.size() <= 1) return NGALORE_ERR_INVALID_ARG;   // no groups: order by the stepping stream itself
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return NGALORE_ERR_CUDA;
+  NG_CUDA(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), st->ev_upd[g], 0));
   return NGALORE_OK;
 }
 

@@ -60,6 +60,14 @@ _lib.ngalore_state_export.restype = ctypes.c_int
 _lib.ngalore_state_export.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_size_t)]
 _lib.ngalore_state_import.restype = ctypes.c_int
 _lib.ngalore_state_import.argtypes = [_vp, _vp, ctypes.c_size_t]
+_lib.ngalore_set_update_groups.restype = ctypes.c_int
+_lib.ngalore_set_update_groups.argtypes = [_vp, ctypes.c_int]
+_lib.ngalore_num_update_groups.restype = ctypes.c_int
+_lib.ngalore_num_update_groups.argtypes = [_vp]
+_lib.ngalore_update_group_range.restype = ctypes.c_int
+_lib.ngalore_update_group_range.argtypes = [_vp, ctypes.c_int, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
+_lib.ngalore_stream_wait_update.restype = ctypes.c_int
+_lib.ngalore_stream_wait_update.argtypes = [_vp, ctypes.c_int, _vp]
 _lib.ngalore_debug_withhold_solution.restype = ctypes.c_int
 _lib.ngalore_debug_withhold_solution.argtypes = [_vp, ctypes.c_int, ctypes.c_int]
 _lib.ngalore_set_lr.restype = ctypes.c_int
@@ -209,6 +217,23 @@ class NGaLore:
 
     def import_state(self, blob: bytes):
         _check(_lib.ngalore_state_import(self._h, blob, len(blob)), "ngalore_state_import")
+
+    def set_update_groups(self, n_groups: int):
+        """Run the weight update in n_groups launches with an event after each (see include/ngalore.h)."""
+        _check(_lib.ngalore_set_update_groups(self._h, n_groups), "ngalore_set_update_groups")
+
+    def update_groups(self):
+        """[(first, last), ...]: the matrix ranges of the update groups (one range when groups are off)."""
+        out = []
+        for g in range(_lib.ngalore_num_update_groups(self._h)):
+            a, b = ctypes.c_int(0), ctypes.c_int(0)
+            _check(_lib.ngalore_update_group_range(self._h, g, ctypes.byref(a), ctypes.byref(b)), "ngalore_update_group_range")
+            out.append((a.value, b.value))
+        return out
+
+    def stream_wait_update(self, g: int, stream):
+        """Make `stream` (a torch.cuda.Stream) wait until the latest enqueued step has updated group g."""
+        _check(_lib.ngalore_stream_wait_update(self._h, g, ctypes.c_void_p(stream.cuda_stream)), "ngalore_stream_wait_update")
 
     def debug_withhold_solution(self, matrix_index: int, polls: int):
         """Testing aid: the next step does not announce matrix_index's solved weights (see include/ngalore.h)."""

@@ -311,3 +311,62 @@ def test_more_buffer_sets_than_cached_descriptor_sets():
     torch.cuda.synchronize()
     assert all(torch.equal(x, y) for x, y in zip(Wa, Wb))
     assert a.poll_status()[0] == 0 and b.poll_status()[0] == 0
+
+
+def test_update_groups_and_overlapped_exchange_with_one_rank():
+    """The weight update in groups with an event after each: same bits as the single launch; a side stream that waits
+    for group g sees that group's weights updated; the sharded wrapper with the overlapped exchange (one rank: it
+    owns everything) gives the bits of the plain optimizer."""
+    import os
+
+    import torch.distributed as dist
+
+    from paper_2410_16029_b200.sharding import ShardedNGaLore
+
+    w = wl.tiny_workload([(136, 264), (264, 136), (72, 40), (200, 96), (128, 512)], r=16, s=3, T=0, inner_rank=4, index=79)
+    dev = torch.device("cuda")
+    shapes = [(M, N) for _, M, N in w.shapes]
+    grads = _grads(w, 4, dev)
+    plain, grouped = _make(w), _make(w)
+    plain.refresh_subspace(grads[0])
+    for i in range(len(shapes)):
+        grouped.set_subspace(i, plain.get_subspace(i))
+    grouped.set_update_groups(3)
+    ranges = grouped.update_groups()
+    assert ranges[0][0] == 0 and ranges[-1][1] == len(shapes) and len(ranges) == 3
+    assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
+    Wa = [wl.initial_weight_device(w, i, dev) for i in range(len(shapes))]
+    Wb = [t.clone() for t in Wa]
+    side = torch.cuda.Stream()
+    copies = []
+    for k in range(4):
+        plain.step(Wa, grads[k])
+        grouped.step(Wb, grads[k])
+        for g, (a, b) in enumerate(ranges):
+            grouped.stream_wait_update(g, side)
+            with torch.cuda.stream(side):
+                copies = [Wb[i].clone() for i in range(a, b)]
+            torch.cuda.synchronize()
+            assert all(torch.equal(c, Wa[i]) for c, i in zip(copies, range(a, b))), (k, g)
+    assert all(torch.equal(x, y) for x, y in zip(Wa, Wb))
+    grouped.set_update_groups(0)
+    assert grouped.update_groups() == [(0, len(shapes))]
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29763")
+    dist.init_process_group("gloo", rank=0, world_size=1)
+    try:
+        kw = dict(lam=w.lam, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, wd=w.wd)
+        sharded = ShardedNGaLore(shapes, w.r, w.s, 0, update_groups=2, **kw)
+        ref = _make(w)
+        for i in range(len(shapes)):
+            ref.set_subspace(i, plain.get_subspace(i))
+            sharded.opt.set_subspace(i, plain.get_subspace(i))
+        Wc = [wl.initial_weight_device(w, i, dev) for i in range(len(shapes))]
+        Wd = [t.clone() for t in Wc]
+        for k in range(3):
+            ref.step(Wc, grads[k])
+            sharded.step(Wd, grads[k])
+        torch.cuda.synchronize()
+        assert all(torch.equal(x, y) for x, y in zip(Wc, Wd))
+    finally:
+        dist.destroy_process_group()

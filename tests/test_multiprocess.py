@@ -125,3 +125,70 @@ def test_two_ranks_exchange_their_shards():
     (ok0, parts0), (ok1, parts1) = got
     assert ok0 and ok1
     assert parts0 == parts1 and sorted(parts0[0] + parts0[1]) == [0, 1, 2, 3, 4]
+
+
+def _overlap_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    from paper_2410_16029_b200 import sharding
+
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    shapes = [(8, 16), (24, 8), (16, 16), (8, 8), (32, 8), (8, 24)]
+    parts = sharding.partition(shapes, 4, 2, world)
+    # each rank's matrices in two update groups, as the library would report them (contiguous in its own order)
+    groups = [[p[: (len(p) + 1) // 2], p[(len(p) + 1) // 2:]] for p in parts]
+    results = {}
+    for wire in ("fp32", "bf16"):
+        W = [torch.full(s, float(i)) + 0.001 * torch.arange(s[0] * s[1], dtype=torch.float32).reshape(s)
+             for i, s in enumerate(shapes)]
+        for i in parts[rank]:
+            W[i] += rank + 1                                   # the stand-in for this rank's optimizer step
+        expect = []
+        own = sharding.owners(parts, len(shapes))
+        for i, s in enumerate(shapes):
+            e = torch.full(s, float(i)) + 0.001 * torch.arange(s[0] * s[1], dtype=torch.float32).reshape(s) + own[i] + 1
+            if wire == "bf16" and own[i] != rank:
+                e = e.to(torch.bfloat16).to(torch.float32)     # the other ranks see the owner's weights rounded
+            expect.append(e)
+        log, waited = [], []
+        sharding.exchange_overlapped(W, groups, wait_update=lambda g: waited.append(g), wire=wire, log=log)
+        ok = all(torch.equal(a, b) for a, b in zip(W, expect))
+        results[wire] = (ok, log, waited)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, (results, groups))
+    if rank == 0:
+        out.put(gathered)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_overlapped_exchange_order_and_wire_formats():
+    """Two gloo ranks: the group-by-group exchange delivers every owner's weights (bit-exact in fp32, the owner's
+    bf16 rounding on the bf16 wire), every rank issues the collectives in the same order, and an owner waits for the
+    update event of a group before it packs that group, never for a later one."""
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_overlap_worker, args=(r, 2, 29751, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (res0, groups0), (res1, groups1) = got
+    assert groups0 == groups1
+    for wire in ("fp32", "bf16"):
+        ok0, log0, waited0 = res0[wire]
+        ok1, log1, waited1 = res1[wire]
+        assert ok0 and ok1
+        bcast0 = [e for e in log0 if e[0] == "bcast"]
+        bcast1 = [e for e in log1 if e[0] == "bcast"]
+        assert bcast0 == bcast1                                # same collectives, same order, on both ranks
+        assert bcast0 == [("bcast", src, g) for src in range(2) for g in range(2) if groups0[src][g]]
+        for rank, log, waited in ((0, log0, waited0), (1, log1, waited1)):
+            mine = [g for g in range(2) if groups0[rank][g]]
+            assert waited == mine                              # one wait per own group, in update order
+            for g in mine:                                     # wait -> pack -> broadcast for every own group
+                i = log.index(("wait", rank, g))
+                assert log[i + 1] == ("pack", rank, g) and log[i + 2] == ("bcast", rank, g)
+            assert all(e[1] != rank for e in log if e[0] == "unpack")
