@@ -26,7 +26,9 @@ the start of Sec. 2.4, that most steps are those of GaLore: project on the
 right, R = G Q with Q the first r' right singular vectors, when M >= N);
 r' = min(r, M, N); ``Hyper.history_bf16`` is the reduced-precision state the paper's
 conclusion names as future work: every stored gradient but the current one is
-rounded to bf16; the empirical Fisher is
+rounded to bf16; ``Hyper.moments_bf16`` is the same idea for the Adam moments: m is stored
+rounded to nearest, v with stochastic rounding from a counter-based generator (round to nearest
+would freeze v, whose relative change per step, 1 - beta2, is below half a bf16 unit); the empirical Fisher is
 the *mean* of outer products plus lambda I (the 1/h of the Sec. 2.2 definition
 carried into Sec. 2.4); exactly s columns, the current gradient among them;
 divide by the number of gradients actually held while the history fills; eps
@@ -157,6 +159,56 @@ def adam_moments(m, v, g, beta1, beta2, eps, *, step_index=0, bias_correction=Fa
     return m, v, u
 
 
+# ----------------------------------------------------------------------------- reduced-precision moments
+
+PHILOX_M0, PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+PHILOX_W0, PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32_10(counter: np.ndarray, key0: int, key1: int) -> np.ndarray:
+    """Philox-4x32 with ten rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3",
+    2011): counter (n, 4) uint32 -> (n, 4) uint32.  One round maps (c0, c1, c2, c3) to
+    (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)); the key is bumped by the Weyl constants
+    between rounds."""
+    c = np.asarray(counter, dtype=np.uint64).reshape(-1, 4).copy()
+    k0, k1 = np.uint64(key0 & 0xFFFFFFFF), np.uint64(key1 & 0xFFFFFFFF)
+    mask = np.uint64(0xFFFFFFFF)
+    for _ in range(10):
+        p0 = np.uint64(PHILOX_M0) * c[:, 0]
+        p1 = np.uint64(PHILOX_M1) * c[:, 2]
+        n0 = ((p1 >> np.uint64(32)) ^ c[:, 1] ^ k0) & mask
+        n1 = p1 & mask
+        n2 = ((p0 >> np.uint64(32)) ^ c[:, 3] ^ k1) & mask
+        n3 = p0 & mask
+        c = np.stack([n0, n1, n2, n3], axis=1)
+        k0 = (k0 + np.uint64(PHILOX_W0)) & mask
+        k1 = (k1 + np.uint64(PHILOX_W1)) & mask
+    return c.astype(np.uint32)
+
+
+def rounding_bits(n_elements: int, matrix_index: int, step_index: int, seed: int) -> np.ndarray:
+    """Sixteen random bits per element of a flattened array for the stochastic rounding of the second moment:
+    elements 4 g .. 4 g + 3 take the upper halves of the four words of Philox(counter = (g mod 2^32, g div 2^32,
+    matrix index, step index), key = (seed mod 2^32, seed div 2^32))."""
+    groups = (n_elements + 3) // 4
+    g = np.arange(groups, dtype=np.uint64)
+    ctr = np.stack([g & np.uint64(0xFFFFFFFF), g >> np.uint64(32),
+                    np.full(groups, matrix_index & 0xFFFFFFFF, dtype=np.uint64),
+                    np.full(groups, step_index & 0xFFFFFFFF, dtype=np.uint64)], axis=1)
+    words = philox4x32_10(ctr, seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)
+    return (words >> np.uint32(16)).reshape(-1)[:n_elements].astype(np.uint32)
+
+
+def stochastic_round_to_bf16(x: np.ndarray, bits16: np.ndarray) -> np.ndarray:
+    """Non-negative values rounded to bf16 up or down with probabilities in proportion to the distances: the
+    sixteen random bits are added below the sixteen bits that bf16 keeps of the float32 pattern, and the sum is
+    truncated.  Returned as float64."""
+    f = np.ascontiguousarray(x, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64).reshape(-1)
+    u = (u + bits16.astype(np.uint64).reshape(-1)) & np.uint64(0xFFFF0000)
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
 # ----------------------------------------------------------------------------- the optimizer state
 
 @dataclasses.dataclass
@@ -176,13 +228,16 @@ class Hyper:
     store_P_as_bf16: bool = True
     projection: str = "left"        # "left": always R = P^T G; "short_side": R = G Q when M >= N
     history_bf16: bool = False      # keep every low-rank gradient but the current one rounded to bf16
+    moments_bf16: bool = False      # store m (round to nearest) and v (stochastic rounding) as bf16
+    rounding_seed: int = 0x9E3779B97F4A7C15   # key of the generator behind the stochastic rounding
 
 
 class MatrixState:
     """Optimizer state of one M x N weight matrix."""
 
-    def __init__(self, M: int, N: int, hp: Hyper):
+    def __init__(self, M: int, N: int, hp: Hyper, matrix_index: int = 0):
         self.M, self.N, self.hp = M, N, hp
+        self.matrix_index = matrix_index      # position in the optimizer's matrix list (keys the rounding stream)
         self.rp = min(hp.r, M, N)
         if hp.projection not in ("left", "short_side"):
             raise ValueError(hp.projection)
@@ -243,6 +298,12 @@ class MatrixState:
         self.m, self.v, u = adam_moments(self.m, self.v, Nt, hp.beta1, hp.beta2, hp.eps,
                                          step_index=self.k, bias_correction=hp.bias_correction,
                                          eps_outside=hp.eps_outside)    # O6
+        if hp.moments_bf16:
+            # Reduced-precision moments: the direction u above came from the unrounded moments of this step;
+            # what the next step starts from is their bf16 storage.
+            self.m = round_to_bf16(self.m)
+            bits = rounding_bits(self.v.size, self.matrix_index, self.k, hp.rounding_seed)
+            self.v = stochastic_round_to_bf16(self.v, bits.reshape(self.v.shape))
         back = u @ self.P.T if self.right else self.P @ u
         dW = -hp.lr * back - hp.lr * hp.wd * W                          # O7
         W += dW

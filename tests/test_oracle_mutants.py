@@ -59,6 +59,13 @@ MUTANTS = [
      "slot = (self.head - 1) % hp.s", "slot = self.head % hp.s"),
     ("history and moments dropped at every refresh", "reset_history_on_refresh: bool = False", "reset_history_on_refresh: bool = True"),
     ("P kept unrounded", "store_P_as_bf16: bool = True", "store_P_as_bf16: bool = False"),
+    ("Philox with nine rounds", "    for _ in range(10):\n        p0 = np.uint64(PHILOX_M0) * c[:, 0]", "    for _ in range(9):\n        p0 = np.uint64(PHILOX_M0) * c[:, 0]"),
+    ("Philox round with the two multipliers swapped", "p0 = np.uint64(PHILOX_M0) * c[:, 0]", "p0 = np.uint64(PHILOX_M1) * c[:, 0]"),
+    ("rounding bits from the lower halves of the words", "return (words >> np.uint32(16)).reshape(-1)[:n_elements]", "return (words & np.uint32(0xFFFF)).reshape(-1)[:n_elements]"),
+    ("second moment rounded to nearest, not stochastically",
+     "self.v = stochastic_round_to_bf16(self.v, bits.reshape(self.v.shape))", "self.v = round_to_bf16(self.v)"),
+    ("stochastic rounding that always rounds down", "u = (u + bits16.astype(np.uint64).reshape(-1)) & np.uint64(0xFFFF0000)", "u = u & np.uint64(0xFFFF0000)"),
+    ("first moment left unrounded under moments_bf16", "            self.m = round_to_bf16(self.m)\n", "            pass\n"),
 ]
 
 

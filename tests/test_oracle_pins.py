@@ -489,3 +489,75 @@ def test_bf16_history_keeps_the_current_gradient_exact_and_rounds_the_rest():
         stored.append(orc.round_to_bf16(R))
         ring = [h for h in st.history()]
         assert all(np.array_equal(h, orc.round_to_bf16(h)) for h in ring)
+
+
+# ----------------------------------------------------------------------------- reduced-precision moments
+
+def test_philox_reproduces_the_published_known_answers():
+    """The generator behind the stochastic rounding against the known-answer vectors published with it."""
+    import os
+
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "philox4x32_10_kat.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 3
+    for row in rows:
+        words = [int(x, 16) for x in row]
+        got = orc.philox4x32_10(np.array([words[:4]], dtype=np.uint64), words[4], words[5])[0]
+        assert [int(x) for x in got] == words[6:], row
+
+
+def test_stochastic_rounding_picks_a_neighbour_with_the_right_odds():
+    """A value goes to one of its two bf16 neighbours, up with probability (x - down) / (up - down); a bf16 value
+    stays; the mean over many draws is the value itself."""
+    x = np.float32(1.0) + np.float32(2.0 ** -7) * np.float32(0.3)           # 30 % of the way from 1 to 1 + 2^-7
+    n = 200000
+    bits = orc.rounding_bits(n, matrix_index=3, step_index=11, seed=12345)
+    assert bits.dtype == np.uint32 and bits.max() < 65536 and bits.min() >= 0
+    out = orc.stochastic_round_to_bf16(np.full(n, x, dtype=np.float64), bits)
+    down, up = 1.0, 1.0 + 2.0 ** -7
+    assert set(np.unique(out)) == {down, up}
+    frac_up = float(np.mean(out == up))
+    assert abs(frac_up - 0.3) <= 4 * np.sqrt(0.3 * 0.7 / n) + 2.0 ** -15
+    assert abs(float(np.mean(out)) - float(x)) <= 5e-6
+    exact = np.array([0.5, 1.0, 1.0 + 2.0 ** -7, 3.0e-5], dtype=np.float64)
+    exact = orc.round_to_bf16(exact)
+    assert np.array_equal(orc.stochastic_round_to_bf16(exact, np.full(4, 65535, dtype=np.uint32)), exact)
+    # the bits of different steps, matrices and seeds are different streams; the same arguments give the same bits
+    a = orc.rounding_bits(64, 0, 0, 1)
+    assert np.array_equal(a, orc.rounding_bits(64, 0, 0, 1))
+    assert not np.array_equal(a, orc.rounding_bits(64, 0, 1, 1))
+    assert not np.array_equal(a, orc.rounding_bits(64, 1, 0, 1))
+    assert not np.array_equal(a, orc.rounding_bits(64, 0, 0, 2))
+    assert np.array_equal(orc.rounding_bits(61, 0, 0, 1), a[:61])
+
+
+def test_bf16_moments_store_rounded_values_and_the_second_moment_does_not_freeze():
+    """moments_bf16: the direction of a step comes from the unrounded moments, the state holds bf16 values
+    (m rounded to nearest), and v keeps following (1 - beta2) g^2 although one step changes it by less than half
+    a bf16 unit: its mean over many elements tracks the full-precision recursion, where rounding to nearest would
+    leave it at its starting value."""
+    M, N, r = 8, 4096, 8
+    hp16 = orc.Hyper(r=r, s=0, T=0, lr=1.0, beta1=0.9, beta2=0.999, eps=1e-8, moments_bf16=True, store_P_as_bf16=False)
+    hp32 = orc.Hyper(r=r, s=0, T=0, lr=1.0, beta1=0.9, beta2=0.999, eps=1e-8, store_P_as_bf16=False)
+    a, b = orc.MatrixState(M, N, hp16, matrix_index=2), orc.MatrixState(M, N, hp32)
+    for st in (a, b):
+        st.set_subspace(np.eye(M))
+    rng = np.random.default_rng(7)
+    G0 = rng.standard_normal((M, N))
+    # first step from zero moments: both see the same unrounded m, v, hence the same direction
+    dWa = a.step(np.zeros((M, N)), G0, auto_refresh=False)
+    dWb = b.step(np.zeros((M, N)), G0, auto_refresh=False)
+    assert np.array_equal(dWa, dWb)
+    assert np.array_equal(a.m, orc.round_to_bf16(b.m))
+    assert np.array_equal(a.v, orc.round_to_bf16(a.v)) and not np.array_equal(a.v, orc.round_to_bf16(b.v))
+    lo = np.floor(b.v / 2.0 ** np.floor(np.log2(b.v)) * 128) / 128 * 2.0 ** np.floor(np.log2(b.v))   # bf16 below
+    assert np.all((a.v == lo) | (a.v == lo + 2.0 ** (np.floor(np.log2(b.v)) - 7)))
+    # a long run with a gradient four times larger: v must climb towards 16 g0^2
+    for k in range(300):
+        a.step(np.zeros((M, N)), 4.0 * G0, auto_refresh=False)
+        b.step(np.zeros((M, N)), 4.0 * G0, auto_refresh=False)
+    ratio = float(np.sum(a.v) / np.sum(b.v))
+    assert abs(ratio - 1.0) <= 2e-3, ratio                      # unbiased: the totals agree
+    frozen = orc.round_to_bf16(1e-3 * G0 * G0)                  # what round-to-nearest would still hold
+    assert float(np.sum(b.v) / np.sum(frozen)) > 3.0            # the full-precision v has moved far from it
+    assert np.array_equal(a.m, orc.round_to_bf16(a.m))
