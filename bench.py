@@ -47,7 +47,8 @@ def config_dict(args, wl, n_matrices, sharded):
     """The workload and protocol of a run; both arms (CUDA path and oracle) describe the same one."""
     grad_bytes = sum(M * N * 2 for _, M, N in wl.shapes)
     return {"workload": wl.name, "matrices": n_matrices, "r": wl.r, "s": wl.s, "T": wl.T,
-            "projection": args.projection, "history": args.history, "gram_fusion": args.gram_fusion,
+            "projection": args.projection, "history": args.history, "moments": args.moments,
+            "gram_fusion": args.gram_fusion,
             "sharded": sharded, "history_filled": True, "refresh_in_timed_region": False,
             "l2": f"inputs larger than L2: {pool_size(args, wl)} gradient sets of {grad_bytes / 1e9:.2f} GB cycled"}
 
@@ -74,19 +75,20 @@ def low_rank_dims(wl, i, projection):
     return rp, (N if right else M), rp * (M if right else N)
 
 
-def byte_model(wl, projection="left", history="fp32"):
+def byte_model(wl, projection="left", history="fp32", moments="fp32"):
     """Algorithmic bytes per step: every datum moved once (G bf16, W fp32, P bf16, history/m/v fp32).
     With a bf16 history the s - 1 older gradients are 2 bytes each, the current one is written and read in
-    fp32, and its bf16 copy is written once."""
+    fp32, and its bf16 copy is written once.  With bf16 moments m and v are 2 bytes each way instead of 4."""
     tot = stream = 0
+    mom = 8 if moments == "bf16" else 16        # m and v, read and written
     for i, (_, M, N) in enumerate(wl.shapes):
         rp, pr, rn = low_rank_dims(wl, i, projection)
         if history == "bf16":
-            tot += 10 * M * N + 2 * pr * rp + (2 * wl.s + 24) * rn
-            stream += (2 * wl.s + 20) * rn      # older slots (bf16) + current (fp32) once, bf16 copy, m and v
+            tot += 10 * M * N + 2 * pr * rp + (2 * wl.s + 8 + mom) * rn
+            stream += (2 * wl.s + 4 + mom) * rn  # older slots (bf16) + current (fp32) once, bf16 copy, m and v
         else:
-            tot += 10 * M * N + 2 * pr * rp + (4 * wl.s + 20) * rn
-            stream += (4 * wl.s + 16) * rn      # history read once + m, v read and written
+            tot += 10 * M * N + 2 * pr * rp + (4 * wl.s + 4 + mom) * rn
+            stream += (4 * wl.s + mom) * rn      # history read once + m, v read and written
     return tot, stream
 
 
@@ -159,8 +161,8 @@ class OracleSampler:
     are made once per shape and kept; every timing starts from a fresh state whose history holds s
     gradients, the steady state of the optimizer."""
 
-    def __init__(self, wl, projection="left", history="fp32"):
-        self.wl, self.projection, self.history = wl, projection, history
+    def __init__(self, wl, projection="left", history="fp32", moments="fp32"):
+        self.wl, self.projection, self.history, self.moments = wl, projection, history, moments
         self.counts = {}
         for _, M, N in wl.shapes:
             self.counts[(M, N)] = self.counts.get((M, N), 0) + 1
@@ -171,7 +173,8 @@ class OracleSampler:
     def _hyper(self, orc):
         wl = self.wl
         return orc.Hyper(r=wl.r, s=wl.s, T=0, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
-                         projection=self.projection, history_bf16=self.history == "bf16")
+                         projection=self.projection, history_bf16=self.history == "bf16",
+                         moments_bf16=self.moments == "bf16")
 
     def time_shape(self, j, seed):
         """One oracle step on matrix shape j (history pre-filled); returns and records its seconds."""
@@ -209,9 +212,9 @@ class OracleSampler:
             return os.cpu_count()
 
 
-def oracle_sample(wl, projection="left", history="fp32"):
+def oracle_sample(wl, projection="left", history="fp32", moments="fp32"):
     """Time the oracle once on every distinct shape.  Returns (seconds per full step, description, threads)."""
-    smp = OracleSampler(wl, projection, history)
+    smp = OracleSampler(wl, projection, history, moments)
     for j in range(len(smp.shapes)):
         smp.time_shape(j, 0)
     desc = (f"one oracle step (full history of {wl.s}) on one matrix of each of the "
@@ -226,7 +229,7 @@ def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    smp = OracleSampler(wl, args.projection, args.history)
+    smp = OracleSampler(wl, args.projection, args.history, args.moments)
     n_shapes = len(smp.shapes)
     times = []
     for k in range(args.warmup + args.steps):
@@ -311,7 +314,7 @@ def run_ours(args, wl):
     # no refresh among them, whatever T is); the refresh is run once before them and timed alone further down.
     opt = NGaLore(shapes, wl.r, wl.s, 0, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
                   wd=wl.wd, seed=1 + rank, projection=args.projection, history_bf16=args.history == "bf16",
-                  gram_fusion=args.gram_fusion == "on")
+                  gram_fusion=args.gram_fusion == "on", moments_bf16=args.moments == "bf16")
     # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
     wl_rank = rank_workload(wl, rank)
     if parts is not None:
@@ -476,7 +479,7 @@ def run_ours(args, wl):
 
     # ---- roofline of the dominant kernel and of the whole step
     peak, tensor_peak, peak_kind = measured_peaks()
-    tot_bytes, stream_bytes = byte_model(wl, args.projection, args.history)
+    tot_bytes, stream_bytes = byte_model(wl, args.projection, args.history, args.moments)
     dims = [low_rank_dims(wl, i, args.projection) for i in range(n)]
     # the library runs the projection with 256-row tiles (tc_project2_kernel) where nearly all of the work has at
     # least 512 output rows and a long K, which of the workloads here are those of rank 512; elsewhere the
@@ -495,7 +498,7 @@ def run_ours(args, wl):
     traffic = None
     per_unit = NCU_TRAFFIC_PER_UNIT.get(names[dom])
     if (per_unit is not None and wl.r == 512 and wl.s == 16 and args.projection == "left" and args.history == "fp32"
-            and not fused_gram):
+            and args.moments == "fp32" and not fused_gram):
         units = sum(d[2] for d in dims) if per_unit[0] == "rn" else sum(M * N for M, N in shapes)
         traffic = per_unit[1] * units
     roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -512,7 +515,7 @@ def run_ours(args, wl):
     # ---- the oracle on the host cores, bounded sample
     cpu = None
     if not args.no_cpu:
-        sec, desc, threads = oracle_sample(wl, projection=args.projection, history=args.history)
+        sec, desc, threads = oracle_sample(wl, projection=args.projection, history=args.history, moments=args.moments)
         cpu = {"value": 1.0 / sec, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -555,6 +558,9 @@ def main():
     ap.add_argument("--history", default="fp32", choices=["fp32", "bf16"],
                     help="fp32: the ring of low-rank gradients in fp32 (the headline configuration); bf16: every "
                          "stored gradient but the current one in bf16 (reduced-precision state option)")
+    ap.add_argument("--moments", default="fp32", choices=["fp32", "bf16"],
+                    help="fp32: the Adam moments in fp32 (the headline configuration); bf16: m rounded to nearest and v "
+                         "rounded stochastically to bf16 (reduced-precision state option)")
     ap.add_argument("--gram-fusion", default="off", choices=["on", "off"],
                     help="off (the library's default): the Gram tiles run in the stream kernel; on: where the workload "
                          "allows it the new Gram row is formed in the projection's epilogue")

@@ -78,7 +78,8 @@ typedef struct {
   int32_t gemm_impl;                /* 0 (default): tensor-core (tcgen05) projection GEMMs; 1: plain SIMT GEMMs (debug) */
   int32_t power_iterations;         /* subspace-iteration sweeps in the refresh; <= 0 selects the default 6 */
   int32_t reset_history_on_refresh; /* default 0: history, m and v survive a refresh */
-  uint64_t seed;                    /* seed of the refresh's random test matrix; 0 selects a fixed default */
+  uint64_t seed;                    /* seed of the refresh's random test matrix and of the stochastic rounding of
+                                       moments_bf16; 0 selects a fixed default (0x9E3779B97F4A7C15) */
   int32_t stream_impl;              /* 0 (default): fused Gram/solve/moment kernel; 1: separate plain kernels (debug) */
   int32_t projection_rule;          /* 0 (default): every matrix is projected on the left, R = P^T G, as the paper
                                        writes it; 1: the short-side rule of GaLore, which the paper's "most steps are
@@ -107,6 +108,14 @@ typedef struct {
                                        hundred columns of an unconverged basis, which is why the default is not
                                        smaller); -1: all r' columns (the full Rayleigh-Ritz step, about 2.5 times the
                                        refresh time at r' = 512). */
+  int32_t moments_bf16;             /* 0 (default): the Adam moments are fp32.  1: reduced-precision state (the paper's
+                                       conclusion names it as future work): m is stored as bf16 rounded to nearest; v is
+                                       stored as bf16 with stochastic rounding (one step changes v by a relative
+                                       1 - beta2, less than half a bf16 unit, so rounding to nearest would freeze it),
+                                       its random bits from Philox-4x32-10 keyed by `seed` with the counter (element
+                                       index / 4, matrix index, step index).  The direction of a step comes from the
+                                       unrounded moments.  Halves the moments' memory and traffic.  Needs the fused
+                                       stream kernel and the left projection. */
 } ngalore_options;
 
 /*

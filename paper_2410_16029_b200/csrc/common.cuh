@@ -22,8 +22,11 @@ struct MatDesc {
   float* H;                   // history ring: s slots of one low-rank matrix, fp32 (one slot when s == 0); with a
                               // bf16 history only the gradient of the current step (one slot, fp32)
   uint16_t* H16;              // bf16 history ring, s slots (null unless the state keeps its history in bf16)
-  float* m;                   // first moment, rp x N
+  float* m;                   // first moment, rp x N (null when the moments are kept in bf16)
   float* v;                   // second moment, rp x N
+  uint16_t* m16;              // bf16 moments (null unless the state keeps them in bf16): m rounded to nearest,
+  uint16_t* v16;              // v rounded stochastically
+  int index;                  // position of the matrix in the state's list (keys the stochastic rounding)
   __half* u16;                // direction u = m / sqrt(v + eps) rounded to fp16, lr_rows x lr_cols
   // Working copies of the projector, both holding the bf16-rounded values of P32 (padding is zero).  The
   // projection GEMM reads bf16 (its other operand G is bf16), the back-projection fp16 (its other operand u is):
@@ -62,7 +65,27 @@ struct Hyper {
   float lr, wd, beta1, beta2, eps;
   float pad;
   double lambda;
+  unsigned int seed_lo, seed_hi;  // key of the generator behind the stochastic rounding of bf16 second moments
 };
+
+// Philox-4x32 with ten rounds (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", 2011).
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned int k0, unsigned int k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const unsigned int hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const unsigned int hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c;
+}
+
+// A non-negative float rounded to bf16 up or down with odds in proportion to the distances: sixteen random bits are
+// added below the sixteen bits bf16 keeps, and the sum is truncated.
+__device__ __forceinline__ unsigned int stochastic_bf16_bits(float x, unsigned int bits16) {
+  return (__float_as_uint(x) + bits16) >> 16;
+}
 
 struct StreamTile {
   int mat;    // matrix index

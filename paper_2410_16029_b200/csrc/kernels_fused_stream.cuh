@@ -35,6 +35,7 @@ struct FusedPlan {
   int n_items = 0;
   int grid = 0;
   bool hist16 = false;  // the state keeps its history ring in bf16
+  bool mom16 = false;   // the state keeps its moments in bf16
 };
 
 constexpr long long kSpinLimit = 4000000;  // polls of ~100 ns each before a flag wait is abandoned
@@ -47,7 +48,8 @@ struct StageMeta {
 
 // Stage layout.  fp32 history: SMAX slots of CE floats, then m, then v.  bf16 history (HIST16): SMAX slots of CE
 // bf16 values (the current slot's place stays unused), then the current gradient, m and v as floats.
-template <int SMAX, bool HIST16>
+// MOM16: the moments are stored as bf16 (half the bytes of their stages).
+template <int SMAX, bool HIST16, bool MOM16 = false>
 struct FusedCfg {
   // Elements per stage and slot.  The bf16 history costs more instructions per byte (conversion, two Gram rows),
   // and the per-stage bookkeeping of a consumer thread weighs as much as its arithmetic on two elements, so its
@@ -60,8 +62,8 @@ struct FusedCfg {
   static constexpr int kHistBytes = SMAX * CE * (HIST16 ? 2 : 4);
   static constexpr int kCurOff = kHistBytes;                          // HIST16: fp32 gradient of this step
   static constexpr int kMOff = kHistBytes + (HIST16 ? CE * 4 : 0);
-  static constexpr int kVOff = kMOff + CE * 4;
-  static constexpr int kStageBytes = kVOff + CE * 4;
+  static constexpr int kVOff = kMOff + CE * (MOM16 ? 2 : 4);
+  static constexpr int kStageBytes = kVOff + CE * (MOM16 ? 2 : 4);
   static constexpr int kStages = HIST16 ? (SMAX <= 8 ? 3 : (SMAX <= 16 ? 2 : 5)) : (SMAX <= 8 ? 5 : 3);
   static constexpr int kBase = kStages * kStageBytes;
   static constexpr int kFullOff = kBase, kEmptyOff = kBase + 64, kMetaOff = kBase + 128, kFlagOff = kBase + 512;
@@ -93,11 +95,15 @@ __device__ __forceinline__ uint32_t float_to_bf16_bits(float x) {
 // (MatDesc::H) and its bf16 rounding is written into ring slot `cur` by the combination pass.  The Gram pass
 // then also recomputes the row of the slot that was current one step ago, now that it is a rounded value, so
 // that Kraw stays the Gram matrix of exactly the values the combination uses.
-template <int SMAX, bool HIST16>
-__global__ void __launch_bounds__((FusedCfg<SMAX, HIST16>::kThreads), 1)
+// MOM16: the moments are read and written as bf16: m rounded to nearest, v rounded stochastically (one step changes
+// v by a relative 1 - beta2, less than half a bf16 unit, so rounding to nearest would freeze it) with bits from a
+// counter-based generator keyed by (element group, matrix, step index); the direction u of the step comes from
+// the unrounded values.
+template <int SMAX, bool HIST16, bool MOM16>
+__global__ void __launch_bounds__((FusedCfg<SMAX, HIST16, MOM16>::kThreads), 1)
 fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restrict__ items, int n_items, Ctrl* ctrl,
                     const Hyper* __restrict__ hyper) {
-  using C = FusedCfg<SMAX, HIST16>;
+  using C = FusedCfg<SMAX, HIST16, MOM16>;
   constexpr int CE = C::CE;
   constexpr int kConsumerThreads = C::kConsumers;
   constexpr int kGroups = kConsumerThreads / 32;
@@ -168,8 +174,10 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
             mt.first = (e == e0) ? 1 : 0; mt.last = (e + CE >= e1) ? 1 : 0; mt.count = cnt; mt.e0 = e;
             mt.cur = cur_slot; mt.c = c;
             meta[stage] = mt;
-            mbar_expect_tx(full_bar + stage, HIST16 ? bytes * static_cast<uint32_t>(ncopies) - (bytes / 2) * static_cast<uint32_t>(c - 1)
-                                                    : bytes * static_cast<uint32_t>(ncopies));
+            const uint32_t hist_bytes = HIST16 ? bytes * static_cast<uint32_t>(c) - (bytes / 2) * static_cast<uint32_t>(c - 1)
+                                               : bytes * static_cast<uint32_t>(c);
+            const uint32_t mom_bytes = item.kind == 1 ? (MOM16 ? bytes : 2u * bytes) : 0u;
+            mbar_expect_tx(full_bar + stage, hist_bytes + mom_bytes);
           }
           __syncwarp();
           for (int j = lane; j < ncopies; j += 32) {
@@ -182,7 +190,10 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
                 bulk_load(sb + j * CE * 2, d.H16 + static_cast<long long>(j) * d.rn + e, bytes / 2, full_bar + stage);
             } else {
               const int k = j - c;  // 0: m, 1: v
-              bulk_load(sb + (k == 0 ? C::kMOff : C::kVOff), (k == 0 ? d.m : d.v) + e, bytes, full_bar + stage);
+              if (MOM16)
+                bulk_load(sb + (k == 0 ? C::kMOff : C::kVOff), (k == 0 ? d.m16 : d.v16) + e, bytes / 2, full_bar + stage);
+              else
+                bulk_load(sb + (k == 0 ? C::kMOff : C::kVOff), (k == 0 ? d.m : d.v) + e, bytes, full_bar + stage);
             }
           }
           if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
@@ -206,7 +217,8 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
     // per-item pointers of the combination pass, fetched once at the item's first stage
     float *it_m = nullptr, *it_v = nullptr, *it_cur = nullptr;
     __half* it_u = nullptr;
-    uint16_t* it_h16 = nullptr;
+    uint16_t *it_h16 = nullptr, *it_m16 = nullptr, *it_v16 = nullptr;
+    unsigned int it_mat = 0, it_step = 0;
     while (true) {
       if (!mbar_wait(full_bar + stage, phase, abort_flag)) break;
       const StageMeta mt = meta[stage];
@@ -235,8 +247,22 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
           }
         }
       };
-      const float* sm_m = reinterpret_cast<const float*>(sbytes + C::kMOff);
-      const float* sm_v = reinterpret_cast<const float*>(sbytes + C::kVOff);
+      // this thread's VEC elements of a moment in this stage
+      auto load_moment = [&](int off, float (&x)[VEC]) {
+        if (!MOM16) {
+          const float* p = reinterpret_cast<const float*>(sbytes + off) + idx;
+#pragma unroll
+          for (int q = 0; q < VEC; ++q) x[q] = p[q];
+        } else {
+          const uint32_t* p = reinterpret_cast<const uint32_t*>(sbytes + off + idx * 2);
+#pragma unroll
+          for (int q = 0; q < VEC; q += 2) {
+            const uint32_t pair = p[q >> 1];
+            x[q] = bf16_bits_to_float(pair & 0xFFFFu);
+            x[q + 1] = bf16_bits_to_float(pair >> 16);
+          }
+        }
+      };
       const bool two_rows = HIST16 && c >= 2;
       const int prev = two_rows ? (cur == 0 ? d.s : cur) - 1 : 0;
       if (mt.kind == 0) {
@@ -374,6 +400,9 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
           if (tid < kMaxHistory) wsm[tid] = __ldcg(d.wsol + tid);
           item_bad = __ldcg(d.step_bad) != 0;
           it_m = d.m; it_v = d.v; it_u = d.u16;
+          it_m16 = d.m16; it_v16 = d.v16;
+          it_mat = static_cast<unsigned int>(d.index);
+          it_step = static_cast<unsigned int>(ctrl->k);
           it_cur = current_gradient(d, cur);
           it_h16 = HIST16 ? d.H16 + static_cast<long long>(cur) * d.rn : nullptr;
           consumer_sync<kConsumerThreads>();
@@ -411,13 +440,35 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
 #pragma unroll
               for (int q = 0; q < VEC; q += 2) dst[q >> 1] = float_to_bf16_bits(x[q]) | (float_to_bf16_bits(x[q + 1]) << 16);
             }
+            load_moment(C::kMOff, mm);
+            load_moment(C::kVOff, vv);
 #pragma unroll
             for (int q = 0; q < VEC; ++q) {
-              mm[q] = hp.beta1 * sm_m[idx + q] + (1.f - hp.beta1) * n[q];
-              vv[q] = hp.beta2 * sm_v[idx + q] + (1.f - hp.beta2) * n[q] * n[q];
+              mm[q] = hp.beta1 * mm[q] + (1.f - hp.beta1) * n[q];
+              vv[q] = hp.beta2 * vv[q] + (1.f - hp.beta2) * n[q] * n[q];
               uu[q] = mm[q] / sqrtf(vv[q] + hp.eps);
             }
-            if (VEC == 4) {
+            if (MOM16) {
+              // elements 4 g .. 4 g + 3 take the upper halves of the four words of one generator call
+              uint32_t* dm = reinterpret_cast<uint32_t*>(it_m16 + e);
+              uint32_t* dv = reinterpret_cast<uint32_t*>(it_v16 + e);
+#pragma unroll
+              for (int q0 = 0; q0 < VEC; q0 += 4) {
+                const unsigned long long grp = static_cast<unsigned long long>(e + q0) >> 2;
+                const uint4 rnd = philox4x32_10(make_uint4(static_cast<unsigned int>(grp), static_cast<unsigned int>(grp >> 32),
+                                                           it_mat, it_step), hp.seed_lo, hp.seed_hi);
+                const unsigned int rb[4] = {rnd.x >> 16, rnd.y >> 16, rnd.z >> 16, rnd.w >> 16};
+#pragma unroll
+                for (int q = q0; q < q0 + 4 && q < VEC; q += 2) {
+                  // (VEC = 2: e is a multiple of 2, the pair is words 0, 1 or words 2, 3 of its group)
+                  const int w0 = VEC == 2 ? static_cast<int>(e & 2) : q - q0;
+                  dm[q >> 1] = float_to_bf16_bits(mm[q]) | (float_to_bf16_bits(mm[q + 1]) << 16);
+                  dv[q >> 1] = stochastic_bf16_bits(vv[q], rb[w0]) | (stochastic_bf16_bits(vv[q + 1], rb[w0 + 1]) << 16);
+                }
+              }
+              if (VEC == 4) *reinterpret_cast<uint2*>(it_u + e) = pack_f16x4(uu[0], uu[1], uu[2 % VEC], uu[3 % VEC]);
+              else *reinterpret_cast<uint32_t*>(it_u + e) = pack_f16x4(uu[0], uu[1], 0.f, 0.f).x;
+            } else if (VEC == 4) {
               *reinterpret_cast<float4*>(it_m + e) = make_float4(mm[0], mm[1], mm[2 % VEC], mm[3 % VEC]);
               *reinterpret_cast<float4*>(it_v + e) = make_float4(vv[0], vv[1], vv[2 % VEC], vv[3 % VEC]);
               *reinterpret_cast<uint2*>(it_u + e) = pack_f16x4(uu[0], uu[1], uu[2 % VEC], uu[3 % VEC]);
@@ -442,10 +493,15 @@ fused_stream_kernel(const MatDesc* __restrict__ mats, const FusedItem* __restric
   }
 }
 
-template <int SMAX, bool HIST16>
+template <int SMAX, bool HIST16, bool MOM16>
 inline cudaError_t fused_set_smem() {
-  return cudaFuncSetAttribute(fused_stream_kernel<SMAX, HIST16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              FusedCfg<SMAX, HIST16>::kTotal);
+  return cudaFuncSetAttribute(fused_stream_kernel<SMAX, HIST16, MOM16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              FusedCfg<SMAX, HIST16, MOM16>::kTotal);
+}
+
+template <bool HIST16, bool MOM16>
+inline cudaError_t fused_set_smem_for(int s) {
+  return s <= 8 ? fused_set_smem<8, HIST16, MOM16>() : (s <= 16 ? fused_set_smem<16, HIST16, MOM16>() : fused_set_smem<32, HIST16, MOM16>());
 }
 
 // skip_gram (optional, one entry per matrix): 1 where the Gram row and the solve of a matrix are done before this
@@ -476,11 +532,9 @@ inline ngalore_status fused_plan_create(FusedPlan& plan, const std::vector<MatDe
   if (cudaMemcpy(plan.d_items, items.data(), sizeof(FusedItem) * items.size(), cudaMemcpyHostToDevice) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   plan.hist16 = !mats.empty() && mats[0].H16 != nullptr;
-  cudaError_t e;
-  if (plan.hist16)
-    e = s <= 8 ? fused_set_smem<8, true>() : (s <= 16 ? fused_set_smem<16, true>() : fused_set_smem<32, true>());
-  else
-    e = s <= 8 ? fused_set_smem<8, false>() : (s <= 16 ? fused_set_smem<16, false>() : fused_set_smem<32, false>());
+  plan.mom16 = !mats.empty() && mats[0].m16 != nullptr;
+  const cudaError_t e = plan.hist16 ? (plan.mom16 ? fused_set_smem_for<true, true>(s) : fused_set_smem_for<true, false>(s))
+                                    : (plan.mom16 ? fused_set_smem_for<false, true>(s) : fused_set_smem_for<false, false>(s));
   return e == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
@@ -489,23 +543,30 @@ inline void fused_plan_destroy(FusedPlan& plan) {
   plan.d_items = nullptr;
 }
 
-template <int SMAX, bool HIST16>
+template <int SMAX, bool HIST16, bool MOM16>
 inline void fused_launch_one(const FusedPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const Hyper* d_hyper,
                              cudaStream_t stream) {
-  fused_stream_kernel<SMAX, HIST16><<<plan.grid, FusedCfg<SMAX, HIST16>::kThreads, FusedCfg<SMAX, HIST16>::kTotal, stream>>>(
-      d_mats, plan.d_items, plan.n_items, d_ctrl, d_hyper);
+  using C = FusedCfg<SMAX, HIST16, MOM16>;
+  fused_stream_kernel<SMAX, HIST16, MOM16><<<plan.grid, C::kThreads, C::kTotal, stream>>>(d_mats, plan.d_items, plan.n_items,
+                                                                                         d_ctrl, d_hyper);
+}
+
+template <bool HIST16, bool MOM16>
+inline void fused_launch_for(const FusedPlan& plan, const MatDesc* d_mats, Ctrl* d_ctrl, const Hyper* d_hyper, int s,
+                             cudaStream_t stream) {
+  if (s <= 8) fused_launch_one<8, HIST16, MOM16>(plan, d_mats, d_ctrl, d_hyper, stream);
+  else if (s <= 16) fused_launch_one<16, HIST16, MOM16>(plan, d_mats, d_ctrl, d_hyper, stream);
+  else fused_launch_one<32, HIST16, MOM16>(plan, d_mats, d_ctrl, d_hyper, stream);
 }
 
 inline ngalore_status fused_stream_launch(FusedPlan& plan, const MatDesc* d_mats, int /*n_mats*/, Ctrl* d_ctrl,
                                           const Hyper* d_hyper, int s, cudaStream_t stream, int64_t* launches) {
   if (plan.hist16) {
-    if (s <= 8) fused_launch_one<8, true>(plan, d_mats, d_ctrl, d_hyper, stream);
-    else if (s <= 16) fused_launch_one<16, true>(plan, d_mats, d_ctrl, d_hyper, stream);
-    else fused_launch_one<32, true>(plan, d_mats, d_ctrl, d_hyper, stream);
+    if (plan.mom16) fused_launch_for<true, true>(plan, d_mats, d_ctrl, d_hyper, s, stream);
+    else fused_launch_for<true, false>(plan, d_mats, d_ctrl, d_hyper, s, stream);
   } else {
-    if (s <= 8) fused_launch_one<8, false>(plan, d_mats, d_ctrl, d_hyper, stream);
-    else if (s <= 16) fused_launch_one<16, false>(plan, d_mats, d_ctrl, d_hyper, stream);
-    else fused_launch_one<32, false>(plan, d_mats, d_ctrl, d_hyper, stream);
+    if (plan.mom16) fused_launch_for<false, true>(plan, d_mats, d_ctrl, d_hyper, s, stream);
+    else fused_launch_for<false, false>(plan, d_mats, d_ctrl, d_hyper, s, stream);
   }
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;

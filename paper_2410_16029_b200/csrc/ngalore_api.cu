@@ -516,6 +516,10 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (opt != nullptr && (opt->history_bf16 < 0 || opt->history_bf16 > 1)) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && (opt->gram_fusion < 0 || opt->gram_fusion > 1)) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && opt->ritz_columns < -1) return NGALORE_ERR_INVALID_ARG;
+  // bf16 moments live in the fused stream kernel only; the rounding stream is keyed by the element's position in
+  // the unpadded low-rank matrix, which the padded layout of right-projected matrices does not keep
+  if (opt != nullptr && (opt->moments_bf16 < 0 || opt->moments_bf16 > 1)) return NGALORE_ERR_INVALID_ARG;
+  if (opt != nullptr && opt->moments_bf16 == 1 && (opt->stream_impl == 1 || opt->projection_rule == 1)) return NGALORE_ERR_INVALID_ARG;
   // the bf16 history lives in the fused stream kernel only
   if (opt != nullptr && opt->history_bf16 == 1 && (s < 1 || opt->stream_impl == 1)) return NGALORE_ERR_INVALID_ARG;
 
@@ -535,6 +539,8 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (opt != nullptr) st->opt = *opt;
   st->opt.struct_size = sizeof(ngalore_options);
   if (st->opt.seed == 0) st->opt.seed = 0x9E3779B97F4A7C15ull;
+  st->hyper.seed_lo = static_cast<unsigned int>(st->opt.seed & 0xFFFFFFFFull);
+  st->hyper.seed_hi = static_cast<unsigned int>(st->opt.seed >> 32);
 
   // ---- streaming tile size.  A work item of the persistent stream kernel carries a fixed cost (table and
   // descriptor loads, the end-of-tile reduction, the completion counter), so tiles are large; measured on the
@@ -560,7 +566,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     total_rn += hm.rn;
     hash = (hash ^ static_cast<uint64_t>(hm.M)) * 1099511628211ull;
     hash = (hash ^ static_cast<uint64_t>(hm.N)) * 1099511628211ull;
-    hash = (hash ^ static_cast<uint64_t>((hm.right ? 2 : 1) + (st->opt.history_bf16 ? 4 : 0))) * 1099511628211ull;
+    hash = (hash ^ static_cast<uint64_t>((hm.right ? 2 : 1) + (st->opt.history_bf16 ? 4 : 0) + (st->opt.moments_bf16 ? 8 : 0))) * 1099511628211ull;
   }
   st->shape_hash = hash;
   // Stream tiles: two per SM and pass on large workloads.  Where that would make them short, one per SM: every tile
@@ -586,6 +592,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   // ---- arena layout
   const int slots = s > 0 ? s : 1;
   const bool hist16 = st->opt.history_bf16 == 1;
+  const bool mom16 = st->opt.moments_bf16 == 1;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
   struct Offs { size_t H, m, v, P32, P16, Pt16, Kraw, wsol; };
@@ -596,8 +603,8 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   for (int i = 0; i < n_matrices; ++i) {
     const HostMat& hm = st->mats[i];
     offs[i].H = hist16 ? take(sizeof(uint16_t) * hm.rn * slots) : take(sizeof(float) * hm.rn * slots);
-    offs[i].m = take(sizeof(float) * hm.rn);
-    offs[i].v = take(sizeof(float) * hm.rn);
+    offs[i].m = take((mom16 ? sizeof(uint16_t) : sizeof(float)) * hm.rn);
+    offs[i].v = take((mom16 ? sizeof(uint16_t) : sizeof(float)) * hm.rn);
     offs[i].P32 = take(sizeof(float) * hm.eM * hm.rp);
     offs[i].P16 = take(sizeof(uint16_t) * hm.eM * ((hm.rp + 7) / 8 * 8));
     offs[i].Pt16 = take(sizeof(uint16_t) * hm.rp * ((hm.eM + 7) / 8 * 8));
@@ -689,8 +696,16 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
       d.H16 = nullptr;
       d.H = reinterpret_cast<float*>(st->arena + offs[i].H);
     }
-    d.m = reinterpret_cast<float*>(st->arena + offs[i].m);
-    d.v = reinterpret_cast<float*>(st->arena + offs[i].v);
+    d.index = i;
+    if (mom16) {
+      d.m = nullptr; d.v = nullptr;
+      d.m16 = reinterpret_cast<uint16_t*>(st->arena + offs[i].m);
+      d.v16 = reinterpret_cast<uint16_t*>(st->arena + offs[i].v);
+    } else {
+      d.m = reinterpret_cast<float*>(st->arena + offs[i].m);
+      d.v = reinterpret_cast<float*>(st->arena + offs[i].v);
+      d.m16 = nullptr; d.v16 = nullptr;
+    }
     d.P32 = reinterpret_cast<float*>(st->arena + offs[i].P32);
     d.P16 = reinterpret_cast<uint16_t*>(st->arena + offs[i].P16);
     d.Pt16 = reinterpret_cast<uint16_t*>(st->arena + offs[i].Pt16);

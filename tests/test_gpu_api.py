@@ -333,7 +333,7 @@ def test_update_groups_and_overlapped_exchange_with_one_rank():
         grouped.set_subspace(i, plain.get_subspace(i))
     grouped.set_update_groups(3)
     ranges = grouped.update_groups()
-    assert ranges[0][0] == 0 and ranges[-1][1] == len(shapes) and len(ranges) == 3
+    assert ranges[0][0] == 0 and ranges[-1][1] == len(shapes) and 2 <= len(ranges) <= 3   # about equal sizes, at most 3
     assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
     Wa = [wl.initial_weight_device(w, i, dev) for i in range(len(shapes))]
     Wb = [t.clone() for t in Wa]
