@@ -178,6 +178,145 @@ inline cudaError_t chol_batched_launch(CholProblem* d_probs, int n, int Lmax, cu
   return cudaGetLastError();
 }
 
+// The same factorisation with one CTA per matrix and no launches between the panels: for a batch of about as many
+// matrices as there are SMs this keeps every SM busy from the first panel to the last, where the launch-per-panel
+// version spends most of its time between kernels (a 512 x 512 factor is 16 panels, i.e. 32 launches of a few
+// tens of microseconds each, for 45 million multiply-adds).  Per panel: one warp factors the diagonal block in
+// shared memory, every thread solves one row of the panel against it (keeping the solved panel in shared memory,
+// column-major), and all threads update the trailing triangle in 4 x 4 register tiles straight in global memory
+// (the matrix stays in L2).  Shared memory: 32 x (L - 32) doubles for the panel.
+constexpr int kCholCtaThreads = 512;
+
+inline size_t chol_cta_smem_bytes(int Lmax) {
+  const int rows = Lmax > kCholNB ? Lmax - kCholNB : 0;
+  return sizeof(double) * static_cast<size_t>(kCholNB) * (rows + 4);
+}
+
+__global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const CholProblem* probs) {
+  constexpr int NB = kCholNB;
+  extern __shared__ __align__(16) double chol_ps[];   // panel, k-major: chol_ps[k * ldp + (row - base)]
+  __shared__ double D[NB][NB + 1];
+  __shared__ double s_tiny;
+  const CholProblem p = probs[blockIdx.x];
+  double* C = p.C;
+  const int L = p.L;
+  const int tid = threadIdx.x;
+  // pivot floor from the diagonal (a pivot that is not above it is replaced by it, see chol_begin_kernel)
+  if (tid < 32) {
+    double md = 0.0;
+    for (int i = tid; i < L; i += 32) md = fmax(md, C[static_cast<long long>(i) * L + i]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) md = fmax(md, __shfl_xor_sync(0xffffffffu, md, o));
+    if (tid == 0) s_tiny = fmax(md, 1e-300) * 1e-28;
+  }
+  __syncthreads();
+  const double tiny = s_tiny;
+  for (int j0 = 0; j0 < L; j0 += NB) {
+    const int nbj = (L - j0 < NB) ? (L - j0) : NB;
+    const int base = j0 + nbj;            // first row / column of the trailing part
+    const int T = L - base;               // its size
+    const int ldp = T + 4 - (T & 1);      // even, so that pairs of rows are 16-byte aligned
+    for (int x = tid; x < NB * NB; x += kCholCtaThreads) {
+      const int a = x / NB, b = x % NB;
+      D[a][b] = (a < nbj && b < nbj) ? C[static_cast<long long>(j0 + a) * L + j0 + b] : 0.0;
+    }
+    __syncthreads();
+    if (tid < 32) {
+      const int lane = tid;
+      for (int k = 0; k < nbj; ++k) {
+        double dkk = D[k][k];
+        if (!(dkk > tiny)) dkk = tiny;
+        const double lkk = sqrt(dkk);
+        __syncwarp();
+        if (lane == k) D[k][k] = lkk;
+        if (lane > k && lane < nbj) D[lane][k] /= lkk;
+        __syncwarp();
+        if (lane > k && lane < nbj) {
+          const double lik = D[lane][k];
+          for (int j = k + 1; j <= lane; ++j) D[lane][j] -= lik * D[j][k];
+        }
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+    for (int x = tid; x < NB * NB; x += kCholCtaThreads) {
+      const int a = x / NB, b = x % NB;
+      if (a < nbj && b <= a) C[static_cast<long long>(j0 + a) * L + j0 + b] = D[a][b];
+    }
+    // panel rows: x D^T = c by forward substitution, one thread per row
+    for (int i = base + tid; i < L; i += kCholCtaThreads) {
+      double xr[NB];
+      double* crow = C + static_cast<long long>(i) * L + j0;
+#pragma unroll
+      for (int jj = 0; jj < NB; ++jj) {
+        if (jj < nbj) {
+          double a = crow[jj];
+#pragma unroll
+          for (int t = 0; t < NB; ++t)
+            if (t < jj) a -= xr[t] * D[jj][t];
+          xr[jj] = a / D[jj][jj];
+        } else {
+          xr[jj] = 0.0;
+        }
+      }
+#pragma unroll
+      for (int jj = 0; jj < NB; ++jj) {
+        if (jj < nbj) crow[jj] = xr[jj];
+        chol_ps[jj * ldp + (i - base)] = xr[jj];
+      }
+    }
+    __syncthreads();
+    // trailing update on the lower triangle: C[i][j] -= sum_k panel[i][k] panel[j][k], 4 x 4 tiles
+    if (T > 0) {
+      const int nt = (T + 3) >> 2;
+      const int ntiles = nt * (nt + 1) / 2;
+      for (int t = tid; t < ntiles; t += kCholCtaThreads) {
+        int ti = static_cast<int>((sqrtf(8.f * t + 1.f) - 1.f) * 0.5f);
+        while ((ti + 1) * (ti + 2) / 2 <= t) ++ti;
+        while (ti * (ti + 1) / 2 > t) --ti;
+        const int tj = t - ti * (ti + 1) / 2;
+        const int i0 = 4 * ti, c0 = 4 * tj;        // relative to base
+        double acc[4][4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+#pragma unroll
+          for (int y = 0; y < 4; ++y) acc[x][y] = 0.0;
+#pragma unroll 4
+        for (int k = 0; k < NB; ++k) {
+          const double* pk = chol_ps + k * ldp;
+          // (rows beyond T inside the last tile read the padding or the next column's start: finite values that
+          // the bounds check below keeps from being stored)
+          const double2 a01 = *reinterpret_cast<const double2*>(pk + i0), a23 = *reinterpret_cast<const double2*>(pk + i0 + 2);
+          const double2 b01 = *reinterpret_cast<const double2*>(pk + c0), b23 = *reinterpret_cast<const double2*>(pk + c0 + 2);
+          const double a[4] = {a01.x, a01.y, a23.x, a23.y}, b[4] = {b01.x, b01.y, b23.x, b23.y};
+#pragma unroll
+          for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) acc[x][y] += a[x] * b[y];
+        }
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const int i = base + i0 + x;
+          if (i >= L) continue;
+#pragma unroll
+          for (int y = 0; y < 4; ++y) {
+            const int j = base + c0 + y;
+            if (j <= i) C[static_cast<long long>(i) * L + j] -= acc[x][y];
+          }
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// Factor n matrices, one CTA each (the list should start with the largest matrices: CTAs are handed out in order).
+inline cudaError_t chol_cta_launch(const CholProblem* d_probs, int n, int Lmax, cudaStream_t stream, int64_t* launches) {
+  chol_cta_kernel<<<n, kCholCtaThreads, chol_cta_smem_bytes(Lmax), stream>>>(d_probs);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
 // ---------------------------------------------------------------- Q = Y Lf^-T (rows are independent)
 
 // One CTA owns 32 rows of Y (rows x L, fp32) and produces the same rows of Q (fp32) with

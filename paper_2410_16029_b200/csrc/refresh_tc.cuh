@@ -323,37 +323,48 @@ __global__ void __launch_bounds__(256) tri_convert_kernel(const TriInverse* prob
 // Scale every column of Y (rows x L, fp32) to unit norm, the norm summed in fp64.  The products of the refresh go
 // through operands split in two bf16 parts; the rounding of the diagonal of a triangular factor or of a rotation
 // (a relative 2^-17) scales a whole column, which is the largest part of what the last product leaves of
-// non-orthonormality.  Block (32, 8): blockIdx.x = strip of 32 columns, blockIdx.y = matrix.
+// non-orthonormality.  Two kernels: partial sums of squares per strip of 32 columns and chunk of rows (added to
+// `sums` with fp64 atomics; `sums` is cleared beforehand), then the scaling.  Block (32, 8): blockIdx.x = strip of
+// 32 columns, blockIdx.y = matrix, blockIdx.z = chunk of kNormRows rows.
 struct NormJob {
   float* Y;
+  double* sums;   // L sums of squares
   int rows, L;
 };
+constexpr int kNormRows = 1024;
 
-__global__ void __launch_bounds__(256) normalize_columns_kernel(const NormJob* jobs) {
+__global__ void __launch_bounds__(256) column_sumsq_kernel(const NormJob* jobs) {
   __shared__ double part[8][33];
-  __shared__ float scale[32];
   const NormJob jb = jobs[blockIdx.y];
   const int col = blockIdx.x * 32 + threadIdx.x;
-  if (blockIdx.x * 32 >= jb.L) return;
+  const int r0 = blockIdx.z * kNormRows;
+  if (blockIdx.x * 32 >= jb.L || r0 >= jb.rows) return;
+  const int r1 = min(jb.rows, r0 + kNormRows);
   double s = 0.0;
   if (col < jb.L)
-    for (int r = threadIdx.y; r < jb.rows; r += 8) {
+    for (int r = r0 + threadIdx.y; r < r1; r += 8) {
       const double v = static_cast<double>(jb.Y[static_cast<long long>(r) * jb.L + col]);
       s += v * v;
     }
   part[threadIdx.y][threadIdx.x] = s;
   __syncthreads();
-  if (threadIdx.y == 0) {
+  if (threadIdx.y == 0 && col < jb.L) {
     double t = 0.0;
 #pragma unroll
     for (int g = 0; g < 8; ++g) t += part[g][threadIdx.x];
-    scale[threadIdx.x] = t > 0.0 ? static_cast<float>(1.0 / sqrt(t)) : 0.f;
+    atomicAdd(jb.sums + col, t);
   }
-  __syncthreads();
-  if (col < jb.L) {
-    const float f = scale[threadIdx.x];
-    for (int r = threadIdx.y; r < jb.rows; r += 8) jb.Y[static_cast<long long>(r) * jb.L + col] *= f;
-  }
+}
+
+__global__ void __launch_bounds__(256) column_scale_kernel(const NormJob* jobs) {
+  const NormJob jb = jobs[blockIdx.y];
+  const int col = blockIdx.x * 32 + threadIdx.x;
+  const int r0 = blockIdx.z * kNormRows;
+  if (col >= jb.L || r0 >= jb.rows) return;
+  const int r1 = min(jb.rows, r0 + kNormRows);
+  const double t = jb.sums[col];
+  const float f = t > 0.0 ? static_cast<float>(1.0 / sqrt(t)) : 0.f;
+  for (int r = r0 + threadIdx.y; r < r1; r += 8) jb.Y[static_cast<long long>(r) * jb.L + col] *= f;
 }
 
 constexpr int kTriMaxLevels = 12;
@@ -400,6 +411,7 @@ struct RefreshPlan {
   char* zero_tables = nullptr;
   GramPrep* d_prep = nullptr;
   CholProblem* d_chol = nullptr;
+  CholProblem* d_chol_sorted = nullptr;  // the same problems, widest first (for the one-CTA-per-matrix kernel)
   int l_max = 0;  // largest basis width L of the set
   TriInverse* d_tri = nullptr;
   TriLeaf* d_leaves = nullptr;
@@ -422,6 +434,8 @@ struct RefreshPlan {
   JacobiSlot* d_jac_slots = nullptr;
   int jac_nblk_max = 0, jac_ld_max = 0;
   NormJob* d_norm = nullptr;
+  ZeroJob* d_zero_d = nullptr;   // clears every matrix's D (as 16-byte words)
+  int m_max = 0;                 // most rows among the matrices
 };
 
 inline void refresh_plan_destroy(RefreshPlan& plan) {
@@ -531,6 +545,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   }
   const size_t o_prep = take(sizeof(GramPrep) * n);
   const size_t o_chol = take(sizeof(CholProblem) * n);
+  const size_t o_chol_sorted = take(sizeof(CholProblem) * n);
   const size_t o_tri = take(sizeof(TriInverse) * n);
   std::vector<SyrkTile> syrk_tiles;
   for (int i = 0; i < n; ++i) {
@@ -549,6 +564,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   const size_t o_jac_init = take(sizeof(JacobiInit) * n);
   const size_t o_jac_out = take(sizeof(JacobiOut) * n);
   const size_t o_norm = take(sizeof(NormJob) * n);
+  const size_t o_zero_d = take(sizeof(ZeroJob) * n);
   const size_t o_jac_flags = take(sizeof(int) * 2 * n);
   int nblk_max_all = 2;
   for (int i = 0; i < n; ++i) nblk_max_all = std::max(nblk_max_all, jacobi_blocks(std::min(mats[i].rp, (ritz_columns + 3) & ~3)));
@@ -596,7 +612,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     const int Lj = std::min(m.L, (ritz_columns + 3) & ~3);
     jac[i] = JacobiMat{reinterpret_cast<float*>(m.T64), m.X64, Lj, Lj, jacobi_blocks(Lj),
                        reinterpret_cast<int*>(plan.buf + o_jac_flags) + 2 * i};
-    norm[i] = NormJob{m.Yf, m.M, m.L};
+    norm[i] = NormJob{m.Yf, m.D, m.M, m.L};   // the column-norm buffer of the orthonormalisations is free by then
     jac_init[i] = JacobiInit{m.C32, nullptr, m.L};
     jac_out[i] = JacobiOut{nullptr, 0, m.Rhi, m.Rlo, m.ldl, m.L};
     plan.jac_nblk_max = std::max(plan.jac_nblk_max, jac[i].nblk);
@@ -692,6 +708,16 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   }
   plan.d_prep = reinterpret_cast<GramPrep*>(plan.buf + o_prep);
   plan.d_chol = reinterpret_cast<CholProblem*>(plan.buf + o_chol);
+  plan.d_chol_sorted = reinterpret_cast<CholProblem*>(plan.buf + o_chol_sorted);
+  {
+    std::vector<CholProblem> sorted(chol);
+    std::stable_sort(sorted.begin(), sorted.end(), [](const CholProblem& a, const CholProblem& b) { return a.L > b.L; });
+    if (cudaMemcpy(plan.d_chol_sorted, sorted.data(), sizeof(CholProblem) * n, cudaMemcpyHostToDevice) != cudaSuccess)
+      return NGALORE_ERR_CUDA;
+    if (cudaFuncSetAttribute(chol_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(chol_cta_smem_bytes(plan.l_max))) != cudaSuccess)
+      return NGALORE_ERR_CUDA;
+  }
   plan.d_tri = reinterpret_cast<TriInverse*>(plan.buf + o_tri);
   plan.d_split_y = reinterpret_cast<SplitJob*>(plan.buf + o_sy);
   plan.d_syrk_mats = reinterpret_cast<SyrkMat*>(plan.buf + o_syrk_m);
@@ -702,6 +728,15 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   plan.d_jac_init = reinterpret_cast<JacobiInit*>(plan.buf + o_jac_init);
   plan.d_jac_out = reinterpret_cast<JacobiOut*>(plan.buf + o_jac_out);
   plan.d_norm = reinterpret_cast<NormJob*>(plan.buf + o_norm);
+  plan.d_zero_d = reinterpret_cast<ZeroJob*>(plan.buf + o_zero_d);
+  {
+    std::vector<ZeroJob> zd(n);
+    for (int i = 0; i < n; ++i) {
+      zd[i] = ZeroJob{reinterpret_cast<float4*>(plan.mats[i].D), static_cast<long long>(plan.mats[i].L) * 8 / 16};  // L is a multiple of 4
+      plan.m_max = std::max(plan.m_max, plan.mats[i].M);
+    }
+    if (cudaMemcpy(plan.d_zero_d, zd.data(), sizeof(ZeroJob) * n, cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
+  }
   plan.d_jac_slots = reinterpret_cast<JacobiSlot*>(plan.buf + o_jac_slots);
   if (cudaMemcpy(plan.d_prep, prep.data(), sizeof(GramPrep) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_chol, chol.data(), sizeof(CholProblem) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -836,7 +871,7 @@ inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ct
   if ((rc = refresh_tc_gemm(plan, y_side ? RG_GRAM_Y : RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
   gram_prep_kernel<<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_prep, shift_scale);
   *launches += 1;
-  if (chol_batched_launch(plan.d_chol, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
+  if (chol_cta_launch(plan.d_chol_sorted, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, y_side ? RG_APPLY_Y : RG_APPLY_Z, d_ctrl, stream, launches))) return rc;
   return refresh_tc_split(plan, y_side, stream, launches);
@@ -854,7 +889,7 @@ inline ngalore_status refresh_tc_final(RefreshPlan& plan, Ctrl* d_ctrl, cudaStre
   syrk_f64_kernel<<<plan.n_syrk_tiles, 256, 0, stream>>>(plan.d_syrk_mats, plan.d_syrk_tiles);
   gram_prep64_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep64);
   *launches += 2;
-  if (chol_batched_launch(plan.d_chol, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
+  if (chol_cta_launch(plan.d_chol_sorted, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
   return refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches);
 }
@@ -918,8 +953,11 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
   *launches += 1;
   // Q orthonormal to about 1e-6 and V orthogonal: so is their product, once its columns are scaled back to unit norm
   if ((rc = refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches))) return rc;
-  normalize_columns_kernel<<<dim3((plan.l_max + 31) / 32, plan.n), dim3(32, 8), 0, stream>>>(plan.d_norm);
-  *launches += 1;
+  zero_jobs_kernel<<<dim3(1, plan.n), 256, 0, stream>>>(plan.d_zero_d);
+  const dim3 norm_grid((plan.l_max + 31) / 32, plan.n, (plan.m_max + kNormRows - 1) / kNormRows);
+  column_sumsq_kernel<<<norm_grid, dim3(32, 8), 0, stream>>>(plan.d_norm);
+  column_scale_kernel<<<norm_grid, dim3(32, 8), 0, stream>>>(plan.d_norm);
+  *launches += 3;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
