@@ -208,75 +208,72 @@ __global__ void __launch_bounds__(kJacThreads) jacobi_gram_kernel(const JacobiMa
   }
 }
 
-// Step 2: one warp per block pair diagonalises its Gram matrix by cyclic two-sided Jacobi rotations, 16 disjoint
-// ones per step: A <- R^T A R, J <- J R.  With partner(j) the column that column j is paired with in a step,
-// column j of A R is ca[j] * column j + cb[j] * column partner(j); rows likewise.  Lane i owns row i of A (in shared
-// memory, because the column update indexes it by partner) and column i of J (in registers).  A few sweeps are
-// enough: the outer iteration comes back to every pair.
-constexpr int kJacInnerWarps = 8;
+// Step 2: one CTA of four warps per block pair diagonalises its Gram matrix by cyclic two-sided Jacobi rotations, 16
+// disjoint ones per step: A <- R^T A R, J <- J R.  With partner(j) the column that column j is paired with in a
+// step, column j of A R is ca[j] * column j + cb[j] * column partner(j); rows likewise.  Sixteen threads find the
+// angles; then every thread (row r, eight columns) forms its entries of B = A R, and after a barrier its entries of
+// R^T B and of J R.  A solve is a chain of dependent steps, so its latency is what a round of the rotation costs:
+// four warps per solve instead of one cut it about fivefold.  A few sweeps are enough: the outer iteration comes
+// back to every pair.
+constexpr int kJacInnerThreads = 128;
 
-__global__ void __launch_bounds__(32 * kJacInnerWarps) jacobi_inner_kernel(JacobiSlot* slots, int n_slots) {
-  __shared__ float As_all[kJacInnerWarps][kJacCols][kJacCols + 1];
-  __shared__ float cab_all[kJacInnerWarps][2][kJacCols];
-  __shared__ unsigned char partner_tab[kJacCols - 1][kJacCols];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int x = threadIdx.x; x < (kJacCols - 1) * kJacBlock; x += blockDim.x) {
-    int p, q;
-    round_robin_pair(kJacCols, x / kJacBlock, x % kJacBlock, p, q);
-    partner_tab[x / kJacBlock][p] = static_cast<unsigned char>(q);
-    partner_tab[x / kJacBlock][q] = static_cast<unsigned char>(p);
+__global__ void __launch_bounds__(kJacInnerThreads) jacobi_inner_kernel(JacobiSlot* slots, int n_slots) {
+  __shared__ float As[kJacCols][kJacCols + 1];
+  __shared__ float Bs[kJacCols][kJacCols + 1];
+  __shared__ float JT[kJacCols][kJacCols + 1];   // JT[a][b] = J[b][a]
+  __shared__ float ca[kJacCols], cb[kJacCols];
+  __shared__ unsigned char partner[kJacCols];
+  JacobiSlot& slot = slots[blockIdx.x];
+  if (slot.active == 0) return;
+  const int tid = threadIdx.x;
+  const int r = tid >> 2, j0 = (tid & 3) * 8;     // this thread: row r, columns j0 .. j0 + 7
+#pragma unroll
+  for (int y = 0; y < 8; ++y) {
+    As[r][j0 + y] = slot.A[r][j0 + y];
+    JT[r][j0 + y] = (r == j0 + y) ? 1.f : 0.f;
   }
   __syncthreads();
-  const int id = blockIdx.x * kJacInnerWarps + warp;
-  if (id >= n_slots) return;
-  JacobiSlot& slot = slots[id];
-  if (slot.active == 0) return;
-  float (*As)[kJacCols + 1] = As_all[warp];
-  float* ca = cab_all[warp][0];
-  float* cb = cab_all[warp][1];
-#pragma unroll 4
-  for (int r = 0; r < kJacCols; ++r) As[r][lane] = slot.A[r][lane];
-  float jt[kJacCols];   // column `lane` of J
-#pragma unroll
-  for (int c = 0; c < kJacCols; ++c) jt[c] = (c == lane) ? 1.f : 0.f;
-  __syncwarp();
   for (int sweep = 0; sweep < kJacInnerSweeps; ++sweep) {
     int rotated = 0;
     for (int step = 0; step < kJacCols - 1; ++step) {
-      const int mate = partner_tab[step][lane];
-      const int p = lane < mate ? lane : mate, q = lane < mate ? mate : lane;
-      const float app = As[p][p], aqq = As[q][q], apq = As[p][q];
-      float c = 1.f, sn = 0.f;
-      if (apq * apq > 1e-12f * app * aqq && apq != 0.f) {
-        const float tau = (aqq - app) / (2.f * apq);
-        const float t = (tau >= 0.f ? 1.f : -1.f) / (fabsf(tau) + sqrtf(1.f + tau * tau));
-        c = rsqrtf(1.f + t * t);
-        sn = t * c;
-        rotated = 1;
+      if (tid < kJacBlock) {
+        int p, q;
+        round_robin_pair(kJacCols, step, tid, p, q);
+        const float app = As[p][p], aqq = As[q][q], apq = As[p][q];
+        float c = 1.f, sn = 0.f;
+        if (apq * apq > 1e-12f * app * aqq && apq != 0.f) {
+          const float tau = (aqq - app) / (2.f * apq);
+          const float t = (tau >= 0.f ? 1.f : -1.f) / (fabsf(tau) + sqrtf(1.f + tau * tau));
+          c = rsqrtf(1.f + t * t);
+          sn = t * c;
+          rotated = 1;
+        }
+        ca[p] = c; cb[p] = -sn; partner[p] = static_cast<unsigned char>(q);
+        ca[q] = c; cb[q] = sn; partner[q] = static_cast<unsigned char>(p);
       }
-      const float my_ca = c, my_cb = (lane == p) ? -sn : sn;
-      ca[lane] = my_ca;
-      cb[lane] = my_cb;
-      __syncwarp();
-      // B = A R: this lane's row
-      float b[kJacCols];
+      __syncthreads();
+      float t[8];
 #pragma unroll
-      for (int j = 0; j < kJacCols; ++j) b[j] = ca[j] * As[lane][j] + cb[j] * As[lane][partner_tab[step][j]];
-      __syncwarp();
-      // A <- R^T B and J <- J R: the mate's row of B and column of J come by shuffle
+      for (int y = 0; y < 8; ++y) t[y] = ca[j0 + y] * As[r][j0 + y] + cb[j0 + y] * As[r][partner[j0 + y]];
 #pragma unroll
-      for (int j = 0; j < kJacCols; ++j) {
-        const float bm = __shfl_sync(0xffffffffu, b[j], mate);
-        As[lane][j] = my_ca * b[j] + my_cb * bm;
-        const float jm = __shfl_sync(0xffffffffu, jt[j], mate);
-        jt[j] = my_ca * jt[j] + my_cb * jm;
+      for (int y = 0; y < 8; ++y) Bs[r][j0 + y] = t[y];                            // B = A R
+      __syncthreads();
+      const float car = ca[r], cbr = cb[r];
+      const int pr = partner[r];
+#pragma unroll
+      for (int y = 0; y < 8; ++y) {
+        As[r][j0 + y] = car * Bs[r][j0 + y] + cbr * Bs[pr][j0 + y];                // A <- R^T B
+        t[y] = car * JT[r][j0 + y] + cbr * JT[pr][j0 + y];                         // row r of JT = column r of J
       }
-      __syncwarp();
+      __syncthreads();
+#pragma unroll
+      for (int y = 0; y < 8; ++y) JT[r][j0 + y] = t[y];
     }
-    if (!__any_sync(0xffffffffu, rotated)) break;
+    if (!__syncthreads_or(rotated)) break;
   }
+  __syncthreads();
 #pragma unroll
-  for (int r = 0; r < kJacCols; ++r) slot.J[lane][r] = jt[r];
+  for (int y = 0; y < 8; ++y) slot.J[r][j0 + y] = JT[r][j0 + y];
 }
 
 // Step 3: the rotation of every active block pair is made orthogonal to second order, J <- J (I - (J^T J - I) / 2),
@@ -445,7 +442,7 @@ inline cudaError_t jacobi_batched_launch(const JacobiMat* d_mats, int n, int nbl
     for (int round = 0; round < nblk_max - 1; ++round) {
       const int r = sweep * (nblk_max - 1) + round;
       jacobi_gram_kernel<<<dim3(tables, n), kJacThreads, smem, stream>>>(d_mats, slots, r);
-      jacobi_inner_kernel<<<(n_slots + kJacInnerWarps - 1) / kJacInnerWarps, 32 * kJacInnerWarps, 0, stream>>>(slots, n_slots);
+      jacobi_inner_kernel<<<n_slots, kJacInnerThreads, 0, stream>>>(slots, n_slots);
       jacobi_polish_kernel<<<n_slots, kJacThreads, 0, stream>>>(slots);
       jacobi_apply_kernel<<<dim3(tables, n, parts), kJacApplyThreads, 0, stream>>>(d_mats, slots, r);
       *launches += 4;
