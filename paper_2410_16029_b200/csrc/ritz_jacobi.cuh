@@ -8,7 +8,7 @@
 // the columns of a working matrix X (started as C, scaled to a unit largest diagonal entry) are rotated against
 // each other until they are mutually orthogonal; the accumulated rotation is V and the column norms are the
 // eigenvalues.  The unit of work is one pair of 16-column blocks of one matrix: a CTA forms the 32 x 32 Gram
-// matrix of its 32 columns, one warp diagonalises that by cyclic two-sided Jacobi rotations, and a CTA applies the
+// matrix of its 32 columns, four warps diagonalise that by cyclic two-sided Jacobi rotations, and a CTA applies the
 // resulting 32 x 32 rotation to the 32 columns of X and of V.  The block pairs of a round are disjoint
 // (round-robin ordering), so a round is a few launches over every matrix; a sweep is (blocks - 1) rounds.
 //
