@@ -48,7 +48,7 @@ def config_dict(args, wl, n_matrices, sharded):
     grad_bytes = sum(M * N * 2 for _, M, N in wl.shapes)
     return {"workload": wl.name, "matrices": n_matrices, "r": wl.r, "s": wl.s, "T": wl.T,
             "projection": args.projection, "history": args.history, "moments": args.moments,
-            "gram_fusion": args.gram_fusion,
+            "gram_fusion": args.gram_fusion, "small_rank_path": args.small_rank_path,
             "sharded": sharded, "history_filled": True, "refresh_in_timed_region": False,
             "l2": f"inputs larger than L2: {pool_size(args, wl)} gradient sets of {grad_bytes / 1e9:.2f} GB cycled"}
 
@@ -314,7 +314,8 @@ def run_ours(args, wl):
     # no refresh among them, whatever T is); the refresh is run once before them and timed alone further down.
     opt = NGaLore(shapes, wl.r, wl.s, 0, lam=wl.lam, lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps,
                   wd=wl.wd, seed=1 + rank, projection=args.projection, history_bf16=args.history == "bf16",
-                  gram_fusion=args.gram_fusion == "on", moments_bf16=args.moments == "bf16")
+                  gram_fusion=args.gram_fusion == "on", moments_bf16=args.moments == "bf16",
+                  small_rank_path=args.small_rank_path == "on")
     # seeded synthetic inputs, resident in HBM: a pool of gradient sets cycled through the steps
     wl_rank = rank_workload(wl, rank)
     if parts is not None:
@@ -493,6 +494,12 @@ def run_ours(args, wl):
     proj_bytes = sum(2 * M * N + 2 * dims[i][1] * dims[i][0] + 4 * dims[i][2] for i, (M, N) in enumerate(shapes))
     back_bytes = sum(8 * M * N + 2 * dims[i][1] * dims[i][0] for i, (M, N) in enumerate(shapes))
     alg = [proj_bytes, stream_bytes, back_bytes]
+    if opt.uses_small_rank_path:
+        # two bandwidth kernels (every r' <= 8): the first reads the history once for the Gram row, the second owns
+        # the moments; there is no separate stream phase
+        names = ["sr_project_gram_kernel", "(no stream phase)", "sr_update_kernel"]
+        hist_once = sum(4 * wl.s * d[2] for d in dims)
+        alg = [proj_bytes + hist_once, 0, back_bytes + sum(16 * d[2] for d in dims)]
     dom = int(np.argmax(phase))
     achieved = alg[dom] / (phase[dom] * 1e-3) / 1e9
     traffic = None
@@ -505,7 +512,8 @@ def run_ours(args, wl):
                 "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
                 "algorithmic_bytes_per_launch": alg[dom], "ms_per_launch": float(phase[dom]),
                 "phases_ms": {names[i]: float(phase[i]) for i in range(3)},
-                "phases_frac_of_peak": {names[i]: alg[i] / (phase[i] * 1e-3) / 1e9 / peak for i in range(3)}}
+                "phases_frac_of_peak": {names[i]: alg[i] / (phase[i] * 1e-3) / 1e9 / peak for i in range(3)
+                                        if phase[i] > 1e-6}}
     flops = flop_model(wl, args.projection)
     step_roofline_ms = max(tot_bytes / (peak * 1e9), flops / (tensor_peak * 1e12)) * 1e3
     step_roof = {"bytes_per_step": tot_bytes, "flops_per_step": flops, "roofline_ms": step_roofline_ms,
@@ -564,6 +572,9 @@ def main():
     ap.add_argument("--gram-fusion", default="off", choices=["on", "off"],
                     help="off (the library's default): the Gram tiles run in the stream kernel; on: where the workload "
                          "allows it the new Gram row is formed in the projection's epilogue")
+    ap.add_argument("--small-rank-path", default="off", choices=["on", "off"],
+                    help="on: where every matrix has r' <= 8 the step runs as two kernels without tensor cores (an "
+                         "option of the library, slower than the default as built)")
     ap.add_argument("--shard", action="store_true",
                     help="with --gpus N > 1: one model's matrices split over the ranks (state memory / N, weights "
                          "exchanged after every step) instead of N independent replicas; rank 0's phases and "

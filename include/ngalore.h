@@ -116,6 +116,15 @@ typedef struct {
                                        index / 4, matrix index, step index).  The direction of a step comes from the
                                        unrounded moments.  Halves the moments' memory and traffic.  Needs the fused
                                        stream kernel and the left projection. */
+  int32_t small_rank_path;          /* 0 (default): the tensor-core kernels at every rank.  1: when every matrix has
+                                       r' <= 8 (the fine-tuning ranks 4 and 8 of Sec. 4.2 and 4.3), the projection is
+                                       on the left, history and moments are fp32 and s <= 16, the step runs as two
+                                       kernels without tensor cores that touch every element of G and W once with
+                                       plain loads and stores (projection + Gram row; solve + moments + weight
+                                       update).  Same results to rounding.  Measured slower than the default as built
+                                       (strips of 64 columns stream G and W in pieces too short for the memory
+                                       system), hence off unless asked for.  The path is left when update groups
+                                       are set. */
 } ngalore_options;
 
 /*
@@ -237,6 +246,7 @@ int64_t ngalore_step_count(const ngalore_state* st);        /* k as the host las
 size_t ngalore_device_bytes(const ngalore_state* st);       /* device memory held by the state */
 /* Kernels launched by the library on behalf of this state since creation. */
 int64_t ngalore_launch_count(const ngalore_state* st);
+int ngalore_uses_small_rank_path(const ngalore_state* st);  /* 1 if the state takes the small-rank path (see options) */
 /* How many times ngalore_step had to encode and upload the TMA descriptors of a (W, G) pair of pointer arrays
  * (see ngalore_step: once per distinct pair while it stays cached). */
 int64_t ngalore_descriptor_uploads(const ngalore_state* st);

@@ -456,6 +456,12 @@ struct TcPlan {
   CUtensorMap* d_maps_all = nullptr;
   CUtensorMap* h_pinned_all = nullptr;
   CUtensorMap* d_maps = nullptr;    // the set of the current call (one of bindings[*].d_maps)
+  // Behind the tensor maps every set also carries the raw pointers (n gradient pointers, then n weight pointers) for
+  // the kernels that read G and W with plain loads (small-rank path).
+  size_t ptr_offset = 0;            // bytes from the start of a set to its pointers
+  size_t set_bytes = 0;
+  const uint16_t* const* d_Gptr = nullptr;   // of the current call
+  float* const* d_Wptr = nullptr;
   TcTile* d_tiles_proj = nullptr;
   TcTile* d_tiles_back = nullptr;
   std::vector<int> back_tile0;     // first back-projection tile of every matrix, plus the total (n + 1 entries)
@@ -644,7 +650,9 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   }
 
   // binding sets: as many as fit in 64 MB, between 2 and 32
-  const size_t set_bytes = sizeof(CUtensorMap) * plan.h_maps.size();
+  plan.ptr_offset = (sizeof(CUtensorMap) * plan.h_maps.size() + 255) / 256 * 256;
+  plan.set_bytes = (plan.ptr_offset + sizeof(void*) * 2 * n + 255) / 256 * 256;
+  const size_t set_bytes = plan.set_bytes;
   int n_sets = static_cast<int>((64u << 20) / set_bytes);
   n_sets = n_sets < 2 ? 2 : (n_sets > 32 ? 32 : n_sets);
   const size_t maps_bytes = set_bytes * n_sets;
@@ -652,8 +660,8 @@ inline ngalore_status tc_plan_create(TcPlan& plan, const std::vector<MatDesc>& m
   if (cudaMallocHost(&plan.h_pinned_all, maps_bytes) != cudaSuccess) { plan.h_pinned_all = nullptr; return NGALORE_ERR_ALLOC; }
   plan.bindings.resize(n_sets);
   for (int b = 0; b < n_sets; ++b) {
-    plan.bindings[b].d_maps = plan.d_maps_all + static_cast<size_t>(b) * plan.h_maps.size();
-    plan.bindings[b].h_pinned = plan.h_pinned_all + static_cast<size_t>(b) * plan.h_maps.size();
+    plan.bindings[b].d_maps = reinterpret_cast<CUtensorMap*>(reinterpret_cast<char*>(plan.d_maps_all) + b * set_bytes);
+    plan.bindings[b].h_pinned = reinterpret_cast<CUtensorMap*>(reinterpret_cast<char*>(plan.h_pinned_all) + b * set_bytes);
     if (cudaEventCreateWithFlags(&plan.bindings[b].uploaded, cudaEventDisableTiming) != cudaSuccess) {
       plan.bindings[b].uploaded = nullptr;
       return NGALORE_ERR_CUDA;
@@ -694,6 +702,8 @@ inline ngalore_status tc_bind_buffers(TcPlan& plan, const uint16_t* const* G, fl
         std::equal(b.W.begin(), b.W.end(), reinterpret_cast<const void* const*>(W))) {
       b.last_use = plan.bind_clock;
       plan.d_maps = b.d_maps;
+      plan.d_Gptr = reinterpret_cast<const uint16_t* const*>(reinterpret_cast<char*>(b.d_maps) + plan.ptr_offset);
+      plan.d_Wptr = reinterpret_cast<float* const*>(reinterpret_cast<char*>(b.d_maps) + plan.ptr_offset) + n;
       return NGALORE_OK;
     }
     if (victim == nullptr || (victim->valid && (!b.valid || b.last_use < victim->last_use))) victim = &b;
@@ -717,8 +727,11 @@ inline ngalore_status tc_bind_buffers(TcPlan& plan, const uint16_t* const* G, fl
         !tc_encode_2d(plan.encode, mp + TC_MAP_W_STORE, W[i], plan.colsN[i], plan.rowsN[i], row_bytes, 32, 32, true))
       return NGALORE_ERR_CUDA;
   }
-  if (cudaMemcpyAsync(b.d_maps, b.h_pinned, sizeof(CUtensorMap) * plan.h_maps.size(), cudaMemcpyHostToDevice, stream) !=
-          cudaSuccess ||
+  {
+    const void** hp = reinterpret_cast<const void**>(reinterpret_cast<char*>(b.h_pinned) + plan.ptr_offset);
+    for (int i = 0; i < n; ++i) { hp[i] = G[i]; hp[n + i] = W[i]; }
+  }
+  if (cudaMemcpyAsync(b.d_maps, b.h_pinned, plan.set_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaEventRecord(b.uploaded, stream) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   b.G.assign(reinterpret_cast<const void* const*>(G), reinterpret_cast<const void* const*>(G) + n);
@@ -728,6 +741,8 @@ inline ngalore_status tc_bind_buffers(TcPlan& plan, const uint16_t* const* G, fl
   b.last_use = plan.bind_clock;
   plan.bind_uploads += 1;
   plan.d_maps = b.d_maps;
+  plan.d_Gptr = reinterpret_cast<const uint16_t* const*>(reinterpret_cast<char*>(b.d_maps) + plan.ptr_offset);
+  plan.d_Wptr = reinterpret_cast<float* const*>(reinterpret_cast<char*>(b.d_maps) + plan.ptr_offset) + n;
   return NGALORE_OK;
 }
 

@@ -19,6 +19,7 @@
 #include "kernels_fused_stream.cuh"
 #include "refresh_tc.cuh"
 #include "static_natural_gradient.cuh"
+#include "small_rank.cuh"
 
 using namespace ngalore;
 
@@ -95,6 +96,8 @@ struct ngalore_state {
   FusedPlan fused;
   // tensor-core refresh plan
   RefreshPlan refresh;
+  // small-rank path (every r' <= 8): the step as two bandwidth kernels
+  SrPlan sr;
   // host-buffer staging; W travels in groups of matrices so that the copies in, the back-projection and the
   // copies out of different groups overlap
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
@@ -381,6 +384,30 @@ ngalore_status step_impl(ngalore_state* st, float* const* W, const uint16_t* con
   if (st->opt.gemm_impl != 1 && (rc = tc_bind_buffers(st->tc, G, W, stream))) return rc;
   const int cur = st->s > 0 ? static_cast<int>(st->n_appended % st->s) : 0;
 
+  if (st->sr.ready && !grouped && st->upd_first.size() <= 1) {
+    // small-rank path: projection with the Gram row, then solve + moments + weight update (small_rank.cuh)
+    if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[0], stream));
+    if ((rc = sr_project_gram(st->sr, st->d_desc, st->tc.d_Gptr, st->d_ctrl, st->s, stream, &st->launches))) return rc;
+    if (st->profiling) {
+      NG_CUDA(cudaEventRecord(st->ev[1], stream));
+      NG_CUDA(cudaEventRecord(st->ev[2], stream));
+    }
+    if ((rc = sr_update(st->sr, st->d_desc, st->tc.d_Wptr, st->d_ctrl, st->d_hyper, st->s, stream, &st->launches))) return rc;
+    advance_kernel<<<1, 1, 0, stream>>>(st->d_ctrl);
+    st->launches += 1;
+    NG_CUDA(cudaGetLastError());
+    if (st->profiling) {
+      NG_CUDA(cudaEventRecord(st->ev[3], stream));
+      st->ev_valid = true;
+    }
+    cudaStreamCaptureStatus cap_sr = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap_sr) != cudaSuccess) cap_sr = cudaStreamCaptureStatusNone;
+    if (cap_sr == cudaStreamCaptureStatusNone) {
+      st->k += 1;
+      st->n_appended += 1;
+    }
+    return NGALORE_OK;
+  }
   if (st->profiling) NG_CUDA(cudaEventRecord(st->ev[0], stream));
   // ---- phase 0: R = P^T G into ring slot `cur`
   if (st->opt.gemm_impl == 1) {
@@ -516,6 +543,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if (opt != nullptr && (opt->history_bf16 < 0 || opt->history_bf16 > 1)) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && (opt->gram_fusion < 0 || opt->gram_fusion > 1)) return NGALORE_ERR_INVALID_ARG;
   if (opt != nullptr && opt->ritz_columns < -1) return NGALORE_ERR_INVALID_ARG;
+  if (opt != nullptr && (opt->small_rank_path < 0 || opt->small_rank_path > 1)) return NGALORE_ERR_INVALID_ARG;
   // bf16 moments live in the fused stream kernel only; the rounding stream is keyed by the element's position in
   // the unpadded low-rank matrix, which the padded layout of right-projected matrices does not keep
   if (opt != nullptr && (opt->moments_bf16 < 0 || opt->moments_bf16 > 1)) return NGALORE_ERR_INVALID_ARG;
@@ -762,6 +790,11 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   if ((rc = tc_backproject_init()) != NGALORE_OK) return fail(rc);
   rc = fused_plan_create(st->fused, st->h_desc, s, prop.multiProcessorCount, &st->tc.gram_fused);
   if (rc != NGALORE_OK) return fail(rc);
+  if (st->opt.gemm_impl != 1 && st->opt.stream_impl != 1 && st->opt.gram_fusion != 1 && st->opt.small_rank_path == 1 &&
+      sr_eligible(st->h_desc, s)) {
+    rc = sr_plan_create(st->sr, st->h_desc, s, prop.multiProcessorCount);
+    if (rc != NGALORE_OK) return fail(rc);
+  }
   if (st->opt.gemm_impl != 1) {
     // the refresh plan sees every matrix it takes in the orientation whose left subspace is wanted
     std::vector<float*> Yf, Zf;
@@ -792,6 +825,7 @@ void ngalore_destroy(ngalore_state* st) {
   tc_plan_destroy(st->tc);
   fused_plan_destroy(st->fused);
   refresh_plan_destroy(st->refresh);
+  sr_plan_destroy(st->sr);
   for (int e = 0; e < 4; ++e)
     if (st->ev[e]) cudaEventDestroy(st->ev[e]);
   for (cudaEvent_t e : st->ev_upd) if (e) cudaEventDestroy(e);
@@ -1093,6 +1127,7 @@ ngalore_status ngalore_debug_withhold_solution(ngalore_state* st, int matrix_ind
   if (st == nullptr || matrix_index < 0 || matrix_index >= st->n || polls < 1 || polls > 1000000) return NGALORE_ERR_INVALID_ARG;
   if (st->s < 1 || st->opt.stream_impl == 1) return NGALORE_ERR_INVALID_ARG;
   if (!st->tc.gram_fused.empty() && st->tc.gram_fused[matrix_index]) return NGALORE_ERR_INVALID_ARG;
+  if (st->sr.ready) return NGALORE_ERR_INVALID_ARG;   // the small-rank path has no wait to run out
   DeviceGuard guard(st->device);
   if (!guard.ok) return NGALORE_ERR_CUDA;
   NG_CUDA(cudaDeviceSynchronize());
@@ -1113,9 +1148,10 @@ int ngalore_rank(const ngalore_state* st, int i) { return (st && i >= 0 && i < s
 int ngalore_projects_right(const ngalore_state* st, int i) { return (st && i >= 0 && i < st->n) ? (st->mats[i].right ? 1 : 0) : -1; }
 int ngalore_subspace_rows(const ngalore_state* st, int i) { return (st && i >= 0 && i < st->n) ? st->mats[i].eM : -1; }
 int64_t ngalore_step_count(const ngalore_state* st) { return st ? st->k : -1; }
-size_t ngalore_device_bytes(const ngalore_state* st) { return st ? st->arena_bytes + st->work_bytes + st->stage_bytes + st->tc.device_bytes + st->refresh.device_bytes : 0; }
+size_t ngalore_device_bytes(const ngalore_state* st) { return st ? st->arena_bytes + st->work_bytes + st->stage_bytes + st->tc.device_bytes + st->refresh.device_bytes + st->sr.device_bytes : 0; }
 int64_t ngalore_launch_count(const ngalore_state* st) { return st ? st->launches : 0; }
 int64_t ngalore_descriptor_uploads(const ngalore_state* st) { return st ? st->tc.bind_uploads : 0; }
+int ngalore_uses_small_rank_path(const ngalore_state* st) { return (st && st->sr.ready) ? 1 : 0; }
 
 ngalore_status ngalore_set_profiling(ngalore_state* st, int on) {
   if (st == nullptr) return NGALORE_ERR_INVALID_ARG;

@@ -36,7 +36,7 @@ class Options(ctypes.Structure):
                 ("power_iterations", ctypes.c_int32), ("reset_history_on_refresh", ctypes.c_int32),
                 ("seed", ctypes.c_uint64), ("stream_impl", ctypes.c_int32), ("projection_rule", ctypes.c_int32),
                 ("history_bf16", ctypes.c_int32), ("gram_fusion", ctypes.c_int32), ("ritz_columns", ctypes.c_int32),
-                ("moments_bf16", ctypes.c_int32)]
+                ("moments_bf16", ctypes.c_int32), ("small_rank_path", ctypes.c_int32)]
 
 
 _vp = ctypes.c_void_p
@@ -84,6 +84,8 @@ _lib.ngalore_device_bytes.restype = ctypes.c_size_t
 _lib.ngalore_device_bytes.argtypes = [_vp]
 _lib.ngalore_launch_count.restype = ctypes.c_int64
 _lib.ngalore_launch_count.argtypes = [_vp]
+_lib.ngalore_uses_small_rank_path.restype = ctypes.c_int
+_lib.ngalore_uses_small_rank_path.argtypes = [_vp]
 _lib.ngalore_descriptor_uploads.restype = ctypes.c_int64
 _lib.ngalore_descriptor_uploads.argtypes = [_vp]
 _lib.ngalore_set_profiling.restype = ctypes.c_int
@@ -127,13 +129,13 @@ class NGaLore:
     def __init__(self, shapes, r, s, T, lam=1e-3, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, wd=0.0, *,
                  gemm_impl=0, stream_impl=0, power_iterations=0, reset_history_on_refresh=False, seed=0,
                  projection="left", history_bf16=False, gram_fusion=False, ritz_columns=0,
-                 moments_bf16=False):
+                 moments_bf16=False, small_rank_path=False):
         self.shapes = [(int(M), int(N)) for M, N in shapes]
         arr = (Shape * len(self.shapes))(*[Shape(M, N) for M, N in self.shapes])
         rule = {"left": 0, "short_side": 1}[projection]
         opt = Options(ctypes.sizeof(Options), gemm_impl, power_iterations, int(reset_history_on_refresh), seed,
                       stream_impl, rule, int(history_bf16), 1 if gram_fusion else 0, ritz_columns,
-                      int(moments_bf16))
+                      int(moments_bf16), 1 if small_rank_path else 0)
         handle = _vp()
         _check(_lib.ngalore_create(arr, len(self.shapes), r, s, T, lam, lr, beta1, beta2, eps, wd,
                                    ctypes.byref(opt), ctypes.byref(handle)), "ngalore_create")
@@ -256,6 +258,10 @@ class NGaLore:
     @property
     def launch_count(self) -> int:
         return _lib.ngalore_launch_count(self._h)
+
+    @property
+    def uses_small_rank_path(self) -> bool:
+        return _lib.ngalore_uses_small_rank_path(self._h) == 1
 
     @property
     def descriptor_uploads(self) -> int:
