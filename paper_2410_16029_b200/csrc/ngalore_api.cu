@@ -83,7 +83,6 @@ struct ngalore_state {
   JacobiMat* d_jac = nullptr;
   JacobiInit* d_jac_init = nullptr;
   JacobiOut* d_jac_out = nullptr;
-  JacobiSlot* d_jac_slots = nullptr;   // one matrix's worth (the plain path diagonalises the matrices one by one)
   int64_t k = 0;
   int64_t n_appended = 0;
   bool has_subspace = false;         // every matrix has a projector
@@ -311,7 +310,7 @@ ngalore_status refresh_simt(ngalore_state* st, const uint16_t* const* G, const s
     jacobi_init_kernel<<<1, 256, 0, stream>>>(st->d_jac + i, st->d_jac_init + i);
     st->launches += 1;
     const int Lj = std::min(hm.rp, ritz_columns(st));
-    NG_CUDA(jacobi_batched_launch(st->d_jac + i, 1, jacobi_blocks(Lj), (Lj + 3) & ~3, st->d_jac_slots, stream, &st->launches));
+    NG_CUDA(jacobi_batched_launch(st->d_jac + i, 1, stream, &st->launches));
     jacobi_finish_kernel<<<dim3(1, kJacFinishSplit), 256, 0, stream>>>(st->d_jac + i, st->d_jac_out + i);
     st->launches += 1;
     SimtGemm a{};
@@ -652,10 +651,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   const size_t o_jac = take(sizeof(JacobiMat) * n_matrices);
   const size_t o_jac_init = take(sizeof(JacobiInit) * n_matrices);
   const size_t o_jac_out = take(sizeof(JacobiOut) * n_matrices);
-  const size_t o_jac_flags = take(sizeof(int) * 2 * n_matrices);
-  int jac_tables = 1;
-  for (const HostMat& hm : st->mats) jac_tables = std::max(jac_tables, jacobi_blocks(std::min(hm.rp, ritz_columns(st))) / 2);
-  const size_t o_jac_slots = take(sizeof(JacobiSlot) * jac_tables);
+  const size_t o_jac_flags = take(sizeof(int) * kJacMaxSweeps * n_matrices);
   int n_tiles = 0;
   std::vector<StreamTile> tiles;
   std::vector<int> tile0(n_matrices), ntl(n_matrices);
@@ -701,7 +697,6 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   st->d_jac = reinterpret_cast<JacobiMat*>(st->work + o_jac);
   st->d_jac_init = reinterpret_cast<JacobiInit*>(st->work + o_jac_init);
   st->d_jac_out = reinterpret_cast<JacobiOut*>(st->work + o_jac_out);
-  st->d_jac_slots = reinterpret_cast<JacobiSlot*>(st->work + o_jac_slots);
   std::vector<JacobiMat> jac(n_matrices);
   std::vector<JacobiInit> jac_init(n_matrices);
   std::vector<JacobiOut> jac_out(n_matrices);
@@ -757,7 +752,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     // doubles) takes over C, which is allocated with that leading dimension
     const int Lj = std::min(hm.rp, ritz_columns(st));
     jac[i] = JacobiMat{hm.Xa, hm.C, Lj, (Lj + 3) & ~3, jacobi_blocks(Lj),
-                       reinterpret_cast<int*>(st->work + o_jac_flags) + 2 * i};
+                       reinterpret_cast<int*>(st->work + o_jac_flags) + kJacMaxSweeps * i};
     jac_init[i] = JacobiInit{nullptr, hm.C, hm.rp};
     jac_out[i] = JacobiOut{hm.Xb, hm.rp, nullptr, nullptr, 0, hm.rp};
     if (s == 0 && cudaMemcpy(d.wsol, w_init.data(), sizeof(float) * kMaxHistory, cudaMemcpyHostToDevice) != cudaSuccess)
@@ -778,9 +773,7 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
   for (const HostMat& hm : st->mats) max_rp = hm.rp > max_rp ? hm.rp : max_rp;
   if (orth_apply_smem_bytes(max_rp) > static_cast<size_t>(prop.sharedMemPerBlockOptin)) return fail(NGALORE_ERR_INVALID_ARG);
   if (cudaFuncSetAttribute(orth_apply_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(orth_apply_smem_bytes(max_rp))) != cudaSuccess ||
-      cudaFuncSetAttribute(jacobi_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(jacobi_smem_bytes(kJacMaxL))) != cudaSuccess)
+                           static_cast<int>(orth_apply_smem_bytes(max_rp))) != cudaSuccess)
     return fail(NGALORE_ERR_CUDA);
 
   const bool allow_gram_fusion = st->opt.gemm_impl != 1 && st->opt.stream_impl != 1 && !hist16 && st->opt.gram_fusion == 1;

@@ -320,6 +320,24 @@ __global__ void __launch_bounds__(256) tri_convert_kernel(const TriInverse* prob
   }
 }
 
+// Second-order orthonormalisation of a basis that is orthonormal to first order already: with C = Q^T Q = I + E,
+// Q (I - E / 2) has Q^T Q = I + O(E^2).  C comes from the tensor cores (its error, about 1e-7 on an entry for columns
+// of unit norm, is what is left of E afterwards); S = I - E / 2 = 1.5 I - C / 2 is written in two bf16 parts where the
+// product Q = Y R^-1 expects R^-1.  blockIdx.x = matrix, blockIdx.y = share of its entries.
+__global__ void __launch_bounds__(256) newton_prep_kernel(const GramPrep* preps, const TriInverse* tris) {
+  const GramPrep g = preps[blockIdx.x];
+  const TriInverse t = tris[blockIdx.x];
+  const long long total = static_cast<long long>(g.L) * g.L;
+  for (long long x = blockIdx.y * 256 + threadIdx.x; x < total; x += 256ll * gridDim.y) {
+    const int j = static_cast<int>(x / g.L), i = static_cast<int>(x % g.L);
+    const float c = 0.5f * (g.C32[x] + g.C32[static_cast<long long>(i) * g.L + j]);
+    const float f = (i == j) ? 1.5f - 0.5f * c : -0.5f * c;
+    const __nv_bfloat16 h = __float2bfloat16_rn(f);
+    t.Rhi[static_cast<long long>(j) * t.ld + i] = h;
+    t.Rlo[static_cast<long long>(j) * t.ld + i] = __float2bfloat16_rn(f - __bfloat162float(h));
+  }
+}
+
 // Scale every column of Y (rows x L, fp32) to unit norm, the norm summed in fp64.  The products of the refresh go
 // through operands split in two bf16 parts; the rounding of the diagonal of a triangular factor or of a rotation
 // (a relative 2^-17) scales a whole column, which is the largest part of what the last product leaves of
@@ -371,8 +389,8 @@ constexpr int kTriMaxLevels = 12;
 
 // ------------------------------------------------------------------------------------------ plan
 
-enum RefreshGemm { RG_Y_FROM_Z = 0, RG_Z_FROM_Y, RG_GRAM_Y, RG_GRAM_Z, RG_APPLY_Y, RG_APPLY_Z, RG_COUNT };
-enum RefreshMap { RM_G_A = 0, RM_G_MN, RM_Z_B, RM_Z_B_LO, RM_Y_B, RM_Y_B_LO, RM_Y_A, RM_Y_A_LO, RM_Z_A, RM_Z_A_LO,
+enum RefreshGemm { RG_Y_FROM_Z = 0, RG_Z_FROM_Y, RG_GRAM_Y, RG_GRAM_Z, RG_APPLY_Y, RG_COUNT };
+enum RefreshMap { RM_G_A = 0, RM_G_MN, RM_Z_B, RM_Z_B_LO, RM_Y_B, RM_Y_B_LO, RM_Y_A, RM_Y_A_LO,
                   RM_RINV, RM_RINV_LO, RM_COUNT };
 
 struct RefreshMat {
@@ -431,8 +449,6 @@ struct RefreshPlan {
   JacobiMat* d_jac = nullptr;
   JacobiInit* d_jac_init = nullptr;
   JacobiOut* d_jac_out = nullptr;
-  JacobiSlot* d_jac_slots = nullptr;
-  int jac_nblk_max = 0, jac_ld_max = 0;
   NormJob* d_norm = nullptr;
   ZeroJob* d_zero_d = nullptr;   // clears every matrix's D (as 16-byte words)
   int m_max = 0;                 // most rows among the matrices
@@ -516,8 +532,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
         case RG_Z_FROM_Y: rows = m.N; cols = m.L; K = m.M; break;
         case RG_GRAM_Y: rows = m.L; cols = m.L; K = m.M; break;
         case RG_GRAM_Z: rows = m.L; cols = m.L; K = m.N; break;
-        case RG_APPLY_Y: rows = m.M; cols = m.L; K = m.L; break;
-        default: rows = m.N; cols = m.L; K = m.L; break;
+        default: rows = m.M; cols = m.L; K = m.L; break;  // RG_APPLY_Y
       }
       total_kb += static_cast<long long>((rows + kTcBM - 1) / kTcBM) * ((cols + kRefBN - 1) / kRefBN) *
                   ((K + kTcBK - 1) / kTcBK);
@@ -532,8 +547,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
         case RG_Z_FROM_Y: rows = m.N; cols = m.L; K = m.M; break;
         case RG_GRAM_Y: rows = m.L; cols = m.L; K = m.M; break;
         case RG_GRAM_Z: rows = m.L; cols = m.L; K = m.N; break;
-        case RG_APPLY_Y: rows = m.M; cols = m.L; K = m.L; break;
-        default: rows = m.N; cols = m.L; K = m.L; break;
+        default: rows = m.M; cols = m.L; K = m.L; break;  // RG_APPLY_Y
       }
       add_tiles(g, i, rows, cols, K, target);
     }
@@ -565,10 +579,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   const size_t o_jac_out = take(sizeof(JacobiOut) * n);
   const size_t o_norm = take(sizeof(NormJob) * n);
   const size_t o_zero_d = take(sizeof(ZeroJob) * n);
-  const size_t o_jac_flags = take(sizeof(int) * 2 * n);
-  int nblk_max_all = 2;
-  for (int i = 0; i < n; ++i) nblk_max_all = std::max(nblk_max_all, jacobi_blocks(std::min(mats[i].rp, (ritz_columns + 3) & ~3)));
-  const size_t o_jac_slots = take(sizeof(JacobiSlot) * n * (nblk_max_all / 2));
+  const size_t o_jac_flags = take(sizeof(int) * kJacMaxSweeps * n);
   if (cudaMalloc(&plan.buf, off) != cudaSuccess) { plan.buf = nullptr; return NGALORE_ERR_ALLOC; }
   if (cudaMemset(plan.buf, 0, off) != cudaSuccess) return NGALORE_ERR_CUDA;
   plan.device_bytes = off;
@@ -611,12 +622,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     // (width of the rotated part: all of the basis, or its leading ritz_columns, kept a multiple of 4)
     const int Lj = std::min(m.L, (ritz_columns + 3) & ~3);
     jac[i] = JacobiMat{reinterpret_cast<float*>(m.T64), m.X64, Lj, Lj, jacobi_blocks(Lj),
-                       reinterpret_cast<int*>(plan.buf + o_jac_flags) + 2 * i};
+                       reinterpret_cast<int*>(plan.buf + o_jac_flags) + kJacMaxSweeps * i};
     norm[i] = NormJob{m.Yf, m.D, m.M, m.L};   // the column-norm buffer of the orthonormalisations is free by then
     jac_init[i] = JacobiInit{m.C32, nullptr, m.L};
     jac_out[i] = JacobiOut{nullptr, 0, m.Rhi, m.Rlo, m.ldl, m.L};
-    plan.jac_nblk_max = std::max(plan.jac_nblk_max, jac[i].nblk);
-    plan.jac_ld_max = std::max(plan.jac_ld_max, Lj);
     CUtensorMap* mp = &plan.h_maps[static_cast<size_t>(i) * RM_COUNT];
     const uint64_t sl = static_cast<uint64_t>(m.ldl) * 2;
     bool ok = true;
@@ -626,8 +635,6 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     ok &= tc_encode_2d(plan.encode, mp + RM_Y_B_LO, m.Ylo, m.L, m.M, sl, 64, kTcBK);
     ok &= tc_encode_2d(plan.encode, mp + RM_Y_A, m.Yhi, m.L, m.M, sl, kTcBK, kTcBM);
     ok &= tc_encode_2d(plan.encode, mp + RM_Y_A_LO, m.Ylo, m.L, m.M, sl, kTcBK, kTcBM);
-    ok &= tc_encode_2d(plan.encode, mp + RM_Z_A, m.Zhi, m.L, m.N, sl, kTcBK, kTcBM);
-    ok &= tc_encode_2d(plan.encode, mp + RM_Z_A_LO, m.Zlo, m.L, m.N, sl, kTcBK, kTcBM);
     ok &= tc_encode_2d(plan.encode, mp + RM_RINV, m.Rhi, m.L, m.L, sl, 64, kTcBK);
     ok &= tc_encode_2d(plan.encode, mp + RM_RINV_LO, m.Rlo, m.L, m.L, sl, 64, kTcBK);
     if (!ok) return NGALORE_ERR_CUDA;
@@ -637,7 +644,6 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     probs[RG_GRAM_Y][i] = TcProblem{m.C32, m.L, m.L, m.L, base + RM_Y_B, base + RM_Y_B, 0};
     probs[RG_GRAM_Z][i] = TcProblem{m.C32, m.L, m.L, m.L, base + RM_Z_B, base + RM_Z_B, 0};
     probs[RG_APPLY_Y][i] = TcProblem{m.Yf, m.M, m.L, m.L, base + RM_Y_A, base + RM_RINV, 0};
-    probs[RG_APPLY_Z][i] = TcProblem{m.Zf, m.N, m.L, m.L, base + RM_Z_A, base + RM_RINV, 0};
   }
   // ---- tables of the blocked triangular inverse
   {
@@ -737,7 +743,6 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     }
     if (cudaMemcpy(plan.d_zero_d, zd.data(), sizeof(ZeroJob) * n, cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
   }
-  plan.d_jac_slots = reinterpret_cast<JacobiSlot*>(plan.buf + o_jac_slots);
   if (cudaMemcpy(plan.d_prep, prep.data(), sizeof(GramPrep) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_chol, chol.data(), sizeof(CholProblem) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_tri, tri.data(), sizeof(TriInverse) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -768,7 +773,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
         float* out; long long bytes;
         switch (g) {
           case RG_Y_FROM_Z: case RG_APPLY_Y: out = m.Yf; bytes = 4ll * m.M * m.L; break;
-          case RG_Z_FROM_Y: case RG_APPLY_Z: out = m.Zf; bytes = 4ll * m.N * m.L; break;
+          case RG_Z_FROM_Y: out = m.Zf; bytes = 4ll * m.N * m.L; break;
           default: out = m.C32; bytes = 4ll * m.L * m.L; break;
         }
         jobs.push_back(ZeroJob{reinterpret_cast<float4*>(out), bytes / 16});  // L is a multiple of 4
@@ -798,9 +803,6 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
                            cudaFuncAttributeMaxDynamicSharedMemorySize, L2::kTotal) != cudaSuccess ||
       cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 2, 2, kRefStages2, TC_EPI_STORE, 4, true>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, L2::kTotal) != cudaSuccess)
-    return NGALORE_ERR_CUDA;
-  if (cudaFuncSetAttribute(jacobi_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(jacobi_smem_bytes(kJacMaxL))) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   plan.ready = true;
   return NGALORE_OK;
@@ -863,18 +865,18 @@ inline ngalore_status refresh_tc_split(RefreshPlan& plan, bool y_side, cudaStrea
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
-// iterate (fp32, in Yf or Zf) -> well-conditioned basis, left both as fp32 and as its bf16 parts.
-inline ngalore_status refresh_tc_orth(RefreshPlan& plan, bool y_side, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches,
+// iterate (fp32, in Yf) -> well-conditioned basis, left both as fp32 and as its bf16 parts.
+inline ngalore_status refresh_tc_orth(RefreshPlan& plan, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches,
                                       double shift_scale = 1.0) {
   ngalore_status rc;
-  if ((rc = refresh_tc_split(plan, y_side, stream, launches))) return rc;
-  if ((rc = refresh_tc_gemm(plan, y_side ? RG_GRAM_Y : RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
+  if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;
+  if ((rc = refresh_tc_gemm(plan, RG_GRAM_Y, d_ctrl, stream, launches))) return rc;
   gram_prep_kernel<<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_prep, shift_scale);
   *launches += 1;
   if (chol_cta_launch(plan.d_chol_sorted, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
-  if ((rc = refresh_tc_gemm(plan, y_side ? RG_APPLY_Y : RG_APPLY_Z, d_ctrl, stream, launches))) return rc;
-  return refresh_tc_split(plan, y_side, stream, launches);
+  if ((rc = refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches))) return rc;
+  return refresh_tc_split(plan, true, stream, launches);
 }
 
 // Final pass: Cholesky QR of the last basis with the Gram matrix accumulated exactly in fp64 (no shift beyond
@@ -891,6 +893,18 @@ inline ngalore_status refresh_tc_final(RefreshPlan& plan, Ctrl* d_ctrl, cudaStre
   *launches += 2;
   if (chol_cta_launch(plan.d_chol_sorted, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
+  return refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches);
+}
+
+// Pass after refresh_tc_final: the basis is orthonormal to first order by then (1e-5, up to 1e-3 for a gradient of
+// low numerical rank), and a Newton step with the tensor-core Gram matrix squares what is missing, down to the
+// accuracy of that Gram matrix; a second exact pass gave the same at ten times the cost.
+inline ngalore_status refresh_tc_refine(RefreshPlan& plan, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
+  ngalore_status rc;
+  if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;
+  if ((rc = refresh_tc_gemm(plan, RG_GRAM_Y, d_ctrl, stream, launches))) return rc;
+  newton_prep_kernel<<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_prep, plan.d_tri);
+  *launches += 1;
   return refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches);
 }
 
@@ -924,19 +938,24 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
   if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_split(plan, false, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches))) return rc;
-  if ((rc = refresh_tc_orth(plan, true, d_ctrl, stream, launches))) return rc;
+  if ((rc = refresh_tc_orth(plan, d_ctrl, stream, launches))) return rc;
+  // A sweep applies G G^T to the basis and orthonormalises the result.  Z = G^T Q is not orthonormalised in between:
+  // its columns are images of orthonormal ones, and the two-part bf16 operands keep 16 bits of every entry whatever
+  // the norm of its column, so the second product loses nothing that an orthonormalisation of Z would have saved
+  // (measured on the 1.1B shapes: the same Ritz vectors to all printed digits, a quarter of the refresh time less).
   for (int it = 0; it < q; ++it) {
     if ((rc = refresh_tc_gemm(plan, RG_Z_FROM_Y, d_ctrl, stream, launches))) return rc;
-    if ((rc = refresh_tc_orth(plan, false, d_ctrl, stream, launches))) return rc;
+    if ((rc = refresh_tc_split(plan, false, stream, launches))) return rc;
     if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches))) return rc;
-    if ((rc = refresh_tc_orth(plan, true, d_ctrl, stream, launches))) return rc;
+    if ((rc = refresh_tc_orth(plan, d_ctrl, stream, launches))) return rc;
   }
-  // Exact orthonormalisation of the basis that leaves the sweeps, twice: the basis can be ill conditioned in its
-  // weak directions, so the product with the first triangular factor leaves it orthonormal to about 1e-5 only; the
-  // second pass starts from that and ends at about 1e-6.  The Rayleigh-Ritz step below relies on it (it solves
-  // C v = lambda v, not C v = lambda (Q^T Q) v, and what Q lacks in orthonormality goes into the Ritz vectors).
+  // Exact orthonormalisation of the basis that leaves the sweeps: the basis can be ill conditioned in its weak
+  // directions, so the product with the exact triangular factor leaves it orthonormal to 1e-5 .. 1e-3 only; two
+  // Newton steps start from that and end at about 1e-6.  The Rayleigh-Ritz step below relies on it (it
+  // solves C v = lambda v, not C v = lambda (Q^T Q) v, and what Q lacks in orthonormality goes into the Ritz vectors).
   if ((rc = refresh_tc_final(plan, d_ctrl, stream, launches))) return rc;
-  if ((rc = refresh_tc_final(plan, d_ctrl, stream, launches))) return rc;
+  if ((rc = refresh_tc_refine(plan, d_ctrl, stream, launches))) return rc;
+  if ((rc = refresh_tc_refine(plan, d_ctrl, stream, launches))) return rc;
   if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;
   // Rayleigh-Ritz: Z = G^T Q, C = Z^T Z (tensor cores: its entries are good to about 2^-17 of the diagonal, far
   // finer than the gaps that decide a Ritz vector), V = eigenvectors of C (or of its leading block, see
@@ -946,8 +965,7 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
   if ((rc = refresh_tc_gemm(plan, RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
   jacobi_init_kernel<<<plan.n, 256, 0, stream>>>(plan.d_jac, plan.d_jac_init);
   *launches += 1;
-  if (jacobi_batched_launch(plan.d_jac, plan.n, plan.jac_nblk_max, plan.jac_ld_max, plan.d_jac_slots, stream, launches) !=
-      cudaSuccess)
+  if (jacobi_batched_launch(plan.d_jac, plan.n, stream, launches) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   jacobi_finish_kernel<<<dim3(plan.n, kJacFinishSplit), 256, 0, stream>>>(plan.d_jac, plan.d_jac_out);
   *launches += 1;

@@ -41,7 +41,7 @@ constexpr int kJacCols = 2 * kJacBlock;
 constexpr int kJacThreads = 256;
 constexpr int kJacMaxSweeps = 12;
 constexpr float kJacTol = 1e-5f;        // a pair of columns counts as orthogonal below this cosine
-constexpr int kJacInnerSweeps = 2;      // sweeps over the 32 x 32 Gram matrix of a block pair per visit
+constexpr int kJacInnerSweeps = 1;      // sweeps over the 32 x 32 Gram matrix of a block pair per visit
 
 struct JacobiMat {
   float* XT;    // L x ld: row i is column i of the working matrix X
@@ -49,7 +49,7 @@ struct JacobiMat {
                 // of jacobi_init_kernel: that kernel reads all of its input before it writes V)
   int L, ld;    // ld >= L, a multiple of 4
   int nblk;     // number of 16-column blocks, rounded up to an even number (>= 2)
-  int* flags;   // [0]: some pair was rotated in the sweep in progress; [1]: converged, nothing left to do
+  int* flags;   // kJacMaxSweeps words: [i] != 0 once some pair was rotated in sweep i
 };
 
 // Circle method: round r of a tournament of n players (n even), table l (0 .. n/2 - 1).
@@ -102,22 +102,28 @@ __global__ void __launch_bounds__(256) jacobi_init_kernel(const JacobiMat* mats,
   }
   __syncthreads();  // V may overwrite the input
   for (long long x = threadIdx.x; x < total; x += 256) m.VT[x] = (x / m.ld == x % m.ld) ? 1.0 : 0.0;
-  if (threadIdx.x < 2) m.flags[threadIdx.x] = 0;
+  if (threadIdx.x < kJacMaxSweeps) m.flags[threadIdx.x] = 0;
 }
 
-inline size_t jacobi_smem_bytes(int ld_max) {
-  return static_cast<size_t>(kJacCols) * (ld_max + 4) * sizeof(float);
-}
+// One launch diagonalises every matrix: a cluster of kJacCluster CTAs per matrix, each CTA working on two block
+// pairs of a round at a time.  The pairs of a round are disjoint, so within a round a CTA reads and writes only the
+// columns of its own pairs; between rounds the blocks change partners, and a cluster barrier (release / acquire)
+// makes the columns the other CTAs wrote visible.  X and V stay in global memory (they live in L2: a quarter and
+// half a megabyte per matrix) and are read past L1.  Per pair: the 32 x 32 Gram matrix of its columns (staged
+// through shared memory 64 rows at a time), its eigenvectors by cyclic two-sided Jacobi rotations on 64 threads (both
+// pairs of the CTA at once), one Newton-Schulz step in double precision that makes the 32 x 32 rotation orthogonal
+// to second order, and the rotation applied to the pair's columns of X (single) and V (double precision).  A sweep
+// in which no pair of any round was rotated ends the matrix; all CTAs of a cluster read the same flag after the same
+// barrier, so they leave together.
+constexpr int kJacCluster = 4;
+constexpr int kJacCtaThreads = 128;
+constexpr int kJacPairsPerCta = 2;
+constexpr int kJacStageRows = 64;                     // rows of the columns staged per Gram chunk
+constexpr int kJacPad = kJacCols + 1;
 
-// Scratch of one block pair of the round in progress: its Gram matrix, the rotation found for it, and whether
-// there is anything to rotate.
-struct JacobiSlot {
-  float A[kJacCols][kJacCols];
-  float J[kJacCols][kJacCols];    // J[a][b] = rotation entry (b, a): new column a = sum_b J[a][b] * old column b
-  double Jd[kJacCols][kJacCols];  // the same, re-orthogonalised in double precision
-  int active;
-  int pad[3];
-};
+__device__ __forceinline__ void jacobi_cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 struct JacobiPairInfo {
   int bi, bj;
@@ -127,250 +133,299 @@ struct JacobiPairInfo {
 __device__ __forceinline__ JacobiPairInfo jacobi_pair_of(const JacobiMat& m, int round, int table) {
   JacobiPairInfo pi{0, 0, false};
   if (table >= m.nblk / 2) return pi;
-  if (*reinterpret_cast<volatile int*>(m.flags + 1)) return pi;
-  round_robin_pair(m.nblk, round % (m.nblk - 1), table, pi.bi, pi.bj);
+  round_robin_pair(m.nblk, round, table, pi.bi, pi.bj);
   // (a block beyond L is padding: its columns load as zeros and never rotate; the columns of its partner are
   // still rotated against each other, which is all there is to do when the matrix has a single block)
   pi.live = !(pi.bi * kJacBlock >= m.L && pi.bj * kJacBlock >= m.L);
   return pi;
 }
 
-// Step 1 of a round: Gram matrix of the 32 columns of every block pair.  blockIdx.y = matrix, blockIdx.x = table
-// of the round-robin round; slot = blockIdx.y * gridDim.x + blockIdx.x.
-__global__ void __launch_bounds__(kJacThreads) jacobi_gram_kernel(const JacobiMat* mats, JacobiSlot* slots, int round) {
-  extern __shared__ __align__(16) float jac_xs[];               // 32 rows x (ld + 4)
-  __shared__ float Ap[4][kJacCols][kJacCols + 1];               // one partial Gram matrix per group of threads
-  __shared__ int s_any;
-  const JacobiMat m = mats[blockIdx.y];
-  JacobiSlot& slot = slots[blockIdx.y * gridDim.x + blockIdx.x];
-  const JacobiPairInfo pi = jacobi_pair_of(m, round, blockIdx.x);
-  const int tid = threadIdx.x;
-  if (!pi.live) {
-    if (tid == 0) slot.active = 0;
-    return;
-  }
-  const int L = m.L, ld = m.ld, lds = ld + 4;
-  const int quads = ld >> 2;
-  for (int a = tid >> 5; a < kJacCols; a += kJacThreads / 32) {       // a warp per row: coalesced, no divisions
-    const int gr = (a < kJacBlock ? pi.bi : pi.bj) * kJacBlock + (a & (kJacBlock - 1));
-    for (int q = tid & 31; q < quads; q += 32) {
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (gr < L) v = *reinterpret_cast<const float4*>(m.XT + static_cast<long long>(gr) * ld + 4 * q);
-      *reinterpret_cast<float4*>(jac_xs + a * lds + 4 * q) = v;
-    }
-  }
-  if (tid == 0) s_any = 0;
-  __syncthreads();
-  // 64 tiles of 4 x 4 entries; four groups of threads share the length of the columns
-  {
-    const int kg = tid >> 6, tile = tid & 63, ta = tile >> 3, tb = tile & 7;
-    const float* ra = jac_xs + (4 * ta) * lds;
-    const float* rb = jac_xs + (4 * tb) * lds;
-    float g[4][4];
-#pragma unroll
-    for (int x = 0; x < 4; ++x)
-#pragma unroll
-      for (int y = 0; y < 4; ++y) g[x][y] = 0.f;
-    for (int q = kg; q < quads; q += 4) {
-      float4 a[4], b[4];
-#pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        a[x] = *reinterpret_cast<const float4*>(ra + x * lds + 4 * q);
-        b[x] = *reinterpret_cast<const float4*>(rb + x * lds + 4 * q);
-      }
-#pragma unroll
-      for (int x = 0; x < 4; ++x)
-#pragma unroll
-        for (int y = 0; y < 4; ++y)
-          g[x][y] += a[x].x * b[y].x + a[x].y * b[y].y + a[x].z * b[y].z + a[x].w * b[y].w;
-    }
-#pragma unroll
-    for (int x = 0; x < 4; ++x)
-#pragma unroll
-      for (int y = 0; y < 4; ++y) Ap[kg][4 * ta + x][4 * tb + y] = g[x][y];
-  }
-  __syncthreads();
-  // add the four partial matrices in a fixed order (entry (p, q) and entry (q, p) then agree to the bit); is any
-  // pair of columns further from orthogonal than the tolerance?
-  auto entry = [&](int p, int q) { return (Ap[0][p][q] + Ap[1][p][q]) + (Ap[2][p][q] + Ap[3][p][q]); };
-  int any = 0;
-  for (int x = tid; x < kJacCols * kJacCols; x += kJacThreads) {
-    const int p = x / kJacCols, q = x % kJacCols;
-    const float v = p <= q ? entry(p, q) : entry(q, p);
-    slot.A[p][q] = v;
-    if (p < q && v * v > kJacTol * kJacTol * entry(p, p) * entry(q, q)) any = 1;
-  }
-  if (any) atomicOr(&s_any, 1);
-  __syncthreads();
-  if (tid == 0) {
-    slot.active = s_any;
-    if (s_any) atomicOr(m.flags, 1);
-  }
-}
+// Shared memory of a CTA, two regions that change hands between the phases of a pair's visit:
+//   region 1: Gram: the staged rows (32 x 64 floats, quads swizzled by row so that the 4 x 4 tiles read them
+//             without bank conflicts) and two partial Gram matrices; eigensolve: the second operand Bs;
+//             polish: J^T in double precision; apply: the rotations in single precision (rows padded to 36)
+//   region 2: eigensolve: As (the Gram matrix, rotated in place) and JT (JT[a][b] = J[b][a]); polish: J^T J - I in
+//             the place of As; then the polished rotations in double precision (rows padded to 34)
+constexpr int kJacLdD = kJacCols + 2;     // row length of the 32 x 32 double-precision matrices (16-byte rows)
+constexpr int kJacLdF = kJacCols + 4;     // the same for the single-precision copy
+constexpr size_t kJacStageBytes = sizeof(float) * kJacCols * kJacStageRows;
+constexpr size_t kJacMat32Bytes = sizeof(float) * kJacCols * kJacPad;
+constexpr size_t kJacMat64Bytes = sizeof(double) * kJacCols * kJacLdD;
+constexpr size_t kJacRegion1Bytes = kJacPairsPerCta * kJacMat64Bytes;
+constexpr size_t kJacRegion2Bytes = kJacPairsPerCta * kJacMat64Bytes;
+static_assert(kJacStageBytes + 2 * kJacMat32Bytes <= kJacRegion1Bytes, "Gram phase fits region 1");
+static_assert(kJacPairsPerCta * sizeof(float) * kJacCols * kJacLdF <= kJacRegion1Bytes, "single-precision rotations fit");
+static_assert(2 * kJacPairsPerCta * kJacMat32Bytes <= kJacRegion2Bytes, "As and JT fit region 2");
 
-// Step 2: one CTA of four warps per block pair diagonalises its Gram matrix by cyclic two-sided Jacobi rotations, 16
-// disjoint ones per step: A <- R^T A R, J <- J R.  With partner(j) the column that column j is paired with in a
-// step, column j of A R is ca[j] * column j + cb[j] * column partner(j); rows likewise.  Sixteen threads find the
-// angles; then every thread (row r, eight columns) forms its entries of B = A R, and after a barrier its entries of
-// R^T B and of J R.  A solve is a chain of dependent steps, so its latency is what a round of the rotation costs:
-// four warps per solve instead of one cut it about fivefold.  A few sweeps are enough: the outer iteration comes
-// back to every pair.
-constexpr int kJacInnerThreads = 128;
+struct JacobiShared {
+  __align__(16) unsigned char r1[kJacRegion1Bytes];
+  __align__(16) unsigned char r2[kJacRegion2Bytes];
+  float ca[kJacPairsPerCta][kJacCols], cb[kJacPairsPerCta][kJacCols];
+  unsigned char partner[kJacPairsPerCta][kJacCols];
+  int active[kJacPairsPerCta];
+};
 
-__global__ void __launch_bounds__(kJacInnerThreads) jacobi_inner_kernel(JacobiSlot* slots, int n_slots) {
-  __shared__ float As[kJacCols][kJacCols + 1];
-  __shared__ float Bs[kJacCols][kJacCols + 1];
-  __shared__ float JT[kJacCols][kJacCols + 1];   // JT[a][b] = J[b][a]
-  __shared__ float ca[kJacCols], cb[kJacCols];
-  __shared__ unsigned char partner[kJacCols];
-  JacobiSlot& slot = slots[blockIdx.x];
-  if (slot.active == 0) return;
-  const int tid = threadIdx.x;
-  const int r = tid >> 2, j0 = (tid & 3) * 8;     // this thread: row r, columns j0 .. j0 + 7
-#pragma unroll
-  for (int y = 0; y < 8; ++y) {
-    As[r][j0 + y] = slot.A[r][j0 + y];
-    JT[r][j0 + y] = (r == j0 + y) ? 1.f : 0.f;
-  }
-  __syncthreads();
-  for (int sweep = 0; sweep < kJacInnerSweeps; ++sweep) {
-    int rotated = 0;
-    for (int step = 0; step < kJacCols - 1; ++step) {
-      if (tid < kJacBlock) {
-        int p, q;
-        round_robin_pair(kJacCols, step, tid, p, q);
-        const float app = As[p][p], aqq = As[q][q], apq = As[p][q];
-        float c = 1.f, sn = 0.f;
-        if (apq * apq > 1e-12f * app * aqq && apq != 0.f) {
-          const float tau = (aqq - app) / (2.f * apq);
-          const float t = (tau >= 0.f ? 1.f : -1.f) / (fabsf(tau) + sqrtf(1.f + tau * tau));
-          c = rsqrtf(1.f + t * t);
-          sn = t * c;
-          rotated = 1;
-        }
-        ca[p] = c; cb[p] = -sn; partner[p] = static_cast<unsigned char>(q);
-        ca[q] = c; cb[q] = sn; partner[q] = static_cast<unsigned char>(p);
-      }
-      __syncthreads();
-      float t[8];
-#pragma unroll
-      for (int y = 0; y < 8; ++y) t[y] = ca[j0 + y] * As[r][j0 + y] + cb[j0 + y] * As[r][partner[j0 + y]];
-#pragma unroll
-      for (int y = 0; y < 8; ++y) Bs[r][j0 + y] = t[y];                            // B = A R
-      __syncthreads();
-      const float car = ca[r], cbr = cb[r];
-      const int pr = partner[r];
-#pragma unroll
-      for (int y = 0; y < 8; ++y) {
-        As[r][j0 + y] = car * Bs[r][j0 + y] + cbr * Bs[pr][j0 + y];                // A <- R^T B
-        t[y] = car * JT[r][j0 + y] + cbr * JT[pr][j0 + y];                         // row r of JT = column r of J
-      }
-      __syncthreads();
-#pragma unroll
-      for (int y = 0; y < 8; ++y) JT[r][j0 + y] = t[y];
-    }
-    if (!__syncthreads_or(rotated)) break;
-  }
-  __syncthreads();
-#pragma unroll
-  for (int y = 0; y < 8; ++y) slot.J[r][j0 + y] = JT[r][j0 + y];
-}
+__global__ void __cluster_dims__(kJacCluster, 1, 1) __launch_bounds__(kJacCtaThreads, 5)
+jacobi_cluster_kernel(const JacobiMat* mats) {
+  extern __shared__ __align__(16) unsigned char jac_smem_raw[];
+  JacobiShared& sh = *reinterpret_cast<JacobiShared*>(jac_smem_raw);
+  typedef float Mat32[kJacCols][kJacPad];
+  typedef double Mat64[kJacCols][kJacLdD];
+  typedef float MatF[kJacCols][kJacLdF];
+  float* stage = reinterpret_cast<float*>(sh.r1);                               // [32][64], swizzled
+  Mat32* Ap = reinterpret_cast<Mat32*>(sh.r1 + kJacStageBytes);                  // [2] partial Gram matrices
+  Mat32* Bs = reinterpret_cast<Mat32*>(sh.r1 + kJacStageBytes);                  // [pair]
+  Mat64* JTd = reinterpret_cast<Mat64*>(sh.r1);                                  // [pair]
+  MatF* Jf = reinterpret_cast<MatF*>(sh.r1);                                     // [pair]
+  Mat32* As = reinterpret_cast<Mat32*>(sh.r2);                                   // [pair]; later J^T J - I
+  Mat32* JT = reinterpret_cast<Mat32*>(sh.r2 + kJacPairsPerCta * kJacMat32Bytes);  // [pair]
+  Mat64* Jd = reinterpret_cast<Mat64*>(sh.r2);                                   // [pair]
 
-// Step 3: the rotation of every active block pair is made orthogonal to second order, J <- J (I - (J^T J - I) / 2),
-// in double precision.  One CTA per slot.
-__global__ void __launch_bounds__(kJacThreads) jacobi_polish_kernel(JacobiSlot* slots) {
-  __shared__ float JT[kJacCols][kJacCols + 1];   // JT[a][b] = J[b][a] as the inner kernel left it
-  __shared__ float Es[kJacCols][kJacCols + 1];   // J^T J - I
-  JacobiSlot& slot = slots[blockIdx.x];
-  if (slot.active == 0) return;
-  const int tid = threadIdx.x;
-  for (int x = tid; x < kJacCols * kJacCols; x += kJacThreads) JT[x / kJacCols][x % kJacCols] = slot.J[x / kJacCols][x % kJacCols];
-  __syncthreads();
-  for (int x = tid; x < kJacCols * kJacCols; x += kJacThreads) {
-    const int a = x / kJacCols, b = x % kJacCols;
-    double e = (a == b) ? -1.0 : 0.0;
-#pragma unroll 8
-    for (int k = 0; k < kJacCols; ++k) e += static_cast<double>(JT[a][k]) * static_cast<double>(JT[b][k]);  // (J^T J)_ab
-    Es[a][b] = static_cast<float>(e);
-  }
-  __syncthreads();
-  for (int x = tid; x < kJacCols * kJacCols; x += kJacThreads) {
-    const int r = x % kJacCols, a = x / kJacCols;
-    double v = static_cast<double>(JT[a][r]);                                                              // J[r][a]
-#pragma unroll 8
-    for (int k = 0; k < kJacCols; ++k) v -= 0.5 * static_cast<double>(JT[k][r]) * static_cast<double>(Es[k][a]);
-    slot.Jd[a][r] = v;
-  }
-}
-
-// Step 4: new column a = sum_b J[a][b] (old column b) for the 32 columns of every active block pair, X in single
-// and V in double precision.  blockIdx.z splits the length of the columns.
-constexpr int kJacApplyThreads = 128;
-
-__global__ void __launch_bounds__(kJacApplyThreads, 3) jacobi_apply_kernel(const JacobiMat* mats, const JacobiSlot* slots, int round) {
-  __shared__ double Jd[kJacCols][kJacCols + 1];
-  __shared__ __align__(16) float Jf[kJacCols][kJacCols + 4];
-  const JacobiMat m = mats[blockIdx.y];
-  const JacobiSlot& slot = slots[blockIdx.y * gridDim.x + blockIdx.x];
-  if (slot.active == 0) return;
-  int bi, bj;
-  round_robin_pair(m.nblk, round % (m.nblk - 1), blockIdx.x, bi, bj);
+  const JacobiMat m = mats[blockIdx.x / kJacCluster];
+  const int crank = blockIdx.x % kJacCluster;
   const int tid = threadIdx.x;
   const int L = m.L, ld = m.ld;
-  auto global_row = [&](int a) { return (a < kJacBlock ? bi : bj) * kJacBlock + (a & (kJacBlock - 1)); };
-  for (int x = tid; x < kJacCols * kJacCols; x += kJacApplyThreads) {
-    const double v = slot.Jd[x / kJacCols][x % kJacCols];
-    Jd[x / kJacCols][x % kJacCols] = v;
-    Jf[x / kJacCols][x % kJacCols] = static_cast<float>(v);
-  }
-  __syncthreads();
-  // one element of every column per thread: 32 loads in flight, then 32 x 32 multiply-adds, then 32 stores
-  const int k = blockIdx.z * kJacApplyThreads + tid;
-  if (k >= ld) return;
-  {
-    float x[kJacCols];
-#pragma unroll
-    for (int b = 0; b < kJacCols; ++b) {
-      const int gr = global_row(b);
-      x[b] = gr < L ? m.XT[static_cast<long long>(gr) * ld + k] : 0.f;
-    }
-#pragma unroll 4
-    for (int a = 0; a < kJacCols; ++a) {
-      float acc = 0.f;
-#pragma unroll
-      for (int b4 = 0; b4 < kJacCols; b4 += 4) {
-        const float4 j = *reinterpret_cast<const float4*>(&Jf[a][b4]);
-        acc += j.x * x[b4] + j.y * x[b4 + 1] + j.z * x[b4 + 2] + j.w * x[b4 + 3];
-      }
-      const int gr = global_row(a);
-      if (gr < L) m.XT[static_cast<long long>(gr) * ld + k] = acc;
-    }
-  }
-  {
-    double v[kJacCols];
-#pragma unroll
-    for (int b = 0; b < kJacCols; ++b) {
-      const int gr = global_row(b);
-      v[b] = gr < L ? m.VT[static_cast<long long>(gr) * ld + k] : 0.0;
-    }
-#pragma unroll 4
-    for (int a = 0; a < kJacCols; ++a) {
-      double acc = 0.0;
-#pragma unroll
-      for (int b = 0; b < kJacCols; ++b) acc += Jd[a][b] * v[b];
-      const int gr = global_row(a);
-      if (gr < L) m.VT[static_cast<long long>(gr) * ld + k] = acc;
-    }
-  }
-}
+  const int tables = m.nblk / 2, rounds = m.nblk - 1;
+  const int groups = (tables + kJacCluster * kJacPairsPerCta - 1) / (kJacCluster * kJacPairsPerCta);
+  auto global_row = [](const JacobiPairInfo& pi, int a) {
+    return (a < kJacBlock ? pi.bi : pi.bj) * kJacBlock + (a & (kJacBlock - 1));
+  };
 
-// End of a sweep: a matrix none of whose pairs was rotated is done.
-__global__ void jacobi_sweep_end_kernel(const JacobiMat* mats, int n) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  int* f = mats[i].flags;
-  if (f[0] == 0) f[1] = 1;
-  f[0] = 0;
+  for (int sweep = 0; sweep < kJacMaxSweeps; ++sweep) {
+    for (int round = 0; round < rounds; ++round) {
+      for (int grp = 0; grp < groups; ++grp) {
+        JacobiPairInfo pis[kJacPairsPerCta];
+#pragma unroll
+        for (int p = 0; p < kJacPairsPerCta; ++p)
+          pis[p] = jacobi_pair_of(m, round, (grp * kJacCluster + crank) * kJacPairsPerCta + p);
+        if (!pis[0].live && !pis[1].live) continue;      // the same for every thread of the CTA
+
+        // ---- Gram matrices ----
+#pragma unroll 1
+        for (int p = 0; p < kJacPairsPerCta; ++p) {
+          const JacobiPairInfo pi = pis[p];
+          if (!pi.live) {
+            if (tid == 0) sh.active[p] = 0;
+            continue;
+          }
+          // 64 tiles of 4 x 4 entries, two groups of threads share the rows of a chunk
+          const int kg = tid >> 6, tile = tid & 63, ta = tile >> 3, tb = tile & 7;
+          float g[4][4];
+#pragma unroll
+          for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) g[x][y] = 0.f;
+          for (int k0 = 0; k0 < ld; k0 += kJacStageRows) {
+            __syncthreads();                                // the previous chunk has been consumed
+            for (int x = tid; x < kJacCols * (kJacStageRows / 4); x += kJacCtaThreads) {
+              const int a = x / (kJacStageRows / 4), q = x % (kJacStageRows / 4);
+              const int gr = global_row(pi, a), k = k0 + 4 * q;
+              float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (gr < L && k < ld) v = __ldcg(reinterpret_cast<const float4*>(m.XT + static_cast<long long>(gr) * ld + k));
+              *reinterpret_cast<float4*>(stage + a * kJacStageRows + 4 * (q ^ ((a >> 2) & 7))) = v;
+            }
+            __syncthreads();
+#pragma unroll 2
+            for (int q = kg; q < kJacStageRows / 4; q += 2) {
+              float4 a[4], b[4];
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                a[x] = *reinterpret_cast<const float4*>(stage + (4 * ta + x) * kJacStageRows + 4 * (q ^ ta));
+                b[x] = *reinterpret_cast<const float4*>(stage + (4 * tb + x) * kJacStageRows + 4 * (q ^ tb));
+              }
+#pragma unroll
+              for (int x = 0; x < 4; ++x)
+#pragma unroll
+                for (int y = 0; y < 4; ++y)
+                  g[x][y] += a[x].x * b[y].x + a[x].y * b[y].y + a[x].z * b[y].z + a[x].w * b[y].w;
+            }
+          }
+#pragma unroll
+          for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) Ap[kg][4 * ta + x][4 * tb + y] = g[x][y];
+          __syncthreads();
+          // the two partial matrices added in a fixed order (entry (a, b) and entry (b, a) then agree to the bit); is
+          // any pair of columns further from orthogonal than the tolerance?
+          auto entry = [&](int a, int b) { return Ap[0][a][b] + Ap[1][a][b]; };
+          int any = 0;
+          for (int x = tid; x < kJacCols * kJacCols; x += kJacCtaThreads) {
+            const int a = x / kJacCols, b = x % kJacCols;
+            const float v = a <= b ? entry(a, b) : entry(b, a);
+            As[p][a][b] = v;
+            if (a < b && v * v > kJacTol * kJacTol * entry(a, a) * entry(b, b)) any = 1;
+          }
+          any = __syncthreads_or(any);
+          if (tid == 0) {
+            sh.active[p] = any;
+            if (any) atomicOr(m.flags + sweep, 1);
+          }
+        }
+        __syncthreads();
+        const bool act0 = sh.active[0] != 0, act1 = sh.active[1] != 0;
+        if (!act0 && !act1) continue;                       // the same for every thread of the CTA
+
+        // ---- eigenvectors of the Gram matrices: 64 threads per pair, both pairs in step ----
+        {
+          const int p = tid >> 6, lt = tid & 63;
+          const int r = lt >> 1, j0 = (lt & 1) * 16;        // this thread: row r, columns j0 .. j0 + 15
+          const bool mine = p == 0 ? act0 : act1;
+          float(&A)[kJacCols][kJacPad] = As[p];
+          float(&B)[kJacCols][kJacPad] = Bs[p];
+          float(&T)[kJacCols][kJacPad] = JT[p];
+#pragma unroll
+          for (int y = 0; y < 16; ++y) T[r][j0 + y] = (r == j0 + y) ? 1.f : 0.f;
+          __syncthreads();
+          for (int isweep = 0; isweep < kJacInnerSweeps; ++isweep) {
+            int rotated = 0;
+            for (int step = 0; step < kJacCols - 1; ++step) {
+              if (lt < kJacBlock) {
+                int a, b;
+                round_robin_pair(kJacCols, step, lt, a, b);
+                const float aaa = A[a][a], abb = A[b][b], aab = A[a][b];
+                float c = 1.f, sn = 0.f;
+                if (mine && aab * aab > 1e-12f * aaa * abb && aab != 0.f) {
+                  const float tau = (abb - aaa) / (2.f * aab);
+                  const float t = (tau >= 0.f ? 1.f : -1.f) / (fabsf(tau) + sqrtf(1.f + tau * tau));
+                  c = rsqrtf(1.f + t * t);
+                  sn = t * c;
+                  rotated = 1;
+                }
+                sh.ca[p][a] = c; sh.cb[p][a] = -sn; sh.partner[p][a] = static_cast<unsigned char>(b);
+                sh.ca[p][b] = c; sh.cb[p][b] = sn; sh.partner[p][b] = static_cast<unsigned char>(a);
+              }
+              __syncthreads();
+              float t[16];
+#pragma unroll
+              for (int y = 0; y < 16; ++y)
+                t[y] = sh.ca[p][j0 + y] * A[r][j0 + y] + sh.cb[p][j0 + y] * A[r][sh.partner[p][j0 + y]];
+#pragma unroll
+              for (int y = 0; y < 16; ++y) B[r][j0 + y] = t[y];                          // B = A R
+              __syncthreads();
+              const float car = sh.ca[p][r], cbr = sh.cb[p][r];
+              const int pr = sh.partner[p][r];
+#pragma unroll
+              for (int y = 0; y < 16; ++y) {
+                A[r][j0 + y] = car * B[r][j0 + y] + cbr * B[pr][j0 + y];                 // A <- R^T B
+                t[y] = car * T[r][j0 + y] + cbr * T[pr][j0 + y];                         // row r of JT = column r of J
+              }
+              __syncthreads();
+#pragma unroll
+              for (int y = 0; y < 16; ++y) T[r][j0 + y] = t[y];
+            }
+            if (!__syncthreads_or(rotated)) break;
+          }
+          __syncthreads();
+        }
+
+        // ---- the rotations made orthogonal to second order, J <- J (I - (J^T J - I) / 2), in double precision.
+        // Thread: pair p, row a, half of the other index.  Operands are widened once, not per product. ----
+        {
+          const int p = tid >> 6, a = (tid & 63) >> 1, h0 = (tid & 1) * 16;
+          for (int x = tid; x < kJacPairsPerCta * kJacCols * kJacCols; x += kJacCtaThreads) {
+            const int pp = x / (kJacCols * kJacCols), aa = (x / kJacCols) % kJacCols, bb = x % kJacCols;
+            JTd[pp][aa][bb] = static_cast<double>(JT[pp][aa][bb]);
+          }
+          __syncthreads();
+          {
+            double row[kJacCols];                                                        // JT[a][.] = column a of J
+#pragma unroll
+            for (int k = 0; k < kJacCols; k += 2) {
+              const double2 v = *reinterpret_cast<const double2*>(&JTd[p][a][k]);
+              row[k] = v.x; row[k + 1] = v.y;
+            }
+#pragma unroll 2
+            for (int y = 0; y < 16; ++y) {
+              const int b = h0 + y;
+              double e = (a == b) ? -1.0 : 0.0;
+#pragma unroll
+              for (int k = 0; k < kJacCols; k += 2) {
+                const double2 v = *reinterpret_cast<const double2*>(&JTd[p][b][k]);
+                e += row[k] * v.x + row[k + 1] * v.y;
+              }
+              As[p][a][b] = static_cast<float>(e);                                       // (J^T J - I)_ab
+            }
+          }
+          __syncthreads();
+          {
+            double ecol[kJacCols];                                                       // (J^T J - I)[.][a]
+#pragma unroll
+            for (int k = 0; k < kJacCols; ++k) ecol[k] = static_cast<double>(As[p][k][a]);
+            __syncthreads();                                                             // region 2 changes hands
+#pragma unroll 2
+            for (int y = 0; y < 16; y += 2) {
+              const int r = h0 + y;
+              double2 acc = *reinterpret_cast<const double2*>(&JTd[p][a][r]);           // J[r][a], J[r + 1][a]
+#pragma unroll
+              for (int k = 0; k < kJacCols; ++k) {
+                const double2 v = *reinterpret_cast<const double2*>(&JTd[p][k][r]);
+                acc.x -= 0.5 * v.x * ecol[k];
+                acc.y -= 0.5 * v.y * ecol[k];
+              }
+              *reinterpret_cast<double2*>(&Jd[p][a][r]) = acc;
+            }
+          }
+          __syncthreads();
+          for (int x = tid; x < kJacPairsPerCta * kJacCols * kJacCols; x += kJacCtaThreads) {
+            const int pp = x / (kJacCols * kJacCols), aa = (x / kJacCols) % kJacCols, bb = x % kJacCols;
+            Jf[pp][aa][bb] = static_cast<float>(Jd[pp][aa][bb]);
+          }
+          __syncthreads();
+        }
+
+        // ---- new column a = sum_b J[a][b] (old column b), X in single and V in double precision ----
+#pragma unroll 1
+        for (int p = 0; p < kJacPairsPerCta; ++p) {
+          if (sh.active[p] == 0) continue;
+          const JacobiPairInfo pi = pis[p];
+          for (int k = tid; k < ld; k += kJacCtaThreads) {
+            {
+              float x[kJacCols];
+#pragma unroll
+              for (int b = 0; b < kJacCols; ++b) {
+                const int gr = global_row(pi, b);
+                x[b] = gr < L ? __ldcg(m.XT + static_cast<long long>(gr) * ld + k) : 0.f;
+              }
+#pragma unroll 4
+              for (int a = 0; a < kJacCols; ++a) {
+                float acc = 0.f;
+#pragma unroll
+                for (int b = 0; b < kJacCols; b += 4) {
+                  const float4 j = *reinterpret_cast<const float4*>(&Jf[p][a][b]);
+                  acc += j.x * x[b] + j.y * x[b + 1] + j.z * x[b + 2] + j.w * x[b + 3];
+                }
+                const int gr = global_row(pi, a);
+                if (gr < L) m.XT[static_cast<long long>(gr) * ld + k] = acc;
+              }
+            }
+            {
+              double v[kJacCols];
+#pragma unroll
+              for (int b = 0; b < kJacCols; ++b) {
+                const int gr = global_row(pi, b);
+                v[b] = gr < L ? __ldcg(m.VT + static_cast<long long>(gr) * ld + k) : 0.0;
+              }
+#pragma unroll 4
+              for (int a = 0; a < kJacCols; ++a) {
+                double acc = 0.0;
+#pragma unroll
+                for (int b = 0; b < kJacCols; b += 2) {
+                  const double2 j = *reinterpret_cast<const double2*>(&Jd[p][a][b]);
+                  acc += j.x * v[b] + j.y * v[b + 1];
+                }
+                const int gr = global_row(pi, a);
+                if (gr < L) m.VT[static_cast<long long>(gr) * ld + k] = acc;
+              }
+            }
+          }
+        }
+        __syncthreads();     // shared memory is reused by the next group of pairs
+      }
+      jacobi_cluster_barrier();
+    }
+    // every rotation of this sweep was flagged before the barrier that ended its last round
+    if (__ldcg(m.flags + sweep) == 0) break;
+  }
 }
 
 // Order the Ritz vectors by falling eigenvalue (the norm of a column of X) and write the rotation of the whole
@@ -431,25 +486,17 @@ __global__ void __launch_bounds__(256) jacobi_finish_kernel(const JacobiMat* mat
   }
 }
 
-// Diagonalise n matrices (descriptors d_mats, already initialised by jacobi_init_kernel); nblk_max and ld_max are
-// the largest block count and leading dimension among them; slots: scratch of n * nblk_max / 2 entries.
-inline cudaError_t jacobi_batched_launch(const JacobiMat* d_mats, int n, int nblk_max, int ld_max, JacobiSlot* slots,
-                                         cudaStream_t stream, int64_t* launches) {
-  const size_t smem = jacobi_smem_bytes(ld_max);
-  const int tables = nblk_max / 2, n_slots = n * tables;
-  const int parts = (ld_max + kJacApplyThreads - 1) / kJacApplyThreads;
-  for (int sweep = 0; sweep < kJacMaxSweeps; ++sweep) {
-    for (int round = 0; round < nblk_max - 1; ++round) {
-      const int r = sweep * (nblk_max - 1) + round;
-      jacobi_gram_kernel<<<dim3(tables, n), kJacThreads, smem, stream>>>(d_mats, slots, r);
-      jacobi_inner_kernel<<<n_slots, kJacInnerThreads, 0, stream>>>(slots, n_slots);
-      jacobi_polish_kernel<<<n_slots, kJacThreads, 0, stream>>>(slots);
-      jacobi_apply_kernel<<<dim3(tables, n, parts), kJacApplyThreads, 0, stream>>>(d_mats, slots, r);
-      *launches += 4;
-    }
-    jacobi_sweep_end_kernel<<<(n + 127) / 128, 128, 0, stream>>>(d_mats, n);
-    *launches += 1;
+// Diagonalise n matrices (descriptors d_mats, already initialised by jacobi_init_kernel).
+inline cudaError_t jacobi_batched_launch(const JacobiMat* d_mats, int n, cudaStream_t stream, int64_t* launches) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    const cudaError_t e = cudaFuncSetAttribute(jacobi_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>(sizeof(JacobiShared)));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
   }
+  jacobi_cluster_kernel<<<n * kJacCluster, kJacCtaThreads, sizeof(JacobiShared), stream>>>(d_mats);
+  *launches += 1;
   return cudaGetLastError();
 }
 
