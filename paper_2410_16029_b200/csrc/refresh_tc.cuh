@@ -405,6 +405,7 @@ struct RefreshMat {
 
 constexpr int kRefBN = 128;
 constexpr int kRefStages1 = 4;  // NA = 1, NB = 2: 48 KB per stage
+constexpr int kRefStages0 = 6;  // NA = 1, NB = 1: 32 KB per stage
 constexpr int kRefStages2 = 3;  // NA = 2, NB = 2: 64 KB per stage
 
 struct RefreshPlan {
@@ -795,7 +796,12 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
 
   using L1 = TcSmem<kRefBN, 1, 2, kRefStages1, 4>;
   using L2 = TcSmem<kRefBN, 2, 2, kRefStages2, 4>;
-  if (cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, false>,
+  using L0 = TcSmem<kRefBN, 1, 1, kRefStages0, 4>;
+  if (cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 1, 1, kRefStages0, TC_EPI_STORE, 4, false>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, L0::kTotal) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 1, 1, kRefStages0, TC_EPI_STORE, 4, true>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, L0::kTotal) != cudaSuccess ||
+      cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, false>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, L1::kTotal) != cudaSuccess ||
       cudaFuncSetAttribute(tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, true>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, L1::kTotal) != cudaSuccess ||
@@ -809,7 +815,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
 }
 
 
-inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
+// high_only: the products with G take only the high bf16 part of the basis (half the tensor-core work; the basis
+// then enters with 8 bits instead of 16, which the early sweeps of the iteration do not notice).
+inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches,
+                                      bool high_only = false) {
   // outputs that several K slices accumulate into start from zero
   if (plan.n_zero[g] > 0) {
     zero_jobs_kernel<<<dim3(32, plan.n_zero[g]), 256, 0, stream>>>(plan.d_zero[g]);
@@ -818,14 +827,23 @@ inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cu
   using L1 = TcSmem<kRefBN, 1, 2, kRefStages1, 4>;
   using L2 = TcSmem<kRefBN, 2, 2, kRefStages2, 4>;
   const int threads = 64 + 32 * 4;
+  using L0 = TcSmem<kRefBN, 1, 1, kRefStages0, 4>;
   switch (g) {
     case RG_Y_FROM_Z:
-      tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, false><<<plan.grid[g], threads, L1::kTotal, stream>>>(
-          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
+      if (high_only)
+        tc_gemm_kernel<kRefBN, 1, 1, kRefStages0, TC_EPI_STORE, 4, false><<<plan.grid[g], threads, L0::kTotal, stream>>>(
+            plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
+      else
+        tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, false><<<plan.grid[g], threads, L1::kTotal, stream>>>(
+            plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
       break;
     case RG_Z_FROM_Y:
-      tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, true><<<plan.grid[g], threads, L1::kTotal, stream>>>(
-          plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
+      if (high_only)
+        tc_gemm_kernel<kRefBN, 1, 1, kRefStages0, TC_EPI_STORE, 4, true><<<plan.grid[g], threads, L0::kTotal, stream>>>(
+            plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
+      else
+        tc_gemm_kernel<kRefBN, 1, 2, kRefStages1, TC_EPI_STORE, 4, true><<<plan.grid[g], threads, L1::kTotal, stream>>>(
+            plan.d_maps, plan.d_tiles[g], plan.n_tiles[g], nullptr, d_ctrl, plan.d_probs[g]);
       break;
     case RG_GRAM_Y:
     case RG_GRAM_Z:
@@ -944,9 +962,13 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
   // the norm of its column, so the second product loses nothing that an orthonormalisation of Z would have saved
   // (measured on the 1.1B shapes: the same Ritz vectors to all printed digits, a quarter of the refresh time less).
   for (int it = 0; it < q; ++it) {
-    if ((rc = refresh_tc_gemm(plan, RG_Z_FROM_Y, d_ctrl, stream, launches))) return rc;
+    // the first half of the sweeps multiplies with the high bf16 part of the basis only: what that rounding adds
+    // (2^-9 of an entry) shrinks with every later sweep like any other component outside the dominant subspace
+    // (not with fewer than four sweeps, where every one of them counts)
+    const bool coarse = q >= 4 && it < q / 2;
+    if ((rc = refresh_tc_gemm(plan, RG_Z_FROM_Y, d_ctrl, stream, launches, coarse))) return rc;
     if ((rc = refresh_tc_split(plan, false, stream, launches))) return rc;
-    if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches))) return rc;
+    if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches, coarse))) return rc;
     if ((rc = refresh_tc_orth(plan, d_ctrl, stream, launches))) return rc;
   }
   // Exact orthonormalisation of the basis that leaves the sweeps: the basis can be ill conditioned in its weak

@@ -7,10 +7,11 @@
 // matrices C (L x L, L = r' <= 875, one per weight matrix, all in one batch) by a one-sided block Jacobi method:
 // the columns of a working matrix X (started as C, scaled to a unit largest diagonal entry) are rotated against
 // each other until they are mutually orthogonal; the accumulated rotation is V and the column norms are the
-// eigenvalues.  The unit of work is one pair of 16-column blocks of one matrix: a CTA forms the 32 x 32 Gram
-// matrix of its 32 columns, four warps diagonalise that by cyclic two-sided Jacobi rotations, and a CTA applies the
-// resulting 32 x 32 rotation to the 32 columns of X and of V.  The block pairs of a round are disjoint
-// (round-robin ordering), so a round is a few launches over every matrix; a sweep is (blocks - 1) rounds.
+// eigenvalues.  The unit of work is one pair of 16-column blocks of one matrix: the 32 x 32 Gram matrix of its 32
+// columns is diagonalised by cyclic two-sided Jacobi rotations, and the resulting 32 x 32 rotation is applied to the
+// 32 columns of X and of V.  The block pairs of a round are disjoint (round-robin ordering); a sweep is
+// (blocks - 1) rounds.  All of it is one launch: a cluster of CTAs per matrix shares the pairs of a round and meets
+// at a cluster barrier between rounds (jacobi_cluster_kernel below).
 //
 // The rotation can be limited to the span of the leading k columns of the basis (JacobiMat::L = k < basis width):
 // the matrix diagonalised is then the leading k x k block of C, the first k columns of P become the Ritz vectors
@@ -38,7 +39,6 @@ namespace ngalore {
 
 constexpr int kJacBlock = 16;           // columns per block; a CTA rotates two blocks against each other
 constexpr int kJacCols = 2 * kJacBlock;
-constexpr int kJacThreads = 256;
 constexpr int kJacMaxSweeps = 12;
 constexpr float kJacTol = 1e-5f;        // a pair of columns counts as orthogonal below this cosine
 constexpr int kJacInnerSweeps = 1;      // sweeps over the 32 x 32 Gram matrix of a block pair per visit

@@ -146,10 +146,13 @@ def test_update_parity_with_the_oracles_own_svd(impl):
     assert opt.poll_status()[0] == 0
 
 
-def test_all_columns_rotated_on_request():
-    """ritz_columns = -1: every column of a 256-wide basis is a Ritz vector, in falling order."""
+@pytest.mark.parametrize("r", [256, 328])
+def test_all_columns_rotated_on_request(r):
+    """ritz_columns = -1: every column of the basis is a Ritz vector, in falling order.  r = 328 has 21 blocks of
+    16 columns (rounded up to 22): more block pairs per round than one pass of the eigensolver's CTAs takes, and a
+    last block that is half padding."""
     shapes = [(768, 1024), (1024, 768)]
-    w = wl.tiny_workload(shapes, r=256, s=2, T=0, inner_rank=16, index=73)
+    w = wl.tiny_workload(shapes, r=r, s=2, T=0, inner_rank=16, index=73)
     dev = torch.device("cuda")
     opt = _make(w, ritz_columns=-1)
     bits = [wl.gradient_bits(w, i, 0) for i in range(2)]
@@ -157,7 +160,7 @@ def test_all_columns_rotated_on_request():
     torch.cuda.synchronize()
     for i in range(2):
         P = opt.get_subspace(i).cpu().numpy().astype(np.float64)
-        assert np.max(np.abs(P.T @ P - np.eye(256))) <= 1e-5
-        n, worst = check_columns(P, wl.bf16_bits_to_f64(bits[i]), 256, shapes[i], rotated=256)
+        assert np.max(np.abs(P.T @ P - np.eye(r))) <= 1e-5
+        n, worst = check_columns(P, wl.bf16_bits_to_f64(bits[i]), r, shapes[i], rotated=r)
         assert n >= 2
     assert opt.poll_status()[0] == 0
