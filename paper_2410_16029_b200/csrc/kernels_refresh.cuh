@@ -187,52 +187,82 @@ inline cudaError_t chol_batched_launch(CholProblem* d_probs, int n, int Lmax, cu
 // (the matrix stays in L2).  Shared memory: 32 x (L - 32) doubles for the panel.
 constexpr int kCholCtaThreads = 512;
 
-inline size_t chol_cta_smem_bytes(int Lmax) {
-  const int rows = Lmax > kCholNB ? Lmax - kCholNB : 0;
-  return sizeof(double) * static_cast<size_t>(kCholNB) * (rows + 4);
+// Row length of the panel in shared memory: a multiple of 16 bytes, so that four consecutive rows load at once.
+template <typename T>
+__host__ __device__ inline int chol_cta_ldp(int trailing) {
+  return sizeof(T) == 8 ? trailing + 4 - (trailing & 1) : (trailing + 7) & ~3;
 }
 
+template <typename T>
+inline size_t chol_cta_smem_bytes(int Lmax) {
+  const int rows = Lmax > kCholNB ? Lmax - kCholNB : 0;
+  return sizeof(T) * static_cast<size_t>(kCholNB) * (chol_cta_ldp<T>(rows) + 4);
+}
+
+__device__ __forceinline__ void chol_load4(const double* p, double (&a)[4]) {
+  const double2 lo = *reinterpret_cast<const double2*>(p), hi = *reinterpret_cast<const double2*>(p + 2);
+  a[0] = lo.x; a[1] = lo.y; a[2] = hi.x; a[3] = hi.y;
+}
+__device__ __forceinline__ void chol_load4(const float* p, float (&a)[4]) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w;
+}
+
+// T = double: the factorisation as described.  T = float: the same on a matrix stored as L x L floats at the same
+// address (CholProblem::C reinterpreted); enough for the orthonormalisations between the products of the subspace
+// iteration, whose Gram matrices come from the tensor cores with 2^-17 of relative accuracy and carry a shift of
+// about 1e-2 on a unit diagonal, and about twice as fast (half the shared-memory traffic per multiply-add, twice
+// the arithmetic rate).
+template <typename T>
 __global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const CholProblem* probs) {
   constexpr int NB = kCholNB;
-  extern __shared__ __align__(16) double chol_ps[];   // panel, k-major: chol_ps[k * ldp + (row - base)]
-  __shared__ double D[NB][NB + 1];
-  __shared__ double s_tiny;
+  extern __shared__ __align__(16) unsigned char chol_ps_raw[];
+  T* chol_ps = reinterpret_cast<T*>(chol_ps_raw);    // panel, k-major: chol_ps[k * ldp + (row - base)]
+  __shared__ T D[NB][NB + 1];
+  __shared__ T s_tiny;
   const CholProblem p = probs[blockIdx.x];
-  double* C = p.C;
+  T* C = reinterpret_cast<T*>(p.C);
   const int L = p.L;
   const int tid = threadIdx.x;
   // pivot floor from the diagonal (a pivot that is not above it is replaced by it, see chol_begin_kernel)
   if (tid < 32) {
-    double md = 0.0;
-    for (int i = tid; i < L; i += 32) md = fmax(md, C[static_cast<long long>(i) * L + i]);
+    T md = 0;
+    for (int i = tid; i < L; i += 32) {
+      const T v = C[static_cast<long long>(i) * L + i];
+      md = v > md ? v : md;
+    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) md = fmax(md, __shfl_xor_sync(0xffffffffu, md, o));
-    if (tid == 0) s_tiny = fmax(md, 1e-300) * 1e-28;
+    for (int o = 16; o > 0; o >>= 1) {
+      const T v = __shfl_xor_sync(0xffffffffu, md, o);
+      md = v > md ? v : md;
+    }
+    if (tid == 0) s_tiny = sizeof(T) == 8 ? static_cast<T>(fmax(static_cast<double>(md), 1e-300) * 1e-28)
+                                          : static_cast<T>(fmax(static_cast<double>(md), 1e-30) * 1e-12);
   }
   __syncthreads();
-  const double tiny = s_tiny;
+  const T tiny = s_tiny;
   for (int j0 = 0; j0 < L; j0 += NB) {
     const int nbj = (L - j0 < NB) ? (L - j0) : NB;
     const int base = j0 + nbj;            // first row / column of the trailing part
-    const int T = L - base;               // its size
-    const int ldp = T + 4 - (T & 1);      // even, so that pairs of rows are 16-byte aligned
+    const int Tn = L - base;              // its size
+    const int ldp = chol_cta_ldp<T>(Tn);
     for (int x = tid; x < NB * NB; x += kCholCtaThreads) {
       const int a = x / NB, b = x % NB;
-      D[a][b] = (a < nbj && b < nbj) ? C[static_cast<long long>(j0 + a) * L + j0 + b] : 0.0;
+      D[a][b] = (a < nbj && b < nbj) ? C[static_cast<long long>(j0 + a) * L + j0 + b] : T(0);
     }
     __syncthreads();
     if (tid < 32) {
       const int lane = tid;
       for (int k = 0; k < nbj; ++k) {
-        double dkk = D[k][k];
+        T dkk = D[k][k];
         if (!(dkk > tiny)) dkk = tiny;
-        const double lkk = sqrt(dkk);
+        const T lkk = sqrt(dkk);
         __syncwarp();
         if (lane == k) D[k][k] = lkk;
         if (lane > k && lane < nbj) D[lane][k] /= lkk;
         __syncwarp();
         if (lane > k && lane < nbj) {
-          const double lik = D[lane][k];
+          const T lik = D[lane][k];
           for (int j = k + 1; j <= lane; ++j) D[lane][j] -= lik * D[j][k];
         }
         __syncwarp();
@@ -245,18 +275,18 @@ __global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const Chol
     }
     // panel rows: x D^T = c by forward substitution, one thread per row
     for (int i = base + tid; i < L; i += kCholCtaThreads) {
-      double xr[NB];
-      double* crow = C + static_cast<long long>(i) * L + j0;
+      T xr[NB];
+      T* crow = C + static_cast<long long>(i) * L + j0;
 #pragma unroll
       for (int jj = 0; jj < NB; ++jj) {
         if (jj < nbj) {
-          double a = crow[jj];
+          T a = crow[jj];
 #pragma unroll
           for (int t = 0; t < NB; ++t)
             if (t < jj) a -= xr[t] * D[jj][t];
           xr[jj] = a / D[jj][jj];
         } else {
-          xr[jj] = 0.0;
+          xr[jj] = T(0);
         }
       }
 #pragma unroll
@@ -267,8 +297,8 @@ __global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const Chol
     }
     __syncthreads();
     // trailing update on the lower triangle: C[i][j] -= sum_k panel[i][k] panel[j][k], 4 x 4 tiles
-    if (T > 0) {
-      const int nt = (T + 3) >> 2;
+    if (Tn > 0) {
+      const int nt = (Tn + 3) >> 2;
       const int ntiles = nt * (nt + 1) / 2;
       for (int t = tid; t < ntiles; t += kCholCtaThreads) {
         int ti = static_cast<int>((sqrtf(8.f * t + 1.f) - 1.f) * 0.5f);
@@ -276,19 +306,19 @@ __global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const Chol
         while (ti * (ti + 1) / 2 > t) --ti;
         const int tj = t - ti * (ti + 1) / 2;
         const int i0 = 4 * ti, c0 = 4 * tj;        // relative to base
-        double acc[4][4];
+        T acc[4][4];
 #pragma unroll
         for (int x = 0; x < 4; ++x)
 #pragma unroll
-          for (int y = 0; y < 4; ++y) acc[x][y] = 0.0;
+          for (int y = 0; y < 4; ++y) acc[x][y] = T(0);
 #pragma unroll 4
         for (int k = 0; k < NB; ++k) {
-          const double* pk = chol_ps + k * ldp;
-          // (rows beyond T inside the last tile read the padding or the next column's start: finite values that
-          // the bounds check below keeps from being stored)
-          const double2 a01 = *reinterpret_cast<const double2*>(pk + i0), a23 = *reinterpret_cast<const double2*>(pk + i0 + 2);
-          const double2 b01 = *reinterpret_cast<const double2*>(pk + c0), b23 = *reinterpret_cast<const double2*>(pk + c0 + 2);
-          const double a[4] = {a01.x, a01.y, a23.x, a23.y}, b[4] = {b01.x, b01.y, b23.x, b23.y};
+          const T* pk = chol_ps + k * ldp;
+          // (rows beyond the trailing part inside the last tile read the padding or the next column's start: finite
+          // values that the bounds check below keeps from being stored)
+          T a[4], b[4];
+          chol_load4(pk + i0, a);
+          chol_load4(pk + c0, b);
 #pragma unroll
           for (int x = 0; x < 4; ++x)
 #pragma unroll
@@ -311,8 +341,9 @@ __global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const Chol
 }
 
 // Factor n matrices, one CTA each (the list should start with the largest matrices: CTAs are handed out in order).
+template <typename T>
 inline cudaError_t chol_cta_launch(const CholProblem* d_probs, int n, int Lmax, cudaStream_t stream, int64_t* launches) {
-  chol_cta_kernel<<<n, kCholCtaThreads, chol_cta_smem_bytes(Lmax), stream>>>(d_probs);
+  chol_cta_kernel<T><<<n, kCholCtaThreads, chol_cta_smem_bytes<T>(Lmax), stream>>>(d_probs);
   *launches += 1;
   return cudaGetLastError();
 }

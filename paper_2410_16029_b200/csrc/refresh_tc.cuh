@@ -90,7 +90,8 @@ __global__ void zero_jobs_kernel(const ZeroJob* jobs) {
 
 struct GramPrep {
   const float* C32;  // L x L Gram matrix from the tensor cores
-  double* C64;       // L x L, lower triangle written: column-scaled, symmetrised Gram + shift I
+  double* C64;       // L x L, lower triangle written: column-scaled, symmetrised Gram + shift I (as doubles, or
+                     // as L x L floats at the same address: gram_prep_kernel<float>)
   double* D;         // L column norms d_i = sqrt(C_ii)
   int L;
 };
@@ -106,6 +107,7 @@ __host__ __device__ inline double gram_shift(int L) { return static_cast<double>
 // Scaling the columns to unit norm first makes the shift act on every column alike, whatever its
 // norm, so weak directions are still orthogonalised against each other and re-normalised.
 // (blockIdx.y shares the entries of a matrix among several CTAs; each of them forms the column norms for itself)
+template <typename T>
 __global__ void __launch_bounds__(256) gram_prep_kernel(const GramPrep* probs, double shift_scale) {
   __shared__ double Ds[880];
   const GramPrep p = probs[blockIdx.x];
@@ -122,7 +124,7 @@ __global__ void __launch_bounds__(256) gram_prep_kernel(const GramPrep* probs, d
     double v = 0.5 * (static_cast<double>(p.C32[x]) + static_cast<double>(p.C32[static_cast<long long>(j) * p.L + i]));
     v /= Ds[i] * Ds[j];
     if (i == j) v = 1.0 + shift_scale * gram_shift(p.L);
-    p.C64[x] = v;
+    reinterpret_cast<T*>(p.C64)[x] = static_cast<T>(v);
   }
 }
 
@@ -218,73 +220,82 @@ struct TriInverse {
 //   [[A, 0], [C, B]]^-1 = [[A^-1, 0], [-B^-1 C A^-1, B^-1]],
 // leaves (<= 32 x 32) by forward substitution, inner nodes by two small batched fp64 GEMMs per level.
 
+// (the pointers of TriLeaf and TriGemm are those of elements of type T, whatever their declared type: the tables
+// exist once for matrices of doubles and once for the same buffers holding floats)
 struct TriLeaf {
-  const double* Lf;  // top-left element of the diagonal block inside the L x L factor
-  double* X;         // same position inside X
+  const void* Lf;  // top-left element of the diagonal block inside the L x L factor
+  void* X;         // same position inside X
   int ld, size;
 };
 
 // One warp per leaf; lane j solves column j of the block by forward substitution in shared memory.
+template <typename T>
 __global__ void __launch_bounds__(128) tri_leaf_kernel(const TriLeaf* leaves, int n_leaves) {
-  __shared__ double blk[4][32][33];
+  __shared__ T blk[4][32][33];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int id = blockIdx.x * 4 + warp;
   if (id >= n_leaves) return;
   const TriLeaf lf = leaves[id];
+  const T* Lf = static_cast<const T*>(lf.Lf);
+  T* X = static_cast<T*>(lf.X);
   for (int i = 0; i < lf.size; ++i)
-    if (lane < lf.size) blk[warp][i][lane] = lf.Lf[static_cast<long long>(i) * lf.ld + lane];
+    if (lane < lf.size) blk[warp][i][lane] = Lf[static_cast<long long>(i) * lf.ld + lane];
   __syncwarp();
   if (lane < lf.size) {
-    double x[32];
+    T x[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-      double acc = (i == lane) ? 1.0 : 0.0;
+      T acc = (i == lane) ? T(1) : T(0);
       if (i < lf.size && i >= lane) {
 #pragma unroll
         for (int k = 0; k < 32; ++k)
           if (k < i && k >= lane) acc -= blk[warp][i][k] * x[k];
         acc /= blk[warp][i][i];
       } else {
-        acc = 0.0;
+        acc = T(0);
       }
       x[i] = acc;
-      if (i < lf.size) lf.X[static_cast<long long>(i) * lf.ld + lane] = acc;
+      if (i < lf.size) X[static_cast<long long>(i) * lf.ld + lane] = acc;
     }
   }
 }
 
 struct TriGemm {
-  const double* A;  // m x k
-  const double* B;  // k x n
-  double* C;        // m x n = (negate ? -1 : 1) * A B
+  const void* A;  // m x k
+  const void* B;  // k x n
+  void* C;        // m x n = (negate ? -1 : 1) * A B
   int lda, ldb, ldc, m, n, k, negate;
 };
 
-// Batched small fp64 GEMM: blockIdx.z selects the problem, (blockIdx.y, blockIdx.x) a 64 x 64 tile of it.
+// Batched small GEMM: blockIdx.z selects the problem, (blockIdx.y, blockIdx.x) a 64 x 64 tile of it.
+template <typename T>
 __global__ void __launch_bounds__(256) tri_gemm_kernel(const TriGemm* probs) {
-  __shared__ double As[16][64 + 1];
-  __shared__ double Bs[16][64 + 1];
+  __shared__ T As[16][64 + 1];
+  __shared__ T Bs[16][64 + 1];
   const TriGemm g = probs[blockIdx.z];
+  const T* gA = static_cast<const T*>(g.A);
+  const T* gB = static_cast<const T*>(g.B);
+  T* gC = static_cast<T*>(g.C);
   const int i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
   if (i0 >= g.m || j0 >= g.n) return;
   const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
-  double acc[4][4];
+  T acc[4][4];
 #pragma unroll
   for (int a = 0; a < 4; ++a)
 #pragma unroll
-    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+    for (int b = 0; b < 4; ++b) acc[a][b] = T(0);
   for (int k0 = 0; k0 < g.k; k0 += 16) {
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
       const int kk = t & 15, i = (t >> 4) + 16 * p;  // A: k contiguous
-      As[kk][i] = (i0 + i < g.m && k0 + kk < g.k) ? g.A[static_cast<long long>(i0 + i) * g.lda + k0 + kk] : 0.0;
+      As[kk][i] = (i0 + i < g.m && k0 + kk < g.k) ? gA[static_cast<long long>(i0 + i) * g.lda + k0 + kk] : T(0);
       const int j = t & 63, kb = (t >> 6) + 4 * p;   // B: n contiguous
-      Bs[kb][j] = (j0 + j < g.n && k0 + kb < g.k) ? g.B[static_cast<long long>(k0 + kb) * g.ldb + j0 + j] : 0.0;
+      Bs[kb][j] = (j0 + j < g.n && k0 + kb < g.k) ? gB[static_cast<long long>(k0 + kb) * g.ldb + j0 + j] : T(0);
     }
     __syncthreads();
 #pragma unroll
     for (int kk = 0; kk < 16; ++kk) {
-      double a[4], b[4];
+      T a[4], b[4];
 #pragma unroll
       for (int x = 0; x < 4; ++x) { a[x] = As[kk][ty * 4 + x]; b[x] = Bs[kk][tx * 4 + x]; }
 #pragma unroll
@@ -301,18 +312,20 @@ __global__ void __launch_bounds__(256) tri_gemm_kernel(const TriGemm* probs) {
 #pragma unroll
     for (int y = 0; y < 4; ++y) {
       const int j = j0 + tx * 4 + y;
-      if (j < g.n) g.C[static_cast<long long>(i) * g.ldc + j] = g.negate ? -acc[x][y] : acc[x][y];
+      if (j < g.n) gC[static_cast<long long>(i) * g.ldc + j] = g.negate ? -acc[x][y] : acc[x][y];
     }
   }
 }
 
 // R^-1 = D^-1 X^T (upper triangular) split into two bf16 parts; blockIdx.x = matrix, blockIdx.y = share of its entries.
+template <typename T>
 __global__ void __launch_bounds__(256) tri_convert_kernel(const TriInverse* probs) {
   const TriInverse p = probs[blockIdx.x];
+  const T* X = reinterpret_cast<const T*>(p.X);
   const long long total = static_cast<long long>(p.L) * p.L;
   for (long long x = blockIdx.y * 256 + threadIdx.x; x < total; x += 256ll * gridDim.y) {
     const int j = static_cast<int>(x / p.L), i = static_cast<int>(x % p.L);  // entry (j, i) of R^-1
-    const double v = (i >= j) ? p.X[static_cast<long long>(i) * p.L + j] / p.D[j] : 0.0;
+    const double v = (i >= j) ? static_cast<double>(X[static_cast<long long>(i) * p.L + j]) / p.D[j] : 0.0;
     const float f = static_cast<float>(fmin(fmax(v, -1e30), 1e30));
     const __nv_bfloat16 h = __float2bfloat16_rn(f);
     p.Rhi[static_cast<long long>(j) * p.ld + i] = h;
@@ -417,7 +430,7 @@ struct RefreshPlan {
   std::vector<CUtensorMap> h_maps;  // RM_COUNT per matrix
   std::vector<const void*> last_G;
   char* buf = nullptr;
-  char* tri_tables = nullptr;
+  char* tri_tables[2] = {nullptr, nullptr};
   CUtensorMap* d_maps = nullptr;
   TcProblem* d_probs[RG_COUNT] = {};
   TcTile* d_tiles[RG_COUNT] = {};
@@ -433,10 +446,10 @@ struct RefreshPlan {
   CholProblem* d_chol_sorted = nullptr;  // the same problems, widest first (for the one-CTA-per-matrix kernel)
   int l_max = 0;  // largest basis width L of the set
   TriInverse* d_tri = nullptr;
-  TriLeaf* d_leaves = nullptr;
+  TriLeaf* d_leaves[2] = {nullptr, nullptr};   // [0]: the buffers hold doubles, [1]: floats
   int n_leaves = 0;
-  TriGemm* d_tg1[kTriMaxLevels] = {};
-  TriGemm* d_tg2[kTriMaxLevels] = {};
+  TriGemm* d_tg1[2][kTriMaxLevels] = {};
+  TriGemm* d_tg2[2][kTriMaxLevels] = {};
   int n_tg[kTriMaxLevels] = {};
   int tg_max[kTriMaxLevels] = {};
   int tri_levels = 0;
@@ -457,11 +470,12 @@ struct RefreshPlan {
 
 inline void refresh_plan_destroy(RefreshPlan& plan) {
   if (plan.buf) cudaFree(plan.buf);
-  if (plan.tri_tables) cudaFree(plan.tri_tables);
+  for (int set = 0; set < 2; ++set)
+    if (plan.tri_tables[set]) cudaFree(plan.tri_tables[set]);
   if (plan.zero_tables) cudaFree(plan.zero_tables);
   plan.zero_tables = nullptr;
   plan.buf = nullptr;
-  plan.tri_tables = nullptr;
+  plan.tri_tables[0] = plan.tri_tables[1] = nullptr;
   plan.ready = false;
 }
 
@@ -646,8 +660,9 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     probs[RG_GRAM_Z][i] = TcProblem{m.C32, m.L, m.L, m.L, base + RM_Z_B, base + RM_Z_B, 0};
     probs[RG_APPLY_Y][i] = TcProblem{m.Yf, m.M, m.L, m.L, base + RM_Y_A, base + RM_RINV, 0};
   }
-  // ---- tables of the blocked triangular inverse
-  {
+  // ---- tables of the blocked triangular inverse, for the buffers holding doubles (set 0) and floats (set 1)
+  for (int set = 0; set < 2; ++set) {
+    const size_t esz = set == 0 ? sizeof(double) : sizeof(float);
     std::vector<TriLeaf> leaves;
     std::vector<TriGemm> g1[kTriMaxLevels], g2[kTriMaxLevels];
     int max_level = 0;
@@ -655,26 +670,30 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
       const RefreshMat& m = plan.mats[i];
       // returns the height of the node covering [lo, hi)
       struct Rec {
-        static int go(const RefreshMat& m, int lo, int hi, std::vector<TriLeaf>& leaves, std::vector<TriGemm>* g1,
-                      std::vector<TriGemm>* g2) {
+        size_t esz;
+        void* at(double* buf, const RefreshMat& m, int row, int col) const {
+          return reinterpret_cast<char*>(buf) + esz * (static_cast<size_t>(row) * m.L + col);
+        }
+        int go(const RefreshMat& m, int lo, int hi, std::vector<TriLeaf>& leaves, std::vector<TriGemm>* g1,
+               std::vector<TriGemm>* g2) const {
           const int len = hi - lo;
           if (len <= 32) {
-            leaves.push_back(TriLeaf{m.C64 + static_cast<long long>(lo) * m.L + lo, m.X64 + static_cast<long long>(lo) * m.L + lo, m.L, len});
+            leaves.push_back(TriLeaf{at(m.C64, m, lo, lo), at(m.X64, m, lo, lo), m.L, len});
             return 0;
           }
           const int mid = lo + ((len / 2 + 31) / 32) * 32;
           const int ha = go(m, lo, mid, leaves, g1, g2), hb = go(m, mid, hi, leaves, g1, g2);
           const int h = (ha > hb ? ha : hb) + 1;
           // T = C A^-1 with C = Lf[mid:hi, lo:mid];  X[mid:hi, lo:mid] = -B^-1 T
-          double* T = m.T64 + static_cast<long long>(mid) * m.L + lo;
-          g1[h].push_back(TriGemm{m.C64 + static_cast<long long>(mid) * m.L + lo, m.X64 + static_cast<long long>(lo) * m.L + lo, T,
-                                  m.L, m.L, m.L, hi - mid, mid - lo, mid - lo, 0});
-          g2[h].push_back(TriGemm{m.X64 + static_cast<long long>(mid) * m.L + mid, T, m.X64 + static_cast<long long>(mid) * m.L + lo,
-                                  m.L, m.L, m.L, hi - mid, mid - lo, hi - mid, 1});
+          void* T = at(m.T64, m, mid, lo);
+          g1[h].push_back(TriGemm{at(m.C64, m, mid, lo), at(m.X64, m, lo, lo), T, m.L, m.L, m.L, hi - mid, mid - lo,
+                                  mid - lo, 0});
+          g2[h].push_back(TriGemm{at(m.X64, m, mid, mid), T, at(m.X64, m, mid, lo), m.L, m.L, m.L, hi - mid, mid - lo,
+                                  hi - mid, 1});
           return h;
         }
       };
-      const int h = Rec::go(m, 0, m.L, leaves, g1, g2);
+      const int h = Rec{esz}.go(m, 0, m.L, leaves, g1, g2);
       if (h > max_level) max_level = h;
     }
     if (max_level >= kTriMaxLevels) return NGALORE_ERR_INVALID_ARG;
@@ -685,10 +704,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     bytes = (bytes + 255) / 256 * 256 + 256;
     char* tb = nullptr;
     if (cudaMalloc(&tb, bytes) != cudaSuccess) return NGALORE_ERR_ALLOC;
-    plan.tri_tables = tb;
+    plan.tri_tables[set] = tb;
     plan.device_bytes += bytes;
     size_t o = 0;
-    plan.d_leaves = reinterpret_cast<TriLeaf*>(tb);
+    plan.d_leaves[set] = reinterpret_cast<TriLeaf*>(tb);
     if (cudaMemcpy(tb, leaves.data(), sizeof(TriLeaf) * leaves.size(), cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
     o = (sizeof(TriLeaf) * leaves.size() + 255) / 256 * 256;
     for (int h = 1; h <= max_level; ++h) {
@@ -697,10 +716,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
       int mx = 1;
       for (const TriGemm& g : g1[h]) { if (g.m > mx) mx = g.m; if (g.n > mx) mx = g.n; }
       plan.tg_max[h] = mx;
-      plan.d_tg1[h] = reinterpret_cast<TriGemm*>(tb + o);
+      plan.d_tg1[set][h] = reinterpret_cast<TriGemm*>(tb + o);
       if (sz && cudaMemcpy(tb + o, g1[h].data(), sz, cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
       o += (sz + 255) / 256 * 256;
-      plan.d_tg2[h] = reinterpret_cast<TriGemm*>(tb + o);
+      plan.d_tg2[set][h] = reinterpret_cast<TriGemm*>(tb + o);
       if (sz && cudaMemcpy(tb + o, g2[h].data(), sz, cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
       o += (sz + 255) / 256 * 256;
     }
@@ -721,8 +740,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     std::stable_sort(sorted.begin(), sorted.end(), [](const CholProblem& a, const CholProblem& b) { return a.L > b.L; });
     if (cudaMemcpy(plan.d_chol_sorted, sorted.data(), sizeof(CholProblem) * n, cudaMemcpyHostToDevice) != cudaSuccess)
       return NGALORE_ERR_CUDA;
-    if (cudaFuncSetAttribute(chol_cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(chol_cta_smem_bytes(plan.l_max))) != cudaSuccess)
+    if (cudaFuncSetAttribute(chol_cta_kernel<double>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(chol_cta_smem_bytes<double>(plan.l_max))) != cudaSuccess ||
+        cudaFuncSetAttribute(chol_cta_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(chol_cta_smem_bytes<float>(plan.l_max))) != cudaSuccess)
       return NGALORE_ERR_CUDA;
   }
   plan.d_tri = reinterpret_cast<TriInverse*>(plan.buf + o_tri);
@@ -859,20 +880,22 @@ inline ngalore_status refresh_tc_gemm(RefreshPlan& plan, int g, Ctrl* d_ctrl, cu
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
-// X = Lf^-1 for every matrix (blocked), then R^-1 = D^-1 X^T in two bf16 parts.
+// X = Lf^-1 for every matrix (blocked), then R^-1 = D^-1 X^T in two bf16 parts.  T: what the buffers hold.
+template <typename T>
 inline ngalore_status refresh_tc_tri_inverse(RefreshPlan& plan, cudaStream_t stream, int64_t* launches) {
+  constexpr int set = sizeof(T) == 8 ? 0 : 1;
   zero_jobs_kernel<<<dim3(32, plan.n_zero[RG_COUNT]), 256, 0, stream>>>(plan.d_zero[RG_COUNT]);
   *launches += 1;
-  tri_leaf_kernel<<<(plan.n_leaves + 3) / 4, 128, 0, stream>>>(plan.d_leaves, plan.n_leaves);
+  tri_leaf_kernel<T><<<(plan.n_leaves + 3) / 4, 128, 0, stream>>>(plan.d_leaves[set], plan.n_leaves);
   *launches += 1;
   for (int h = 1; h <= plan.tri_levels; ++h) {
     if (plan.n_tg[h] == 0) continue;
     const int tiles = (plan.tg_max[h] + 63) / 64;
-    tri_gemm_kernel<<<dim3(tiles, tiles, plan.n_tg[h]), 256, 0, stream>>>(plan.d_tg1[h]);
-    tri_gemm_kernel<<<dim3(tiles, tiles, plan.n_tg[h]), 256, 0, stream>>>(plan.d_tg2[h]);
+    tri_gemm_kernel<T><<<dim3(tiles, tiles, plan.n_tg[h]), 256, 0, stream>>>(plan.d_tg1[set][h]);
+    tri_gemm_kernel<T><<<dim3(tiles, tiles, plan.n_tg[h]), 256, 0, stream>>>(plan.d_tg2[set][h]);
     *launches += 2;
   }
-  tri_convert_kernel<<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_tri);
+  tri_convert_kernel<T><<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_tri);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
@@ -889,10 +912,11 @@ inline ngalore_status refresh_tc_orth(RefreshPlan& plan, Ctrl* d_ctrl, cudaStrea
   ngalore_status rc;
   if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, RG_GRAM_Y, d_ctrl, stream, launches))) return rc;
-  gram_prep_kernel<<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_prep, shift_scale);
+  // single precision from here to R^-1: the Gram matrix has 2^-17 of relative accuracy and a shift of about 1e-2
+  gram_prep_kernel<float><<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_prep, shift_scale);
   *launches += 1;
-  if (chol_cta_launch(plan.d_chol_sorted, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
-  if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
+  if (chol_cta_launch<float>(plan.d_chol_sorted, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
+  if ((rc = refresh_tc_tri_inverse<float>(plan, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches))) return rc;
   return refresh_tc_split(plan, true, stream, launches);
 }
@@ -909,8 +933,8 @@ inline ngalore_status refresh_tc_final(RefreshPlan& plan, Ctrl* d_ctrl, cudaStre
   syrk_f64_kernel<<<plan.n_syrk_tiles, 256, 0, stream>>>(plan.d_syrk_mats, plan.d_syrk_tiles);
   gram_prep64_kernel<<<plan.n, 256, 0, stream>>>(plan.d_prep64);
   *launches += 2;
-  if (chol_cta_launch(plan.d_chol_sorted, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
-  if ((rc = refresh_tc_tri_inverse(plan, stream, launches))) return rc;
+  if (chol_cta_launch<double>(plan.d_chol_sorted, plan.n, plan.l_max, stream, launches) != cudaSuccess) return NGALORE_ERR_CUDA;
+  if ((rc = refresh_tc_tri_inverse<double>(plan, stream, launches))) return rc;
   return refresh_tc_gemm(plan, RG_APPLY_Y, d_ctrl, stream, launches);
 }
 
