@@ -37,7 +37,11 @@ struct TcProblem {
   float* out;
   int out_rows, out_cols, ld_out;
   int map_a, map_b;
-  int pad;
+  int ld16 = 0;
+  // if set (problems whose K is not split only): the result is written as two bf16 parts, hi = bf16(x) and
+  // lo = bf16(x - hi), rows of ld16 elements, instead of as fp32 into `out`
+  __nv_bfloat16* out_hi = nullptr;
+  __nv_bfloat16* out_lo = nullptr;
 };
 
 struct TcTile {
@@ -318,13 +322,17 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
       if (kGroups == 2 && (local & 1) != group) continue;
       const TcTile tile = tiles[t];
       float* out;
-      int rows_total, out_cols, ld_out;
+      __nv_bfloat16 *out_hi = nullptr, *out_lo = nullptr;
+      int rows_total, out_cols, ld_out, ld16 = 0;
       if (EPI == TC_EPI_STORE) {
         const TcProblem pr = probs[tile.mat];
         out = pr.out;
         rows_total = pr.out_rows;
         out_cols = pr.out_cols;
         ld_out = pr.ld_out;
+        out_hi = pr.out_hi;
+        out_lo = pr.out_lo;
+        ld16 = pr.ld16;
       } else {
         const MatDesc& d = mats[tile.mat];
         out_cols = tile.cols;
@@ -366,7 +374,17 @@ tc_gemm_kernel(const CUtensorMap* __restrict__ tmaps, const TcTile* __restrict__
               if (row < rows_total) {
                 const float4 acc = *reinterpret_cast<const float4*>(stg + rr * 36 + sub_col);
                 float* p = out + static_cast<long long>(row) * ld_out + col;
-                if (tile.atomic) {
+                if (EPI == TC_EPI_STORE && out_hi != nullptr) {
+                  const __nv_bfloat162 h01 = __floats2bfloat162_rn(acc.x, acc.y), h23 = __floats2bfloat162_rn(acc.z, acc.w);
+                  const __nv_bfloat162 l01 = __floats2bfloat162_rn(acc.x - __low2float(h01), acc.y - __high2float(h01));
+                  const __nv_bfloat162 l23 = __floats2bfloat162_rn(acc.z - __low2float(h23), acc.w - __high2float(h23));
+                  uint2 hv, lv;
+                  hv.x = *reinterpret_cast<const uint32_t*>(&h01); hv.y = *reinterpret_cast<const uint32_t*>(&h23);
+                  lv.x = *reinterpret_cast<const uint32_t*>(&l01); lv.y = *reinterpret_cast<const uint32_t*>(&l23);
+                  const long long o = static_cast<long long>(row) * ld16 + col;
+                  *reinterpret_cast<uint2*>(out_hi + o) = hv;
+                  *reinterpret_cast<uint2*>(out_lo + o) = lv;
+                } else if (tile.atomic) {
                   atomicAdd(reinterpret_cast<float4*>(p), acc);
                 } else {
                   *reinterpret_cast<float4*>(p) = acc;

@@ -17,6 +17,8 @@
 #include <cstring>
 #include <vector>
 
+#include <algorithm>
+
 #include "gemm_tcgen05.cuh"
 #include "kernels_refresh.cuh"
 #include "ritz_jacobi.cuh"
@@ -454,6 +456,11 @@ struct RefreshPlan {
   int tg_max[kTriMaxLevels] = {};
   int tri_levels = 0;
   SplitJob* d_split_y = nullptr;
+  // the matrices whose product with G splits K (their result arrives as fp32 and is split afterwards; all others
+  // leave the product as bf16 parts already)
+  SplitJob* d_split_y_rest = nullptr;
+  SplitJob* d_split_z_rest = nullptr;
+  int n_split_y_rest = 0, n_split_z_rest = 0;
   SyrkMat* d_syrk_mats = nullptr;
   SyrkTile* d_syrk_tiles = nullptr;
   int n_syrk_tiles = 0;
@@ -589,6 +596,8 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   const size_t o_prep64 = take(sizeof(GramPrep64) * n);
   const size_t o_sy = take(sizeof(SplitJob) * n);
   const size_t o_sz = take(sizeof(SplitJob) * n);
+  const size_t o_sy_rest = take(sizeof(SplitJob) * n);
+  const size_t o_sz_rest = take(sizeof(SplitJob) * n);
   const size_t o_jac = take(sizeof(JacobiMat) * n);
   const size_t o_jac_init = take(sizeof(JacobiInit) * n);
   const size_t o_jac_out = take(sizeof(JacobiOut) * n);
@@ -604,7 +613,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   plan.l_max = 0;
   for (const RefreshMat& m : plan.mats) plan.l_max = m.L > plan.l_max ? m.L : plan.l_max;
   std::vector<TriInverse> tri(n);
-  std::vector<SplitJob> sy(n), sz(n);
+  std::vector<SplitJob> sy(n), sz(n), sy_rest, sz_rest;
   std::vector<SyrkMat> syrk_m(n);
   std::vector<GramPrep64> prep64(n);
   std::vector<JacobiMat> jac(n);
@@ -633,6 +642,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     prep64[i] = GramPrep64{m.X64, m.C64, m.D, m.L};
     sy[i] = SplitJob{m.Yf, m.Yhi, m.Ylo, static_cast<long long>(m.M) * m.L, m.L, m.ldl};
     sz[i] = SplitJob{m.Zf, m.Zhi, m.Zlo, static_cast<long long>(m.N) * m.L, m.L, m.ldl};
+    if (std::find(plan.atomic_mats[RG_Y_FROM_Z].begin(), plan.atomic_mats[RG_Y_FROM_Z].end(), i) != plan.atomic_mats[RG_Y_FROM_Z].end())
+      sy_rest.push_back(sy[i]);
+    if (std::find(plan.atomic_mats[RG_Z_FROM_Y].begin(), plan.atomic_mats[RG_Z_FROM_Y].end(), i) != plan.atomic_mats[RG_Z_FROM_Y].end())
+      sz_rest.push_back(sz[i]);
     // the Jacobi rotation keeps X (fp32) in the memory of T64 and V (fp64) in X64 (L is a multiple of 4 on this path)
     // (width of the rotated part: all of the basis, or its leading ritz_columns, kept a multiple of 4)
     const int Lj = std::min(m.L, (ritz_columns + 3) & ~3);
@@ -656,6 +669,16 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
     const int base = i * RM_COUNT;
     probs[RG_Y_FROM_Z][i] = TcProblem{m.Yf, m.M, m.L, m.L, base + RM_G_A, base + RM_Z_B, 0};
     probs[RG_Z_FROM_Y][i] = TcProblem{m.Zf, m.N, m.L, m.L, base + RM_G_MN, base + RM_Y_B, 0};
+    {
+      const std::vector<int>& ay = plan.atomic_mats[RG_Y_FROM_Z];
+      const std::vector<int>& az = plan.atomic_mats[RG_Z_FROM_Y];
+      if (std::find(ay.begin(), ay.end(), i) == ay.end()) {
+        probs[RG_Y_FROM_Z][i].ld16 = m.ldl; probs[RG_Y_FROM_Z][i].out_hi = m.Yhi; probs[RG_Y_FROM_Z][i].out_lo = m.Ylo;
+      }
+      if (std::find(az.begin(), az.end(), i) == az.end()) {
+        probs[RG_Z_FROM_Y][i].ld16 = m.ldl; probs[RG_Z_FROM_Y][i].out_hi = m.Zhi; probs[RG_Z_FROM_Y][i].out_lo = m.Zlo;
+      }
+    }
     probs[RG_GRAM_Y][i] = TcProblem{m.C32, m.L, m.L, m.L, base + RM_Y_B, base + RM_Y_B, 0};
     probs[RG_GRAM_Z][i] = TcProblem{m.C32, m.L, m.L, m.L, base + RM_Z_B, base + RM_Z_B, 0};
     probs[RG_APPLY_Y][i] = TcProblem{m.Yf, m.M, m.L, m.L, base + RM_Y_A, base + RM_RINV, 0};
@@ -752,6 +775,10 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   plan.d_syrk_tiles = reinterpret_cast<SyrkTile*>(plan.buf + o_syrk_t);
   plan.d_prep64 = reinterpret_cast<GramPrep64*>(plan.buf + o_prep64);
   plan.d_split_z = reinterpret_cast<SplitJob*>(plan.buf + o_sz);
+  plan.d_split_y_rest = reinterpret_cast<SplitJob*>(plan.buf + o_sy_rest);
+  plan.d_split_z_rest = reinterpret_cast<SplitJob*>(plan.buf + o_sz_rest);
+  plan.n_split_y_rest = static_cast<int>(sy_rest.size());
+  plan.n_split_z_rest = static_cast<int>(sz_rest.size());
   plan.d_jac = reinterpret_cast<JacobiMat*>(plan.buf + o_jac);
   plan.d_jac_init = reinterpret_cast<JacobiInit*>(plan.buf + o_jac_init);
   plan.d_jac_out = reinterpret_cast<JacobiOut*>(plan.buf + o_jac_out);
@@ -773,6 +800,8 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
       cudaMemcpy(plan.d_prep64, prep64.data(), sizeof(GramPrep64) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_split_y, sy.data(), sizeof(SplitJob) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_split_z, sz.data(), sizeof(SplitJob) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_split_y_rest, sy_rest.data(), sizeof(SplitJob) * sy_rest.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(plan.d_split_z_rest, sz_rest.data(), sizeof(SplitJob) * sz_rest.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_jac, jac.data(), sizeof(JacobiMat) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_jac_init, jac_init.data(), sizeof(JacobiInit) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemcpy(plan.d_jac_out, jac_out.data(), sizeof(JacobiOut) * n, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -900,17 +929,27 @@ inline ngalore_status refresh_tc_tri_inverse(RefreshPlan& plan, cudaStream_t str
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
-inline ngalore_status refresh_tc_split(RefreshPlan& plan, bool y_side, cudaStream_t stream, int64_t* launches) {
-  split_hilo_grouped_kernel<<<dim3(64, plan.n), 256, 0, stream>>>(y_side ? plan.d_split_y : plan.d_split_z);
+// after_product: the iterate has just left a product with G, which wrote the bf16 parts itself except for the
+// matrices whose K it splits.
+inline ngalore_status refresh_tc_split(RefreshPlan& plan, bool y_side, cudaStream_t stream, int64_t* launches,
+                                       bool after_product = false) {
+  const SplitJob* jobs = y_side ? plan.d_split_y : plan.d_split_z;
+  int n_jobs = plan.n;
+  if (after_product) {
+    jobs = y_side ? plan.d_split_y_rest : plan.d_split_z_rest;
+    n_jobs = y_side ? plan.n_split_y_rest : plan.n_split_z_rest;
+    if (n_jobs == 0) return NGALORE_OK;
+  }
+  split_hilo_grouped_kernel<<<dim3(64, n_jobs), 256, 0, stream>>>(jobs);
   *launches += 1;
   return cudaGetLastError() == cudaSuccess ? NGALORE_OK : NGALORE_ERR_CUDA;
 }
 
-// iterate (fp32, in Yf) -> well-conditioned basis, left both as fp32 and as its bf16 parts.
+// iterate (as it leaves the product Y = G Z) -> well-conditioned basis, left both as fp32 and as its bf16 parts.
 inline ngalore_status refresh_tc_orth(RefreshPlan& plan, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches,
                                       double shift_scale = 1.0) {
   ngalore_status rc;
-  if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;
+  if ((rc = refresh_tc_split(plan, true, stream, launches, true))) return rc;
   if ((rc = refresh_tc_gemm(plan, RG_GRAM_Y, d_ctrl, stream, launches))) return rc;
   // single precision from here to R^-1: the Gram matrix has 2^-17 of relative accuracy and a shift of about 1e-2
   gram_prep_kernel<float><<<dim3(plan.n, 8), 256, 0, stream>>>(plan.d_prep, shift_scale);
@@ -927,7 +966,7 @@ inline ngalore_status refresh_tc_orth(RefreshPlan& plan, Ctrl* d_ctrl, cudaStrea
 // the caller.
 inline ngalore_status refresh_tc_final(RefreshPlan& plan, Ctrl* d_ctrl, cudaStream_t stream, int64_t* launches) {
   ngalore_status rc;
-  if ((rc = refresh_tc_split(plan, true, stream, launches))) return rc;  // bf16 parts of the basis for the apply
+  // (the bf16 parts of the basis, which the apply below multiplies, are current: refresh_tc_orth ends with a split)
   zero_jobs_kernel<<<dim3(32, plan.n_zero[RG_COUNT]), 256, 0, stream>>>(plan.d_zero[RG_COUNT]);
   *launches += 1;
   syrk_f64_kernel<<<plan.n_syrk_tiles, 256, 0, stream>>>(plan.d_syrk_mats, plan.d_syrk_tiles);
@@ -991,7 +1030,7 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
     // (not with fewer than four sweeps, where every one of them counts)
     const bool coarse = q >= 4 && it < q / 2;
     if ((rc = refresh_tc_gemm(plan, RG_Z_FROM_Y, d_ctrl, stream, launches, coarse))) return rc;
-    if ((rc = refresh_tc_split(plan, false, stream, launches))) return rc;
+    if ((rc = refresh_tc_split(plan, false, stream, launches, true))) return rc;
     if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches, coarse))) return rc;
     if ((rc = refresh_tc_orth(plan, d_ctrl, stream, launches))) return rc;
   }
@@ -1007,7 +1046,7 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
   // finer than the gaps that decide a Ritz vector), V = eigenvectors of C (or of its leading block, see
   // ritz_jacobi.cuh), P = Q V.
   if ((rc = refresh_tc_gemm(plan, RG_Z_FROM_Y, d_ctrl, stream, launches))) return rc;
-  if ((rc = refresh_tc_split(plan, false, stream, launches))) return rc;
+  if ((rc = refresh_tc_split(plan, false, stream, launches, true))) return rc;
   if ((rc = refresh_tc_gemm(plan, RG_GRAM_Z, d_ctrl, stream, launches))) return rc;
   jacobi_init_kernel<<<plan.n, 256, 0, stream>>>(plan.d_jac, plan.d_jac_init);
   *launches += 1;
