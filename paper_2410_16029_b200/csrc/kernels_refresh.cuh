@@ -28,6 +28,26 @@ __global__ void fill_normal_kernel(float* X, long long n, unsigned long long see
   X[i] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
 }
 
+// The same values for a list of matrices in one launch: blockIdx.y selects the matrix (its stream of random numbers
+// is stream_base + blockIdx.y), blockIdx.x strides over its entries.
+struct FillJob {
+  float* X;
+  long long n;
+};
+
+__global__ void fill_normal_grouped_kernel(const FillJob* jobs, unsigned long long seed, unsigned long long stream_base) {
+  const FillJob jb = jobs[blockIdx.y];
+  const unsigned long long stream_id = stream_base + blockIdx.y;
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < jb.n; i += stride) {
+    const unsigned long long h =
+        splitmix64(seed ^ splitmix64(stream_id * 0x100000001B3ull + static_cast<unsigned long long>(i)));
+    const float u1 = (static_cast<float>(h >> 40) + 1.0f) * (1.0f / 16777217.0f);
+    const float u2 = static_cast<float>((h >> 8) & 0xFFFFFFull) * (1.0f / 16777216.0f);
+    jb.X[i] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+  }
+}
+
 // ---------------------------------------------------------------- batched Cholesky (fp64, right-looking, blocked)
 
 struct CholProblem {
@@ -456,6 +476,46 @@ __global__ void working_copies_kernel(const float* P32, uint16_t* P16, uint16_t*
   for (int a = threadIdx.y; a < 32; a += blockDim.y) {
     const int j = j0 + a, i = i0 + threadIdx.x;
     if (i < rows && j < rp) Pt16[static_cast<long long>(j) * ldpt + i] = working_bits(tile[threadIdx.x][a], p16_is_half == 0);
+  }
+}
+
+// The same for a list of matrices in one launch, reading the new basis where the refresh left it (src) and writing
+// the fp32 master as well.  CTA t works on a 32 x 32 tile; tile_start[j] is the first tile of job j (n_jobs + 1
+// entries, ascending).
+struct WorkingJob {
+  const float* src;   // rows x rp, dense
+  float* P32;
+  uint16_t* P16;
+  uint16_t* Pt16;
+  int rows, rp, ldp, ldpt;
+  int p16_is_half;
+  int tiles_x;        // tiles along the rp columns
+};
+
+__global__ void working_copies_grouped_kernel(const WorkingJob* jobs, const int* tile_start, int n_jobs) {
+  __shared__ float tile[32][33];
+  int lo = 0, hi = n_jobs;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (tile_start[mid] <= static_cast<int>(blockIdx.x)) lo = mid; else hi = mid;
+  }
+  const WorkingJob jb = jobs[lo];
+  const int t = static_cast<int>(blockIdx.x) - tile_start[lo];
+  const int i0 = (t / jb.tiles_x) * 32, j0 = (t % jb.tiles_x) * 32;
+  for (int a = threadIdx.y; a < 32; a += blockDim.y) {
+    const int i = i0 + a, j = j0 + threadIdx.x;
+    float val = 0.f;
+    if (i < jb.rows && j < jb.rp) {
+      val = jb.src[static_cast<long long>(i) * jb.rp + j];
+      jb.P32[static_cast<long long>(i) * jb.rp + j] = val;
+      jb.P16[static_cast<long long>(i) * jb.ldp + j] = working_bits(val, jb.p16_is_half != 0);
+    }
+    tile[a][threadIdx.x] = val;
+  }
+  __syncthreads();
+  for (int a = threadIdx.y; a < 32; a += blockDim.y) {
+    const int j = j0 + a, i = i0 + threadIdx.x;
+    if (i < jb.rows && j < jb.rp) jb.Pt16[static_cast<long long>(j) * jb.ldpt + i] = working_bits(tile[threadIdx.x][a], jb.p16_is_half == 0);
   }
 }
 

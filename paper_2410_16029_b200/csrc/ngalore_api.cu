@@ -95,6 +95,10 @@ struct ngalore_state {
   FusedPlan fused;
   // tensor-core refresh plan
   RefreshPlan refresh;
+  // working copies of the projectors of refresh_tc_idx in one launch (finish_refresh)
+  WorkingJob* d_wjobs = nullptr;
+  int* d_wtile_start = nullptr;
+  int n_wjobs = 0, n_wtiles = 0;
   // small-rank path (every r' <= 8): the step as two bandwidth kernels
   SrPlan sr;
   // host-buffer staging; W travels in groups of matrices so that the copies in, the back-projection and the
@@ -245,11 +249,18 @@ ngalore_status apply_gradient(ngalore_state* st, const std::vector<int>& idx, co
 ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bool basis_in_a, cudaStream_t stream,
                               bool whole_set) {
   ngalore_status rc;
-  for (int i : idx) {
-    const HostMat& hm = st->mats[i];
-    NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, basis_in_a ? hm.Ya : hm.Yb, sizeof(float) * hm.eM * hm.rp,
-                            cudaMemcpyDeviceToDevice, stream));
-    if ((rc = make_working_copies(st, i, stream))) return rc;
+  if (basis_in_a && st->n_wjobs > 0 && &idx == &st->refresh_tc_idx) {
+    // the whole tensor-core set: master and working copies of every projector in one launch
+    working_copies_grouped_kernel<<<st->n_wtiles, dim3(32, 8), 0, stream>>>(st->d_wjobs, st->d_wtile_start, st->n_wjobs);
+    st->launches += 1;
+    NG_CUDA(cudaGetLastError());
+  } else {
+    for (int i : idx) {
+      const HostMat& hm = st->mats[i];
+      NG_CUDA(cudaMemcpyAsync(st->h_desc[i].P32, basis_in_a ? hm.Ya : hm.Yb, sizeof(float) * hm.eM * hm.rp,
+                              cudaMemcpyDeviceToDevice, stream));
+      if ((rc = make_working_copies(st, i, stream))) return rc;
+    }
   }
   if (st->opt.reset_history_on_refresh && whole_set) {
     st->n_appended = 0;
@@ -802,6 +813,23 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
     if (!eff.empty()) {
       rc = refresh_plan_create(st->refresh, eff, Yf, Zf, prop.multiProcessorCount, ritz_columns(st));
       if (rc != NGALORE_OK) return fail(rc);
+      std::vector<WorkingJob> jobs;
+      std::vector<int> start(1, 0);
+      for (int i : st->refresh_tc_idx) {
+        const HostMat& hm = st->mats[i];
+        const MatDesc& d = st->h_desc[i];
+        const int tx = (hm.rp + 31) / 32, ty = (hm.eM + 31) / 32;
+        jobs.push_back(WorkingJob{hm.Ya, d.P32, d.P16, d.Pt16, hm.eM, hm.rp, d.ldp, d.ldpt, hm.right ? 0 : 1, tx});
+        start.push_back(start.back() + tx * ty);
+      }
+      st->n_wjobs = static_cast<int>(jobs.size());
+      st->n_wtiles = start.back();
+      if (cudaMalloc(&st->d_wjobs, sizeof(WorkingJob) * jobs.size()) != cudaSuccess ||
+          cudaMalloc(&st->d_wtile_start, sizeof(int) * start.size()) != cudaSuccess)
+        return fail(NGALORE_ERR_ALLOC);
+      if (cudaMemcpy(st->d_wjobs, jobs.data(), sizeof(WorkingJob) * jobs.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemcpy(st->d_wtile_start, start.data(), sizeof(int) * start.size(), cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(NGALORE_ERR_CUDA);
     }
   }
   for (int e = 0; e < 4; ++e)
@@ -831,6 +859,8 @@ void ngalore_destroy(ngalore_state* st) {
   if (st->copy_out) cudaStreamDestroy(st->copy_out);
   if (st->stage) cudaFree(st->stage);
   if (st->work) cudaFree(st->work);
+  if (st->d_wjobs) cudaFree(st->d_wjobs);
+  if (st->d_wtile_start) cudaFree(st->d_wtile_start);
   if (st->arena) cudaFree(st->arena);
   delete st;
 }

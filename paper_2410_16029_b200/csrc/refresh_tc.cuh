@@ -471,6 +471,7 @@ struct RefreshPlan {
   JacobiInit* d_jac_init = nullptr;
   JacobiOut* d_jac_out = nullptr;
   NormJob* d_norm = nullptr;
+  FillJob* d_fill = nullptr;   // the random start Z = Omega of every matrix
   ZeroJob* d_zero_d = nullptr;   // clears every matrix's D (as 16-byte words)
   int m_max = 0;                 // most rows among the matrices
 };
@@ -602,6 +603,7 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   const size_t o_jac_init = take(sizeof(JacobiInit) * n);
   const size_t o_jac_out = take(sizeof(JacobiOut) * n);
   const size_t o_norm = take(sizeof(NormJob) * n);
+  const size_t o_fill = take(sizeof(FillJob) * n);
   const size_t o_zero_d = take(sizeof(ZeroJob) * n);
   const size_t o_jac_flags = take(sizeof(int) * kJacMaxSweeps * n);
   if (cudaMalloc(&plan.buf, off) != cudaSuccess) { plan.buf = nullptr; return NGALORE_ERR_ALLOC; }
@@ -783,6 +785,12 @@ inline ngalore_status refresh_plan_create(RefreshPlan& plan, const std::vector<M
   plan.d_jac_init = reinterpret_cast<JacobiInit*>(plan.buf + o_jac_init);
   plan.d_jac_out = reinterpret_cast<JacobiOut*>(plan.buf + o_jac_out);
   plan.d_norm = reinterpret_cast<NormJob*>(plan.buf + o_norm);
+  plan.d_fill = reinterpret_cast<FillJob*>(plan.buf + o_fill);
+  {
+    std::vector<FillJob> fill(n);
+    for (int i = 0; i < n; ++i) fill[i] = FillJob{plan.mats[i].Zf, static_cast<long long>(plan.mats[i].N) * plan.mats[i].L};
+    if (cudaMemcpy(plan.d_fill, fill.data(), sizeof(FillJob) * n, cudaMemcpyHostToDevice) != cudaSuccess) return NGALORE_ERR_CUDA;
+  }
   plan.d_zero_d = reinterpret_cast<ZeroJob*>(plan.buf + o_zero_d);
   {
     std::vector<ZeroJob> zd(n);
@@ -1009,13 +1017,8 @@ inline ngalore_status refresh_tc_run(RefreshPlan& plan, const uint16_t* const* G
                                  cudaMemcpyHostToDevice, stream) != cudaSuccess)
     return NGALORE_ERR_CUDA;
   ngalore_status rc;
-  for (int i = 0; i < plan.n; ++i) {
-    const RefreshMat& m = plan.mats[i];
-    const long long cnt = static_cast<long long>(m.N) * m.L;
-    fill_normal_kernel<<<static_cast<unsigned>((cnt + 255) / 256), 256, 0, stream>>>(m.Zf, cnt, seed,
-                                                                                     stream_base + static_cast<unsigned>(i));
-    *launches += 1;
-  }
+  fill_normal_grouped_kernel<<<dim3(64, plan.n), 256, 0, stream>>>(plan.d_fill, seed, stream_base);
+  *launches += 1;
   if (cudaGetLastError() != cudaSuccess) return NGALORE_ERR_CUDA;
   if ((rc = refresh_tc_split(plan, false, stream, launches))) return rc;
   if ((rc = refresh_tc_gemm(plan, RG_Y_FROM_Z, d_ctrl, stream, launches))) return rc;
