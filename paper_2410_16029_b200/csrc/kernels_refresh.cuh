@@ -202,7 +202,7 @@ inline cudaError_t chol_batched_launch(CholProblem* d_probs, int n, int Lmax, cu
 // matrices as there are SMs this keeps every SM busy from the first panel to the last, where the launch-per-panel
 // version spends most of its time between kernels (a 512 x 512 factor is 16 panels, i.e. 32 launches of a few
 // tens of microseconds each, for 45 million multiply-adds).  Per panel: one warp factors the diagonal block in
-// shared memory, every thread solves one row of the panel against it (keeping the solved panel in shared memory,
+// registers, every thread solves one row of the panel against it (keeping the solved panel in shared memory,
 // column-major), and all threads update the trailing triangle in 4 x 4 register tiles straight in global memory
 // (the matrix stays in L2).  Shared memory: 32 x (L - 32) doubles for the panel.
 constexpr int kCholCtaThreads = 512;
@@ -228,6 +228,60 @@ __device__ __forceinline__ void chol_load4(const float* p, float (&a)[4]) {
   a[0] = v.x; a[1] = v.y; a[2] = v.z; a[3] = v.w;
 }
 
+// The diagonal block of a panel, by one warp: D (nbj x nbj, zero beyond) is replaced by its lower Cholesky factor
+// and rdiag receives the reciprocals of the factor's diagonal (zero beyond the block).  Lane i holds row i in
+// registers: step k takes the pivot from lane k, scales column k, and every lane subtracts its share of the
+// rank-one update with one shuffle per entry.  A function of its own so that its 32 row entries get registers
+// whatever the caller needs elsewhere.
+template <typename T>
+__device__ __noinline__ void chol_diag_block(T (*D)[kCholNB + 1], T* rdiag, int nbj, T tiny, int lane) {
+  constexpr int NB = kCholNB;
+  T r[NB];
+#pragma unroll
+  for (int j = 0; j < NB; ++j) r[j] = D[lane][j];
+#pragma unroll
+  for (int k = 0; k < NB; ++k) {
+    T dkk = __shfl_sync(0xffffffffu, r[k], k);
+    if (!(dkk > tiny)) dkk = tiny;
+    const T lkk = sqrt(dkk);
+    const T inv = T(1) / lkk;
+    if (lane == k) {
+      r[k] = lkk;
+      rdiag[k] = k < nbj ? inv : T(0);
+    }
+    if (lane > k) r[k] = r[k] * inv;
+    const T lik = r[k];
+#pragma unroll
+    for (int j = k + 1; j < NB; ++j) {
+      const T ljk = __shfl_sync(0xffffffffu, r[k], j);
+      if (lane >= j) r[j] -= lik * ljk;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < NB; ++j) D[lane][j] = (j <= lane && lane < nbj && j < nbj) ? r[j] : T(0);
+}
+
+// One row of the panel, held as entries p[jj * ldp] (jj = 0 .. 31) of the k-major panel in shared memory:
+// x D^T = c by forward substitution in place.  As soon as x_t is known every later entry takes its share of it, so
+// the dependent chain is one multiply and one multiply-add per t.
+template <typename T>
+__device__ __noinline__ void chol_panel_row(T* p, int ldp, const T (*D)[kCholNB + 1], const T* rdiag) {
+  constexpr int NB = kCholNB;
+  T a[NB];
+#pragma unroll
+  for (int jj = 0; jj < NB; ++jj) a[jj] = p[jj * ldp];
+#pragma unroll
+  for (int t = 0; t < NB; ++t) {
+    const T xt = a[t] * rdiag[t];
+    a[t] = xt;
+#pragma unroll
+    for (int jj = t + 1; jj < NB; ++jj) a[jj] -= xt * D[jj][t];
+    if ((t & 3) == 3) asm volatile("" ::: "memory");   // keeps the 496 loads of D from being lifted to the front
+  }
+#pragma unroll
+  for (int jj = 0; jj < NB; ++jj) p[jj * ldp] = a[jj];
+}
+
 // T = double: the factorisation as described.  T = float: the same on a matrix stored as L x L floats at the same
 // address (CholProblem::C reinterpreted); enough for the orthonormalisations between the products of the subspace
 // iteration, whose Gram matrices come from the tensor cores with 2^-17 of relative accuracy and carry a shift of
@@ -238,7 +292,8 @@ __global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const Chol
   constexpr int NB = kCholNB;
   extern __shared__ __align__(16) unsigned char chol_ps_raw[];
   T* chol_ps = reinterpret_cast<T*>(chol_ps_raw);    // panel, k-major: chol_ps[k * ldp + (row - base)]
-  __shared__ T D[NB][NB + 1];
+  __shared__ T D[NB][NB + 1];      // the diagonal block, then its lower Cholesky factor
+  __shared__ T rdiag[NB];          // reciprocals of the factor's diagonal
   __shared__ T s_tiny;
   const CholProblem p = probs[blockIdx.x];
   T* C = reinterpret_cast<T*>(p.C);
@@ -271,49 +326,24 @@ __global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const Chol
       D[a][b] = (a < nbj && b < nbj) ? C[static_cast<long long>(j0 + a) * L + j0 + b] : T(0);
     }
     __syncthreads();
-    if (tid < 32) {
-      const int lane = tid;
-      for (int k = 0; k < nbj; ++k) {
-        T dkk = D[k][k];
-        if (!(dkk > tiny)) dkk = tiny;
-        const T lkk = sqrt(dkk);
-        __syncwarp();
-        if (lane == k) D[k][k] = lkk;
-        if (lane > k && lane < nbj) D[lane][k] /= lkk;
-        __syncwarp();
-        if (lane > k && lane < nbj) {
-          const T lik = D[lane][k];
-          for (int j = k + 1; j <= lane; ++j) D[lane][j] -= lik * D[j][k];
-        }
-        __syncwarp();
-      }
-    }
+    if (tid < 32) chol_diag_block<T>(D, rdiag, nbj, tiny, tid);
     __syncthreads();
     for (int x = tid; x < NB * NB; x += kCholCtaThreads) {
       const int a = x / NB, b = x % NB;
       if (a < nbj && b <= a) C[static_cast<long long>(j0 + a) * L + j0 + b] = D[a][b];
     }
-    // panel rows: x D^T = c by forward substitution, one thread per row
-    for (int i = base + tid; i < L; i += kCholCtaThreads) {
-      T xr[NB];
-      T* crow = C + static_cast<long long>(i) * L + j0;
-#pragma unroll
-      for (int jj = 0; jj < NB; ++jj) {
-        if (jj < nbj) {
-          T a = crow[jj];
-#pragma unroll
-          for (int t = 0; t < NB; ++t)
-            if (t < jj) a -= xr[t] * D[jj][t];
-          xr[jj] = a / D[jj][jj];
-        } else {
-          xr[jj] = T(0);
-        }
-      }
-#pragma unroll
-      for (int jj = 0; jj < NB; ++jj) {
-        if (jj < nbj) crow[jj] = xr[jj];
-        chol_ps[jj * ldp + (i - base)] = xr[jj];
-      }
+    // panel rows: x D^T = c.  The rows come in through shared memory (a warp reads one row of 32
+    // entries at a time, so that global memory sees whole lines), one thread per row then works in place on its
+    // column of the k-major panel, and the solved rows go out the same way.
+    {
+      const int warp = tid >> 5, lane = tid & 31;
+      for (int r = warp; r < Tn; r += kCholCtaThreads / 32)
+        chol_ps[lane * ldp + r] = (lane < nbj) ? C[static_cast<long long>(base + r) * L + j0 + lane] : T(0);
+      __syncthreads();
+      for (int r = tid; r < Tn; r += kCholCtaThreads) chol_panel_row<T>(chol_ps + r, ldp, D, rdiag);
+      __syncthreads();
+      for (int r = warp; r < Tn; r += kCholCtaThreads / 32)
+        if (lane < nbj) C[static_cast<long long>(base + r) * L + j0 + lane] = chol_ps[lane * ldp + r];
     }
     __syncthreads();
     // trailing update on the lower triangle: C[i][j] -= sum_k panel[i][k] panel[j][k], 4 x 4 tiles
