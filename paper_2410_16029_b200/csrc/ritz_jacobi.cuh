@@ -119,7 +119,7 @@ constexpr int kJacCluster = 4;
 constexpr int kJacCtaThreads = 128;
 constexpr int kJacPairsPerCta = 2;
 constexpr int kJacStageRows = 64;                     // rows of the columns staged per Gram chunk
-constexpr int kJacPad = kJacCols + 1;
+constexpr int kJacPad = kJacCols + 4;
 
 __device__ __forceinline__ void jacobi_cluster_barrier() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -142,26 +142,29 @@ __device__ __forceinline__ JacobiPairInfo jacobi_pair_of(const JacobiMat& m, int
 
 // Shared memory of a CTA, two regions that change hands between the phases of a pair's visit:
 //   region 1: Gram: the staged rows (32 x 64 floats, quads swizzled by row so that the 4 x 4 tiles read them
-//             without bank conflicts) and two partial Gram matrices; eigensolve: the second operand Bs;
-//             polish: J^T in double precision; apply: the rotations in single precision (rows padded to 36)
-//   region 2: eigensolve: As (the Gram matrix, rotated in place) and JT (JT[a][b] = J[b][a]); polish: J^T J - I in
-//             the place of As; then the polished rotations in double precision (rows padded to 34)
+//             without bank conflicts) and two partial Gram matrices; eigensolve: the intermediate Bs = A R;
+//             polish: J^T in double precision; apply: the rotations in single precision
+//   region 2: eigensolve: As (the Gram matrix, rotated in place) and Js (the accumulated rotation, Js[b][a] =
+//             coefficient of old column b in new column a); polish: J^T J - I in the place of As; then the polished
+//             rotations in double precision (rows padded to 34)
+// The 32 x 32 single-precision matrices have rows of 36 floats: 16-byte rows whose quarter-warp accesses fall into
+// different banks.
 constexpr int kJacLdD = kJacCols + 2;     // row length of the 32 x 32 double-precision matrices (16-byte rows)
 constexpr int kJacLdF = kJacCols + 4;     // the same for the single-precision copy
 constexpr size_t kJacStageBytes = sizeof(float) * kJacCols * kJacStageRows;
 constexpr size_t kJacMat32Bytes = sizeof(float) * kJacCols * kJacPad;
 constexpr size_t kJacMat64Bytes = sizeof(double) * kJacCols * kJacLdD;
-constexpr size_t kJacRegion1Bytes = kJacPairsPerCta * kJacMat64Bytes;
-constexpr size_t kJacRegion2Bytes = kJacPairsPerCta * kJacMat64Bytes;
-static_assert(kJacStageBytes + 2 * kJacMat32Bytes <= kJacRegion1Bytes, "Gram phase fits region 1");
+constexpr size_t kJacRegion1Bytes = kJacStageBytes + 2 * kJacMat32Bytes;
+constexpr size_t kJacRegion2Bytes = 2 * kJacPairsPerCta * kJacMat32Bytes;
+static_assert(kJacPairsPerCta * kJacMat64Bytes <= kJacRegion1Bytes, "double-precision J^T fits region 1");
+static_assert(kJacPairsPerCta * kJacMat64Bytes <= kJacRegion2Bytes, "double-precision rotations fit region 2");
+static_assert(kJacPairsPerCta * kJacMat32Bytes <= kJacRegion1Bytes, "Bs fits region 1");
 static_assert(kJacPairsPerCta * sizeof(float) * kJacCols * kJacLdF <= kJacRegion1Bytes, "single-precision rotations fit");
-static_assert(2 * kJacPairsPerCta * kJacMat32Bytes <= kJacRegion2Bytes, "As and JT fit region 2");
 
 struct JacobiShared {
   __align__(16) unsigned char r1[kJacRegion1Bytes];
   __align__(16) unsigned char r2[kJacRegion2Bytes];
-  float ca[kJacPairsPerCta][kJacCols], cb[kJacPairsPerCta][kJacCols];
-  unsigned char partner[kJacPairsPerCta][kJacCols];
+  __align__(16) float2 cs[kJacPairsPerCta][kJacBlock];   // cosine and sine of the 16 rotations of a step
   int active[kJacPairsPerCta];
 };
 
@@ -174,11 +177,11 @@ jacobi_cluster_kernel(const JacobiMat* mats) {
   typedef float MatF[kJacCols][kJacLdF];
   float* stage = reinterpret_cast<float*>(sh.r1);                               // [32][64], swizzled
   Mat32* Ap = reinterpret_cast<Mat32*>(sh.r1 + kJacStageBytes);                  // [2] partial Gram matrices
-  Mat32* Bs = reinterpret_cast<Mat32*>(sh.r1 + kJacStageBytes);                  // [pair]
+  Mat32* Bs = reinterpret_cast<Mat32*>(sh.r1);                                   // [pair]
   Mat64* JTd = reinterpret_cast<Mat64*>(sh.r1);                                  // [pair]
   MatF* Jf = reinterpret_cast<MatF*>(sh.r1);                                     // [pair]
   Mat32* As = reinterpret_cast<Mat32*>(sh.r2);                                   // [pair]; later J^T J - I
-  Mat32* JT = reinterpret_cast<Mat32*>(sh.r2 + kJacPairsPerCta * kJacMat32Bytes);  // [pair]
+  Mat32* Js = reinterpret_cast<Mat32*>(sh.r2 + kJacPairsPerCta * kJacMat32Bytes);  // [pair]
   Mat64* Jd = reinterpret_cast<Mat64*>(sh.r2);                                   // [pair]
 
   const JacobiMat m = mats[blockIdx.x / kJacCluster];
@@ -265,23 +268,61 @@ jacobi_cluster_kernel(const JacobiMat* mats) {
         const bool act0 = sh.active[0] != 0, act1 = sh.active[1] != 0;
         if (!act0 && !act1) continue;                       // the same for every thread of the CTA
 
-        // ---- eigenvectors of the Gram matrices: 64 threads per pair, both pairs in step ----
+        // ---- eigenvectors of the Gram matrices: 64 threads per pair, both pairs in step.  Cyclic two-sided
+        // Jacobi in the ordering of Brent and Luk: the 16 rotations of a step act on the columns (and rows) at
+        // positions (2i, 2i + 1), and every step ends by moving the columns and rows to the positions of their
+        // next partners (position 0 stays, the even positions move up by two, the odd ones down by two, the ends
+        // turn around).  After the 31 steps of a sweep every pair has met once and everything is back in its
+        // place.  A thread holds 16 consecutive entries of one row, i.e. eight whole pairs, so the column
+        // rotation and the move happen in registers (one shuffle with the thread that holds the other half of the
+        // row) and all shared-memory traffic is 16-byte accesses. ----
         {
           const int p = tid >> 6, lt = tid & 63;
-          const int r = lt >> 1, j0 = (lt & 1) * 16;        // this thread: row r, columns j0 .. j0 + 15
+          const int r = lt >> 1, h = lt & 1;                // this thread: row r, positions 16 h .. 16 h + 15
           const bool mine = p == 0 ? act0 : act1;
           float(&A)[kJacCols][kJacPad] = As[p];
           float(&B)[kJacCols][kJacPad] = Bs[p];
-          float(&T)[kJacCols][kJacPad] = JT[p];
+          float(&J)[kJacCols][kJacPad] = Js[p];
+          // where row (or column) r goes at the end of a step
+          const int r_next = r == 0 ? 0 : (r == 1 ? 2 : (r == kJacCols - 2 ? kJacCols - 1 : ((r & 1) ? r - 2 : r + 2)));
 #pragma unroll
-          for (int y = 0; y < 16; ++y) T[r][j0 + y] = (r == j0 + y) ? 1.f : 0.f;
+          for (int y = 0; y < 16; ++y) J[r][16 * h + y] = (r == 16 * h + y) ? 1.f : 0.f;
           __syncthreads();
+          auto load16 = [&](const float* src, float (&v)[16]) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float4 x = *reinterpret_cast<const float4*>(src + 4 * q);
+              v[4 * q] = x.x; v[4 * q + 1] = x.y; v[4 * q + 2] = x.z; v[4 * q + 3] = x.w;
+            }
+          };
+          auto store16 = [&](float* dst, const float (&v)[16]) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              *reinterpret_cast<float4*>(dst + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+          };
+          // v <- (v R) moved: rotate the eight pairs, then shift the even entries up and the odd ones down by one
+          // pair; the entry that leaves this half of the row is traded for the one that enters it
+          auto rotate_and_move = [&](float (&v)[16], const float2 (&c)[8]) {
+            float t[16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              t[2 * i] = c[i].x * v[2 * i] - c[i].y * v[2 * i + 1];
+              t[2 * i + 1] = c[i].y * v[2 * i] + c[i].x * v[2 * i + 1];
+            }
+            const float recv = __shfl_xor_sync(0xffffffffu, h ? t[1] : t[14], 1);
+            v[0] = h ? recv : t[0];
+            v[2] = h ? t[0] : t[1];
+#pragma unroll
+            for (int i = 2; i < 8; ++i) v[2 * i] = t[2 * i - 2];
+#pragma unroll
+            for (int i = 0; i < 7; ++i) v[2 * i + 1] = t[2 * i + 3];
+            v[15] = h ? t[14] : recv;
+          };
           for (int isweep = 0; isweep < kJacInnerSweeps; ++isweep) {
             int rotated = 0;
             for (int step = 0; step < kJacCols - 1; ++step) {
               if (lt < kJacBlock) {
-                int a, b;
-                round_robin_pair(kJacCols, step, lt, a, b);
+                const int a = 2 * lt, b = 2 * lt + 1;
                 const float aaa = A[a][a], abb = A[b][b], aab = A[a][b];
                 float c = 1.f, sn = 0.f;
                 if (mine && aab * aab > 1e-12f * aaa * abb && aab != 0.f) {
@@ -291,27 +332,32 @@ jacobi_cluster_kernel(const JacobiMat* mats) {
                   sn = t * c;
                   rotated = 1;
                 }
-                sh.ca[p][a] = c; sh.cb[p][a] = -sn; sh.partner[p][a] = static_cast<unsigned char>(b);
-                sh.ca[p][b] = c; sh.cb[p][b] = sn; sh.partner[p][b] = static_cast<unsigned char>(a);
+                sh.cs[p][lt] = make_float2(c, sn);
               }
               __syncthreads();
-              float t[16];
+              float2 c8[8];
 #pragma unroll
-              for (int y = 0; y < 16; ++y)
-                t[y] = sh.ca[p][j0 + y] * A[r][j0 + y] + sh.cb[p][j0 + y] * A[r][sh.partner[p][j0 + y]];
-#pragma unroll
-              for (int y = 0; y < 16; ++y) B[r][j0 + y] = t[y];                          // B = A R
-              __syncthreads();
-              const float car = sh.ca[p][r], cbr = sh.cb[p][r];
-              const int pr = sh.partner[p][r];
-#pragma unroll
-              for (int y = 0; y < 16; ++y) {
-                A[r][j0 + y] = car * B[r][j0 + y] + cbr * B[pr][j0 + y];                 // A <- R^T B
-                t[y] = car * T[r][j0 + y] + cbr * T[pr][j0 + y];                         // row r of JT = column r of J
+              for (int q = 0; q < 4; ++q) {
+                const float4 x = *reinterpret_cast<const float4*>(&sh.cs[p][8 * h + 2 * q]);
+                c8[2 * q] = make_float2(x.x, x.y);
+                c8[2 * q + 1] = make_float2(x.z, x.w);
               }
+              float v[16];
+              load16(&A[r][16 * h], v);
+              rotate_and_move(v, c8);
+              store16(&B[r][16 * h], v);                                                   // B = (A R) moved
+              load16(&J[r][16 * h], v);
+              rotate_and_move(v, c8);
+              store16(&J[r][16 * h], v);                                                   // J <- (J R) moved
               __syncthreads();
+              const float2 cr = sh.cs[p][r >> 1];
+              float w[16];
+              load16(&B[r][16 * h], v);
+              load16(&B[r ^ 1][16 * h], w);
 #pragma unroll
-              for (int y = 0; y < 16; ++y) T[r][j0 + y] = t[y];
+              for (int y = 0; y < 16; ++y) v[y] = (r & 1) ? cr.y * w[y] + cr.x * v[y] : cr.x * v[y] - cr.y * w[y];
+              store16(&A[r_next][16 * h], v);                                              // A <- (R^T B) moved
+              __syncthreads();
             }
             if (!__syncthreads_or(rotated)) break;
           }
@@ -324,7 +370,7 @@ jacobi_cluster_kernel(const JacobiMat* mats) {
           const int p = tid >> 6, a = (tid & 63) >> 1, h0 = (tid & 1) * 16;
           for (int x = tid; x < kJacPairsPerCta * kJacCols * kJacCols; x += kJacCtaThreads) {
             const int pp = x / (kJacCols * kJacCols), aa = (x / kJacCols) % kJacCols, bb = x % kJacCols;
-            JTd[pp][aa][bb] = static_cast<double>(JT[pp][aa][bb]);
+            JTd[pp][aa][bb] = static_cast<double>(Js[pp][bb][aa]);
           }
           __syncthreads();
           {
