@@ -51,7 +51,11 @@ def check_columns(P, G64, rp, label, rotated=256):
     return len(cols), worst
 
 
-@pytest.mark.parametrize("impl", [pytest.param(dict(gemm_impl=0), id="tcgen05"), pytest.param(dict(gemm_impl=1), id="simt")])
+@pytest.mark.parametrize("impl", [pytest.param(dict(gemm_impl=0), id="tcgen05"), pytest.param(dict(gemm_impl=1), id="simt"),
+                                  # fewer than four sweeps: every product takes both bf16 parts of the basis;
+                                  # eight: the first four take the high part only
+                                  pytest.param(dict(gemm_impl=0, power_iterations=3), id="tcgen05-3-sweeps"),
+                                  pytest.param(dict(gemm_impl=0, power_iterations=8), id="tcgen05-8-sweeps")])
 def test_config0_columns_are_singular_vectors(impl):
     w = wl.WORKLOADS[0]
     dev = torch.device("cuda")
