@@ -106,8 +106,8 @@ typedef struct {
                                        iteration orders its basis by strength, so the determined singular vectors sit
                                        at the front; a weak one close to the noise level is still spread over a few
                                        hundred columns of an unconverged basis, which is why the default is not
-                                       smaller); -1: all r' columns (the full Rayleigh-Ritz step, about 2.5 times the
-                                       refresh time at r' = 512). */
+                                       smaller); -1: all r' columns (the full Rayleigh-Ritz step; the cost of the
+                                       eigensolve grows with the cube of the number of columns). */
   int32_t moments_bf16;             /* 0 (default): the Adam moments are fp32.  1: reduced-precision state (the paper's
                                        conclusion names it as future work): m is stored as bf16 rounded to nearest; v is
                                        stored as bf16 with stochastic rounding (one step changes v by a relative
