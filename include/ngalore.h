@@ -170,6 +170,9 @@ ngalore_status ngalore_step(ngalore_state* st, float* const* W, const uint16_t* 
  * (G is still the full array of n_matrices pointers; only entry matrix_index is read).
  * Uses a randomized subspace iteration; P is orthonormal to fp32 accuracy and is
  * stored both as an fp32 master and as the working copies the step reads (the master's values rounded to bf16).
+ * Degenerate gradients: a gradient of zeros (a frozen layer) has no leading subspace; its matrix gets the first r'
+ * unit vectors as P and no status.  A gradient with entries that are not finite gets the same P and
+ * NGALORE_ERR_NONFINITE in its status word; the other matrices are refreshed as usual.
  */
 ngalore_status ngalore_refresh_subspace(ngalore_state* st, const uint16_t* const* G, int matrix_index,
                                         void* stream);

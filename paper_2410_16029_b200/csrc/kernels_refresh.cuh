@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(32) chol_begin_kernel(CholProblem* probs) {
   for (int i = threadIdx.x; i < p.L; i += 32) md = fmax(md, p.C[static_cast<long long>(i) * p.L + i]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) md = fmax(md, __shfl_xor_sync(0xffffffffu, md, o));
-  if (threadIdx.x == 0) p.tiny = fmax(md, 1e-300) * 1e-28;
+  if (threadIdx.x == 0) p.tiny = fmax(md * 1e-28, 1e-300);   // never zero: a matrix of zeros still factors
 }
 
 // Panel step at column j0, one CTA per matrix: factor the diagonal block in shared memory (one warp, lane = row),
@@ -311,8 +311,8 @@ __global__ void __launch_bounds__(kCholCtaThreads, 1) chol_cta_kernel(const Chol
       const T v = __shfl_xor_sync(0xffffffffu, md, o);
       md = v > md ? v : md;
     }
-    if (tid == 0) s_tiny = sizeof(T) == 8 ? static_cast<T>(fmax(static_cast<double>(md), 1e-300) * 1e-28)
-                                          : static_cast<T>(fmax(static_cast<double>(md), 1e-30) * 1e-12);
+    if (tid == 0) s_tiny = sizeof(T) == 8 ? static_cast<T>(fmax(static_cast<double>(md) * 1e-28, 1e-300))
+                                          : static_cast<T>(fmax(static_cast<double>(md) * 1e-12, 1e-30));
   }
   __syncthreads();
   const T tiny = s_tiny;
@@ -547,6 +547,58 @@ __global__ void working_copies_grouped_kernel(const WorkingJob* jobs, const int*
     const int j = j0 + a, i = i0 + threadIdx.x;
     if (i < jb.rows && j < jb.rp) jb.Pt16[static_cast<long long>(j) * jb.ldpt + i] = working_bits(tile[threadIdx.x][a], jb.p16_is_half == 0);
   }
+}
+
+// A refreshed basis that is no basis: all zeros (the gradient of a frozen layer: every product of the iteration is
+// zero and nothing can be normalised) or with entries that are not finite (a gradient with such entries).  Any
+// orthonormal basis serves a zero gradient, so such a matrix gets the first r' unit vectors; the second case also
+// raises the matrix's status word.  Two launches over a list of matrices: sums, then the repair.
+struct BasisJob {
+  float* Ya;       // rows x rp, dense: the basis, in one of the two buffers of the refresh
+  float* Yb;
+  double* acc;     // [0]: sum of squares, [1]: number of entries that are not finite (cleared by the caller)
+  int* status;
+  int rows, rp;
+};
+
+__global__ void __launch_bounds__(256) basis_check_kernel(const BasisJob* jobs, int in_a) {
+  __shared__ double red[8];
+  __shared__ int bad_any;
+  const BasisJob jb = jobs[blockIdx.y];
+  const float* Y = in_a ? jb.Ya : jb.Yb;
+  const long long n = static_cast<long long>(jb.rows) * jb.rp;
+  if (threadIdx.x == 0) bad_any = 0;
+  __syncthreads();
+  double s = 0.0;
+  int bad = 0;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += 256ll * gridDim.x) {
+    const float x = Y[i];
+    if (isfinite(x)) s += static_cast<double>(x) * static_cast<double>(x);
+    else bad = 1;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+  if (bad) bad_any = 1;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) t += red[w];
+    if (t != 0.0) atomicAdd(jb.acc, t);
+    if (bad_any) atomicAdd(jb.acc + 1, 1.0);
+  }
+}
+
+__global__ void __launch_bounds__(256) basis_repair_kernel(const BasisJob* jobs, int in_a) {
+  const BasisJob jb = jobs[blockIdx.y];
+  const bool nonfinite = jb.acc[1] > 0.0;
+  if (!nonfinite && jb.acc[0] > 0.0) return;
+  float* Y = in_a ? jb.Ya : jb.Yb;
+  const long long n = static_cast<long long>(jb.rows) * jb.rp;
+  for (long long i = blockIdx.x * 256ll + threadIdx.x; i < n; i += 256ll * gridDim.x)
+    Y[i] = (i / jb.rp == i % jb.rp) ? 1.f : 0.f;
+  if (nonfinite && blockIdx.x == 0 && threadIdx.x == 0) atomicCAS(jb.status, 0, 7 /* NGALORE_ERR_NONFINITE */);
 }
 
 // dst (rows x cols, dense fp32) = src (rows x cols, leading dimension ld; fp16 or bf16 bits)

@@ -95,6 +95,11 @@ struct ngalore_state {
   FusedPlan fused;
   // tensor-core refresh plan
   RefreshPlan refresh;
+  // check and repair of a refreshed basis (finish_refresh): one job per matrix, and the jobs of refresh_tc_idx again
+  // in that order
+  BasisJob* d_bjobs = nullptr;
+  BasisJob* d_bjobs_tc = nullptr;
+  double* d_bacc = nullptr;
   // working copies of the projectors of refresh_tc_idx in one launch (finish_refresh)
   WorkingJob* d_wjobs = nullptr;
   int* d_wtile_start = nullptr;
@@ -246,10 +251,27 @@ ngalore_status apply_gradient(ngalore_state* st, const std::vector<int>& idx, co
 }
 
 // whole_set: this call completes a refresh of every matrix (even when idx lists only part of them).
+// tc_set: idx is the whole list of matrices refreshed on the tensor-core path (ngalore_state::refresh_tc_idx), for
+// which the copies of all projectors are one prepared launch.
 ngalore_status finish_refresh(ngalore_state* st, const std::vector<int>& idx, bool basis_in_a, cudaStream_t stream,
-                              bool whole_set) {
+                              bool whole_set, bool tc_set = false) {
   ngalore_status rc;
-  if (basis_in_a && st->n_wjobs > 0 && &idx == &st->refresh_tc_idx) {
+  // a basis of zeros (zero gradient) or with entries that are not finite becomes the first r' unit vectors
+  NG_CUDA(cudaMemsetAsync(st->d_bacc, 0, sizeof(double) * 2 * st->n, stream));
+  if (tc_set) {
+    const dim3 grid(32, static_cast<unsigned>(idx.size()));
+    basis_check_kernel<<<grid, 256, 0, stream>>>(st->d_bjobs_tc, basis_in_a ? 1 : 0);
+    basis_repair_kernel<<<grid, 256, 0, stream>>>(st->d_bjobs_tc, basis_in_a ? 1 : 0);
+    st->launches += 2;
+  } else {
+    for (int i : idx) {
+      basis_check_kernel<<<dim3(32, 1), 256, 0, stream>>>(st->d_bjobs + i, basis_in_a ? 1 : 0);
+      basis_repair_kernel<<<dim3(32, 1), 256, 0, stream>>>(st->d_bjobs + i, basis_in_a ? 1 : 0);
+      st->launches += 2;
+    }
+  }
+  NG_CUDA(cudaGetLastError());
+  if (tc_set && basis_in_a && st->n_wjobs > 0) {
     // the whole tensor-core set: master and working copies of every projector in one launch
     working_copies_grouped_kernel<<<st->n_wtiles, dim3(32, 8), 0, stream>>>(st->d_wjobs, st->d_wtile_start, st->n_wjobs);
     st->launches += 1;
@@ -376,7 +398,7 @@ ngalore_status refresh_impl(ngalore_state* st, const uint16_t* const* G_in, cons
       NG_CUDA(cudaMemcpyAsync(hm.Ya, hm.Yb, sizeof(float) * hm.eM * hm.rp, cudaMemcpyDeviceToDevice, stream));
     }
   }
-  return finish_refresh(st, st->refresh_tc_idx, true, stream, true);
+  return finish_refresh(st, st->refresh_tc_idx, true, stream, true, true);
 }
 
 // grouped: the caller delivers W in the groups of ngalore_state::group_first; the back-projection of a group waits
@@ -832,6 +854,22 @@ ngalore_status ngalore_create(const ngalore_shape* shapes, int n_matrices, int r
         return fail(NGALORE_ERR_CUDA);
     }
   }
+  {
+    if (cudaMalloc(&st->d_bacc, sizeof(double) * 2 * n_matrices) != cudaSuccess ||
+        cudaMalloc(&st->d_bjobs, sizeof(BasisJob) * n_matrices) != cudaSuccess ||
+        cudaMalloc(&st->d_bjobs_tc, sizeof(BasisJob) * (st->refresh_tc_idx.size() + 1)) != cudaSuccess)
+      return fail(NGALORE_ERR_ALLOC);
+    std::vector<BasisJob> jobs(n_matrices), jobs_tc;
+    for (int i = 0; i < n_matrices; ++i) {
+      const HostMat& hm = st->mats[i];
+      jobs[i] = BasisJob{hm.Ya, hm.Yb, st->d_bacc + 2 * i, st->d_status + i, hm.eM, hm.rp};
+    }
+    for (int i : st->refresh_tc_idx) jobs_tc.push_back(jobs[i]);
+    if (cudaMemcpy(st->d_bjobs, jobs.data(), sizeof(BasisJob) * jobs.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+        (!jobs_tc.empty() && cudaMemcpy(st->d_bjobs_tc, jobs_tc.data(), sizeof(BasisJob) * jobs_tc.size(),
+                                        cudaMemcpyHostToDevice) != cudaSuccess))
+      return fail(NGALORE_ERR_CUDA);
+  }
   for (int e = 0; e < 4; ++e)
     if (cudaEventCreate(&st->ev[e]) != cudaSuccess) return fail(NGALORE_ERR_CUDA);
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(NGALORE_ERR_CUDA);
@@ -859,6 +897,9 @@ void ngalore_destroy(ngalore_state* st) {
   if (st->copy_out) cudaStreamDestroy(st->copy_out);
   if (st->stage) cudaFree(st->stage);
   if (st->work) cudaFree(st->work);
+  if (st->d_bjobs) cudaFree(st->d_bjobs);
+  if (st->d_bjobs_tc) cudaFree(st->d_bjobs_tc);
+  if (st->d_bacc) cudaFree(st->d_bacc);
   if (st->d_wjobs) cudaFree(st->d_wjobs);
   if (st->d_wtile_start) cudaFree(st->d_wtile_start);
   if (st->arena) cudaFree(st->arena);

@@ -504,7 +504,10 @@ __global__ void __launch_bounds__(256) jacobi_finish_kernel(const JacobiMat* mat
     }
 #pragma unroll
     for (int of = 16; of > 0; of >>= 1) s += __shfl_xor_sync(0xffffffffu, s, of);
-    if (lane == 0) nrm[i] = s;
+    if (lane == 0) {
+      nrm[i] = (s == s) ? s : -1.f;   // a norm that is no number goes last: the order below stays total
+      rank_of[i] = i;                 // (every entry holds a valid column whatever happens below)
+    }
   }
   __syncthreads();
   // position of column i in the falling order (ties by index); position -> column

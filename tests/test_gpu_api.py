@@ -370,3 +370,65 @@ def test_update_groups_and_overlapped_exchange_with_one_rank():
         assert all(torch.equal(x, y) for x, y in zip(Wc, Wd))
     finally:
         dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("impl", [pytest.param(dict(gemm_impl=0), id="tcgen05"), pytest.param(dict(gemm_impl=1), id="simt")])
+def test_refresh_and_step_on_a_zero_gradient(impl):
+    """A frozen layer: its gradient is all zeros, at the refresh and in the steps.  There is no subspace to find; what
+    is asked of the library is that the projector stays finite, no status is raised for it or for its neighbours, its
+    weights only see the decay, and the other matrix is updated as if it were alone."""
+    from paper_2410_16029_b200.ngalore import NGaLore
+
+    shapes = [(264, 520), (136, 264)]
+    w = wl.tiny_workload(shapes, r=16, s=3, T=0, inner_rank=4, index=91, wd=0.1)
+    dev = torch.device("cuda")
+    both = _make(w, **impl)
+    alone = NGaLore([shapes[1]], w.r, w.s, 0, lam=w.lam, lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps, wd=w.wd, **impl)
+    zero = torch.zeros(shapes[0], dtype=torch.bfloat16, device=dev)
+    g1 = [wl.gradient_device(w, 1, k, dev) for k in range(4)]
+    both.refresh_subspace([zero, g1[0]])
+    alone.refresh_subspace([g1[0]])
+    torch.cuda.synchronize()
+    P0 = both.get_subspace(0)
+    assert torch.isfinite(P0).all()
+    alone.set_subspace(0, both.get_subspace(1))          # same projector for the live matrix on both sides
+    W = [wl.initial_weight_device(w, i, dev) for i in range(2)]
+    Wl = [W[1].clone()]
+    W0 = W[0].clone()
+    for k in range(4):
+        both.step(W, [zero, g1[k]])
+        alone.step(Wl, [g1[k]])
+    torch.cuda.synchronize()
+    assert both.poll_status() == (0, [0, 0])
+    assert torch.isfinite(W[0]).all()
+    expect = W0 * (1.0 - w.lr * w.wd) ** 4
+    assert torch.allclose(W[0], expect, rtol=1e-5, atol=1e-7)     # u = 0 / sqrt(0 + eps) = 0: decay only
+    assert torch.equal(W[1], Wl[0])
+
+
+def test_refresh_on_a_gradient_that_is_not_finite():
+    """A NaN in the gradient a refresh is given: that matrix's status says so, its projector becomes the first r' unit
+    vectors (finite, orthonormal), the other matrix is refreshed as usual, and a later refresh on a clean gradient is
+    regular again."""
+    shapes = [(264, 520), (136, 264)]
+    w = wl.tiny_workload(shapes, r=16, s=3, T=0, inner_rank=4, index=92)
+    dev = torch.device("cuda")
+    opt = _make(w)
+    good = [wl.gradient_device(w, i, 0, dev) for i in range(2)]
+    bad = good[0].clone()
+    bad[7, 11] = float("nan")
+    opt.refresh_subspace([bad, good[1]])
+    torch.cuda.synchronize()
+    code, per = opt.poll_status()
+    assert code == 7 and per == [7, 0], (code, per)
+    P0 = opt.get_subspace(0)
+    expect = torch.zeros_like(P0)
+    expect[:16, :16] = torch.eye(16, device=dev)
+    assert torch.equal(P0, expect)
+    P1 = opt.get_subspace(1).double()
+    assert torch.allclose(P1.T @ P1, torch.eye(16, device=dev, dtype=torch.float64), atol=1e-5)
+    opt.refresh_subspace(good)
+    torch.cuda.synchronize()
+    assert opt.poll_status() == (0, [0, 0])
+    P0 = opt.get_subspace(0).double()
+    assert torch.allclose(P0.T @ P0, torch.eye(16, device=dev, dtype=torch.float64), atol=1e-5)
