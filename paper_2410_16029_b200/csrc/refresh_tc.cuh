@@ -156,15 +156,26 @@ __global__ void __launch_bounds__(256) syrk_f64_kernel(const SyrkMat* mats, cons
   for (int a = 0; a < 4; ++a)
 #pragma unroll
     for (int b = 0; b < 4; ++b) acc[a][b] = 0.0;
+  // the next 16 rows are fetched into registers while the current ones are multiplied
+  const int lc = threadIdx.x & 63, lk = threadIdx.x >> 6;
+  float pa[4], pb[4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      const int k = k0 + lk + 4 * p;
+      pa[p] = (k < k1 && i0 + lc < m.L) ? m.Y[static_cast<long long>(k) * m.L + i0 + lc] : 0.f;
+      pb[p] = (k < k1 && j0 + lc < m.L) ? m.Y[static_cast<long long>(k) * m.L + j0 + lc] : 0.f;
+    }
+  };
+  fetch(t.k0);
   for (int k0 = t.k0; k0 < k1; k0 += 16) {
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
-      const int kk = (threadIdx.x >> 6) + 4 * p, c = threadIdx.x & 63;
-      const int k = k0 + kk;
-      As[kk][c] = (k < k1 && i0 + c < m.L) ? m.Y[static_cast<long long>(k) * m.L + i0 + c] : 0.f;
-      Bs[kk][c] = (k < k1 && j0 + c < m.L) ? m.Y[static_cast<long long>(k) * m.L + j0 + c] : 0.f;
+      As[lk + 4 * p][lc] = pa[p];
+      Bs[lk + 4 * p][lc] = pb[p];
     }
     __syncthreads();
+    if (k0 + 16 < k1) fetch(k0 + 16);
 #pragma unroll
     for (int kk = 0; kk < 16; ++kk) {
       double a[4], b[4];
